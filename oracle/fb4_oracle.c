@@ -1,0 +1,362 @@
+/*
+ * fb4_oracle.c -- TEST INFRASTRUCTURE, not product code.
+ *
+ * A plain, slow, table-free CPU statement of what the FB4 online activation
+ * quantizer computes (SemanticDialect, Sec. 3.1-3.4), used only to check the
+ * CUDA library and to time a CPU baseline.  Only the tests, the smoke check and
+ * the benchmark's cpu-baseline/reference legs may call it; the CUDA library
+ * never does, and the two share no code, headers, tables or constants.
+ *
+ * Everything is done by direct arithmetic in double precision / integers, one
+ * block at a time, in the order the paper gives:
+ *   Sec. 3.1  block normalisation: power-of-two scale from floor(log2(amax)),
+ *             exponent offset by 3 so normalised magnitudes v lie in [0,16)
+ *             with the block maximum in [8,16); 1 sign bit + 3-bit index into
+ *             the block's dialect (8 integer magnitudes 0..15).
+ *   Sec. 3.2  group-wise maxima (num_groups contiguous groups), approximate
+ *             error of a dialect = sum over group maxima of the absolute error
+ *             at the midpoint of the maximum's 0.5-wide bin; two-stage
+ *             selection (sub-formatbook by block maximum, then argmin); every
+ *             element then rounds to the nearest magnitude of the chosen dialect.
+ *   Sec. 3.3  activation decomposition: residual Delta = Act - Q(Act) of the
+ *             salient tokens is quantized again; one salient token per tile,
+ *             the highest-scoring one.
+ *   Sec. 3.4  SeDA: the candidate set of a token is its cluster's sub-formatbook.
+ *
+ * No lookup tables are used anywhere: each rounding searches the 8 magnitudes,
+ * each error term is computed from the explicit bin midpoint.
+ *
+ * Readings taken where the paper is silent (the same list is in the design notes):
+ *   - rounding ties (v exactly half-way between two magnitudes) go to the LARGER
+ *     magnitude: bins are half-open [k/2,(k+1)/2) and a boundary is the left
+ *     edge of its bin (Sec. 3.2, "shift-and-truncate");
+ *   - dialect ties go to the LOWEST dialect id;
+ *   - the exponent is clamped to [exp_min, exp_max]; an all-zero block gets exp_min;
+ *   - the sign bit is copied even when the magnitude rounds to 0;
+ *   - stage 1: the candidate group is looked up by the bin floor(2*vmax) of the
+ *     block maximum (32 entries); by default entry k holds the dialects whose
+ *     largest magnitude equals max(8, floor(k/2)); an empty intersection with
+ *     the SeDA mask falls back to the SeDA mask alone;
+ *   - the residual is the fp32 value of x - xhat (exact for the default exponent
+ *     range) and is quantized from that value, never rounded to bf16;
+ *   - the scale byte is e + 124, i.e. the E8M0 code of the element scale 2^(e-3).
+ *
+ * Pins (tests/test_oracle_*.py): every representable value of every dialect
+ * round-trips; closed form for the uniform dialect; exact-rational brute force
+ * on tiny blocks and on all 65536 bf16 patterns; |E_d - exact error| <= G/4;
+ * argmin invariant; decomposition never increases any element's error; SeDA
+ * choices lie in the mask; per-tile argmax by brute force.
+ * Parity unpinned: the formatbook VALUES (the paper's table is only in Fig. 2a)
+ * and any worked numeric example (the paper prints none).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+typedef struct {
+  int block_size;   /* B: 32 or 16 (any multiple of num_groups up to 64 works here) */
+  int num_groups;   /* G: 8, or B */
+  int exp_min;      /* clamp of the block exponent e */
+  int exp_max;
+  int select_mode;  /* 0 = two-stage (Sec. 3.2), 1 = score every allowed dialect */
+} fb4o_config;
+
+#define FB4O_MAXB 64
+
+static double bf16_to_double(uint16_t b) {
+  uint32_t u = (uint32_t)b << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+static int formatbook_ok(const uint8_t *F) {
+  for (int d = 0; d < 32; ++d) {
+    if (F[d * 8] != 0) return 0;
+    for (int j = 1; j < 8; ++j)
+      if (F[d * 8 + j] <= F[d * 8 + j - 1] || F[d * 8 + j] > 15) return 0;
+  }
+  return 1;
+}
+
+/* floor(2v) capped at 31: the 0.5-wide bin of a normalised magnitude (Sec. 3.2). */
+static int bin_of(double v) {
+  double b = floor(2.0 * v);
+  return b > 31.0 ? 31 : (int)b;
+}
+
+/* index of the magnitude of dialect row Fd nearest to u; ties -> larger magnitude */
+static int nearest_index(const uint8_t *Fd, double u) {
+  int best = 0;
+  double bestd = fabs(u - (double)Fd[0]);
+  for (int j = 1; j < 8; ++j) {
+    double dj = fabs(u - (double)Fd[j]);
+    if (dj <= bestd) { bestd = dj; best = j; }
+  }
+  return best;
+}
+
+/* Default stage-1 table: entry k (bin of the block maximum) -> dialects whose
+ * largest magnitude is max(8, k/2)  (Sec. 3.2 two-stage; Sec. 3.4 "block maxima 8-15"). */
+void fb4o_default_stage1(const uint8_t *F, uint32_t *stage1 /*32*/) {
+  for (int k = 0; k < 32; ++k) {
+    int bucket = k / 2 < 8 ? 8 : k / 2;
+    uint32_t m = 0;
+    for (int d = 0; d < 32; ++d)
+      if (F[d * 8 + 7] == bucket) m |= 1u << d;
+    stage1[k] = m;
+  }
+}
+
+/*
+ * One block.  x[B] are the real input values, sgn[B] their sign bits.
+ * allowed = SeDA mask (all ones when unconstrained).
+ * Outputs: code[B] (sign<<3 | idx), *did, *e.  If err_q4 != NULL it receives,
+ * for every dialect, the approximate error in quarter units (-1 for dialects
+ * that were not candidates).
+ */
+static void quantize_block(const double *x, const uint8_t *sgn, const fb4o_config *cfg,
+                           const uint8_t *F, const uint32_t *stage1, uint32_t allowed,
+                           uint8_t *code, int *did, int *e_out, int32_t *err_q4) {
+  const int B = cfg->block_size, G = cfg->num_groups, gs = B / G;
+  /* Sec. 3.1: shared power-of-two scale from floor(log2(max magnitude)) */
+  double amax = 0.0;
+  for (int i = 0; i < B; ++i) if (fabs(x[i]) > amax) amax = fabs(x[i]);
+  int e;
+  if (amax == 0.0) {
+    e = cfg->exp_min;
+  } else {
+    int ex;
+    (void)frexp(amax, &ex);          /* amax = m * 2^ex, m in [0.5,1)  =>  floor(log2) = ex-1 */
+    e = ex - 1;
+    if (e < cfg->exp_min) e = cfg->exp_min;
+    if (e > cfg->exp_max) e = cfg->exp_max;
+  }
+  /* normalise: v = |x| * 2^(3-e), in [0,16) unless the exponent was clamped from above */
+  double v[FB4O_MAXB];
+  for (int i = 0; i < B; ++i) v[i] = ldexp(fabs(x[i]), 3 - e);
+  /* Sec. 3.2: group-wise maxima */
+  double gmax[FB4O_MAXB];
+  double vmax = 0.0;
+  for (int g = 0; g < G; ++g) {
+    double m = 0.0;
+    for (int i = 0; i < gs; ++i) if (v[g * gs + i] > m) m = v[g * gs + i];
+    gmax[g] = m;
+    if (m > vmax) vmax = m;
+  }
+  /* stage 1: sub-formatbook by the block maximum, intersected with the SeDA set */
+  uint32_t cand = allowed;
+  if (cfg->select_mode == 0) {
+    cand = stage1[bin_of(vmax)] & allowed;
+    if (cand == 0) cand = allowed;
+  }
+  /* stage 2: approximate error = sum over group maxima of |bin midpoint - nearest value| */
+  int best = -1;
+  double best_err = 0.0;
+  for (int d = 0; d < 32; ++d) {
+    if (err_q4) err_q4[d] = -1;
+    if (!((cand >> d) & 1u)) continue;
+    double err = 0.0;
+    for (int g = 0; g < G; ++g) {
+      double mid = 0.5 * (double)bin_of(gmax[g]) + 0.25;
+      err += fabs(mid - (double)F[d * 8 + nearest_index(F + d * 8, mid)]);
+    }
+    if (err_q4) err_q4[d] = (int32_t)(4.0 * err);
+    if (best < 0 || err < best_err) { best = d; best_err = err; }   /* ties keep the lowest id */
+  }
+  /* quantize every element to the nearest magnitude of the chosen dialect */
+  for (int i = 0; i < B; ++i)
+    code[i] = (uint8_t)((sgn[i] << 3) | nearest_index(F + best * 8, v[i]));
+  *did = best;
+  *e_out = e;
+}
+
+static double dequant_value(const uint8_t *F, int did, int e, uint8_t code) {
+  double mag = ldexp((double)F[did * 8 + (code & 7)], e - 3);
+  return (code & 8) ? -mag : mag;
+}
+
+static void store_block(const uint8_t *code, int B, int did, int e, uint8_t *codes_row, uint16_t *meta_row,
+                        int64_t blk) {
+  for (int i = 0; i < B; i += 2)
+    codes_row[(blk * B + i) / 2] = (uint8_t)(code[i] | (code[i + 1] << 4));
+  meta_row[blk] = (uint16_t)((e + 124) | (did << 8));
+}
+
+static int config_ok(const fb4o_config *cfg, int64_t C) {
+  if (cfg->block_size <= 0 || cfg->block_size > FB4O_MAXB || (cfg->block_size & 1)) return 0;
+  if (cfg->num_groups <= 0 || cfg->block_size % cfg->num_groups) return 0;
+  if (cfg->exp_min < -124 || cfg->exp_max > 127 || cfg->exp_min > cfg->exp_max) return 0;
+  if (C <= 0 || C % cfg->block_size) return 0;
+  return 1;
+}
+
+static uint32_t row_mask(const int32_t *cluster_id, const uint32_t *cluster_mask, int32_t n_clusters, int64_t t) {
+  if (!cluster_id || cluster_id[t] < 0) return 0xffffffffu;
+  if (cluster_id[t] >= n_clusters) return 0;   /* caller error; reported by the entry points */
+  return cluster_mask[cluster_id[t]];
+}
+
+/* Salient-token set, Sec. 3.3: the highest-scoring token of every tile of `tile`
+ * consecutive tokens (ties -> lowest index); ascending list; returns its length. */
+int64_t fb4o_select_salient(const float *score, int64_t T, int32_t tile, int32_t *salient_idx) {
+  if (tile <= 0 || T < 0) return -1;
+  int64_t n = 0;
+  for (int64_t t0 = 0; t0 < T; t0 += tile) {
+    int64_t t1 = t0 + tile < T ? t0 + tile : T, arg = t0;
+    for (int64_t t = t0 + 1; t < t1; ++t) if (score[t] > score[arg]) arg = t;
+    salient_idx[n++] = (int32_t)arg;
+  }
+  return n;
+}
+
+/*
+ * Quantize a T x C bf16 tensor (bit patterns, `ld` elements between rows).
+ * Optional SeDA tables (cluster_id NULL => unconstrained).  Optional residual
+ * pass for the rows listed (ascending) in salient_idx: residual codes/meta are
+ * written compactly, row s of res_* belonging to token salient_idx[s].
+ * err_q4 (optional, T*C/B*32 int32) receives the per-dialect approximate errors
+ * of the main pass.
+ * Returns 0, or a negative code for invalid arguments.
+ */
+int fb4o_quantize(const uint16_t *x, int64_t T, int64_t C, int64_t ld,
+                  const fb4o_config *cfg, const uint8_t *F, const uint32_t *stage1_in,
+                  const int32_t *cluster_id, const uint32_t *cluster_mask, int32_t n_clusters,
+                  const int32_t *salient_idx, int64_t n_salient,
+                  uint8_t *codes, uint16_t *meta, uint8_t *res_codes, uint16_t *res_meta,
+                  int32_t *err_q4) {
+  if (!config_ok(cfg, C) || T < 0 || ld < C) return -1;
+  if (!formatbook_ok(F)) return -2;
+  uint32_t stage1[32];
+  if (stage1_in) memcpy(stage1, stage1_in, sizeof stage1); else fb4o_default_stage1(F, stage1);
+  const int B = cfg->block_size;
+  const int64_t nblk = C / B;
+  int bad = 0;
+  if (cluster_id)
+    for (int64_t t = 0; t < T; ++t)
+      if (cluster_id[t] >= n_clusters || (cluster_id[t] >= 0 && cluster_mask[cluster_id[t]] == 0)) bad = 1;
+  for (int64_t s = 0; s < n_salient; ++s) {
+    if (salient_idx[s] < 0 || salient_idx[s] >= T) bad = 1;
+    if (s > 0 && salient_idx[s] <= salient_idx[s - 1]) bad = 1;
+  }
+  if (bad) return -3;
+
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < T; ++t) {
+    const uint32_t allowed = row_mask(cluster_id, cluster_mask, n_clusters, t);
+    /* is this row salient?  (ascending list => binary search) */
+    int64_t srow = -1;
+    {
+      int64_t lo = 0, hi = n_salient - 1;
+      while (lo <= hi) {
+        int64_t mid = (lo + hi) / 2;
+        if (salient_idx[mid] == t) { srow = mid; break; }
+        if (salient_idx[mid] < t) lo = mid + 1; else hi = mid - 1;
+      }
+    }
+    for (int64_t blk = 0; blk < nblk; ++blk) {
+      double xv[FB4O_MAXB];
+      uint8_t sg[FB4O_MAXB], code[FB4O_MAXB];
+      for (int i = 0; i < B; ++i) {
+        uint16_t b = x[t * ld + blk * B + i];
+        xv[i] = bf16_to_double(b);
+        sg[i] = (uint8_t)(b >> 15);
+      }
+      int did, e;
+      quantize_block(xv, sg, cfg, F, stage1, allowed, code, &did, &e,
+                     err_q4 ? err_q4 + (t * nblk + blk) * 32 : NULL);
+      store_block(code, B, did, e, codes + t * (C / 2), meta + t * nblk, blk);
+      if (srow >= 0) {
+        /* Sec. 3.3: Act = Q(Act) + Delta; quantize Delta again with the same candidate set */
+        double dv[FB4O_MAXB];
+        uint8_t dsg[FB4O_MAXB], dcode[FB4O_MAXB];
+        for (int i = 0; i < B; ++i) {
+          float df = (float)(xv[i] - dequant_value(F, did, e, code[i]));
+          dv[i] = (double)df;
+          dsg[i] = (uint8_t)(signbit(df) ? 1 : 0);
+        }
+        int rdid, re;
+        quantize_block(dv, dsg, cfg, F, stage1, allowed, dcode, &rdid, &re, NULL);
+        store_block(dcode, B, rdid, re, res_codes + srow * (C / 2), res_meta + srow * nblk, blk);
+      }
+    }
+  }
+  return 0;
+}
+
+static uint16_t f32_to_bf16_rne(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7fffu + lsb;
+  return (uint16_t)(u >> 16);
+}
+
+/*
+ * Decode: xhat = (-1)^s * F[did][idx] * 2^(e-3); salient rows add the decoded
+ * residual, the sum being rounded once to fp32.  out_dtype 0: float32 out,
+ * 1: bf16 bit patterns (round-to-nearest-even of the fp32 result).
+ */
+int fb4o_dequantize(const uint8_t *codes, const uint16_t *meta, int64_t T, int64_t C, int block_size,
+                    const uint8_t *F, const int32_t *salient_idx, int64_t n_salient,
+                    const uint8_t *res_codes, const uint16_t *res_meta, void *out, int out_dtype) {
+  if (block_size <= 0 || C % block_size || !formatbook_ok(F)) return -1;
+  const int B = block_size;
+  const int64_t nblk = C / B;
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < T; ++t) {
+    int64_t srow = -1;
+    for (int64_t s = 0; s < n_salient; ++s) if (salient_idx[s] == t) { srow = s; break; }
+    for (int64_t c = 0; c < C; ++c) {
+      int64_t blk = c / B;
+      uint16_t m = meta[t * nblk + blk];
+      uint8_t byte = codes[t * (C / 2) + c / 2];
+      uint8_t code = (c & 1) ? (byte >> 4) : (byte & 15);
+      float val = (float)dequant_value(F, m >> 8, (int)(m & 0xff) - 124, code);
+      if (srow >= 0) {
+        uint16_t rm = res_meta[srow * nblk + blk];
+        uint8_t rb = res_codes[srow * (C / 2) + c / 2];
+        uint8_t rc = (c & 1) ? (rb >> 4) : (rb & 15);
+        double r = dequant_value(F, rm >> 8, (int)(rm & 0xff) - 124, rc);
+        val = (float)((double)val + r);
+      }
+      if (out_dtype == 0) ((float *)out)[t * C + c] = val;
+      else ((uint16_t *)out)[t * C + c] = f32_to_bf16_rne(val);
+    }
+  }
+  return 0;
+}
+
+/* mean squared error between the bf16 input and a reconstruction, accumulated in fp64 */
+double fb4o_mse(const uint16_t *x, int64_t ld, const float *recon, int64_t T, int64_t C) {
+  double acc = 0.0;
+  for (int64_t t = 0; t < T; ++t) {
+    double row = 0.0;
+    for (int64_t c = 0; c < C; ++c) {
+      double d = bf16_to_double(x[t * ld + c]) - (double)recon[t * C + c];
+      row += d * d;
+    }
+    acc += row;
+  }
+  return T * C ? acc / ((double)T * (double)C) : 0.0;
+}
+
+/*
+ * One block given as doubles (for pins and brute-force comparisons on values
+ * that are not bf16, e.g. residuals).  code[B], err_q4[32] may be inspected.
+ */
+int fb4o_quantize_block_f64(const double *x, const fb4o_config *cfg, const uint8_t *F,
+                            const uint32_t *stage1_in, uint32_t allowed,
+                            uint8_t *code, int32_t *did, int32_t *e, int32_t *err_q4) {
+  if (!config_ok(cfg, cfg->block_size) || !formatbook_ok(F) || allowed == 0) return -1;
+  uint32_t stage1[32];
+  if (stage1_in) memcpy(stage1, stage1_in, sizeof stage1); else fb4o_default_stage1(F, stage1);
+  uint8_t sg[FB4O_MAXB];
+  for (int i = 0; i < cfg->block_size; ++i) sg[i] = (uint8_t)(signbit(x[i]) ? 1 : 0);
+  int d_, e_;
+  quantize_block(x, sg, cfg, F, stage1, allowed, code, &d_, &e_, err_q4);
+  *did = d_;
+  *e = e_;
+  return 0;
+}

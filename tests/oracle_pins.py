@@ -1,0 +1,421 @@
+"""Pins for the CPU oracle: facts the paper and plain mathematics fix, checked with exact
+rational arithmetic (fractions.Fraction) or closed forms, never with the oracle itself.
+
+Every function asserts; the mutation tests call the same functions against deliberately
+broken builds of the oracle and expect at least one of them to fail.
+"""
+from __future__ import annotations
+
+import math
+from fractions import Fraction
+
+import numpy as np
+
+from oracle import fb4_oracle as orc
+from paper_2603_02883_b200 import synth
+
+FB = synth.STANDIN_FORMATBOOK
+
+
+def bf16_value(bits: int) -> Fraction:
+    """Exact value of a finite bf16 bit pattern."""
+    s, e, m = bits >> 15, (bits >> 7) & 0xFF, bits & 0x7F
+    assert e != 0xFF
+    mag = Fraction(m, 128) * Fraction(2) ** (-126) if e == 0 else (1 + Fraction(m, 128)) * Fraction(2) ** (e - 127)
+    return -mag if s else mag
+
+
+def f32_value(x) -> Fraction:
+    return Fraction(float(x))
+
+
+def floor_log2(a: Fraction) -> int:
+    assert a > 0
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1
+    assert Fraction(2) ** e <= a < Fraction(2) ** (e + 1)
+    return e
+
+
+def unpack_codes(row: np.ndarray) -> np.ndarray:
+    out = np.empty(row.shape[-1] * 2, dtype=np.uint8)
+    out[0::2] = row & 15
+    out[1::2] = row >> 4
+    return out
+
+
+def rand_block_bits(rng, B, scale_exp_range=(-20, 20), zero_frac=0.1):
+    """Random bf16 block as bit patterns: mixed magnitudes, some zeros, both signs."""
+    e = rng.integers(*scale_exp_range)
+    vals = rng.standard_t(3, size=B) * 2.0 ** e
+    vals[rng.random(B) < zero_frac] = 0.0
+    return synth.f32_to_bf16_bits(vals.astype(np.float32))
+
+
+# ---------------------------------------------------------------- sizes / metadata (Table 1)
+
+def pin_effective_bits(golden_path):
+    for line in open(golden_path):
+        if line.startswith("#") or not line.strip():
+            continue
+        B, printed = line.split()
+        B, printed = int(B), float(printed)
+        C = 4 * B
+        x = synth.f32_to_bf16_bits(np.linspace(-3, 3, 2 * C, dtype=np.float32).reshape(2, C))
+        q = orc.quantize(x, FB, orc.Config(block_size=B))
+        # 4-bit codes + 10 bits of metadata (5-bit dialect id, 5-bit exponent) per block
+        bits = (q.codes.size * 8 + (q.meta.size) * 10) / x.size
+        assert q.codes.shape == (2, C // 2) and q.meta.shape == (2, C // B)
+        assert abs(bits - (4 + 10 / B)) < 1e-12
+        assert abs(bits - printed) < 0.006       # the table prints two decimals
+        assert int(q.did.max()) < 32 and int(q.did.min()) >= 0
+
+
+# ---------------------------------------------------------------- normalisation (Sec. 3.1)
+
+def pin_scale_is_floor_log2(seed=0, n=300):
+    rng = np.random.default_rng(seed)
+    for _ in range(n):
+        bits = rand_block_bits(rng, 32, (-100, 100))
+        q = orc.quantize(bits.reshape(1, 32), FB)
+        vals = [abs(bf16_value(int(b))) for b in bits]
+        amax = max(vals)
+        e = int(q.exponent[0, 0])
+        if amax == 0:
+            assert e == -124
+            continue
+        assert e == max(-124, floor_log2(amax))
+        if floor_log2(amax) >= -124:
+            vmax = amax * Fraction(2) ** (3 - e)
+            assert 8 <= vmax < 16          # "maximum in [8,16)"
+        assert int(q.meta[0, 0] & 0xFF) == e + 124   # E8M0 code of 2^(e-3)
+
+
+def pin_exponent_clamp():
+    cfg = orc.Config(exp_min=-15, exp_max=16)
+    big = synth.f32_to_bf16_bits(np.full(32, 2.0 ** 40, dtype=np.float32))
+    small = synth.f32_to_bf16_bits(np.full(32, 2.0 ** -40, dtype=np.float32))
+    qb = orc.quantize(big.reshape(1, 32), FB, cfg)
+    qs = orc.quantize(small.reshape(1, 32), FB, cfg)
+    assert int(qb.exponent[0, 0]) == 16 and int(qs.exponent[0, 0]) == -15
+    # clamped from above: every element saturates at the largest magnitude of the dialect
+    d = int(qb.did[0, 0])
+    y = orc.dequantize(qb, FB)
+    assert np.all(y == float(FB[d, 7]) * 2.0 ** 13)
+    assert np.all(orc.dequantize(qs, FB) == 0.0)
+
+
+def pin_zero_block():
+    """All-zero block (silent in the paper): exponent = exp_min, every dialect of the lowest
+    dynamic range ties so the lowest id wins, sign bits of -0 are kept, decode gives +-0."""
+    bits = np.zeros(32, dtype=np.uint16)
+    bits[[3, 17]] = 0x8000
+    for cfg in (orc.Config(), orc.Config(exp_min=-15, exp_max=16)):
+        q = orc.quantize(bits.reshape(1, 32), FB, cfg)
+        assert int(q.exponent[0, 0]) == cfg.exp_min
+        assert int(q.did[0, 0]) == min(d for d in range(32) if int(FB[d, 7]) == 8)
+        codes = unpack_codes(q.codes[0])
+        assert np.array_equal(codes, np.where(bits == 0x8000, 8, 0))
+        y = orc.dequantize(q, FB)[0]
+        assert np.all(y == 0) and np.array_equal(np.signbit(y), bits == 0x8000)
+
+
+# ---------------------------------------------------------------- rounding (Sec. 3.2)
+
+def pin_rounding_is_nearest(seed=1, n=200):
+    """Every code is a nearest magnitude of the chosen dialect (exact rationals); exact
+    half-way cases go to the larger magnitude."""
+    rng = np.random.default_rng(seed)
+    for it in range(n):
+        B = 32 if it % 2 == 0 else 16
+        bits = rand_block_bits(rng, B)
+        q = orc.quantize(bits.reshape(1, B), FB, orc.Config(block_size=B))
+        d, e = int(q.did[0, 0]), int(q.exponent[0, 0])
+        codes = unpack_codes(q.codes[0])
+        for b, c in zip(bits, codes):
+            v = abs(bf16_value(int(b))) * Fraction(2) ** (3 - e)
+            chosen = int(FB[d, c & 7])
+            dist = abs(v - chosen)
+            for m in FB[d]:
+                assert dist <= abs(v - int(m))
+                if abs(v - int(m)) == dist:
+                    assert int(m) <= chosen
+            assert (c >> 3) == (int(b) >> 15)        # sign bit copied, also for zeros
+
+
+def pin_uniform_dialect_closed_form():
+    """For the uniform dialect {0,2,...,14} nearest-with-ties-up is floor((v+1)/2), capped at 7."""
+    d = next(i for i in range(32) if list(FB[i]) == [0, 2, 4, 6, 8, 10, 12, 14])
+    # all bf16 magnitudes v in [0,15): block = that value + one element pinning the scale (v=14 -> e=0, 14*2^-3)
+    pats = [p for p in range(0x0000, 0x7F80) if bf16_value(p) * 8 < 15]
+    pats = pats[:: max(1, len(pats) // 4000)] + [synth.f32_to_bf16_bits(np.array([k / 16], np.float32))[0] for k in range(0, 30)]
+    setter = synth.f32_to_bf16_bits(np.array([14 / 8], np.float32))[0]
+    for p in pats:
+        p = int(p)
+        blk = np.zeros(32, dtype=np.uint16)
+        blk[0], blk[5] = setter, p
+        q = orc.quantize(blk.reshape(1, 32), FB, cluster_id=np.zeros(1, np.int32),
+                         cluster_mask=np.array([1 << d], np.uint32))
+        assert int(q.did[0, 0]) == d and int(q.exponent[0, 0]) == 0
+        v = bf16_value(p) * 8
+        want = min(7, math.floor((v + 1) / 2))
+        assert int(unpack_codes(q.codes[0])[5] & 7) == want
+
+
+def pin_representable_values_roundtrip():
+    """Every representable value of every dialect, both signs, several exponents, decodes to itself."""
+    for d in range(32):
+        top = int(FB[d, 7])
+        for e in (-124, -60, -3, 0, 5, 100, 127):
+            for j in range(8):
+                for sgn in (1.0, -1.0):
+                    mag = int(FB[d, j])
+                    vals = np.zeros(32, dtype=np.float64)
+                    vals[31] = math.ldexp(top, e - 3)       # fixes the block exponent and dynamic range
+                    vals[7] = sgn * math.ldexp(mag, e - 3)
+                    bits = synth.f32_to_bf16_bits(vals.astype(np.float32))
+                    assert np.all(synth.bf16_bits_to_f32(bits).astype(np.float64) == vals)
+                    q = orc.quantize(bits.reshape(1, 32), FB, cluster_id=np.zeros(1, np.int32),
+                                     cluster_mask=np.array([1 << d], np.uint32))
+                    assert int(q.did[0, 0]) == d and int(q.exponent[0, 0]) == e
+                    y = orc.dequantize(q, FB)[0]
+                    assert y[7] == vals[7] and y[31] == vals[31] and np.all(y[:7] == 0)
+                    assert np.signbit(y[7]) == (sgn < 0)
+
+
+def pin_single_nonzero_block_truncates(patterns=None):
+    """A block with one nonzero element x: two-stage selection picks a dialect whose largest
+    magnitude is floor(v), so xhat keeps the leading 4 significant bits of x (truncation);
+    checked for bf16 bit patterns against exact rational arithmetic."""
+    if patterns is None:
+        patterns = range(0, 0x10000)
+    pats = np.array([p for p in patterns if ((p >> 7) & 0xFF) != 0xFF], dtype=np.uint16)
+    x = np.zeros((len(pats), 32), dtype=np.uint16)
+    pos = np.arange(len(pats)) % 32
+    x[np.arange(len(pats)), pos] = pats
+    q = orc.quantize(x, FB)
+    y = orc.dequantize(q, FB)
+    for i, p in enumerate(pats):
+        p = int(p)
+        a = abs(bf16_value(p))
+        got = f32_value(y[i, pos[i]])
+        if a == 0:
+            assert got == 0 and int(q.exponent[i, 0]) == -124
+        else:
+            e = max(-124, floor_log2(a))
+            v = a * Fraction(2) ** (3 - e)
+            want = math.floor(v) * Fraction(2) ** (e - 3) if v >= 8 else None
+            assert int(q.exponent[i, 0]) == e
+            if want is not None:
+                assert abs(got) == want, (hex(p), got, want)
+                assert int(FB[int(q.did[i, 0]), 7]) == math.floor(v)
+            else:   # below the clamp: nearest value of a dialect whose top is 8
+                assert int(FB[int(q.did[i, 0]), 7]) == 8
+                dd = FB[int(q.did[i, 0])]
+                assert abs(abs(got) * Fraction(2) ** (3 - e) - v) == min(abs(int(m) - v) for m in dd)
+        assert bool(np.signbit(y[i, pos[i]])) == bool(p >> 15)
+        assert np.count_nonzero(y[i]) <= 1
+
+
+# ---------------------------------------------------------------- approximate error and selection (Sec. 3.2)
+
+def _group_max_v(bits, e, B, G):
+    v = [abs(bf16_value(int(b))) * Fraction(2) ** (3 - e) for b in bits]
+    gs = B // G
+    return v, [max(v[g * gs:(g + 1) * gs]) for g in range(G)]
+
+
+def pin_error_terms_and_argmin(seed=2, n=150):
+    """err_q4[d] = sum over the G contiguous group maxima of |bin midpoint - nearest magnitude|
+    (exact, in quarter units); it stays within G/4 of the true absolute error of the group
+    maxima; the chosen dialect is the lowest-id minimiser inside the stage-1 group."""
+    rng = np.random.default_rng(seed)
+    for it in range(n):
+        B, G = [(32, 8), (16, 8), (32, 32), (16, 16)][it % 4]
+        cfg = orc.Config(block_size=B, num_groups=G)
+        bits = rand_block_bits(rng, B)
+        if it % 7 == 0:                       # few distinct values => ties between dialects
+            bits[:] = bits[rng.integers(0, 2, size=B)]
+        q = orc.quantize(bits.reshape(1, B), FB, cfg, want_errors=True)
+        d_star, e = int(q.did[0, 0]), int(q.exponent[0, 0])
+        v, gm = _group_max_v(bits, e, B, G)
+        vmax = max(v)
+        bucket = max(8, math.floor(vmax)) if vmax < 16 else 15
+        cands = [d for d in range(32) if int(FB[d, 7]) == bucket]
+        err = q.err_q4[0, 0]
+        assert [d for d in range(32) if err[d] >= 0] == cands
+        for d in cands:
+            total, exact = Fraction(0), Fraction(0)
+            for m in gm:
+                k = min(31, math.floor(2 * m))
+                mid = Fraction(2 * k + 1, 4)
+                t = min(abs(mid - int(f)) for f in FB[d])
+                # closed form of the midpoint error: |2k+1-4r|/4 with r the nearest magnitude
+                r = min((int(f) for f in FB[d]), key=lambda f: abs(mid - f))
+                assert t == Fraction(abs(2 * k + 1 - 4 * r), 4)
+                true = min(abs(m - int(f)) for f in FB[d])
+                assert abs(t - true) <= Fraction(1, 4)
+                total += t
+                exact += true
+            assert Fraction(int(err[d]), 4) == total
+            assert abs(total - exact) <= Fraction(G, 4)
+        best = min(int(err[d]) for d in cands)
+        assert int(err[d_star]) == best and d_star == min(d for d in cands if int(err[d]) == best)
+        # the block maximum always lands on the top magnitude of the chosen dialect
+        if 8 <= vmax < 16:
+            codes = unpack_codes(q.codes[0])
+            imax = max(range(B), key=lambda i: v[i])
+            assert int(codes[imax] & 7) == 7
+
+
+def pin_groups_are_contiguous():
+    """Two blocks with the same multiset of values but different grouping must see different
+    group maxima: contiguous groups of B/G elements."""
+    cfg = orc.Config()
+    base = np.full(32, 0.25, dtype=np.float32)
+    a = base.copy(); a[0:4] = [15, 9.5, 9.5, 9.5]          # all large values in ONE contiguous group
+    b = base.copy(); b[[0, 4, 8, 12]] = [15, 9.5, 9.5, 9.5]  # spread over four groups
+    qa = orc.quantize(synth.f32_to_bf16_bits(a).reshape(1, 32), FB, cfg, want_errors=True)
+    qb = orc.quantize(synth.f32_to_bf16_bits(b).reshape(1, 32), FB, cfg, want_errors=True)
+    for d in range(25, 32):    # dialects with top magnitude 15
+        def term(u, d=d):
+            k = math.floor(2 * u)
+            return min(abs(Fraction(2 * k + 1, 4) - int(f)) for f in FB[d])
+        ea = term(Fraction(15)) + 7 * term(Fraction(1, 4))
+        eb = term(Fraction(15)) + 3 * term(Fraction(19, 2)) + 4 * term(Fraction(1, 4))
+        assert Fraction(int(qa.err_q4[0, 0, d]), 4) == ea
+        assert Fraction(int(qb.err_q4[0, 0, d]), 4) == eb
+
+
+def pin_select_all_mode(seed=3, n=60):
+    rng = np.random.default_rng(seed)
+    cfg = orc.Config(select_mode=1)
+    for _ in range(n):
+        bits = rand_block_bits(rng, 32)
+        q = orc.quantize(bits.reshape(1, 32), FB, cfg, want_errors=True)
+        err = q.err_q4[0, 0]
+        assert np.all(err >= 0)
+        assert int(q.did[0, 0]) == int(np.argmin(err))      # numpy argmin returns the first minimum
+
+
+# ---------------------------------------------------------------- SeDA (Sec. 3.4)
+
+def pin_seda_choice_inside_mask(seed=4, n=120):
+    rng = np.random.default_rng(seed)
+    w = synth.Workload("t", T=8, C=64, seed=9, kind=1, n_outlier=0, outlier_gain=1.0,
+                       seda=True, n_clusters=4, cluster_seed=5)
+    cid, masks = synth.clusters(w)
+    for m in masks:
+        assert bin(int(m)).count("1") == 8
+        assert sorted(int(FB[d, 7]) for d in range(32) if (int(m) >> d) & 1) == list(range(8, 16))
+    for it in range(n):
+        bits = rand_block_bits(rng, 32)
+        if it % 3 == 0:
+            mask = int(masks[it % 4])           # paper-structured: one dialect per bucket
+        else:
+            mask = int(rng.integers(1, 2 ** 32))
+        q = orc.quantize(bits.reshape(1, 32), FB, cluster_id=np.zeros(1, np.int32),
+                         cluster_mask=np.array([mask], np.uint32), want_errors=True)
+        d, e = int(q.did[0, 0]), int(q.exponent[0, 0])
+        assert (mask >> d) & 1
+        v, _ = _group_max_v(bits, e, 32, 8)
+        bucket = max(8, math.floor(max(v)))
+        inter = [dd for dd in range(32) if (mask >> dd) & 1 and int(FB[dd, 7]) == bucket]
+        err = q.err_q4[0, 0]
+        cands = inter if inter else [dd for dd in range(32) if (mask >> dd) & 1]
+        assert [dd for dd in range(32) if err[dd] >= 0] == cands
+        if it % 3 == 0:
+            assert cands == [d]                 # exactly one candidate remains after stage 1
+        assert int(err[d]) == min(int(err[dd]) for dd in cands)
+    # cluster id -1 means unconstrained
+    bits = rand_block_bits(rng, 32)
+    qa = orc.quantize(bits.reshape(1, 32), FB)
+    qb = orc.quantize(bits.reshape(1, 32), FB, cluster_id=np.array([-1], np.int32),
+                      cluster_mask=np.array([1], np.uint32))
+    assert np.array_equal(qa.codes, qb.codes) and np.array_equal(qa.meta, qb.meta)
+
+
+# ---------------------------------------------------------------- decomposition (Sec. 3.3)
+
+def pin_salient_is_per_tile_argmax(seed=5):
+    rng = np.random.default_rng(seed)
+    for T, tile in [(40, 20), (47, 20), (5, 20), (64, 1), (33, 7)]:
+        s = rng.random(T).astype(np.float32)
+        s[rng.integers(0, T, size=T // 3)] = s[0]          # ties
+        idx = orc.select_salient(s, tile)
+        assert len(idx) == -(-T // tile)
+        for k, t0 in enumerate(range(0, T, tile)):
+            assert int(idx[k]) == t0 + int(np.argmax(s[t0:t0 + tile]))   # numpy: first maximum
+        assert np.all(np.diff(idx) > 0)
+
+
+def pin_decomposition(seed=6, n=40):
+    """Act = Q(Act) + Delta exactly; Q(Act) + Q(Delta) is never farther from Act than Q(Act)
+    in any element; the residual codes decode to the sign of Delta."""
+    rng = np.random.default_rng(seed)
+    for it in range(n):
+        T, C = 4, 64
+        x = np.stack([rand_block_bits(rng, C, (-30, 30)) for _ in range(T)])
+        sal = np.array([1, 3], dtype=np.int32)
+        q = orc.quantize(x, FB, salient_idx=sal)
+        q_plain = orc.quantize(x, FB)
+        assert np.array_equal(q.codes, q_plain.codes) and np.array_equal(q.meta, q_plain.meta)
+        main = orc.dequantize(q_plain, FB)
+        full = orc.dequantize(q, FB)
+        assert np.array_equal(full[[0, 2]], main[[0, 2]])
+        for s, t in enumerate(sal):
+            # residual block quantized like any other block, from the exact difference
+            for blk in range(C // 32):
+                sl = slice(blk * 32, blk * 32 + 32)
+                delta = [bf16_value(int(b)) - f32_value(m) for b, m in zip(x[t, sl], main[t, sl])]
+                assert all(Fraction(float(np.float32(float(dl)))) == dl for dl in delta)   # exact in fp32
+                code, did, e, _ = orc.quantize_block_f64(np.array([float(dl) for dl in delta]), FB)
+                assert np.array_equal(unpack_codes(q.res_codes[s, blk * 16:(blk + 1) * 16]), code)
+                assert int(q.res_meta[s, blk]) == (e + 124) | (did << 8)
+            rcodes = unpack_codes(q.res_codes[s])
+            for c in range(C):
+                xv = bf16_value(int(x[t, c]))
+                # decoded sum = Q(Act) + Q(Delta), the residual decoded by the same formula
+                rm = int(q.res_meta[s, c // 32])
+                rmag = int(FB[rm >> 8, rcodes[c] & 7]) * Fraction(2) ** ((rm & 0xFF) - 127)
+                rval = -rmag if rcodes[c] & 8 else rmag
+                assert f32_value(full[t, c]) == f32_value(main[t, c]) + rval
+                e0 = abs(xv - f32_value(main[t, c]))
+                e1 = abs(xv - f32_value(full[t, c]))
+                assert e1 <= e0
+                rq = f32_value(full[t, c]) - f32_value(main[t, c])       # decoded residual (sum is exact)
+                dl = xv - f32_value(main[t, c])
+                assert rq == 0 or (rq > 0) == (dl > 0)
+
+
+def pin_dequantize_formula(seed=7):
+    rng = np.random.default_rng(seed)
+    codes = rng.integers(0, 256, size=(3, 32), dtype=np.uint8)
+    did = rng.integers(0, 32, size=(3, 2))
+    sb = np.array([[0, 1], [121, 124], [250, 251]])
+    meta = (sb | (did << 8)).astype(np.uint16)
+    y = orc.dequantize(orc.Quantized(codes, meta), FB)
+    yb = orc.dequantize(orc.Quantized(codes, meta), FB, out_dtype="bf16")
+    for t in range(3):
+        cc = unpack_codes(codes[t])
+        for c in range(64):
+            m = int(FB[did[t, c // 32], cc[c] & 7])
+            want = math.ldexp(m, int(sb[t, c // 32]) - 127)       # F * 2^(e-3), e = byte - 124
+            want = -want if cc[c] & 8 else want
+            assert float(y[t, c]) == want and bool(np.signbit(y[t, c])) == bool(cc[c] & 8)
+            assert float(synth.bf16_bits_to_f32(yb[t:t + 1, c])[0]) == want   # 4-bit magnitudes are exact in bf16
+
+
+def pin_mse():
+    x = synth.f32_to_bf16_bits(np.array([[1.0, 2.0, -3.0, 0.5]], np.float32))
+    r = np.array([[1.5, 2.0, -1.0, 0.5]], np.float32)
+    assert orc.mse(x, r) == (0.25 + 4.0) / 4
+
+
+ALL_PINS = [
+    pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
+    pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
+    pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_decomposition,
+    pin_dequantize_formula, pin_mse,
+]

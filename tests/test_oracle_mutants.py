@@ -1,0 +1,64 @@
+"""Do the pins notice a mistake?  Each case compiles a copy of the oracle source with ONE
+planted error (wrong tie direction, dropped term, wrong offset, transposed grouping, ...)
+and requires at least one pin to fail.  The mistakes are planted in the oracle, on the CPU."""
+import os
+import subprocess
+
+import pytest
+
+import oracle_pins as pins
+from oracle import fb4_oracle as orc
+
+SRC = os.path.join(os.path.dirname(orc.__file__), "fb4_oracle.c")
+
+MUTANTS = {
+    "round_ties_down": ("if (dj <= bestd) { bestd = dj; best = j; }", "if (dj < bestd) { bestd = dj; best = j; }"),
+    "dialect_ties_to_highest": ("if (best < 0 || err < best_err)", "if (best < 0 || err <= best_err)"),
+    "exponent_offset_2": ("v[i] = ldexp(fabs(x[i]), 3 - e);", "v[i] = ldexp(fabs(x[i]), 2 - e);"),
+    "floor_log2_off_by_one": ("e = ex - 1;", "e = ex;"),
+    "midpoint_dropped": ("+ 0.25;", "+ 0.0;"),
+    "squared_error": ("err += fabs(mid - (double)F[d * 8 + nearest_index(F + d * 8, mid)]);",
+                      "{ double q_ = mid - (double)F[d * 8 + nearest_index(F + d * 8, mid)]; err += q_ * q_; }"),
+    "strided_groups": ("if (v[g * gs + i] > m) m = v[g * gs + i];", "if (v[g + i * G] > m) m = v[g + i * G];"),
+    "one_group_missing": ("for (int g = 0; g < G; ++g) {\n      double mid", "for (int g = 1; g < G; ++g) {\n      double mid"),
+    "bin_width_one": ("double b = floor(2.0 * v);", "double b = 2.0 * floor(v);"),
+    "stage1_ignored": ("cand = stage1[bin_of(vmax)] & allowed;", "cand = allowed;"),
+    "seda_mask_ignored": ("cand = stage1[bin_of(vmax)] & allowed;", "cand = stage1[bin_of(vmax)];"),
+    "sign_dropped": ("code[i] = (uint8_t)((sgn[i] << 3) |", "code[i] = (uint8_t)((0 << 3) |"),
+    "nibbles_swapped": ("(uint8_t)(code[i] | (code[i + 1] << 4));", "(uint8_t)(code[i + 1] | (code[i] << 4));"),
+    "scale_byte_bias": ("(uint16_t)((e + 124) | (did << 8));", "(uint16_t)((e + 127) | (did << 8));"),
+    "dequant_exponent": ("ldexp((double)F[did * 8 + (code & 7)], e - 3);", "ldexp((double)F[did * 8 + (code & 7)], e - 4);"),
+    "residual_from_rounded_input": ("float df = (float)(xv[i] - dequant_value(F, did, e, code[i]));",
+                                    "float df = (float)(xv[i] - 0.5 * dequant_value(F, did, e, code[i]));"),
+    "residual_not_added": ("val = (float)((double)val + r);", "val = (float)((double)val + 0.0 * r);"),
+    "salient_last_on_tie": ("if (score[t] > score[arg]) arg = t;", "if (score[t] >= score[arg]) arg = t;"),
+    "salient_min": ("if (score[t] > score[arg]) arg = t;", "if (score[t] < score[arg]) arg = t;"),
+    "clamp_min_ignored": ("if (e < cfg->exp_min) e = cfg->exp_min;", ";"),
+    "zero_block_exponent": ("e = cfg->exp_min;\n  } else {", "e = 0;\n  } else {"),
+    "stage1_bucket_shift": ("int bucket = k / 2 < 8 ? 8 : k / 2;", "int bucket = k / 2 < 9 ? 9 : k / 2;"),
+    "mse_not_squared": ("row += d * d;", "row += fabs(d);"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_pins_catch(name, tmp_path):
+    old, new = MUTANTS[name]
+    src = open(SRC).read()
+    assert src.count(old) == 1, f"mutation site for {name} not unique/found"
+    msrc = tmp_path / "mutant.c"
+    msrc.write_text(src.replace(old, new))
+    so = tmp_path / f"mutant_{name}.so"
+    subprocess.check_call(["gcc", "-O1", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+                           "-o", str(so), str(msrc), "-lm"])
+    orc.use_library(str(so))
+    caught = []
+    try:
+        for pin in pins.ALL_PINS:
+            try:
+                pin()
+            except (AssertionError, ValueError, IndexError, StopIteration, ZeroDivisionError):
+                caught.append(pin.__name__)
+                break
+    finally:
+        orc.use_library(None)
+    assert caught, f"no pin noticed the planted mistake '{name}'"
