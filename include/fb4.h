@@ -1,0 +1,194 @@
+/*
+ * fb4.h -- C ABI of the B200 (sm_100a) FB4 online activation quantizer.
+ *
+ * FB4 is the 4-bit block format of SemanticDialect: every block of B contiguous
+ * channels of a token shares a power-of-two scale and one of 32 "dialects"
+ * (8 integer magnitudes out of 0..15); an element is a sign bit plus a 3-bit
+ * index into the block's dialect (Sec. 3.1).  The dialect is chosen online, per
+ * block, by summing a lookup-table estimate of the quantization error over the
+ * block's group-wise maxima and taking the minimum inside the sub-formatbook
+ * that matches the block's dynamic range (Sec. 3.2).
+ *
+ * Conventions for every call
+ *   - Return value: FB4_OK (0) or a negative FB4_ERR_* code.  Nothing is printed,
+ *     nothing aborts.  fb4_strerror() names a code.
+ *   - Unless a parameter says "host", data pointers are DEVICE pointers owned by
+ *     the caller; the library never frees or retains them.  The library owns only
+ *     the opaque context (a few KB of lookup tables on the device).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls enqueue work on it and return without synchronising; launch errors
+ *     that CUDA reports synchronously come back as FB4_ERR_CUDA.
+ *   - Tensors are row-major [T tokens][C channels]; blocks run along the
+ *     contiguous channel axis.  C must be a multiple of the block size.
+ *     `ld_elems` is the distance between rows of x in elements (>= C).
+ *   - x is bfloat16.  Inputs must be finite (NaN/Inf are not checked and give
+ *     meaningless, but in-bounds, output).
+ *   - Alignment: x and every output pointer must be 16-byte aligned and
+ *     ld_elems a multiple of 8; otherwise FB4_ERR_ALIGN.
+ *   - Device code has no wait loops; a call cannot hang.
+ *
+ * Output layout
+ *   codes : uint8 [T][C/2].  Byte j of a row holds element 2j in its low nibble
+ *           and element 2j+1 in its high nibble; nibble = sign<<3 | index.
+ *   meta  : uint16 [T][C/B].  bits 0-7 = scale byte = e + 124 where e is the
+ *           block exponent floor(log2(amax)) (clamped); this is the E8M0 code of
+ *           the element scale 2^(e-3).  bits 8-12 = dialect id.  bits 13-15 = 0.
+ *   value : (-1)^sign * formatbook[dialect][index] * 2^(e-3).
+ */
+#ifndef FB4_H_
+#define FB4_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FB4_OK 0
+#define FB4_ERR_INVALID_ARG (-1) /* null pointer, bad enum, negative count, empty dialect mask */
+#define FB4_ERR_SHAPE (-2)       /* C not a multiple of the block size, ld_elems < C, T < 0 */
+#define FB4_ERR_ALIGN (-3)       /* pointer not 16-byte aligned or ld_elems not a multiple of 8 */
+#define FB4_ERR_FORMATBOOK (-4)  /* dialect not strictly ascending from 0 within 0..15 */
+#define FB4_ERR_CUDA (-5)        /* a CUDA runtime call failed; fb4_last_cuda_error() has the code */
+#define FB4_ERR_NO_DEVICE (-6)   /* no usable CUDA device / wrong architecture (needs sm_100) */
+
+typedef struct fb4_ctx fb4_ctx;
+
+/* Quantizer parameters (Sec. 4.1: block sizes 16 and 32, num_groups = 8 by default;
+ * Table 2 also evaluates num_groups = block size). */
+typedef struct {
+  uint32_t block_size;  /* 32 (default) or 16 */
+  uint32_t num_groups;  /* 8 (default) or block_size; contiguous groups of block_size/num_groups */
+  int32_t exp_min;      /* clamp of the block exponent e; default -124 (>= -124) */
+  int32_t exp_max;      /* default 127 (<= 127); the paper's 5-bit exponent is e.g. [-15,16] */
+  uint32_t select_mode; /* 0 = two-stage selection (Sec. 3.2); 1 = score every allowed dialect */
+} fb4_config;
+
+/* Defaults: {32, 8, -124, 127, 0}. */
+void fb4_default_config(fb4_config* cfg);
+
+/*
+ * Build a context on CUDA device `device`: validates the formatbook, builds the
+ * Qvalue / Qerror lookup tables (Sec. 3.2: 0.5-wide bins; Qvalue = exact index of
+ * the nearest magnitude, Qerror = absolute error at the bin midpoint) and the
+ * stage-1 table, and uploads them.  Synchronous; may allocate device memory.
+ *   formatbook  : host, 32*8 bytes, dialect-major; NULL = the built-in stand-in
+ *                 table (the paper gives its table only as Fig. 2a).
+ *   stage1_mask : host, 32 words; entry k = bit mask of the dialects compared when
+ *                 the block maximum falls in bin k = floor(2*vmax) (Sec. 3.2,
+ *                 "sub-formatbook based on the block maximum").  NULL = dialects
+ *                 whose largest magnitude equals max(8, k/2).
+ *   cfg         : NULL = defaults.
+ * On success *out owns device memory until fb4_destroy().
+ */
+int fb4_init(fb4_ctx** out, int device, const uint8_t* formatbook, const uint32_t* stage1_mask,
+             const fb4_config* cfg);
+int fb4_destroy(fb4_ctx* ctx);
+
+/* Host copies of the tables a context was built with (any pointer may be NULL):
+ * formatbook[32*8], stage1_mask[32], qvalue[32 dialects][32 bins] (index 0..7),
+ * qerror_q4[32][32] (error in quarter units).  For tests and diagnostics. */
+int fb4_get_tables(const fb4_ctx* ctx, uint8_t* formatbook, uint32_t* stage1_mask, uint8_t* qvalue,
+                   uint8_t* qerror_q4);
+
+/*
+ * Plain FB4 quantization of x[T][C] (Sec. 3.1-3.2): per block, scale -> group
+ * maxima -> LUT error sums over the stage-1 candidates -> argmin (ties: lowest
+ * dialect id) -> LUT quantization.  Writes codes[T][C/2] and meta[T][C/B].
+ * T == 0 is a no-op.
+ */
+int fb4_quantize(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems, uint8_t* codes,
+                 uint16_t* meta, void* stream);
+
+/*
+ * SeDA-constrained quantization (Sec. 3.4): token t may only use the dialects in
+ * cluster_mask[cluster_id[t]] (its cluster's sub-formatbook); cluster_id[t] == -1
+ * means unconstrained.  Stage 1 is intersected with the mask; if the intersection
+ * is empty the whole mask is scored.
+ *   cluster_id   : device int32 [T], values in [-1, n_clusters)
+ *   cluster_mask : device uint32 [n_clusters], every entry non-zero (precondition;
+ *                  a zero mask yields dialect 0 for the affected tokens)
+ */
+int fb4_quantize_seda(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems,
+                      const int32_t* cluster_id, const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* codes,
+                      uint16_t* meta, void* stream);
+
+/*
+ * Salient-token selection for activation decomposition (Sec. 3.3: "one salient
+ * token per tile ... the highest-scoring token in each tile"): for every tile of
+ * `tile` consecutive tokens, the index of the largest score (ties: lowest index).
+ *   score       : device float [T] (finite)
+ *   salient_idx : device int32 [ceil(T/tile)], ascending on return
+ */
+int fb4_select_salient(fb4_ctx* ctx, const float* score, int64_t T, int32_t tile, int32_t* salient_idx,
+                       void* stream);
+
+/*
+ * Quantization with activation decomposition (Sec. 3.3): every token is quantized
+ * as in fb4_quantize[_seda]; for the salient tokens the residual
+ * Delta = x - dequant(Q(x)) is formed in registers (exactly, in fp32), quantized
+ * again with the same candidate set, and written compactly: row s of res_codes /
+ * res_meta belongs to token salient_idx[s].  The salient set is selected first
+ * from `score` (see fb4_select_salient) and returned in salient_idx.
+ *   cluster_id   : NULL = no SeDA restriction (then cluster_mask is ignored)
+ *   salient_idx  : device int32 [ceil(T/tile)] (out)
+ *   res_codes    : device uint8  [ceil(T/tile)][C/2] (out)
+ *   res_meta     : device uint16 [ceil(T/tile)][C/B] (out)
+ */
+int fb4_quantize_decomposed(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems,
+                            const float* score, int32_t tile, const int32_t* cluster_id,
+                            const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* codes, uint16_t* meta,
+                            int32_t* salient_idx, uint8_t* res_codes, uint16_t* res_meta, void* stream);
+
+/*
+ * The same with a salient set given by the caller (App. C: layers that precede the
+ * attention computation reuse the previous timestep's salient tokens).
+ *   salient_idx : device int32 [n_salient] (in), strictly ascending, each in [0,T)
+ *                 (precondition; not checked on the device)
+ */
+int fb4_quantize_decomposed_idx(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems,
+                                const int32_t* salient_idx, int64_t n_salient, const int32_t* cluster_id,
+                                const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* codes,
+                                uint16_t* meta, uint8_t* res_codes, uint16_t* res_meta, void* stream);
+
+/*
+ * Decode (App. D.2: 4-bit codes are decoded on the fly with the block scale applied):
+ * out[t][c] = value(codes, meta); for tokens listed in salient_idx the decoded
+ * residual is added, the sum rounded once to fp32 (Sec. 3.3: Q(Act)+Q(Delta)).
+ *   salient_idx : NULL / n_salient = 0 for plain tensors; else device int32
+ *                 [n_salient], strictly ascending
+ *   out         : device, [T][C] contiguous; out_dtype 0 = float32, 1 = bfloat16
+ *                 (round-to-nearest-even of the fp32 result)
+ */
+int fb4_dequantize(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T, int64_t C,
+                   const int32_t* salient_idx, int64_t n_salient, const uint8_t* res_codes,
+                   const uint16_t* res_meta, void* out, int out_dtype, void* stream);
+
+/*
+ * Host-buffer form of fb4_quantize for callers whose tensors live in host memory:
+ * copies x from the host, quantizes, and copies codes and meta back, in row
+ * chunks pipelined over the context's own streams, then waits for completion.
+ *   x_host, codes_host, meta_host : HOST pointers (pinned memory overlaps copies
+ *                                   with compute; pageable memory works, slower)
+ *   d_x, d_codes, d_meta          : DEVICE staging buffers of the full tensor
+ *                                   sizes, provided by the caller
+ */
+int fb4_quantize_host(fb4_ctx* ctx, const void* x_host, int64_t T, int64_t C, void* d_x, uint8_t* d_codes,
+                      uint16_t* d_meta, uint8_t* codes_host, uint16_t* meta_host);
+
+/* Number of kernel launches this context has enqueued so far (diagnostic counter). */
+int64_t fb4_launch_count(const fb4_ctx* ctx);
+
+/* Name of the kernel variant the last quantize call on this context used
+ * ("fast" = TMA-staged sm_100a path, "generic" = fallback for other shapes). */
+const char* fb4_last_variant(const fb4_ctx* ctx);
+
+/* cudaError_t of the last failing CUDA call made through this library (0 if none). */
+int fb4_last_cuda_error(void);
+
+const char* fb4_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FB4_H_ */

@@ -1,0 +1,53 @@
+// Internal declarations shared by the translation units of libfb4 (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fb4.h"
+
+// Lookup tables as they sit in device global memory (copied to shared memory by each CTA).
+struct Fb4DeviceTables {
+  uint8_t qvalue[32][32];   // [dialect][bin] -> index 0..7 of the nearest magnitude   (Sec. 3.2)
+  uint8_t qerror[32][32];   // [dialect][bin] -> |bin midpoint - nearest magnitude| in quarter units
+  uint8_t formatbook[32][8];
+  uint32_t stage1[32];      // [bin of block maximum] -> candidate dialect mask
+};
+
+// Per-row extras of one quantize launch (all pointers device, nullable).
+struct Fb4RowExtras {
+  const int32_t* cluster_id;    // SeDA: token -> cluster, -1 = unconstrained
+  const uint32_t* cluster_mask; // SeDA: cluster -> allowed dialect mask
+  const int32_t* salient_idx;   // ascending token ids whose residual is quantized too
+  int64_t n_salient;
+  int32_t tile;                 // > 0: salient_idx[t / tile] is the only possible match for token t
+  uint8_t* res_codes;           // [n_salient][C/2]
+  uint16_t* res_meta;           // [n_salient][C/B]
+};
+
+struct fb4_ctx {
+  int device;
+  fb4_config cfg;
+  Fb4DeviceTables host_tables;   // host copy
+  Fb4DeviceTables* d_tables;     // device copy
+  void* d_fast_tables;           // packed tables of the TMA-staged kernel (NULL if not eligible)
+  int fast_ok;                   // formatbook/stage-1 table fit the fast kernel's packed layout
+  int sm_count;
+  int64_t launches;
+  const char* last_variant;
+  cudaStream_t pipe_stream[3];   // fb4_quantize_host pipeline
+  cudaEvent_t pipe_event[3];
+};
+
+int fb4_set_cuda_error(cudaError_t e);   // records e, returns FB4_ERR_CUDA
+
+// generic kernels (any supported config)
+cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
+                                        const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
+                                        cudaStream_t stream);
+cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T,
+                                  int64_t C, const int32_t* salient_idx, int64_t n_salient,
+                                  const uint8_t* res_codes, const uint16_t* res_meta, void* out, int out_dtype,
+                                  cudaStream_t stream);
+cudaError_t fb4_launch_select_salient(const float* score, int64_t T, int32_t tile, int32_t* salient_idx,
+                                      cudaStream_t stream);

@@ -1,0 +1,192 @@
+"""GPU parity: the CUDA library (through its C-ABI binding) against the CPU oracle, bit for bit,
+on the same seeded inputs.  Sizes span several tiles and ragged tails; the five workloads run at
+full size (the largest on sampled rows).  Run with -m gpu on a B200."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import FB, assert_same_bits_f32, assert_same_quantized, meta_np, to_dev_bf16
+from oracle import fb4_oracle as orc
+from paper_2603_02883_b200 import fb4, synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q32():
+    q = fb4.Fb4()
+    yield q
+    q.close()
+
+
+def heavy(T, C, seed, kind=1):
+    w = synth.Workload("t", T=T, C=C, seed=seed, kind=kind, n_outlier=max(1, C // 200), outlier_gain=50.0)
+    return synth.activation(w)
+
+
+def edge_blocks():
+    """Hand-made blocks: zeros, -0, subnormals, extreme exponents, exact rounding ties, dialect ties."""
+    f = np.zeros((40, 64), dtype=np.float32)
+    f[1, :] = -0.0
+    f[2, 5] = 1e-40
+    f[2, 6] = -3e-39                       # bf16 subnormals
+    f[3, :32] = 2.0 ** -126
+    f[3, 32:] = 2.0 ** -130
+    f[4, 0] = 3.0e38
+    f[4, 1:8] = 1.5e38                     # top of the bf16 range
+    f[5, :] = 2.0 ** 127
+    f[6, :32] = np.arange(32) / 2.0        # every half-integer: exact ties at v = k/2 (max 15.5 -> e = 3)
+    f[6, 32:] = -np.arange(32) / 4.0
+    f[7, :] = 1.0                          # all equal: every element is the block maximum
+    f[8, ::4] = [8, 9, 10, 11, 12, 13, 14, 15, 8.5, 9.5, 10.5, 11.5, 12.5, 13.5, 14.5, 15.5]
+    f[9, 0], f[9, 33] = 12.0, -12.0
+    f[9, 1:32] = 0.25
+    rng = np.random.default_rng(11)
+    f[10:] = rng.standard_normal((30, 64)).astype(np.float32) * (2.0 ** rng.integers(-140, 120, size=(30, 1)))
+    bits = synth.f32_to_bf16_bits(f)
+    bits[11, :] = 0x0001                   # smallest subnormal everywhere
+    bits[12, 3] = 0x7F7F                   # largest finite bf16
+    bits[12, 4] = 0xFF7F
+    return bits
+
+
+CONFIGS = [dict(block_size=32, num_groups=8), dict(block_size=16, num_groups=8),
+           dict(block_size=32, num_groups=32), dict(block_size=16, num_groups=16),
+           dict(block_size=32, num_groups=8, select_mode=1),
+           dict(block_size=32, num_groups=8, exp_min=-15, exp_max=16),
+           dict(block_size=16, num_groups=8, exp_min=-8, exp_max=3, select_mode=1)]
+
+
+@pytest.mark.parametrize("cfg", CONFIGS, ids=lambda c: "-".join(f"{k[:3]}{v}" for k, v in c.items()))
+def test_edge_blocks_and_random_small(cfg):
+    q = fb4.Fb4(**cfg)
+    ocfg = orc.Config(**cfg)
+    for bits in (edge_blocks(), heavy(37, 96, 5), heavy(3, 2048 + 64, 6), heavy(130, 1024, 7, kind=0)):
+        ref = orc.quantize(bits, FB, ocfg)
+        got = q.quantize(to_dev_bf16(bits))
+        assert_same_quantized(got, ref, f"{cfg}")
+        out = q.dequantize(got)
+        assert_same_bits_f32(out, orc.dequantize(ref, FB, cfg["block_size"]), f"{cfg} dequant")
+        outb = q.dequantize(got, torch.bfloat16)
+        refb = orc.dequantize(ref, FB, cfg["block_size"], out_dtype="bf16")
+        assert np.array_equal(outb.view(torch.int16).cpu().numpy().view(np.uint16), refb)
+    q.close()
+
+
+def test_tables_match_direct_rounding(q32):
+    """Qvalue/Qerror built at init against exhaustive direct rounding over every bf16 v in [0,16)."""
+    fbk, s1, qv, qe = fb4.fb4_get_tables(q32.ctx)
+    assert np.array_equal(fbk, FB)
+    assert np.array_equal(s1, orc.default_stage1(FB))
+    pats = np.arange(0, 0x4180, dtype=np.uint16)                 # 0 .. 16.0 (exclusive)
+    v = synth.bf16_bits_to_f32(pats).astype(np.float64)
+    assert v.max() < 16
+    bins = np.floor(2 * v).astype(int)
+    for d in range(32):
+        mags = FB[d].astype(np.float64)
+        dist = np.abs(v[:, None] - mags[None, :])
+        near = 7 - np.argmin(dist[:, ::-1], axis=1)             # ties -> larger magnitude
+        assert np.array_equal(qv[d][bins], near)
+        mid = np.arange(32) / 2 + 0.25
+        assert np.array_equal(qe[d], (4 * np.min(np.abs(mid[:, None] - mags[None, :]), axis=1)).astype(int))
+
+
+def test_strided_rows(q32):
+    bits = heavy(50, 256 + 64, 8)
+    x = to_dev_bf16(bits)
+    view = x[:, :256]                                            # ld = 320
+    ref = orc.quantize(bits[:, :256], FB)
+    assert_same_quantized(q32.quantize(view), ref, "strided")
+
+
+def test_seda_masks(q32):
+    bits = heavy(64, 512, 9)
+    rng = np.random.default_rng(3)
+    w = synth.Workload("t", T=64, C=512, seed=9, kind=1, n_outlier=0, outlier_gain=1.0, seda=True, n_clusters=6,
+                       cluster_seed=12)
+    cid, masks = synth.clusters(w)
+    masks = masks.copy()
+    masks[1] = rng.integers(1, 2 ** 32)          # arbitrary masks: partial / empty stage-1 intersections
+    masks[2] = 1 << 31
+    masks[3] = 0x00000003                        # only the narrowest dynamic range
+    cid = cid.copy()
+    cid[5:9] = -1                                # unconstrained tokens
+    ref = orc.quantize(bits, FB, cluster_id=cid, cluster_mask=masks)
+    got = q32.quantize(to_dev_bf16(bits), torch.from_numpy(cid).cuda(),
+                       torch.from_numpy(masks.view(np.int32)).cuda())
+    assert_same_quantized(got, ref, "seda")
+    did = meta_np(got.meta) >> 8
+    for t in range(64):
+        if cid[t] >= 0:
+            assert np.all((int(masks[cid[t]]) >> did[t]) & 1)
+
+
+@pytest.mark.parametrize("T,tile", [(40, 20), (47, 20), (7, 20), (64, 1), (100, 7)])
+def test_decomposed_small(q32, T, tile):
+    bits = heavy(T, 256, 10 + T)
+    w = synth.Workload("t", T=T, C=256, seed=1, kind=1, n_outlier=0, outlier_gain=1.0, score_seed=T)
+    score = synth.scores(w)
+    score[T // 2:T // 2 + 3] = score[T // 2]                    # ties inside a tile
+    sal = orc.select_salient(score, tile)
+    ref = orc.quantize(bits, FB, salient_idx=sal)
+    got = q32.quantize_decomposed(to_dev_bf16(bits), torch.from_numpy(score).cuda(), tile)
+    assert_same_quantized(got, ref, "decomposed")
+    assert np.array_equal(q32.select_salient(torch.from_numpy(score).cuda(), tile).cpu().numpy(), sal)
+    assert_same_bits_f32(q32.dequantize(got), orc.dequantize(ref, FB), "decomposed dequant")
+    # caller-given salient set (reused from an earlier step): arbitrary ascending list
+    mine = np.unique(np.random.default_rng(T).integers(0, T, size=max(1, T // 3))).astype(np.int32)
+    ref2 = orc.quantize(bits, FB, salient_idx=mine)
+    got2 = q32.quantize_decomposed(to_dev_bf16(bits), salient_idx=torch.from_numpy(mine).cuda())
+    assert_same_quantized(got2, ref2, "decomposed idx")
+    assert_same_bits_f32(q32.dequantize(got2), orc.dequantize(ref2, FB), "decomposed idx dequant")
+
+
+def test_decomposed_with_seda_and_b16():
+    q = fb4.Fb4(block_size=16)
+    bits = heavy(60, 128, 21)
+    w = synth.Workload("t", T=60, C=128, seed=1, kind=1, n_outlier=0, outlier_gain=1.0, score_seed=3, seda=True,
+                       n_clusters=5, cluster_seed=4)
+    score = synth.scores(w)
+    cid, masks = synth.clusters(w)
+    sal = orc.select_salient(score, 20)
+    ref = orc.quantize(bits, FB, orc.Config(block_size=16), cluster_id=cid, cluster_mask=masks, salient_idx=sal)
+    got = q.quantize_decomposed(to_dev_bf16(bits), torch.from_numpy(score).cuda(), 20,
+                                cluster_id=torch.from_numpy(cid).cuda(),
+                                cluster_mask=torch.from_numpy(masks.view(np.int32)).cuda())
+    assert_same_quantized(got, ref, "decomposed+seda b16")
+    assert_same_bits_f32(q.dequantize(got), orc.dequantize(ref, FB, 16), "b16 dequant")
+    q.close()
+
+
+def test_argument_checks(q32):
+    x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
+    codes = torch.empty((4, 32), dtype=torch.uint8, device="cuda")
+    meta = torch.empty((4, 2), dtype=torch.int16, device="cuda")
+    L = fb4.lib()
+    import ctypes
+    p = lambda t, off=0: ctypes.c_void_p(t.data_ptr() + off)
+    assert L.fb4_quantize(q32.ctx, p(x), 4, 48, 64, p(codes), p(meta), None) == fb4.ERR_SHAPE       # C % B
+    assert L.fb4_quantize(q32.ctx, p(x), 4, 64, 32, p(codes), p(meta), None) == fb4.ERR_SHAPE       # ld < C
+    assert L.fb4_quantize(q32.ctx, p(x), -1, 64, 64, p(codes), p(meta), None) == fb4.ERR_SHAPE
+    assert L.fb4_quantize(q32.ctx, p(x, 2), 3, 64, 64, p(codes), p(meta), None) == fb4.ERR_ALIGN
+    assert L.fb4_quantize(q32.ctx, p(x), 4, 32, 36, p(codes), p(meta), None) == fb4.ERR_ALIGN       # ld % 8
+    assert L.fb4_quantize(q32.ctx, p(x), 4, 64, 64, None, p(meta), None) == fb4.ERR_INVALID_ARG
+    assert L.fb4_quantize(q32.ctx, None, 0, 64, 64, None, None, None) == fb4.OK                      # empty
+    assert L.fb4_quantize_seda(q32.ctx, p(x), 4, 64, 64, None, None, 0, p(codes), p(meta), None) == fb4.ERR_INVALID_ARG
+    assert L.fb4_dequantize(q32.ctx, p(codes), p(meta), 4, 64, None, 0, None, None, p(x), 7, None) == fb4.ERR_INVALID_ARG
+    assert L.fb4_select_salient(q32.ctx, p(x), 4, 0, p(meta), None) == fb4.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+
+
+def test_host_buffer_entry_point(q32):
+    w = synth.workloads()["c1"]
+    bits = synth.activation(w)
+    ref = orc.quantize(bits, FB)
+    xh = torch.from_numpy(bits.view(np.int16)).pin_memory()
+    ch = torch.empty((w.T, w.C // 2), dtype=torch.uint8).pin_memory()
+    mh = torch.empty((w.T, w.C // 32), dtype=torch.int16).pin_memory()
+    dx = torch.empty((w.T, w.C), dtype=torch.int16, device="cuda")
+    dc = torch.empty((w.T, w.C // 2), dtype=torch.uint8, device="cuda")
+    dm = torch.empty((w.T, w.C // 32), dtype=torch.int16, device="cuda")
+    fb4.fb4_quantize_host(q32.ctx, xh, w.T, w.C, dx, dc, dm, ch, mh)
+    assert np.array_equal(ch.numpy(), ref.codes) and np.array_equal(mh.numpy().view(np.uint16), ref.meta)

@@ -1,0 +1,131 @@
+"""The five benchmark workloads at full size against the oracle (bit-exact codes, dialect ids,
+scale bytes, salient indices; decoded fp32 at 0 ULP; MSE within 1e-6 relative).  The largest
+tensor is quantized in full on the GPU and compared on sampled rows (every row is quantized
+independently, so a row sample is a complete check of those rows)."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import FB, assert_same_bits_f32, assert_same_quantized, meta_np, to_dev_bf16
+from oracle import fb4_oracle as orc
+from paper_2603_02883_b200 import fb4, synth
+
+pytestmark = pytest.mark.gpu
+
+MSE_RTOL = 1e-6
+
+
+@pytest.fixture(scope="module")
+def q32():
+    q = fb4.Fb4()
+    yield q
+    q.close()
+
+
+@pytest.fixture(scope="module")
+def c2_bits():
+    return synth.activation(synth.workloads()["c2"])
+
+
+def gpu_mse(x: torch.Tensor, recon: torch.Tensor, chunk: int = 4096) -> float:
+    acc = 0.0
+    for r in range(0, x.shape[0], chunk):
+        d = x[r:r + chunk].double() - recon[r:r + chunk].double()
+        acc += float((d * d).sum())
+    return acc / x.numel()
+
+
+def test_c1_quantize_dequantize(q32):
+    w = synth.workloads()["c1"]
+    bits = synth.activation(w)
+    ref = orc.quantize(bits, FB)
+    x = to_dev_bf16(bits)
+    got = q32.quantize(x)
+    assert_same_quantized(got, ref, "c1")
+    out = q32.dequantize(got)
+    ref_out = orc.dequantize(ref, FB)
+    assert_same_bits_f32(out, ref_out, "c1 dequant")
+    m_ref = orc.mse(bits, ref_out)
+    assert abs(gpu_mse(x, out) - m_ref) <= MSE_RTOL * m_ref
+
+
+def test_c2_plain(q32, c2_bits):
+    ref = orc.quantize(c2_bits, FB)
+    x = to_dev_bf16(c2_bits)
+    got = q32.quantize(x)
+    assert_same_quantized(got, ref, "c2")
+    out = q32.dequantize(got)
+    ref_out = orc.dequantize(ref, FB)
+    assert_same_bits_f32(out, ref_out, "c2 dequant")
+    m_ref = orc.mse(c2_bits, ref_out)
+    assert abs(gpu_mse(x, out) - m_ref) <= MSE_RTOL * m_ref
+
+
+def test_c3_decomposed(q32, c2_bits):
+    w = synth.workloads()["c3"]
+    score = synth.scores(w)
+    sal = orc.select_salient(score, w.tile)
+    assert len(sal) == 1638
+    ref = orc.quantize(c2_bits, FB, salient_idx=sal)
+    x = to_dev_bf16(c2_bits)
+    got = q32.quantize_decomposed(x, torch.from_numpy(score).cuda(), w.tile)
+    assert_same_quantized(got, ref, "c3")
+    out = q32.dequantize(got)
+    ref_out = orc.dequantize(ref, FB)
+    assert_same_bits_f32(out, ref_out, "c3 dequant")
+    m_ref = orc.mse(c2_bits, ref_out)
+    assert abs(gpu_mse(x, out) - m_ref) <= MSE_RTOL * m_ref
+
+
+def test_c4_seda(q32, c2_bits):
+    w = synth.workloads()["c4"]
+    cid, masks = synth.clusters(w)
+    ref = orc.quantize(c2_bits, FB, cluster_id=cid, cluster_mask=masks)
+    got = q32.quantize(to_dev_bf16(c2_bits), torch.from_numpy(cid).cuda(),
+                       torch.from_numpy(masks.view(np.int32)).cuda())
+    assert_same_quantized(got, ref, "c4")
+    did = meta_np(got.meta) >> 8
+    allowed = masks[cid][:, None]
+    assert np.all((allowed >> did) & 1)
+
+
+def test_c5_decomposed_seda_and_plain_sampled_rows(q32):
+    w = synth.workloads()["c5"]
+    bits = synth.activation(w)                       # 1.86 GB on the host
+    score = synth.scores(w)
+    cid, masks = synth.clusters(w)
+    sal = orc.select_salient(score, w.tile)
+    assert len(sal) == 3780
+    x = to_dev_bf16(bits)
+    got = q32.quantize_decomposed(x, torch.from_numpy(score).cuda(), w.tile,
+                                  cluster_id=torch.from_numpy(cid).cuda(),
+                                  cluster_mask=torch.from_numpy(masks.view(np.int32)).cuda())
+    assert np.array_equal(got.salient_idx.cpu().numpy(), sal)
+    plain = q32.quantize(x)
+    out = q32.dequantize(got, torch.bfloat16)        # bf16 keeps the decoded tensor at 1.86 GB
+    # sampled rows: three slabs (start, middle with a cluster boundary, ragged end) + 300 salient rows
+    rng = np.random.default_rng(0)
+    rows = np.unique(np.concatenate([np.arange(0, 256), np.arange(37000, 37256), np.arange(w.T - 200, w.T),
+                                     rng.choice(sal, 300, replace=False), rng.integers(0, w.T, 300)]))
+    sub = np.ascontiguousarray(bits[rows])
+    sub_sal = np.flatnonzero(np.isin(rows, sal)).astype(np.int32)
+    ref = orc.quantize(sub, FB, cluster_id=cid[rows], cluster_mask=masks, salient_idx=sub_sal)
+    ridx = torch.from_numpy(rows).cuda()
+    assert np.array_equal(got.codes[ridx].cpu().numpy(), ref.codes)
+    assert np.array_equal(meta_np(got.meta[ridx]), ref.meta)
+    srows = torch.from_numpy(np.searchsorted(sal, rows[sub_sal])).cuda()
+    assert np.array_equal(got.res_codes[srows].cpu().numpy(), ref.res_codes)
+    assert np.array_equal(meta_np(got.res_meta[srows]), ref.res_meta)
+    ref_out = orc.dequantize(ref, FB, out_dtype="bf16")
+    assert np.array_equal(out[ridx].view(torch.int16).cpu().numpy().view(np.uint16), ref_out)
+    refp = orc.quantize(sub, FB)
+    assert np.array_equal(plain.codes[ridx].cpu().numpy(), refp.codes)
+    assert np.array_equal(meta_np(plain.meta[ridx]), refp.meta)
+    # properties that hold at any size: SeDA choices inside the mask, scale byte = exponent of the block maximum
+    did = (got.meta.view(torch.int16).to(torch.int32) >> 8) & 31
+    allowed = torch.from_numpy(masks.view(np.int32)).cuda()[torch.from_numpy(cid).cuda().long()].to(torch.int64) & 0xFFFFFFFF
+    assert bool((((allowed[:, None] >> did.to(torch.int64)) & 1) == 1).all())
+    amax = x.view(w.T, w.C // 32, 32).abs().amax(dim=2).float()
+    e = torch.floor(torch.log2(amax.clamp_min(2.0 ** -124))).to(torch.int32)
+    sb = plain.meta.view(torch.int16).to(torch.int32) & 0xFF
+    assert bool((sb == e + 124).all())
