@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the FB4 online activation quantizer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one plain FB4 quantization (fb4_quantize) of the 75600 x 12288 bf16 activation tensor
+(the largest workload; 1.86 GB in, so every step streams from HBM, far beyond the 126 MB L2).
+`value` is algorithmic GB/s (2 B read + 0.5 B codes + 2 B per 32-element block of metadata per
+element) over all ranks; with N > 1 every rank quantizes its own tensor of that shape (no
+data-path collective; weak scaling).  The other paths of the library (SeDA, decomposition,
+decode, the smaller tensor) are timed the same way and reported under "variants".  One JSON
+line is printed by rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "fb4_quantize_throughput"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this
+# workload, from the ncu capture summarised under profiles/ (None until a capture exists).
+NCU_TRAFFIC_BYTES = None
+
+
+def algorithmic_bytes(T: int, C: int, B: int = 32, n_res_rows: int = 0, seda: bool = False,
+                      decomposed: bool = False) -> float:
+    b = T * C * (2 + 0.5) + T * (C // B) * 2
+    if seda:
+        b += 4 * T
+    if decomposed:
+        b += n_res_rows * (C * 0.5 + (C // B) * 2) + 4 * T + 4 * n_res_rows
+    return float(b)
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+                 "sw_power_cap": 0x4, "hw_power_brake": 0x80}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            time.sleep(0.02)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread:
+            self._thread.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def visible_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def time_steps(fn, steps: int, warmup: int, torch, barrier=None):
+    """W untimed calls, then K calls timed with CUDA events on the current stream (per-launch
+    events too); returns (total ms, list of per-call ms)."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+        torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record()
+    for i in range(steps):
+        fn()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+    return ev[0].elapsed_time(ev[steps]), per
+
+
+def run_reference(args):
+    """The CPU oracle, as it stands, on the host cores: each step is a bounded row sample of the
+    same workload and metric."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import fb4_oracle as orc
+    from paper_2603_02883_b200 import synth
+    w = synth.workloads()["c5_plain"]
+    rows = 4096
+    bits = synth.activation_rows(w, 0, rows)
+    fbk = synth.STANDIN_FORMATBOOK
+    for _ in range(args.warmup):
+        orc.quantize(bits, fbk)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        orc.quantize(bits, fbk)
+    dt = (time.perf_counter() - t0) / args.steps
+    gbs = algorithmic_bytes(rows, w.C) / dt / 1e9
+    cores = os.cpu_count()
+    sample = f"first {rows} of {w.T} rows of the 75600x12288 tensor per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "gelem_per_s": rows * w.C / dt / 1e9,
+        "config": {"workload": "plain FB4 quantize, 75600x12288 bf16 (config-5 tensor), block 32, full formatbook",
+                   "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c5_plain", help="c5_plain (default) or c2 (smaller tensor, for profiling)")
+    ap.add_argument("--no-variants", action="store_true", help="time only the headline step")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2603_02883_b200 import fb4, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the quantizer has no CPU path")
+    torch.cuda.set_device(local_rank)
+    barrier = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        barrier = dist.barrier
+
+    ws = synth.workloads()
+    w = ws[args.workload]
+    if world > 1:   # every rank its own tensor of the same shape
+        w = synth.Workload(**{**w.__dict__, "seed": w.seed + 1000 * rank})
+    bits = synth.activation(w)
+    x = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+    q = fb4.Fb4(device=local_rank)
+    T, C, B = w.T, w.C, 32
+    codes = torch.empty((T, C // 2), dtype=torch.uint8, device="cuda")
+    meta = torch.empty((T, C // B), dtype=torch.int16, device="cuda")
+
+    def step():
+        fb4.fb4_quantize(q.ctx, x, T, C, C, codes, meta)
+
+    l0 = q.launch_count
+    for _ in range(args.warmup):
+        step()
+    launches_warm = q.launch_count - l0
+    with ClockSampler(visible_index(local_rank)) as clk:
+        total_ms, per = time_steps(step, args.steps, 0, torch, barrier)
+    launches = (q.launch_count - l0 - launches_warm)
+    variant = q.last_variant
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms = total_ms / args.steps
+    alg = algorithmic_bytes(T, C)
+    value = world * alg / (ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    kernel_ms = float(np.mean(per))
+    achieved = alg / (kernel_ms * 1e-3) / 1e9
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "gelem_per_s": world * T * C / (ms * 1e-3) / 1e9,
+        "frac_hbm_measured": value / world / peak, "frac_hbm_nominal_8000": value / world / 8000.0,
+        "config": {"workload": f"plain FB4 quantize, {T}x{C} bf16 "
+                               f"({'config-5' if args.workload == 'c5_plain' else args.workload} tensor), block 32, "
+                               "full formatbook, two-stage selection",
+                   "per_gpu_tokens": T, "channels": C, "block_size": B, "kernel_variant": variant,
+                   "l2": "input 1.86 GB per step, larger than L2; no flush needed" if T * C * 2 > 2.5e8
+                         else "input larger than L2 only marginally"},
+        "gpu_launches": launches,
+        "clocks": clk.summary(),
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": NCU_TRAFFIC_BYTES, "peak_kind": f"{peak_kind} copy bandwidth",
+                     "kernel": f"fb4 quantize ({variant})", "algorithmic_bytes_per_launch": alg,
+                     "launch_ms_mean": kernel_ms, "launch_ms_min": float(np.min(per))},
+    }
+
+    if rank == 0 and not args.no_variants:
+        out["variants"] = run_variants(q, x, w, args, torch, fb4, synth, peak)
+    if not args.no_e2e:
+        e2e = run_e2e(q, bits, w, args, torch, fb4, barrier)
+        if world > 1:
+            t = torch.tensor([e2e["seconds_per_step"]], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e["seconds_per_step"] = float(t.item())
+        e2e["value"] = world * alg / e2e["seconds_per_step"] / 1e9
+        out["e2e"] = e2e
+    if rank == 0 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = run_cpu_baseline(w, synth)
+    if rank == 0:
+        print(json.dumps(out))
+    q.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_variants(q, x, w, args, torch, fb4, synth, peak):
+    """The other library paths on the same device, each timed like the headline step."""
+    T, C, B = w.T, w.C, 32
+    res = {}
+    steps, warm = max(3, args.steps // 2), 3
+    big = synth.Workload(**{**w.__dict__, "decomposed": True, "score_seed": 4, "seda": True, "n_clusters": 256,
+                            "cluster_seed": 4})
+    score = torch.from_numpy(synth.scores(big)).cuda()
+    cid_np, mask_np = synth.clusters(big)
+    cid = torch.from_numpy(cid_np).cuda()
+    cmask = torch.from_numpy(mask_np.view(np.int32)).cuda()
+    n_sal = -(-T // big.tile)
+    codes = torch.empty((T, C // 2), dtype=torch.uint8, device="cuda")
+    meta = torch.empty((T, C // B), dtype=torch.int16, device="cuda")
+    rc = torch.empty((n_sal, C // 2), dtype=torch.uint8, device="cuda")
+    rm = torch.empty((n_sal, C // B), dtype=torch.int16, device="cuda")
+    sal = torch.empty(n_sal, dtype=torch.int32, device="cuda")
+
+    def rec(name, fn, alg):
+        total, per = time_steps(fn, steps, warm, torch)
+        ms = total / steps
+        res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
+                     "kernel_variant": q.last_variant}
+
+    rec("seda", lambda: fb4.fb4_quantize_seda(q.ctx, x, T, C, C, cid, cmask, cmask.numel(), codes, meta),
+        algorithmic_bytes(T, C, seda=True))
+    rec("decomposed", lambda: fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, big.tile, None, None, 0, codes,
+                                                          meta, sal, rc, rm),
+        algorithmic_bytes(T, C, n_res_rows=n_sal, decomposed=True))
+    rec("decomposed_seda", lambda: fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, big.tile, cid, cmask,
+                                                               cmask.numel(), codes, meta, sal, rc, rm),
+        algorithmic_bytes(T, C, n_res_rows=n_sal, seda=True, decomposed=True))
+    out32 = torch.empty((T, C), dtype=torch.float32, device="cuda")
+    rec("dequantize_f32", lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, sal, n_sal, rc, rm, out32, 0),
+        T * C * (0.5 + 4) + T * (C // B) * 2 + n_sal * (C * 0.5 + (C // B) * 2))
+    del out32
+    out16 = torch.empty((T, C), dtype=torch.bfloat16, device="cuda")
+    rec("dequantize_bf16", lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, None, 0, None, None, out16, 1),
+        T * C * (0.5 + 2) + T * (C // B) * 2)
+    del out16
+    if w.name != "c2":
+        w2 = synth.workloads()["c2"]
+        x2 = torch.from_numpy(synth.activation(w2).view(np.int16)).cuda().view(torch.bfloat16)
+        c2 = torch.empty((w2.T, w2.C // 2), dtype=torch.uint8, device="cuda")
+        m2 = torch.empty((w2.T, w2.C // B), dtype=torch.int16, device="cuda")
+        # 258 MB per step is not far above the 126 MB L2: flush with a 512 MB write between steps
+        flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+        evs = []
+        for i in range(warm + steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fb4.fb4_quantize(q.ctx, x2, w2.T, w2.C, w2.C, c2, m2)
+            b.record()
+            evs.append((a, b))
+        torch.cuda.synchronize()
+        ms = float(np.mean([a.elapsed_time(b) for a, b in evs[warm:]]))
+        alg = algorithmic_bytes(w2.T, w2.C)
+        res["c2_plain_32760x3072_l2_flushed"] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9,
+                                                 "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
+                                                 "kernel_variant": q.last_variant}
+    return res
+
+
+def run_e2e(q, bits, w, args, torch, fb4, barrier):
+    """Same step through fb4_quantize_host: pinned host input -> device -> pinned host codes/meta,
+    copies inside the timed region."""
+    T, C, B = w.T, w.C, 32
+    xh = torch.from_numpy(bits.view(np.int16)).pin_memory()
+    ch = torch.empty((T, C // 2), dtype=torch.uint8).pin_memory()
+    mh = torch.empty((T, C // B), dtype=torch.int16).pin_memory()
+    dx = torch.empty((T, C), dtype=torch.int16, device="cuda")
+    dc = torch.empty((T, C // 2), dtype=torch.uint8, device="cuda")
+    dm = torch.empty((T, C // B), dtype=torch.int16, device="cuda")
+    steps = max(2, min(args.steps, 5))
+    fb4.fb4_quantize_host(q.ctx, xh, T, C, dx, dc, dm, ch, mh)
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        fb4.fb4_quantize_host(q.ctx, xh, T, C, dx, dc, dm, ch, mh)
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / steps
+    return {"value": None, "unit": UNIT, "h2d_bytes_per_step": T * C * 2,
+            "d2h_bytes_per_step": T * C // 2 + T * (C // B) * 2, "seconds_per_step": dt, "steps": steps,
+            "api": "fb4_quantize_host (pinned host buffers, chunked copies pipelined with the kernel)"}
+
+
+def run_cpu_baseline(w, synth):
+    from oracle import fb4_oracle as orc
+    rows = min(w.T, 16384)
+    bits = synth.activation_rows(w, 0, rows)
+    fbk = synth.STANDIN_FORMATBOOK
+    orc.quantize(bits[:256], fbk)
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        orc.quantize(bits, fbk)
+        reps += 1
+        if time.perf_counter() - t0 > 10.0 or reps >= 20:
+            break
+    dt = (time.perf_counter() - t0) / reps
+    return {"value": algorithmic_bytes(rows, w.C) / dt / 1e9, "unit": UNIT, "cores": os.cpu_count(),
+            "kind": "oracle", "gelem_per_s": rows * w.C / dt / 1e9,
+            "sample": f"first {rows} of {w.T} rows, {reps} passes, OpenMP over rows on all host cores"}
+
+
+if __name__ == "__main__":
+    main()

@@ -118,7 +118,7 @@ def test_seda_masks(q32):
     did = meta_np(got.meta) >> 8
     for t in range(64):
         if cid[t] >= 0:
-            assert np.all((int(masks[cid[t]]) >> did[t]) & 1)
+            assert np.all((int(masks[cid[t]]) >> did[t].astype(np.int64)) & 1)
 
 
 @pytest.mark.parametrize("T,tile", [(40, 20), (47, 20), (7, 20), (64, 1), (100, 7)])

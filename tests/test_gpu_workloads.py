@@ -84,8 +84,8 @@ def test_c4_seda(q32, c2_bits):
     got = q32.quantize(to_dev_bf16(c2_bits), torch.from_numpy(cid).cuda(),
                        torch.from_numpy(masks.view(np.int32)).cuda())
     assert_same_quantized(got, ref, "c4")
-    did = meta_np(got.meta) >> 8
-    allowed = masks[cid][:, None]
+    did = (meta_np(got.meta) >> 8).astype(np.int64)
+    allowed = masks[cid][:, None].astype(np.int64)
     assert np.all((allowed >> did) & 1)
 
 
