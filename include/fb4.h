@@ -25,7 +25,10 @@
  *     meaningless, but in-bounds, output).
  *   - Alignment: x and every output pointer must be 16-byte aligned and
  *     ld_elems a multiple of 8; otherwise FB4_ERR_ALIGN.
- *   - Device code has no wait loops; a call cannot hang.
+ *   - The device of the context must be the current device of the calling thread.
+ *   - Device code has no unbounded wait loops: the only waits (for asynchronous loads into
+ *     shared memory) give up after a fixed number of tries and raise a status bit
+ *     (fb4_device_status); a call cannot hang.
  *
  * Output layout
  *   codes : uint8 [T][C/2].  Byte j of a row holds element 2j in its low nibble
@@ -175,6 +178,16 @@ int fb4_dequantize(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int
  */
 int fb4_quantize_host(fb4_ctx* ctx, const void* x_host, int64_t T, int64_t C, void* d_x, uint8_t* d_codes,
                       uint16_t* d_meta, uint8_t* codes_host, uint16_t* meta_host);
+
+/* Kernel choice: 0 (default) = the TMA-staged kernel whenever the call qualifies (default
+ * configuration, C a multiple of 64), else the generic kernel; 1 = always the generic kernel.
+ * Both produce identical output; this exists for tests and measurements. */
+int fb4_set_kernel_variant(fb4_ctx* ctx, int variant);
+
+/* Device-side status word of the context, read back with a blocking copy: 0 = fine; bit 0 =
+ * a bounded wait on an asynchronous (TMA) load inside a kernel ran out of tries, in which case
+ * the affected warp stopped early and the outputs of that call are incomplete. */
+int fb4_device_status(fb4_ctx* ctx, uint32_t* status);
 
 /* Number of kernel launches this context has enqueued so far (diagnostic counter). */
 int64_t fb4_launch_count(const fb4_ctx* ctx);

@@ -66,10 +66,6 @@ void build_tables(Fb4DeviceTables& t, const uint8_t* fb, const uint32_t* stage1)
   }
 }
 
-struct Shape {
-  int64_t nblk;
-};
-
 int check_quantize_args(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const void* codes,
                         const void* meta) {
   if (!ctx) return FB4_ERR_INVALID_ARG;
@@ -96,8 +92,14 @@ struct DeviceGuard {
 int run_quantize(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const Fb4RowExtras& ex,
                  uint8_t* codes, uint16_t* meta, cudaStream_t stream) {
   if (T == 0) return FB4_OK;
-  cudaError_t e = fb4_launch_quantize_generic(ctx, x, T, C, ld, ex, codes, meta, stream);
-  ctx->last_variant = "generic";
+  cudaError_t e;
+  if (!ctx->force_generic && fb4_fast_eligible(ctx, x, T, C, ld)) {
+    e = fb4_launch_quantize_fast(ctx, x, T, C, ld, ex, codes, meta, stream);
+    ctx->last_variant = "fast";
+  } else {
+    e = fb4_launch_quantize_generic(ctx, x, T, C, ld, ex, codes, meta, stream);
+    ctx->last_variant = "generic";
+  }
   if (e != cudaSuccess) return fb4_set_cuda_error(e);
   ctx->launches += 1;
   return FB4_OK;
@@ -154,6 +156,8 @@ int fb4_init(fb4_ctx** out, int device, const uint8_t* formatbook, const uint32_
   ctx->d_tables = nullptr;
   ctx->d_fast_tables = nullptr;
   ctx->fast_ok = 0;
+  ctx->force_generic = 0;
+  ctx->d_status = nullptr;
   for (int i = 0; i < 3; ++i) { ctx->pipe_stream[i] = nullptr; ctx->pipe_event[i] = nullptr; }
   build_tables(ctx->host_tables, fb, stage1_mask);
 
@@ -162,11 +166,19 @@ int fb4_init(fb4_ctx** out, int device, const uint8_t* formatbook, const uint32_
   cudaError_t e = cudaMalloc(&ctx->d_tables, sizeof(Fb4DeviceTables));
   if (e == cudaSuccess)
     e = cudaMemcpy(ctx->d_tables, &ctx->host_tables, sizeof(Fb4DeviceTables), cudaMemcpyHostToDevice);
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(uint32_t));
   if (e != cudaSuccess) {
+    if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_tables) cudaFree(ctx->d_tables);
     delete ctx;
     return fb4_set_cuda_error(e);
   }
+  size_t fast_bytes = 0;
+  if (fb4_fast_build_tables(ctx->host_tables, &ctx->d_fast_tables, &fast_bytes) &&
+      fb4_fast_prepare_device() == cudaSuccess)
+    ctx->fast_ok = 1;
+  cudaGetLastError();
   *out = ctx;
   return FB4_OK;
 }
@@ -179,6 +191,7 @@ int fb4_destroy(fb4_ctx* ctx) {
     if (ctx->pipe_stream[i]) cudaStreamDestroy(ctx->pipe_stream[i]);
   }
   if (ctx->d_fast_tables) cudaFree(ctx->d_fast_tables);
+  if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->d_tables) cudaFree(ctx->d_tables);
   delete ctx;
   return FB4_OK;
@@ -331,6 +344,20 @@ int fb4_quantize_host(fb4_ctx* ctx, const void* x_host, int64_t T, int64_t C, vo
     cudaError_t e = cudaStreamSynchronize(ctx->pipe_stream[i]);
     if (e != cudaSuccess) return fb4_set_cuda_error(e);
   }
+  return FB4_OK;
+}
+
+int fb4_set_kernel_variant(fb4_ctx* ctx, int variant) {
+  if (!ctx || variant < 0 || variant > 1) return FB4_ERR_INVALID_ARG;
+  ctx->force_generic = variant;
+  return FB4_OK;
+}
+
+int fb4_device_status(fb4_ctx* ctx, uint32_t* status) {
+  if (!ctx || !status) return FB4_ERR_INVALID_ARG;
+  DeviceGuard guard(ctx->device);
+  cudaError_t e = cudaMemcpy(status, ctx->d_status, sizeof(uint32_t), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
   return FB4_OK;
 }
 

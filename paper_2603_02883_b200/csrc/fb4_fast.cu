@@ -1,0 +1,531 @@
+// TMA-staged FB4 quantize kernel for sm_100a (default configuration: block 32, 8 groups,
+// two-stage selection, exponent range [-124,127]).
+//
+// Work unit: a tile of 1024 consecutive channels of one token (2 KB of bf16 = 32 blocks).
+// Every warp owns a ring of shared-memory stages; lane 0 keeps the ring full with 3-D TMA
+// loads (tensor view [T][C/64][64], box 1 x 16 x 64, 128-byte swizzle) that complete on
+// per-stage mbarriers.  Lane i then quantizes block i of the tile entirely in registers:
+// it reads its 64 bytes with four conflict-free 16-byte shared loads, and the warp writes
+// 512 B of codes and 64 B of metadata with one coalesced store each.
+//
+// Arithmetic (all exact):
+//  * magnitudes are compared as 15-bit integers (bf16 patterns are monotone), two per register;
+//  * bin = floor(2 * |x| * 2^(3-e)) is read from the low mantissa bits of a round-toward-zero
+//    FMA against a power-of-two constant; for the upper bf16 of a register pair the lower
+//    half may stay in place as extra mantissa bits because truncation discards it;
+//  * Qerror: one 64-bit word per (stage-1 group, bin) holds the error of up to 8 candidate
+//    dialects as bytes, so 8 loads + packed adds score all candidates; argmin on (err<<3|j);
+//  * Qvalue: a per-dialect table indexed by the bins of TWO elements returns a finished code
+//    byte; its address comes out of one integer multiply-add of the two FMA results, whose
+//    exponent bits are chosen to cancel modulo 2^32.
+#include <cuda.h>
+
+#include <cstring>
+
+#include "fb4_internal.h"
+
+namespace {
+
+constexpr int kWarps = 16;           // warps per CTA
+constexpr int kStages = 4;           // ring depth per warp
+constexpr int kTileBytes = 2048;     // 1024 bf16
+constexpr int kPairStride = 1060;    // bytes between per-dialect pair tables (1024 + bank rotation)
+constexpr int kMaxGroups = 8;        // distinct stage-1 groups the packed tables hold
+constexpr uint32_t kSpinLimit = 1u << 20;   // tries per wait before a warp gives up
+
+struct FastTables {
+  uint8_t pairlut[32 * kPairStride];     // [dialect][bin_hi*32 + bin_lo] -> idx_lo | idx_hi<<4
+  uint64_t qerr64[kMaxGroups][32];       // [group][bin] -> byte j = Qerror of candidate j (pad 31)
+  uint8_t did_of[kMaxGroups][8];         // [group][candidate] -> dialect id
+  uint8_t group_of_bin[32];              // [bin of block maximum] -> group
+  uint32_t stage1[32];                   // [bin of block maximum] -> candidate mask
+  uint8_t qerror[32][32];                // [dialect][bin], for masks that cut a group
+  uint8_t fb[32][8];
+};
+static_assert(sizeof(FastTables) % 16 == 0, "copied with 16-byte accesses");
+
+struct FastParams {
+  int64_t T, C;
+  int64_t tiles_per_row, n_tiles;
+  uint8_t* codes;
+  uint16_t* meta;
+  uint32_t* status;   // device word: bit 0 = a TMA wait ran out
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c_outer,
+                                              int row) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(0), "r"(c_outer), "r"(row) : "memory");
+}
+__device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
+  uint32_t v;
+  asm("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
+  uint2 v;
+  asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+
+// prmt.b32 in its default mode: selector nibble bit 3 replicates the sign of the chosen byte
+// (the __byte_perm intrinsic only honours the low three bits).
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+  uint32_t d;
+  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+  return d;
+}
+
+__device__ __forceinline__ float pow2f(int k) {   // 2^k, k in [-149,127]
+  return k >= -126 ? __int_as_float((k + 127) << 23) : __int_as_float(1 << (k + 149));
+}
+
+// Score an arbitrary candidate mask over 8 group bins with the byte table (SeDA masks that
+// cut a stage-1 group, and the residual pass).  Ascending ids: ties keep the lowest.
+__device__ __forceinline__ int select_general(uint32_t cand, const uint8_t* gb, const FastTables* tb) {
+  int best = 0, best_err = 0x7fffffff;
+  for (uint32_t m = cand; m; m &= m - 1) {
+    const int d = __ffs((int)m) - 1;
+    int err = 0;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) err += tb->qerror[d][gb[g]];
+    if (err < best_err) { best_err = err; best = d; }
+  }
+  return best;
+}
+
+// Residual pass of one block (Sec. 3.3): Delta = x - Q(x) in fp32 (exact), quantized again.
+// w = the 16 input registers (2 bf16 each), cw = the block's 4 code words.
+__device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t* cw, int did, int e, uint32_t allowed,
+                                            const FastTables* tb, uint32_t* rcw, int* rdid, int* re) {
+  const float sc = pow2f(e - 3);
+  float ax[32];
+  uint32_t sgn = 0;
+  float amax = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    const uint32_t word = w[i >> 1];
+    const float x = __uint_as_float((i & 1) ? (word & 0xffff0000u) : (word << 16));
+    const uint32_t nib = (cw[i >> 3] >> (4 * (i & 7))) & 15u;
+    const float mag = (float)tb->fb[did][nib & 7u] * sc;
+    const float delta = __fsub_rn(x, (nib & 8u) ? -mag : mag);
+    sgn |= (__float_as_uint(delta) >> 31) << i;
+    ax[i] = fabsf(delta);
+    amax = fmaxf(amax, ax[i]);
+  }
+  int er = amax == 0.f ? -124 : (int)((__float_as_uint(amax) >> 23) & 0xff) - 127;
+  er = max(er, -124);
+  const float s = pow2f(3 - er);
+  uint8_t bin[32], gb[8];
+  int bmax = 0;
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    int m = 0;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int b = min(31, __float2int_rd(2.0f * (ax[g * 4 + i] * s)));
+      bin[g * 4 + i] = (uint8_t)b;
+      m = max(m, b);
+    }
+    gb[g] = (uint8_t)m;
+    bmax = max(bmax, m);
+  }
+  uint32_t cand = tb->stage1[bmax] & allowed;
+  if (cand == 0) cand = allowed;
+  const int d = select_general(cand, gb, tb);
+  const uint8_t* qv = tb->pairlut + d * kPairStride;   // entry [0*32 + bin] low nibble = Qvalue[d][bin]
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint32_t word = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int k = q * 8 + i;
+      word |= ((qv[bin[k]] & 7u) | (((sgn >> k) & 1u) << 3)) << (4 * i);
+    }
+    rcw[q] = word;
+  }
+  *rdid = d;
+  *re = er;
+}
+
+template <bool SEDA, bool DECOMP>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTables* __restrict__ g_tables,
+                         FastParams p, Fb4RowExtras ex) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // [ring: kWarps*kStages*2048 B][tables][mbarriers]
+  uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // 128-byte swizzle needs 1 KB alignment
+  FastTables* tb = reinterpret_cast<FastTables*>(ring + kWarps * kStages * kTileBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(FastTables));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t gwarp = (int64_t)blockIdx.x * kWarps + warp;
+  const int64_t wstride = (int64_t)gridDim.x * kWarps;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kWarps * kStages; ++i) mbar_init(smem_u32(bars + i), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytes);
+  const uint32_t my_bars = smem_u32(bars + warp * kStages);
+  // prologue: fill the ring
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < kStages; ++s) {
+      const int64_t g = gwarp + (int64_t)s * wstride;
+      if (g < p.n_tiles) {
+        const int64_t row = g / p.tiles_per_row;
+        const int col = (int)(g - row * p.tiles_per_row);
+        mbar_expect_tx(my_bars + 8 * s, kTileBytes);
+        tma_load_tile(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, col * 16, (int)row);
+      }
+    }
+  }
+  // tables -> shared memory (overlaps the first loads)
+  {
+    const uint4* src = reinterpret_cast<const uint4*>(g_tables);
+    uint4* dst = reinterpret_cast<uint4*>(tb);
+    for (int i = threadIdx.x; i < (int)(sizeof(FastTables) / 16); i += kWarps * 32) dst[i] = src[i];
+  }
+  __syncthreads();
+
+  const uint32_t pair_base = smem_u32(tb->pairlut);
+  const uint32_t qerr_base = smem_u32(tb->qerr64);
+  // this lane's 64 bytes inside a stage: row r = lane/2 of 128 B, chunks (lane&1)*4 + j, swizzled by r&7
+  const uint32_t r = (uint32_t)lane >> 1, c0 = ((uint32_t)lane & 1u) * 4u;
+  uint32_t chunk_off[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) chunk_off[j] = r * 128u + (((c0 + j) ^ (r & 7u)) << 4);
+
+  const int64_t nblk = p.C >> 5;
+  int64_t k = 0;
+  for (int64_t g = gwarp; g < p.n_tiles; g += wstride, ++k) {
+    const int s = (int)(k % kStages);
+    const uint32_t parity = (uint32_t)((k / kStages) & 1);
+    const uint32_t bar = my_bars + 8 * s;
+    uint32_t spins = 0;
+    bool ready = mbar_try_wait(bar, parity);
+    while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(bar, parity);
+    if (!__all_sync(0xffffffffu, ready)) {
+      // A load never arrived: raise the status bit, give the loads still in flight for this warp a
+      // bounded chance to land (so none writes into shared memory after the CTA has gone), stop.
+      if (lane == 0) atomicOr(p.status, 1u);
+      for (int j = 1; j < kStages; ++j) {
+        if (g + (int64_t)j * wstride >= p.n_tiles) break;
+        const int sj = (int)((k + j) % kStages);
+        const uint32_t pj = (uint32_t)(((k + j) / kStages) & 1);
+        uint32_t tries = 0;
+        while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
+      }
+      break;
+    }
+    const int64_t row = g / p.tiles_per_row;
+    const int col = (int)(g - row * p.tiles_per_row);
+    const int64_t blk = (int64_t)col * 32 + lane;
+    const bool active = blk < nblk;
+
+    uint32_t w[16];
+    {
+      const uint32_t base = my_ring + s * kTileBytes;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint4 v = lds_v4(base + chunk_off[j]);
+        w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
+      }
+    }
+    // ---- magnitudes, group maxima (4 elements = 2 registers), block maximum
+    uint32_t a[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a[i] = w[i] & 0x7fff7fffu;
+    uint32_t g2[4];   // (group 2q+1 max << 16) | group 2q max
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint32_t m0 = __vmaxu2(a[4 * q], a[4 * q + 1]);
+      const uint32_t m1 = __vmaxu2(a[4 * q + 2], a[4 * q + 3]);
+      g2[q] = __vmaxu2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));
+    }
+    const uint32_t mm = __vmaxu2(__vmaxu2(g2[0], g2[1]), __vmaxu2(g2[2], g2[3]));
+    const uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
+    // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
+    const uint32_t Ec = max(amax16 >> 7, 3u);
+    const float s2 = __uint_as_float((257u - Ec) << 23);   // 2^(3-e)
+    const float sG = s2 * 0x1p-21f;                        // bins land in the mantissa of 2.0 + ...
+    const float sH = s2 * 0x1p-25f;                        // ... and of 0.125 + ...
+    const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax16 << 16), sG, 2.0f)) & 31u;
+
+    uint32_t allowed = 0xffffffffu;
+    if (SEDA) {
+      if (ex.cluster_id) {
+        const int32_t cid = ex.cluster_id[row];
+        if (cid >= 0) allowed = ex.cluster_mask[cid];
+        if (allowed == 0) allowed = 1u;
+      }
+    }
+    // ---- dialect selection
+    int did;
+    {
+      const uint32_t grp = tb->group_of_bin[bmax];
+      bool packed_path = true;
+      uint32_t cand = 0;
+      if (SEDA) {
+        const uint32_t st1 = tb->stage1[bmax];
+        cand = st1 & allowed;
+        if (cand == 0) cand = allowed;
+        packed_path = (cand == st1);
+      }
+      if (!SEDA || packed_path) {
+        const uint32_t qb = qerr_base + grp * 256u;
+        uint32_t lo = 0, hi = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint32_t t0 = __float_as_uint(__fmaf_rz(__uint_as_float(g2[q] << 16), sG, 2.0f));
+          const uint32_t t1 = __float_as_uint(__fmaf_rz(__uint_as_float(g2[q]), sG, 2.0f));
+          const uint2 e0 = lds_v2((t0 << 3) + qb);   // 0x40000000 << 3 vanishes mod 2^32
+          const uint2 e1 = lds_v2((t1 << 3) + qb);
+          lo += e0.x + e1.x;
+          hi += e0.y + e1.y;
+        }
+        // argmin over 8 byte sums, ties to the lowest candidate: keys (err << 3 | j) in 16-bit lanes
+        const uint32_t k02 = (lo & 0x00ff00ffu) * 8u + 0x00020000u;
+        const uint32_t k13 = ((lo >> 8) & 0x00ff00ffu) * 8u + 0x00030001u;
+        const uint32_t k46 = (hi & 0x00ff00ffu) * 8u + 0x00060004u;
+        const uint32_t k57 = ((hi >> 8) & 0x00ff00ffu) * 8u + 0x00070005u;
+        const uint32_t km = __vminu2(__vminu2(k02, k13), __vminu2(k46, k57));
+        const uint32_t key = min(km & 0xffffu, km >> 16);
+        did = tb->did_of[grp][key & 7u];
+      } else if (__popc(cand) == 1) {
+        did = __ffs((int)cand) - 1;
+      } else {
+        uint8_t gb[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          gb[2 * q] = (uint8_t)(__float_as_uint(__fmaf_rz(__uint_as_float(g2[q] << 16), sG, 2.0f)) & 31u);
+          gb[2 * q + 1] = (uint8_t)(__float_as_uint(__fmaf_rz(__uint_as_float(g2[q]), sG, 2.0f)) & 31u);
+        }
+        did = select_general(cand, gb, tb);
+      }
+    }
+    // ---- Qvalue: one lookup per element pair
+    const float magic_lo = __uint_as_float(0x40000000u + pair_base + (uint32_t)did * kPairStride);
+    uint32_t cw[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t b[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t av = a[4 * q + j];
+        const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sH, 0.125f));        // 0x3E000000 + bin_hi
+        const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sG, magic_lo));  // 0x40000000 + table + bin_lo
+        b[j] = lds_u8(th * 32u + tl);   // 0x3E000000*32 + 0x40000000 == 0 (mod 2^32)
+      }
+      const uint32_t idx = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+      // sign bits: byte masks by sign replication, then to bit 3 of every nibble
+      const uint32_t sa = prmt(w[4 * q], w[4 * q + 1], 0xfdb9u);
+      const uint32_t sb = prmt(w[4 * q + 2], w[4 * q + 3], 0xfdb9u);
+      const uint32_t ev = __byte_perm(sa, sb, 0x6420), od = __byte_perm(sa, sb, 0x7531);
+      cw[q] = idx | (((ev & 0x0f0f0f0fu) | (od & 0xf0f0f0f0u)) & 0x88888888u);
+    }
+    if (active) {
+      *reinterpret_cast<uint4*>(p.codes + row * (p.C >> 1) + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      p.meta[row * nblk + blk] = (uint16_t)((Ec - 3u) | ((uint32_t)did << 8));
+    }
+    if (DECOMP) {
+      int64_t srow = -1;
+      if (ex.tile > 0) {
+        const int64_t sidx = row / ex.tile;
+        if (sidx < ex.n_salient && ex.salient_idx[sidx] == (int32_t)row) srow = sidx;
+      } else {
+        int64_t lo = 0, hi = ex.n_salient - 1;
+        while (lo <= hi) {
+          const int64_t mid = (lo + hi) >> 1;
+          const int32_t v = ex.salient_idx[mid];
+          if (v == (int32_t)row) { srow = mid; break; }
+          if (v < (int32_t)row) lo = mid + 1; else hi = mid - 1;
+        }
+      }
+      if (srow >= 0) {   // warp-uniform: a tile lies inside one token
+        uint32_t rcw[4];
+        int rdid, re;
+        residual_block(w, cw, did, (int)Ec - 127, allowed, tb, rcw, &rdid, &re);
+        if (active) {
+          *reinterpret_cast<uint4*>(ex.res_codes + srow * (p.C >> 1) + blk * 16) =
+              make_uint4(rcw[0], rcw[1], rcw[2], rcw[3]);
+          ex.res_meta[srow * nblk + blk] = (uint16_t)((re + 124) | (rdid << 8));
+        }
+      }
+    }
+    // ---- refill this stage (all lanes have consumed their registers from it)
+    __syncwarp();
+    if (lane == 0) {
+      const int64_t gn = g + (int64_t)kStages * wstride;
+      if (gn < p.n_tiles) {
+        const int64_t rown = gn / p.tiles_per_row;
+        const int coln = (int)(gn - rown * p.tiles_per_row);
+        mbar_expect_tx(bar, kTileBytes);
+        tma_load_tile(my_ring + s * kTileBytes, &tmap, bar, coln * 16, (int)rown);
+      }
+    }
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+constexpr size_t kSmemBytes = 1024 + (size_t)kWarps * kStages * kTileBytes + sizeof(FastTables) + kWarps * kStages * 8;
+
+template <bool SEDA, bool DECOMP>
+cudaError_t launch(const CUtensorMap& map, const FastTables* tables, const FastParams& p, const Fb4RowExtras& ex,
+                   int grid, cudaStream_t stream) {
+  fb4_quantize_fast_kernel<SEDA, DECOMP><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+// Builds the packed tables of this kernel from the plain ones; returns false when the formatbook /
+// stage-1 table does not fit them (more than 8 groups, a group with 0 or more than 8 dialects, or
+// error sums that could overflow a byte): those contexts use the generic kernel.
+bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes) {
+  static FastTables ft;   // ~37 KB: keep it off the stack (fb4_init is not re-entrant per context anyway)
+  std::memset(&ft, 0, sizeof ft);
+  uint32_t groups[kMaxGroups];
+  int ngroups = 0;
+  for (int k = 0; k < 32; ++k) {
+    const uint32_t m = t.stage1[k];
+    const int pc = __builtin_popcount(m);
+    if (pc == 0 || pc > 8) return false;
+    int gi = -1;
+    for (int i = 0; i < ngroups; ++i) if (groups[i] == m) gi = i;
+    if (gi < 0) {
+      if (ngroups == kMaxGroups) return false;
+      gi = ngroups;
+      groups[ngroups++] = m;
+    }
+    ft.group_of_bin[k] = (uint8_t)gi;
+    ft.stage1[k] = m;
+  }
+  for (int gi = 0; gi < ngroups; ++gi) {
+    int j = 0;
+    for (int d = 0; d < 32; ++d) {
+      if (!((groups[gi] >> d) & 1u)) continue;
+      ft.did_of[gi][j] = (uint8_t)d;
+      for (int k = 0; k < 32; ++k) {
+        if (t.qerror[d][k] > 31) return false;
+        ft.qerr64[gi][k] |= (uint64_t)t.qerror[d][k] << (8 * j);
+      }
+      ++j;
+    }
+    for (; j < 8; ++j)
+      for (int k = 0; k < 32; ++k) ft.qerr64[gi][k] |= (uint64_t)31 << (8 * j);   // never beats a real candidate
+  }
+  for (int d = 0; d < 32; ++d)
+    for (int bh = 0; bh < 32; ++bh)
+      for (int bl = 0; bl < 32; ++bl)
+        ft.pairlut[d * kPairStride + bh * 32 + bl] = (uint8_t)(t.qvalue[d][bl] | (t.qvalue[d][bh] << 4));
+  std::memcpy(ft.qerror, t.qerror, sizeof ft.qerror);
+  std::memcpy(ft.fb, t.formatbook, sizeof ft.fb);
+  void* d = nullptr;
+  if (cudaMalloc(&d, sizeof ft) != cudaSuccess) return false;
+  if (cudaMemcpy(d, &ft, sizeof ft, cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaFree(d);
+    return false;
+  }
+  *d_out = d;
+  *bytes = sizeof ft;
+  return true;
+}
+
+// Opt in to the kernel's dynamic shared memory on the current device (once per context).
+cudaError_t fb4_fast_prepare_device() {
+  cudaError_t e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, false>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSmemBytes);
+  return e;
+}
+
+bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {
+  const fb4_config& c = ctx->cfg;
+  if (!ctx->fast_ok || !ctx->d_fast_tables) return false;
+  if (c.block_size != 32 || c.num_groups != 8 || c.select_mode != 0 || c.exp_min != -124 || c.exp_max != 127)
+    return false;
+  if (C % 64 != 0 || (ld & 7) || (reinterpret_cast<uintptr_t>(x) & 15)) return false;
+  if (T > 0x7fffffffLL || C / 64 > 0x7fffffffLL) return false;
+  return encode_tiled_fn() != nullptr;
+}
+
+cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
+                                     const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta, cudaStream_t stream) {
+  CUtensorMap map;
+  const cuuint64_t dims[3] = {64, (cuuint64_t)(C / 64), (cuuint64_t)T};
+  const cuuint64_t strides[2] = {128, (cuuint64_t)ld * 2};
+  const cuuint32_t box[3] = {64, 16, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = encode_tiled_fn()(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides,
+                                       box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  FastParams p;
+  p.T = T;
+  p.C = C;
+  p.tiles_per_row = (C + 1023) / 1024;
+  p.n_tiles = T * p.tiles_per_row;
+  p.codes = codes;
+  p.meta = meta;
+  p.status = ctx->d_status;
+  const int64_t want = (p.n_tiles + kWarps - 1) / kWarps;
+  const int grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
+  const FastTables* tables = static_cast<const FastTables*>(ctx->d_fast_tables);
+  const bool seda = ex.cluster_id != nullptr, decomp = ex.n_salient > 0;
+  if (seda && decomp) return launch<true, true>(map, tables, p, ex, grid, stream);
+  if (seda) return launch<true, false>(map, tables, p, ex, grid, stream);
+  if (decomp) return launch<false, true>(map, tables, p, ex, grid, stream);
+  return launch<false, false>(map, tables, p, ex, grid, stream);
+}

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 
 #include "fb4.h"
@@ -31,8 +32,10 @@ struct fb4_ctx {
   Fb4DeviceTables host_tables;   // host copy
   Fb4DeviceTables* d_tables;     // device copy
   void* d_fast_tables;           // packed tables of the TMA-staged kernel (NULL if not eligible)
+  int force_generic;             // fb4_set_kernel_variant(ctx, 1): always take the generic kernel
   int fast_ok;                   // formatbook/stage-1 table fit the fast kernel's packed layout
   int sm_count;
+  uint32_t* d_status;            // device status word (bit 0: a TMA wait ran out of tries)
   int64_t launches;
   const char* last_variant;
   cudaStream_t pipe_stream[3];   // fb4_quantize_host pipeline
@@ -40,6 +43,13 @@ struct fb4_ctx {
 };
 
 int fb4_set_cuda_error(cudaError_t e);   // records e, returns FB4_ERR_CUDA
+
+// TMA-staged kernel of the default configuration (fb4_fast.cu)
+bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes);
+cudaError_t fb4_fast_prepare_device();
+bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld);
+cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
+                                     const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta, cudaStream_t stream);
 
 // generic kernels (any supported config)
 cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,

@@ -21,7 +21,7 @@ ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_FORMATBOOK, ERR_CUDA, ERR_NO_DEVICE =
 EXPORTS = [
     "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_seda",
     "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
-    "fb4_quantize_host", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
+    "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
 
 
@@ -77,6 +77,10 @@ def lib() -> ctypes.CDLL:
                  "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx",
                  "fb4_dequantize", "fb4_quantize_host", "fb4_last_cuda_error"):
         getattr(L, name).restype = ci
+    L.fb4_set_kernel_variant.argtypes = [vp, ci]
+    L.fb4_set_kernel_variant.restype = ci
+    L.fb4_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    L.fb4_device_status.restype = ci
     L.fb4_launch_count.argtypes = [vp]
     L.fb4_launch_count.restype = i64
     L.fb4_last_variant.argtypes = [vp]
@@ -180,6 +184,16 @@ def fb4_quantize_host(ctx, x_host, T, C, d_x, d_codes, d_meta, codes_host, meta_
                                    _ptr(codes_host), _ptr(meta_host)), "fb4_quantize_host")
 
 
+def fb4_set_kernel_variant(ctx, variant: int) -> None:
+    _check(lib().fb4_set_kernel_variant(ctx, variant), "fb4_set_kernel_variant")
+
+
+def fb4_device_status(ctx) -> int:
+    st = ctypes.c_uint32(0)
+    _check(lib().fb4_device_status(ctx, ctypes.byref(st)), "fb4_device_status")
+    return int(st.value)
+
+
 def fb4_launch_count(ctx) -> int:
     return int(lib().fb4_launch_count(ctx))
 
@@ -277,6 +291,13 @@ class Fb4:
                        q.res_codes if n else None, q.res_meta if n else None, out,
                        0 if dtype == torch.float32 else 1)
         return out
+
+    def set_kernel_variant(self, variant: int) -> None:
+        fb4_set_kernel_variant(self.ctx, variant)
+
+    @property
+    def device_status(self) -> int:
+        return fb4_device_status(self.ctx)
 
     @property
     def launch_count(self) -> int:

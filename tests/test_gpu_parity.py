@@ -12,10 +12,28 @@ from paper_2603_02883_b200 import fb4, synth
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module")
-def q32():
+@pytest.fixture(scope="module", params=["auto", "generic"])
+def q32(request):
+    """Default-configuration context; 'auto' takes the TMA-staged kernel whenever the call
+    qualifies, 'generic' forces the fallback kernel, so both are checked on every case."""
     q = fb4.Fb4()
+    q.set_kernel_variant(1 if request.param == "generic" else 0)
     yield q
+    assert q.device_status == 0
+    q.close()
+
+
+def test_kernel_choice():
+    q = fb4.Fb4()
+    x = torch.zeros((8, 1024), dtype=torch.bfloat16, device="cuda")
+    q.quantize(x)
+    assert q.last_variant == "fast"
+    q.quantize(x[:, :96])            # 96 channels: not a multiple of 64
+    assert q.last_variant == "generic"
+    q.set_kernel_variant(1)
+    q.quantize(x)
+    assert q.last_variant == "generic"
+    assert q.device_status == 0
     q.close()
 
 

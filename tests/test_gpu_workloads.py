@@ -19,6 +19,7 @@ MSE_RTOL = 1e-6
 def q32():
     q = fb4.Fb4()
     yield q
+    assert q.last_variant == "fast" and q.device_status == 0
     q.close()
 
 
