@@ -29,12 +29,14 @@ namespace {
 constexpr int kWarps = 16;           // warps per CTA
 constexpr int kStages = 4;           // ring depth per warp
 constexpr int kTileBytes = 2048;     // 1024 bf16
-constexpr int kPairStride = 1060;    // bytes between per-dialect pair tables (1024 + bank rotation)
+constexpr int kPairMul = 36;         // pair-table address = 36*bin_hi + bin_lo: spreads small bins over the banks
+constexpr int kPairStride = 1148;    // 36*31 + 32 bytes per dialect; 287 words: one bank of rotation per dialect
 constexpr int kMaxGroups = 8;        // distinct stage-1 groups the packed tables hold
 constexpr uint32_t kSpinLimit = 1u << 20;   // tries per wait before a warp gives up
 
+// Compact tables in global memory (built at init); the kernel expands them into shared memory.
 struct FastTables {
-  uint8_t pairlut[32 * kPairStride];     // [dialect][bin_hi*32 + bin_lo] -> idx_lo | idx_hi<<4
+  uint8_t qvalue[32][32];                // [dialect][bin] -> index of the nearest magnitude
   uint64_t qerr64[kMaxGroups][32];       // [group][bin] -> byte j = Qerror of candidate j (pad 31)
   uint8_t did_of[kMaxGroups][8];         // [group][candidate] -> dialect id
   uint8_t group_of_bin[32];              // [bin of block maximum] -> group
@@ -44,9 +46,20 @@ struct FastTables {
 };
 static_assert(sizeof(FastTables) % 16 == 0, "copied with 16-byte accesses");
 
+// Expanded tables in shared memory.
+struct SmemTables {
+  // [group][bin][lane & 15] -> the 8 candidate errors: each lane of a half-warp has its own
+  // 8-byte column, so the 64-bit loads of a warp never conflict
+  uint64_t qerr_private[kMaxGroups][32][16];
+  uint8_t pairlut[32 * kPairStride];     // [dialect][36*bin_hi + bin_lo] -> idx_lo | idx_hi<<4
+  FastTables c;
+};
+
 struct FastParams {
   int64_t T, C;
   int64_t tiles_per_row, n_tiles;
+  int64_t step_rows;    // gridDim.x*kWarps tiles ahead = step_rows rows + step_cols tile columns
+  int32_t step_cols;
   uint8_t* codes;
   uint16_t* meta;
   uint32_t* status;   // device word: bit 0 = a TMA wait ran out
@@ -105,13 +118,13 @@ __device__ __forceinline__ float pow2f(int k) {   // 2^k, k in [-149,127]
 
 // Score an arbitrary candidate mask over 8 group bins with the byte table (SeDA masks that
 // cut a stage-1 group, and the residual pass).  Ascending ids: ties keep the lowest.
-__device__ __forceinline__ int select_general(uint32_t cand, const uint8_t* gb, const FastTables* tb) {
+__device__ __forceinline__ int select_general(uint32_t cand, const uint8_t* gb, const SmemTables* tb) {
   int best = 0, best_err = 0x7fffffff;
   for (uint32_t m = cand; m; m &= m - 1) {
     const int d = __ffs((int)m) - 1;
     int err = 0;
 #pragma unroll
-    for (int g = 0; g < 8; ++g) err += tb->qerror[d][gb[g]];
+    for (int g = 0; g < 8; ++g) err += tb->c.qerror[d][gb[g]];
     if (err < best_err) { best_err = err; best = d; }
   }
   return best;
@@ -120,7 +133,7 @@ __device__ __forceinline__ int select_general(uint32_t cand, const uint8_t* gb, 
 // Residual pass of one block (Sec. 3.3): Delta = x - Q(x) in fp32 (exact), quantized again.
 // w = the 16 input registers (2 bf16 each), cw = the block's 4 code words.
 __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t* cw, int did, int e, uint32_t allowed,
-                                            const FastTables* tb, uint32_t* rcw, int* rdid, int* re) {
+                                               const SmemTables* tb, uint32_t* rcw, int* rdid, int* re) {
   const float sc = pow2f(e - 3);
   float ax[32];
   uint32_t sgn = 0;
@@ -130,7 +143,7 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
     const uint32_t word = w[i >> 1];
     const float x = __uint_as_float((i & 1) ? (word & 0xffff0000u) : (word << 16));
     const uint32_t nib = (cw[i >> 3] >> (4 * (i & 7))) & 15u;
-    const float mag = (float)tb->fb[did][nib & 7u] * sc;
+    const float mag = (float)tb->c.fb[did][nib & 7u] * sc;
     const float delta = __fsub_rn(x, (nib & 8u) ? -mag : mag);
     sgn |= (__float_as_uint(delta) >> 31) << i;
     ax[i] = fabsf(delta);
@@ -153,17 +166,16 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
     gb[g] = (uint8_t)m;
     bmax = max(bmax, m);
   }
-  uint32_t cand = tb->stage1[bmax] & allowed;
+  uint32_t cand = tb->c.stage1[bmax] & allowed;
   if (cand == 0) cand = allowed;
   const int d = select_general(cand, gb, tb);
-  const uint8_t* qv = tb->pairlut + d * kPairStride;   // entry [0*32 + bin] low nibble = Qvalue[d][bin]
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     uint32_t word = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int k = q * 8 + i;
-      word |= ((qv[bin[k]] & 7u) | (((sgn >> k) & 1u) << 3)) << (4 * i);
+      word |= ((uint32_t)tb->c.qvalue[d][bin[k]] | (((sgn >> k) & 1u) << 3)) << (4 * i);
     }
     rcw[q] = word;
   }
@@ -171,19 +183,31 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
   *re = er;
 }
 
+// Tile index -> (token row, tile column) without a division per tile: advance by a fixed step.
+struct TilePos {
+  int64_t row;
+  int32_t col;
+  __device__ __forceinline__ void advance(int64_t step_rows, int32_t step_cols, int32_t tiles_per_row) {
+    row += step_rows;
+    col += step_cols;
+    if (col >= tiles_per_row) { col -= tiles_per_row; ++row; }
+  }
+};
+
 template <bool SEDA, bool DECOMP>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTables* __restrict__ g_tables,
                          FastParams p, Fb4RowExtras ex) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  // [ring: kWarps*kStages*2048 B][tables][mbarriers]
-  uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);   // 128-byte swizzle needs 1 KB alignment
-  FastTables* tb = reinterpret_cast<FastTables*>(ring + kWarps * kStages * kTileBytes);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(FastTables));
+  // [ring: kWarps*kStages*2048 B, 1 KB aligned for the 128-byte swizzle][tables][mbarriers]
+  uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t gwarp = (int64_t)blockIdx.x * kWarps + warp;
   const int64_t wstride = (int64_t)gridDim.x * kWarps;
+  const int32_t tpr = (int32_t)p.tiles_per_row;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < kWarps * kStages; ++i) mbar_init(smem_u32(bars + i), 1);
@@ -193,29 +217,44 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
 
   const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytes);
   const uint32_t my_bars = smem_u32(bars + warp * kStages);
+  TilePos cur, pre;   // tile being quantized; next tile to request
+  cur.row = gwarp / tpr;
+  cur.col = (int32_t)(gwarp - cur.row * tpr);
+  pre = cur;
+  int64_t g_pre = gwarp;
   // prologue: fill the ring
   if (lane == 0) {
 #pragma unroll
     for (int s = 0; s < kStages; ++s) {
-      const int64_t g = gwarp + (int64_t)s * wstride;
-      if (g < p.n_tiles) {
-        const int64_t row = g / p.tiles_per_row;
-        const int col = (int)(g - row * p.tiles_per_row);
+      if (g_pre < p.n_tiles) {
         mbar_expect_tx(my_bars + 8 * s, kTileBytes);
-        tma_load_tile(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, col * 16, (int)row);
+        tma_load_tile(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, pre.col * 16, (int)pre.row);
       }
+      g_pre += wstride;
+      pre.advance(p.step_rows, p.step_cols, tpr);
     }
   }
-  // tables -> shared memory (overlaps the first loads)
+  // ---- expand the tables into shared memory (overlaps the first loads)
   {
     const uint4* src = reinterpret_cast<const uint4*>(g_tables);
-    uint4* dst = reinterpret_cast<uint4*>(tb);
+    uint4* dst = reinterpret_cast<uint4*>(&tb->c);
     for (int i = threadIdx.x; i < (int)(sizeof(FastTables) / 16); i += kWarps * 32) dst[i] = src[i];
+    // every (group, bin) entry replicated into 16 lane-private columns
+    const uint64_t* q64 = reinterpret_cast<const uint64_t*>(g_tables->qerr64);
+    uint64_t* qp = &tb->qerr_private[0][0][0];
+    for (int i = threadIdx.x; i < kMaxGroups * 32 * 16; i += kWarps * 32) qp[i] = q64[i >> 4];
+    // pair tables, one 32-bit word (4 consecutive bin_lo) at a time
+    for (int i = threadIdx.x; i < 32 * 32 * 8; i += kWarps * 32) {
+      const int d = i >> 8, bh = (i >> 3) & 31, bl4 = (i & 7) * 4;
+      const uint32_t lo4 = *reinterpret_cast<const uint32_t*>(&g_tables->qvalue[d][bl4]);
+      const uint32_t hi = g_tables->qvalue[d][bh];
+      *reinterpret_cast<uint32_t*>(&tb->pairlut[d * kPairStride + bh * kPairMul + bl4]) = lo4 | (hi * 0x10101010u);
+    }
   }
   __syncthreads();
 
   const uint32_t pair_base = smem_u32(tb->pairlut);
-  const uint32_t qerr_base = smem_u32(tb->qerr64);
+  const uint32_t qerr_base = smem_u32(tb->qerr_private) + ((uint32_t)lane & 15u) * 8u;
   // this lane's 64 bytes inside a stage: row r = lane/2 of 128 B, chunks (lane&1)*4 + j, swizzled by r&7
   const uint32_t r = (uint32_t)lane >> 1, c0 = ((uint32_t)lane & 1u) * 4u;
   uint32_t chunk_off[4];
@@ -223,10 +262,10 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
   for (int j = 0; j < 4; ++j) chunk_off[j] = r * 128u + (((c0 + j) ^ (r & 7u)) << 4);
 
   const int64_t nblk = p.C >> 5;
-  int64_t k = 0;
-  for (int64_t g = gwarp; g < p.n_tiles; g += wstride, ++k) {
-    const int s = (int)(k % kStages);
-    const uint32_t parity = (uint32_t)((k / kStages) & 1);
+  const int64_t code_row_bytes = p.C >> 1;
+  int s = 0;
+  uint32_t parity = 0;
+  for (int64_t g = gwarp; g < p.n_tiles; g += wstride) {
     const uint32_t bar = my_bars + 8 * s;
     uint32_t spins = 0;
     bool ready = mbar_try_wait(bar, parity);
@@ -235,18 +274,18 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
       // A load never arrived: raise the status bit, give the loads still in flight for this warp a
       // bounded chance to land (so none writes into shared memory after the CTA has gone), stop.
       if (lane == 0) atomicOr(p.status, 1u);
+      int sj = s;
+      uint32_t pj = parity;
       for (int j = 1; j < kStages; ++j) {
         if (g + (int64_t)j * wstride >= p.n_tiles) break;
-        const int sj = (int)((k + j) % kStages);
-        const uint32_t pj = (uint32_t)(((k + j) / kStages) & 1);
+        if (++sj == kStages) { sj = 0; pj ^= 1u; }
         uint32_t tries = 0;
         while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
       }
       break;
     }
-    const int64_t row = g / p.tiles_per_row;
-    const int col = (int)(g - row * p.tiles_per_row);
-    const int64_t blk = (int64_t)col * 32 + lane;
+    const int64_t row = cur.row;
+    const int64_t blk = (int64_t)cur.col * 32 + lane;
     const bool active = blk < nblk;
 
     uint32_t w[16];
@@ -274,8 +313,9 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
     const uint32_t Ec = max(amax16 >> 7, 3u);
     const float s2 = __uint_as_float((257u - Ec) << 23);   // 2^(3-e)
-    const float sG = s2 * 0x1p-21f;                        // bins land in the mantissa of 2.0 + ...
-    const float sH = s2 * 0x1p-25f;                        // ... and of 0.125 + ...
+    const float sG = s2 * 0x1p-21f;                        // bin in the mantissa of 2.0 + x
+    const float sH = s2 * 0x1p-25f;                        // bin in the mantissa of 0.125 + x
+    const float sL = s2 * 0x1p-5f;                         // bin in the mantissa of 2^17 + x
     const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax16 << 16), sG, 2.0f)) & 31u;
 
     uint32_t allowed = 0xffffffffu;
@@ -289,24 +329,24 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     // ---- dialect selection
     int did;
     {
-      const uint32_t grp = tb->group_of_bin[bmax];
+      const uint32_t grp = tb->c.group_of_bin[bmax];
       bool packed_path = true;
       uint32_t cand = 0;
       if (SEDA) {
-        const uint32_t st1 = tb->stage1[bmax];
+        const uint32_t st1 = tb->c.stage1[bmax];
         cand = st1 & allowed;
         if (cand == 0) cand = allowed;
         packed_path = (cand == st1);
       }
       if (!SEDA || packed_path) {
-        const uint32_t qb = qerr_base + grp * 256u;
+        const uint32_t qb = qerr_base + grp * 4096u;
         uint32_t lo = 0, hi = 0;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const uint32_t t0 = __float_as_uint(__fmaf_rz(__uint_as_float(g2[q] << 16), sG, 2.0f));
           const uint32_t t1 = __float_as_uint(__fmaf_rz(__uint_as_float(g2[q]), sG, 2.0f));
-          const uint2 e0 = lds_v2((t0 << 3) + qb);   // 0x40000000 << 3 vanishes mod 2^32
-          const uint2 e1 = lds_v2((t1 << 3) + qb);
+          const uint2 e0 = lds_v2((t0 << 7) + qb);   // 0x40000000 << 7 vanishes mod 2^32: 128 B per bin
+          const uint2 e1 = lds_v2((t1 << 7) + qb);
           lo += e0.x + e1.x;
           hi += e0.y + e1.y;
         }
@@ -317,7 +357,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
         const uint32_t k57 = ((hi >> 8) & 0x00ff00ffu) * 8u + 0x00070005u;
         const uint32_t km = __vminu2(__vminu2(k02, k13), __vminu2(k46, k57));
         const uint32_t key = min(km & 0xffffu, km >> 16);
-        did = tb->did_of[grp][key & 7u];
+        did = tb->c.did_of[grp][key & 7u];
       } else if (__popc(cand) == 1) {
         did = __ffs((int)cand) - 1;
       } else {
@@ -330,8 +370,9 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
         did = select_general(cand, gb, tb);
       }
     }
-    // ---- Qvalue: one lookup per element pair
-    const float magic_lo = __uint_as_float(0x40000000u + pair_base + (uint32_t)did * kPairStride);
+    // ---- Qvalue: one lookup per element pair.  124*36 + 144 = 9*512, so the exponent fields of
+    // 36*bits(0.125 + ..) + bits(2^17 + ..) cancel mod 2^32 and leave table + 36*bin_hi + bin_lo.
+    const float magic_lo = __uint_as_float(0x48000000u + pair_base + (uint32_t)did * kPairStride);
     uint32_t cw[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
@@ -339,9 +380,9 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const uint32_t av = a[4 * q + j];
-        const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sH, 0.125f));        // 0x3E000000 + bin_hi
-        const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sG, magic_lo));  // 0x40000000 + table + bin_lo
-        b[j] = lds_u8(th * 32u + tl);   // 0x3E000000*32 + 0x40000000 == 0 (mod 2^32)
+        const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sH, 0.125f));
+        const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sL, magic_lo));
+        b[j] = lds_u8(th * (uint32_t)kPairMul + tl);
       }
       const uint32_t idx = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
       // sign bits: byte masks by sign replication, then to bit 3 of every nibble
@@ -351,7 +392,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
       cw[q] = idx | (((ev & 0x0f0f0f0fu) | (od & 0xf0f0f0f0u)) & 0x88888888u);
     }
     if (active) {
-      *reinterpret_cast<uint4*>(p.codes + row * (p.C >> 1) + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
       p.meta[row * nblk + blk] = (uint16_t)((Ec - 3u) | ((uint32_t)did << 8));
     }
     if (DECOMP) {
@@ -373,7 +414,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
         int rdid, re;
         residual_block(w, cw, did, (int)Ec - 127, allowed, tb, rcw, &rdid, &re);
         if (active) {
-          *reinterpret_cast<uint4*>(ex.res_codes + srow * (p.C >> 1) + blk * 16) =
+          *reinterpret_cast<uint4*>(ex.res_codes + srow * code_row_bytes + blk * 16) =
               make_uint4(rcw[0], rcw[1], rcw[2], rcw[3]);
           ex.res_meta[srow * nblk + blk] = (uint16_t)((re + 124) | (rdid << 8));
         }
@@ -381,15 +422,14 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     }
     // ---- refill this stage (all lanes have consumed their registers from it)
     __syncwarp();
-    if (lane == 0) {
-      const int64_t gn = g + (int64_t)kStages * wstride;
-      if (gn < p.n_tiles) {
-        const int64_t rown = gn / p.tiles_per_row;
-        const int coln = (int)(gn - rown * p.tiles_per_row);
-        mbar_expect_tx(bar, kTileBytes);
-        tma_load_tile(my_ring + s * kTileBytes, &tmap, bar, coln * 16, (int)rown);
-      }
+    if (lane == 0 && g_pre < p.n_tiles) {
+      mbar_expect_tx(bar, kTileBytes);
+      tma_load_tile(my_ring + s * kTileBytes, &tmap, bar, pre.col * 16, (int)pre.row);
     }
+    g_pre += wstride;
+    pre.advance(p.step_rows, p.step_cols, tpr);
+    cur.advance(p.step_rows, p.step_cols, tpr);
+    if (++s == kStages) { s = 0; parity ^= 1u; }
   }
 }
 
@@ -411,7 +451,9 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-constexpr size_t kSmemBytes = 1024 + (size_t)kWarps * kStages * kTileBytes + sizeof(FastTables) + kWarps * kStages * 8;
+constexpr size_t kSmemBytes = 1024 + (size_t)kWarps * kStages * kTileBytes + sizeof(SmemTables) + kWarps * kStages * 8;
+static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
+static_assert(sizeof(SmemTables) % 16 == 0, "mbarriers behind the tables stay 8-byte aligned");
 
 template <bool SEDA, bool DECOMP>
 cudaError_t launch(const CUtensorMap& map, const FastTables* tables, const FastParams& p, const Fb4RowExtras& ex,
@@ -426,7 +468,7 @@ cudaError_t launch(const CUtensorMap& map, const FastTables* tables, const FastP
 // stage-1 table does not fit them (more than 8 groups, a group with 0 or more than 8 dialects, or
 // error sums that could overflow a byte): those contexts use the generic kernel.
 bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes) {
-  static FastTables ft;   // ~37 KB: keep it off the stack (fb4_init is not re-entrant per context anyway)
+  FastTables ft;
   std::memset(&ft, 0, sizeof ft);
   uint32_t groups[kMaxGroups];
   int ngroups = 0;
@@ -458,10 +500,7 @@ bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes
     for (; j < 8; ++j)
       for (int k = 0; k < 32; ++k) ft.qerr64[gi][k] |= (uint64_t)31 << (8 * j);   // never beats a real candidate
   }
-  for (int d = 0; d < 32; ++d)
-    for (int bh = 0; bh < 32; ++bh)
-      for (int bl = 0; bl < 32; ++bl)
-        ft.pairlut[d * kPairStride + bh * 32 + bl] = (uint8_t)(t.qvalue[d][bl] | (t.qvalue[d][bh] << 4));
+  std::memcpy(ft.qvalue, t.qvalue, sizeof ft.qvalue);
   std::memcpy(ft.qerror, t.qerror, sizeof ft.qerror);
   std::memcpy(ft.fb, t.formatbook, sizeof ft.fb);
   void* d = nullptr;
@@ -522,6 +561,9 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   p.status = ctx->d_status;
   const int64_t want = (p.n_tiles + kWarps - 1) / kWarps;
   const int grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
+  const int64_t wstride = (int64_t)grid * kWarps;
+  p.step_rows = wstride / p.tiles_per_row;
+  p.step_cols = (int32_t)(wstride % p.tiles_per_row);
   const FastTables* tables = static_cast<const FastTables*>(ctx->d_fast_tables);
   const bool seda = ex.cluster_id != nullptr, decomp = ex.n_salient > 0;
   if (seda && decomp) return launch<true, true>(map, tables, p, ex, grid, stream);
