@@ -82,7 +82,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            time.sleep(0.02)
+            time.sleep(0.001)   # the timed region can be a few milliseconds long
 
     def __enter__(self):
         if self.nv is not None:
@@ -165,6 +165,83 @@ def run_reference(args):
     }))
 
 
+class Ops:
+    """Every library path on one resident tensor: name -> (callable, algorithmic bytes per call).
+    Buffers are allocated on first use and kept (the decoded fp32 tensor alone is 3.7 GB)."""
+
+    def __init__(self, q, x, w, torch, fb4, synth):
+        self.q, self.x, self.w, self.torch, self.fb4, self.synth = q, x, w, torch, fb4, synth
+        self.T, self.C, self.B = w.T, w.C, 32
+        self._buf = {}
+
+    def buf(self, name, shape, dtype):
+        if name not in self._buf:
+            self._buf[name] = self.torch.empty(shape, dtype=dtype, device="cuda")
+        return self._buf[name]
+
+    def drop(self, name):
+        self._buf.pop(name, None)
+
+    def extras(self):
+        if "extras" not in self._buf:
+            w, torch, synth = self.w, self.torch, self.synth
+            big = synth.Workload(**{**w.__dict__, "decomposed": True, "score_seed": 4, "seda": True,
+                                    "n_clusters": 256 if w.T > 40000 else 64, "cluster_seed": 4})
+            cid_np, mask_np = synth.clusters(big)
+            self._buf["extras"] = dict(
+                tile=big.tile, n_sal=-(-w.T // big.tile), score=torch.from_numpy(synth.scores(big)).cuda(),
+                cid=torch.from_numpy(cid_np).cuda(), cmask=torch.from_numpy(mask_np.view(np.int32)).cuda())
+        return self._buf["extras"]
+
+    def get(self, name):
+        q, x, T, C, B, torch, fb4 = self.q, self.x, self.T, self.C, self.B, self.torch, self.fb4
+        codes = self.buf("codes", (T, C // 2), torch.uint8)
+        meta = self.buf("meta", (T, C // B), torch.int16)
+        if name == "plain":
+            return (lambda: fb4.fb4_quantize(q.ctx, x, T, C, C, codes, meta)), algorithmic_bytes(T, C)
+        ex = self.extras()
+        n_sal, tile, cid, cmask, score = ex["n_sal"], ex["tile"], ex["cid"], ex["cmask"], ex["score"]
+        rc = self.buf("rc", (n_sal, C // 2), torch.uint8)
+        rm = self.buf("rm", (n_sal, C // B), torch.int16)
+        sal = self.buf("sal", (n_sal,), torch.int32)
+        if name == "seda":
+            return (lambda: fb4.fb4_quantize_seda(q.ctx, x, T, C, C, cid, cmask, cmask.numel(), codes, meta)), \
+                algorithmic_bytes(T, C, seda=True)
+        if name == "decomposed":
+            return (lambda: fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, tile, None, None, 0, codes, meta,
+                                                        sal, rc, rm)), \
+                algorithmic_bytes(T, C, n_res_rows=n_sal, decomposed=True)
+        if name == "decomposed_seda":
+            return (lambda: fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, tile, cid, cmask, cmask.numel(),
+                                                        codes, meta, sal, rc, rm)), \
+                algorithmic_bytes(T, C, n_res_rows=n_sal, seda=True, decomposed=True)
+        # the decode ops read what a decomposed quantization left in codes/meta/sal/rc/rm
+        fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, tile, None, None, 0, codes, meta, sal, rc, rm)
+        plain_bytes = T * C * 0.5 + T * (C // B) * 2
+        res_bytes = n_sal * (C * 0.5 + (C // B) * 2) + 4 * n_sal
+        if name == "dequantize_f32_decomposed":
+            out = self.buf("out32", (T, C), torch.float32)
+            return (lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, sal, n_sal, rc, rm, out, 0)), \
+                plain_bytes + res_bytes + T * C * 4
+        if name == "dequantize_f32_plain":
+            out = self.buf("out32", (T, C), torch.float32)
+            return (lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, None, 0, None, None, out, 0)), \
+                plain_bytes + T * C * 4
+        if name == "dequantize_bf16_plain":
+            out = self.buf("out16", (T, C), torch.bfloat16)
+            return (lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, None, 0, None, None, out, 1)), \
+                plain_bytes + T * C * 2
+        if name == "dequantize_bf16_decomposed":
+            out = self.buf("out16", (T, C), torch.bfloat16)
+            return (lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, sal, n_sal, rc, rm, out, 1)), \
+                plain_bytes + res_bytes + T * C * 2
+        raise KeyError(name)
+
+
+OP_NAMES = ["plain", "seda", "decomposed", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
+            "dequantize_bf16_plain", "dequantize_bf16_decomposed"]
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -172,7 +249,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5_plain", help="c5_plain (default) or c2 (smaller tensor, for profiling)")
-    ap.add_argument("--no-variants", action="store_true", help="time only the headline step")
+    ap.add_argument("--op", default="plain", choices=OP_NAMES,
+                    help="library path timed as the step (default: plain fb4_quantize, the headline metric)")
+    ap.add_argument("--no-variants", action="store_true", help="time only the step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -204,39 +283,37 @@ def main():
     x = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
     q = fb4.Fb4(device=local_rank)
     T, C, B = w.T, w.C, 32
-    codes = torch.empty((T, C // 2), dtype=torch.uint8, device="cuda")
-    meta = torch.empty((T, C // B), dtype=torch.int16, device="cuda")
+    ops = Ops(q, x, w, torch, fb4, synth)
+    step, alg = ops.get(args.op)
 
-    def step():
-        fb4.fb4_quantize(q.ctx, x, T, C, C, codes, meta)
-
-    l0 = q.launch_count
     for _ in range(args.warmup):
         step()
-    launches_warm = q.launch_count - l0
+    torch.cuda.synchronize()
+    l0 = q.launch_count
     with ClockSampler(visible_index(local_rank)) as clk:
         total_ms, per = time_steps(step, args.steps, 0, torch, barrier)
-    launches = (q.launch_count - l0 - launches_warm)
+    launches = q.launch_count - l0
     variant = q.last_variant
     t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     total_ms = float(t.item())
     ms = total_ms / args.steps
-    alg = algorithmic_bytes(T, C)
     value = world * alg / (ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
     kernel_ms = float(np.mean(per))
     achieved = alg / (kernel_ms * 1e-3) / 1e9
+    tensor_name = "config-5" if args.workload == "c5_plain" else args.workload
+    op_text = "plain FB4 quantize" if args.op == "plain" else f"FB4 {args.op}"
 
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "metric": METRIC if args.op == "plain" else f"fb4_{args.op}_throughput",
+        "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "gelem_per_s": world * T * C / (ms * 1e-3) / 1e9,
         "frac_hbm_measured": value / world / peak, "frac_hbm_nominal_8000": value / world / 8000.0,
-        "config": {"workload": f"plain FB4 quantize, {T}x{C} bf16 "
-                               f"({'config-5' if args.workload == 'c5_plain' else args.workload} tensor), block 32, "
+        "config": {"workload": f"{op_text}, {T}x{C} bf16 ({tensor_name} tensor), block 32, "
                                "full formatbook, two-stage selection",
                    "per_gpu_tokens": T, "channels": C, "block_size": B, "kernel_variant": variant,
                    "l2": "input 1.86 GB per step, larger than L2; no flush needed" if T * C * 2 > 2.5e8
@@ -244,20 +321,22 @@ def main():
         "gpu_launches": launches,
         "clocks": clk.summary(),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_TRAFFIC_BYTES, "peak_kind": f"{peak_kind} copy bandwidth",
-                     "kernel": f"fb4 quantize ({variant})", "algorithmic_bytes_per_launch": alg,
+                     "traffic": NCU_TRAFFIC_BYTES if (args.op == "plain" and args.workload == "c5_plain") else None,
+                     "peak_kind": f"{peak_kind} copy bandwidth",
+                     "kernel": f"fb4 {args.op} ({variant})", "algorithmic_bytes_per_launch": alg,
                      "launch_ms_mean": kernel_ms, "launch_ms_min": float(np.min(per))},
     }
 
     if rank == 0 and not args.no_variants:
-        out["variants"] = run_variants(q, x, w, args, torch, fb4, synth, peak)
+        out["variants"] = run_variants(ops, args, torch, fb4, synth, peak)
+    del ops
     if not args.no_e2e:
         e2e = run_e2e(q, bits, w, args, torch, fb4, barrier)
         if world > 1:
             t = torch.tensor([e2e["seconds_per_step"]], dtype=torch.float64, device="cuda")
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
             e2e["seconds_per_step"] = float(t.item())
-        e2e["value"] = world * alg / e2e["seconds_per_step"] / 1e9
+        e2e["value"] = world * algorithmic_bytes(T, C) / e2e["seconds_per_step"] / 1e9
         out["e2e"] = e2e
     if rank == 0 and not args.no_cpu_baseline:
         out["cpu_baseline"] = run_cpu_baseline(w, synth)
@@ -268,46 +347,22 @@ def main():
         dist.destroy_process_group()
 
 
-def run_variants(q, x, w, args, torch, fb4, synth, peak):
+def run_variants(ops, args, torch, fb4, synth, peak):
     """The other library paths on the same device, each timed like the headline step."""
-    T, C, B = w.T, w.C, 32
+    q, w, B = ops.q, ops.w, 32
     res = {}
     steps, warm = max(3, args.steps // 2), 3
-    big = synth.Workload(**{**w.__dict__, "decomposed": True, "score_seed": 4, "seda": True, "n_clusters": 256,
-                            "cluster_seed": 4})
-    score = torch.from_numpy(synth.scores(big)).cuda()
-    cid_np, mask_np = synth.clusters(big)
-    cid = torch.from_numpy(cid_np).cuda()
-    cmask = torch.from_numpy(mask_np.view(np.int32)).cuda()
-    n_sal = -(-T // big.tile)
-    codes = torch.empty((T, C // 2), dtype=torch.uint8, device="cuda")
-    meta = torch.empty((T, C // B), dtype=torch.int16, device="cuda")
-    rc = torch.empty((n_sal, C // 2), dtype=torch.uint8, device="cuda")
-    rm = torch.empty((n_sal, C // B), dtype=torch.int16, device="cuda")
-    sal = torch.empty(n_sal, dtype=torch.int32, device="cuda")
-
-    def rec(name, fn, alg):
+    for name in OP_NAMES:
+        if name == args.op:
+            continue
+        fn, alg = ops.get(name)
         total, per = time_steps(fn, steps, warm, torch)
         ms = total / steps
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
-                     "kernel_variant": q.last_variant}
-
-    rec("seda", lambda: fb4.fb4_quantize_seda(q.ctx, x, T, C, C, cid, cmask, cmask.numel(), codes, meta),
-        algorithmic_bytes(T, C, seda=True))
-    rec("decomposed", lambda: fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, big.tile, None, None, 0, codes,
-                                                          meta, sal, rc, rm),
-        algorithmic_bytes(T, C, n_res_rows=n_sal, decomposed=True))
-    rec("decomposed_seda", lambda: fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, big.tile, cid, cmask,
-                                                               cmask.numel(), codes, meta, sal, rc, rm),
-        algorithmic_bytes(T, C, n_res_rows=n_sal, seda=True, decomposed=True))
-    out32 = torch.empty((T, C), dtype=torch.float32, device="cuda")
-    rec("dequantize_f32", lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, sal, n_sal, rc, rm, out32, 0),
-        T * C * (0.5 + 4) + T * (C // B) * 2 + n_sal * (C * 0.5 + (C // B) * 2))
-    del out32
-    out16 = torch.empty((T, C), dtype=torch.bfloat16, device="cuda")
-    rec("dequantize_bf16", lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, None, 0, None, None, out16, 1),
-        T * C * (0.5 + 2) + T * (C // B) * 2)
-    del out16
+                     "kernel_variant": q.last_variant if not name.startswith("dequantize") else "decode"}
+        if name == "dequantize_f32_decomposed":
+            ops.drop("out32")
+    ops.drop("out16")
     if w.name != "c2":
         w2 = synth.workloads()["c2"]
         x2 = torch.from_numpy(synth.activation(w2).view(np.int16)).cuda().view(torch.bfloat16)

@@ -60,7 +60,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     with ThreadPoolExecutor(max_workers=min(8, len(sources()))) as ex:
         objs = list(ex.map(compile_one, sources()))
     tmp = LIB + f".{os.getpid()}.tmp"
-    subprocess.check_call([nvcc, "-shared", "-o", tmp, *objs, "-cudart", "static"])
+    subprocess.check_call([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp, *objs,
+                           "-cudart", "static"])
     os.replace(tmp, LIB)
     return LIB
 

@@ -117,7 +117,7 @@ __device__ __forceinline__ float pow2f(int k) {   // 2^k, k in [-149,127]
 }
 
 // Score an arbitrary candidate mask over 8 group bins with the byte table (SeDA masks that
-// cut a stage-1 group, and the residual pass).  Ascending ids: ties keep the lowest.
+// cut a stage-1 group).  Ascending ids: ties keep the lowest.
 __device__ __forceinline__ int select_general(uint32_t cand, const uint8_t* gb, const SmemTables* tb) {
   int best = 0, best_err = 0x7fffffff;
   for (uint32_t m = cand; m; m &= m - 1) {
@@ -130,57 +130,105 @@ __device__ __forceinline__ int select_general(uint32_t cand, const uint8_t* gb, 
   return best;
 }
 
-// Residual pass of one block (Sec. 3.3): Delta = x - Q(x) in fp32 (exact), quantized again.
-// w = the 16 input registers (2 bf16 each), cw = the block's 4 code words.
-__device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t* cw, int did, int e, uint32_t allowed,
-                                               const SmemTables* tb, uint32_t* rcw, int* rdid, int* re) {
-  const float sc = pow2f(e - 3);
-  float ax[32];
-  uint32_t sgn = 0;
-  float amax = 0.f;
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    const uint32_t word = w[i >> 1];
-    const float x = __uint_as_float((i & 1) ? (word & 0xffff0000u) : (word << 16));
-    const uint32_t nib = (cw[i >> 3] >> (4 * (i & 7))) & 15u;
-    const float mag = (float)tb->c.fb[did][nib & 7u] * sc;
-    const float delta = __fsub_rn(x, (nib & 8u) ? -mag : mag);
-    sgn |= (__float_as_uint(delta) >> 31) << i;
-    ax[i] = fabsf(delta);
-    amax = fmaxf(amax, ax[i]);
+// Dialect selection of one block (Sec. 3.2 two-stage; Sec. 3.4 restriction).  gm = the 8 group
+// maxima as fp32 magnitudes (mantissa bits below the bin resolution are truncated away),
+// sG = 2^(3-e) * 2^-21, bmax = bin of the block maximum, qerr_lane = this lane's column of the
+// packed error table.
+template <bool SEDA>
+__device__ __forceinline__ int choose_dialect(const float (&gm)[8], float sG, uint32_t bmax, uint32_t allowed,
+                                              const SmemTables* tb, uint32_t qerr_lane) {
+  const uint32_t grp = tb->c.group_of_bin[bmax];
+  bool packed_path = true;
+  uint32_t cand = 0;
+  if (SEDA) {
+    const uint32_t st1 = tb->c.stage1[bmax];
+    cand = st1 & allowed;
+    if (cand == 0) cand = allowed;
+    packed_path = (cand == st1);
   }
-  int er = amax == 0.f ? -124 : (int)((__float_as_uint(amax) >> 23) & 0xff) - 127;
-  er = max(er, -124);
-  const float s = pow2f(3 - er);
-  uint8_t bin[32], gb[8];
-  int bmax = 0;
+  if (!SEDA || packed_path) {
+    const uint32_t qb = qerr_lane + grp * 4096u;
+    uint32_t lo = 0, hi = 0;
 #pragma unroll
-  for (int g = 0; g < 8; ++g) {
-    int m = 0;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int b = min(31, __float2int_rd(2.0f * (ax[g * 4 + i] * s)));
-      bin[g * 4 + i] = (uint8_t)b;
-      m = max(m, b);
+    for (int g = 0; g < 8; ++g) {
+      const uint32_t t = __float_as_uint(__fmaf_rz(gm[g], sG, 2.0f));
+      const uint2 e = lds_v2((t << 7) + qb);   // 0x40000000 << 7 vanishes mod 2^32: 128 B per bin
+      lo += e.x;
+      hi += e.y;
     }
-    gb[g] = (uint8_t)m;
-    bmax = max(bmax, m);
+    // argmin over 8 byte sums, ties to the lowest candidate: keys (err << 3 | j) in 16-bit lanes
+    const uint32_t k02 = (lo & 0x00ff00ffu) * 8u + 0x00020000u;
+    const uint32_t k13 = ((lo >> 8) & 0x00ff00ffu) * 8u + 0x00030001u;
+    const uint32_t k46 = (hi & 0x00ff00ffu) * 8u + 0x00060004u;
+    const uint32_t k57 = ((hi >> 8) & 0x00ff00ffu) * 8u + 0x00070005u;
+    const uint32_t km = __vminu2(__vminu2(k02, k13), __vminu2(k46, k57));
+    const uint32_t key = min(km & 0xffffu, km >> 16);
+    return tb->c.did_of[grp][key & 7u];
   }
-  uint32_t cand = tb->c.stage1[bmax] & allowed;
-  if (cand == 0) cand = allowed;
-  const int d = select_general(cand, gb, tb);
+  if (__popc(cand) == 1) return __ffs((int)cand) - 1;
+  uint8_t gb[8];
+#pragma unroll
+  for (int g = 0; g < 8; ++g) gb[g] = (uint8_t)(__float_as_uint(__fmaf_rz(gm[g], sG, 2.0f)) & 31u);
+  return select_general(cand, gb, tb);
+}
+
+// Residual pass of one block (Sec. 3.3): Delta = x - Q(x) in fp32 (exact), quantized again with
+// the same tables as the main pass; the fp32 magnitudes take the place of the bf16 ones.
+// w = the 16 input registers (2 bf16 each), cw = the block's 4 code words, Ec = biased exponent.
+template <bool SEDA>
+__device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t* cw, int did, uint32_t Ec,
+                                               uint32_t allowed, const SmemTables* tb, uint32_t qerr_lane,
+                                               uint32_t pair_base, uint32_t* rcw, uint32_t* rmeta) {
+  const float sc = pow2f((int)Ec - 130);   // element scale 2^(e-3)
+  const uint2 fbd = *reinterpret_cast<const uint2*>(tb->c.fb[did]);
+  uint32_t a[32];      // |Delta| bit patterns
+  uint32_t sg[4];      // sign bits at bit 3 of every nibble
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    uint32_t word = 0;
+    uint32_t sq = 0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int k = q * 8 + i;
-      word |= ((uint32_t)tb->c.qvalue[d][bin[k]] | (((sgn >> k) & 1u) << 3)) << (4 * i);
+      const uint32_t word = w[k >> 1];
+      const uint32_t xb = (k & 1) ? (word & 0xffff0000u) : (word << 16);
+      const uint32_t nib = cw[q] >> (4 * i);
+      const float mag = (float)(__byte_perm(fbd.x, fbd.y, nib & 7u) & 0xffu) * sc;
+      // Q(x) carries the sign of x
+      const float xhat = __uint_as_float(__float_as_uint(mag) | (xb & 0x80000000u));
+      const uint32_t db = __float_as_uint(__fsub_rn(__uint_as_float(xb), xhat));
+      a[k] = db & 0x7fffffffu;
+      sq |= (db >> 31) << (4 * i + 3);
     }
-    rcw[q] = word;
+    sg[q] = sq;
   }
-  *rdid = d;
-  *re = er;
+  uint32_t gmx[8];
+  uint32_t amax = 0;
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    gmx[g] = max(max(a[4 * g], a[4 * g + 1]), max(a[4 * g + 2], a[4 * g + 3]));
+    amax = max(amax, gmx[g]);
+  }
+  const uint32_t Er = max(amax >> 23, 3u);
+  const float s2 = __uint_as_float((257u - Er) << 23);   // 2^(3-e)
+  const float sG = s2 * 0x1p-21f, sH = s2 * 0x1p-25f, sL = s2 * 0x1p-5f;
+  const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax), sG, 2.0f)) & 31u;
+  float gm[8];
+#pragma unroll
+  for (int g = 0; g < 8; ++g) gm[g] = __uint_as_float(gmx[g]);
+  const int rdid = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
+  const float magic_lo = __uint_as_float(0x48000000u + pair_base + (uint32_t)rdid * kPairStride);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint32_t idx = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j + 1]), sH, 0.125f));
+      const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j]), sL, magic_lo));
+      idx |= lds_u8(th * (uint32_t)kPairMul + tl) << (8 * j);
+    }
+    rcw[q] = idx | sg[q];
+  }
+  *rmeta = (Er - 3u) | ((uint32_t)rdid << 8);
 }
 
 // Tile index -> (token row, tile column) without a division per tile: advance by a fixed step.
@@ -263,9 +311,51 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
 
   const int64_t nblk = p.C >> 5;
   const int64_t code_row_bytes = p.C >> 1;
+  const bool use_seda = SEDA && ex.cluster_id != nullptr;
+  const bool use_tile = DECOMP && ex.tile > 0;
+
+  // Per-token extras (cluster mask, salient slot) are fetched ahead of use so that their latency
+  // hides behind the tile being quantized: the cluster id two tiles ahead, the mask and the
+  // salient candidate one tile ahead.
+  TilePos n1 = cur, n2;
+  n1.advance(p.step_rows, p.step_cols, tpr);
+  n2 = n1;
+  n2.advance(p.step_rows, p.step_cols, tpr);
+  int32_t cid_n1 = -1;
+  uint32_t allowed_cur = 0xffffffffu;
+  if (use_seda) {
+    if (gwarp < p.n_tiles) {
+      const int32_t cid = ex.cluster_id[cur.row];
+      if (cid >= 0) allowed_cur = ex.cluster_mask[cid];
+    }
+    if (gwarp + wstride < p.n_tiles) cid_n1 = ex.cluster_id[n1.row];
+  }
+  int32_t sal_cur = -1;   // token id stored in the salient slot of the current row's tile
+  if (use_tile && gwarp < p.n_tiles) {
+    const uint32_t sidx = (uint32_t)cur.row / (uint32_t)ex.tile;
+    if ((int64_t)sidx < ex.n_salient) sal_cur = ex.salient_idx[sidx];
+  }
+
   int s = 0;
   uint32_t parity = 0;
   for (int64_t g = gwarp; g < p.n_tiles; g += wstride) {
+    // ---- prefetch the extras of the following tiles
+    uint32_t allowed_n1 = 0xffffffffu;
+    int32_t cid_n2 = -1;
+    int32_t sal_n1 = -1;
+    if (SEDA) {
+      if (use_seda) {
+        if (cid_n1 >= 0) allowed_n1 = ex.cluster_mask[cid_n1];
+        if (g + 2 * wstride < p.n_tiles) cid_n2 = ex.cluster_id[n2.row];
+      }
+    }
+    if (DECOMP) {
+      if (use_tile && g + wstride < p.n_tiles) {
+        const uint32_t sidx = (uint32_t)n1.row / (uint32_t)ex.tile;
+        if ((int64_t)sidx < ex.n_salient) sal_n1 = ex.salient_idx[sidx];
+      }
+    }
+
     const uint32_t bar = my_bars + 8 * s;
     uint32_t spins = 0;
     bool ready = mbar_try_wait(bar, parity);
@@ -320,56 +410,18 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
 
     uint32_t allowed = 0xffffffffu;
     if (SEDA) {
-      if (ex.cluster_id) {
-        const int32_t cid = ex.cluster_id[row];
-        if (cid >= 0) allowed = ex.cluster_mask[cid];
-        if (allowed == 0) allowed = 1u;
-      }
+      allowed = allowed_cur;
+      if (allowed == 0) allowed = 1u;   // precondition violated: stay in bounds
     }
-    // ---- dialect selection
-    int did;
-    {
-      const uint32_t grp = tb->c.group_of_bin[bmax];
-      bool packed_path = true;
-      uint32_t cand = 0;
-      if (SEDA) {
-        const uint32_t st1 = tb->c.stage1[bmax];
-        cand = st1 & allowed;
-        if (cand == 0) cand = allowed;
-        packed_path = (cand == st1);
-      }
-      if (!SEDA || packed_path) {
-        const uint32_t qb = qerr_base + grp * 4096u;
-        uint32_t lo = 0, hi = 0;
+    // ---- dialect selection; the upper bf16 of a pair keeps the lower one as extra mantissa bits,
+    // which truncation discards
+    float gm[8];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint32_t t0 = __float_as_uint(__fmaf_rz(__uint_as_float(g2[q] << 16), sG, 2.0f));
-          const uint32_t t1 = __float_as_uint(__fmaf_rz(__uint_as_float(g2[q]), sG, 2.0f));
-          const uint2 e0 = lds_v2((t0 << 7) + qb);   // 0x40000000 << 7 vanishes mod 2^32: 128 B per bin
-          const uint2 e1 = lds_v2((t1 << 7) + qb);
-          lo += e0.x + e1.x;
-          hi += e0.y + e1.y;
-        }
-        // argmin over 8 byte sums, ties to the lowest candidate: keys (err << 3 | j) in 16-bit lanes
-        const uint32_t k02 = (lo & 0x00ff00ffu) * 8u + 0x00020000u;
-        const uint32_t k13 = ((lo >> 8) & 0x00ff00ffu) * 8u + 0x00030001u;
-        const uint32_t k46 = (hi & 0x00ff00ffu) * 8u + 0x00060004u;
-        const uint32_t k57 = ((hi >> 8) & 0x00ff00ffu) * 8u + 0x00070005u;
-        const uint32_t km = __vminu2(__vminu2(k02, k13), __vminu2(k46, k57));
-        const uint32_t key = min(km & 0xffffu, km >> 16);
-        did = tb->c.did_of[grp][key & 7u];
-      } else if (__popc(cand) == 1) {
-        did = __ffs((int)cand) - 1;
-      } else {
-        uint8_t gb[8];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          gb[2 * q] = (uint8_t)(__float_as_uint(__fmaf_rz(__uint_as_float(g2[q] << 16), sG, 2.0f)) & 31u);
-          gb[2 * q + 1] = (uint8_t)(__float_as_uint(__fmaf_rz(__uint_as_float(g2[q]), sG, 2.0f)) & 31u);
-        }
-        did = select_general(cand, gb, tb);
-      }
+    for (int q = 0; q < 4; ++q) {
+      gm[2 * q] = __uint_as_float(g2[q] << 16);
+      gm[2 * q + 1] = __uint_as_float(g2[q]);
     }
+    const int did = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_base);
     // ---- Qvalue: one lookup per element pair.  124*36 + 144 = 9*512, so the exponent fields of
     // 36*bits(0.125 + ..) + bits(2^17 + ..) cancel mod 2^32 and leave table + 36*bin_hi + bin_lo.
     const float magic_lo = __uint_as_float(0x48000000u + pair_base + (uint32_t)did * kPairStride);
@@ -397,9 +449,8 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     }
     if (DECOMP) {
       int64_t srow = -1;
-      if (ex.tile > 0) {
-        const int64_t sidx = row / ex.tile;
-        if (sidx < ex.n_salient && ex.salient_idx[sidx] == (int32_t)row) srow = sidx;
+      if (use_tile) {
+        if (sal_cur == (int32_t)row) srow = (int64_t)((uint32_t)row / (uint32_t)ex.tile);
       } else {
         int64_t lo = 0, hi = ex.n_salient - 1;
         while (lo <= hi) {
@@ -410,13 +461,12 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
         }
       }
       if (srow >= 0) {   // warp-uniform: a tile lies inside one token
-        uint32_t rcw[4];
-        int rdid, re;
-        residual_block(w, cw, did, (int)Ec - 127, allowed, tb, rcw, &rdid, &re);
+        uint32_t rcw[4], rmeta;
+        residual_block<SEDA>(w, cw, did, Ec, allowed, tb, qerr_base, pair_base, rcw, &rmeta);
         if (active) {
           *reinterpret_cast<uint4*>(ex.res_codes + srow * code_row_bytes + blk * 16) =
               make_uint4(rcw[0], rcw[1], rcw[2], rcw[3]);
-          ex.res_meta[srow * nblk + blk] = (uint16_t)((re + 124) | (rdid << 8));
+          ex.res_meta[srow * nblk + blk] = (uint16_t)rmeta;
         }
       }
     }
@@ -429,6 +479,11 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     g_pre += wstride;
     pre.advance(p.step_rows, p.step_cols, tpr);
     cur.advance(p.step_rows, p.step_cols, tpr);
+    n1.advance(p.step_rows, p.step_cols, tpr);
+    n2.advance(p.step_rows, p.step_cols, tpr);
+    allowed_cur = allowed_n1;
+    cid_n1 = cid_n2;
+    sal_cur = sal_n1;
     if (++s == kStages) { s = 0; parity ^= 1u; }
   }
 }
