@@ -297,10 +297,11 @@ int fb4_dequantize(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int
   if (n_salient > 0 && (!salient_idx || !res_codes || !res_meta)) return FB4_ERR_INVALID_ARG;
   if (!aligned16(codes) || !aligned16(meta) || !aligned16(out)) return FB4_ERR_ALIGN;
   if (n_salient > 0 && (!aligned16(res_codes) || !aligned16(res_meta))) return FB4_ERR_ALIGN;
+  int launches = 0;
   cudaError_t e = fb4_launch_dequantize(ctx, codes, meta, T, C, salient_idx, n_salient, res_codes, res_meta, out,
-                                        out_dtype, static_cast<cudaStream_t>(stream));
+                                        out_dtype, static_cast<cudaStream_t>(stream), &launches);
+  ctx->launches += launches;
   if (e != cudaSuccess) return fb4_set_cuda_error(e);
-  ctx->launches += 1;
   return FB4_OK;
 }
 

@@ -1,8 +1,12 @@
 // FB4 decode (4-bit codes + block metadata -> fp32 / bf16, optionally adding the decoded
 // residual of salient tokens) and the per-tile salient-token selection.
+#include "fb4_device.cuh"
 #include "fb4_internal.h"
 
 namespace {
+
+using fb4dev::decode_word;
+using fb4dev::scale_bf16x2;
 
 __device__ __forceinline__ uint32_t f32_to_bf16_rne(float f) {
   const uint32_t u = __float_as_uint(f);
@@ -11,18 +15,6 @@ __device__ __forceinline__ uint32_t f32_to_bf16_rne(float f) {
 
 constexpr int kDecodeThreads = 256;
 constexpr int kDecodeUnroll = 2;          // blocks in flight per thread
-
-__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-// prmt.b32 in its default mode (selector bit 3 of a nibble replicates the sign of the chosen byte)
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-  uint32_t d;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-  return d;
-}
 
 // 32 bytes per store: a lane writes whole 32-byte sectors.  p must be 32-byte aligned when wide.
 __device__ __forceinline__ void store_b32x8(void* p, const uint32_t* v, bool wide) {
@@ -33,32 +25,6 @@ __device__ __forceinline__ void store_b32x8(void* p, const uint32_t* v, bool wid
     reinterpret_cast<uint4*>(p)[0] = make_uint4(v[0], v[1], v[2], v[3]);
     reinterpret_cast<uint4*>(p)[1] = make_uint4(v[4], v[5], v[6], v[7]);
   }
-}
-
-// One code word (8 elements) -> 4 registers of two bf16 values each.
-// dt = the dialect's magnitudes as bf16 bit patterns, split into a table of high bytes (x,y) and
-// a table of low bytes (z,w): a byte permute with the four 3-bit indices as selector looks up
-// four magnitudes at once, no memory access per element.  One packed multiply applies the scale
-// sc2 (the block scale as two bf16).  Exact: a magnitude 0..15 times a power of two >= 2^-127 is
-// a bf16 value (subnormals included).
-__device__ __forceinline__ void decode_word(uint32_t cw, const uint4& dt, uint32_t sc2, uint32_t* pr) {
-  const uint32_t sel = cw & 0x77777777u;
-  const uint32_t hi_a = prmt(dt.x, dt.y, sel), lo_a = prmt(dt.z, dt.w, sel);              // elements 0..3
-  const uint32_t hi_b = prmt(dt.x, dt.y, sel >> 16), lo_b = prmt(dt.z, dt.w, sel >> 16);  // elements 4..7
-  // byte masks of the sign bits: bit 7 of a code byte is the sign of its odd element
-  const uint32_t s_odd = prmt(cw, 0u, 0xba98u), s_even = prmt(cw << 4, 0u, 0xba98u);
-  const uint32_t mag[4] = {__byte_perm(lo_a, hi_a, 0x5140), __byte_perm(lo_a, hi_a, 0x7362),
-                           __byte_perm(lo_b, hi_b, 0x5140), __byte_perm(lo_b, hi_b, 0x7362)};
-  const uint32_t sgn[4] = {__byte_perm(s_even, s_odd, 0x4000), __byte_perm(s_even, s_odd, 0x5010),
-                           __byte_perm(s_even, s_odd, 0x6020), __byte_perm(s_even, s_odd, 0x7030)};
-#pragma unroll
-  for (int j = 0; j < 4; ++j) pr[j] = mul_bf16x2(mag[j], sc2) | (sgn[j] & 0x80008000u);
-}
-
-// block scale 2^(sb-127) as two bf16: sb << 7, or the subnormal 2^-127 = 0x0040 for sb = 0
-__device__ __forceinline__ uint32_t scale_bf16x2(uint32_t m) {
-  const uint32_t sb = m & 0xffu;
-  return (sb ? (sb << 7) : 0x40u) * 0x10001u;
 }
 
 template <int WPB>
@@ -115,12 +81,7 @@ __global__ void __launch_bounds__(kDecodeThreads)
 fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restrict__ meta, int64_t total_blocks,
                           const Fb4DeviceTables* __restrict__ tables, void* __restrict__ out, int out_aligned32) {
   __shared__ uint4 fb_bf16[32];   // per dialect: high bytes (8) then low bytes (8) of its magnitudes as bf16
-  {
-    const uint32_t bits = __float_as_uint((float)tables->formatbook[threadIdx.x >> 3][threadIdx.x & 7]) >> 16;
-    uint8_t* row = reinterpret_cast<uint8_t*>(&fb_bf16[threadIdx.x >> 3]);
-    row[threadIdx.x & 7] = (uint8_t)(bits >> 8);
-    row[8 + (threadIdx.x & 7)] = (uint8_t)bits;
-  }
+  fb4dev::fill_fb_bf16(fb_bf16, &tables->formatbook[0][0], threadIdx.x);
   __syncthreads();
   const bool wide = out_aligned32 != 0;
   const int lane = threadIdx.x & 31;
@@ -170,27 +131,18 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
   }
 }
 
-// Flat decode, general form: thread <-> one block (WPB code words of 8 elements, one metadata
-// record); block size 16, and rows that add their decoded residual.  A thread keeps kDecodeUnroll
-// blocks in flight, a CTA covers kDecodeThreads * kDecodeUnroll consecutive blocks per step, the
-// grid strides.  codes and out are contiguous [T][C].
-// RESID: rows listed in salient_idx (ascending) add their decoded residual (binary search per block).
-template <int OUT_BF16, bool RESID, int WPB>
+// Flat decode, general form (block size 16): thread <-> one block (WPB code words of 8 elements,
+// one metadata record).  A thread keeps kDecodeUnroll blocks in flight, a CTA covers
+// kDecodeThreads * kDecodeUnroll consecutive blocks per step, the grid strides.
+template <int OUT_BF16, int WPB>
 __global__ void __launch_bounds__(kDecodeThreads)
 fb4_dequantize_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restrict__ meta, int64_t total_blocks,
-                      uint32_t blocks_per_row, const Fb4DeviceTables* __restrict__ tables,
-                      const int32_t* __restrict__ salient_idx, int32_t n_salient,
-                      const uint32_t* __restrict__ res_codes, const uint16_t* __restrict__ res_meta,
-                      void* __restrict__ out, int out_aligned32) {
+                      const Fb4DeviceTables* __restrict__ tables, void* __restrict__ out, int out_aligned32) {
   __shared__ uint4 fb_bf16[32];   // per dialect: high bytes (8) then low bytes (8) of its magnitudes as bf16
-  if (threadIdx.x < 256) {
-    const uint32_t bits = __float_as_uint((float)tables->formatbook[threadIdx.x >> 3][threadIdx.x & 7]) >> 16;
-    uint8_t* row = reinterpret_cast<uint8_t*>(&fb_bf16[threadIdx.x >> 3]);
-    row[threadIdx.x & 7] = (uint8_t)(bits >> 8);
-    row[8 + (threadIdx.x & 7)] = (uint8_t)bits;
-  }
+  fb4dev::fill_fb_bf16(fb_bf16, &tables->formatbook[0][0], threadIdx.x);
   __syncthreads();
   const bool wide = out_aligned32 != 0;
+  constexpr int kWordBytes = OUT_BF16 ? 16 : 32;
   constexpr int64_t kStep = (int64_t)kDecodeThreads * kDecodeUnroll;
   for (int64_t base = (int64_t)blockIdx.x * kStep; base < total_blocks; base += (int64_t)gridDim.x * kStep) {
     uint32_t cw[kDecodeUnroll][WPB], m[kDecodeUnroll];
@@ -206,61 +158,66 @@ fb4_dequantize_kernel(const uint32_t* __restrict__ codes, const uint16_t* __rest
     for (int u = 0; u < kDecodeUnroll; ++u) {
       const int64_t b = base + u * kDecodeThreads + threadIdx.x;
       if (b >= total_blocks) continue;
-      uint32_t pr[WPB * 4];   // two bf16 per register
-      {
-        const uint4 dt = fb_bf16[(m[u] >> 8) & 31u];
-        const uint32_t sc2 = scale_bf16x2(m[u]);
+      const uint4 dt = fb_bf16[(m[u] >> 8) & 31u];
+      const uint32_t sc2 = scale_bf16x2(m[u]);
 #pragma unroll
-        for (int k = 0; k < WPB; ++k) decode_word(cw[u][k], dt, sc2, pr + 4 * k);
+      for (int k = 0; k < WPB; ++k) {
+        uint32_t pr[4];
+        decode_word(cw[u][k], dt, sc2, pr);
+        store_word<OUT_BF16>(reinterpret_cast<uint8_t*>(out) + (b * WPB + k) * kWordBytes, pr, wide);
       }
-      int32_t srow = -1;
-      int64_t rb = 0;
-      if (RESID) {
-        const int64_t t = b / blocks_per_row;
-        int32_t lo = 0, hi = n_salient - 1;
-        while (lo <= hi) {
-          const int32_t mid = (lo + hi) >> 1;
-          const int32_t sv = __ldg(salient_idx + mid);
-          if (sv == (int32_t)t) { srow = mid; break; }
-          if (sv < (int32_t)t) lo = mid + 1; else hi = mid - 1;
-        }
-        rb = (int64_t)srow * blocks_per_row + (b - t * blocks_per_row);
+    }
+  }
+}
+
+// Rows with a residual (Sec. 3.3: Q(Act) + Q(Delta), the sum rounded once to fp32): thread <-> one
+// block of one salient row; decodes the main and the residual codes and writes the row of `out`
+// again.  Runs after the flat decode on the same stream.
+template <int OUT_BF16, int WPB>
+__global__ void __launch_bounds__(kDecodeThreads)
+fb4_dequantize_residual_rows_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restrict__ meta,
+                                    uint32_t blocks_per_row, const Fb4DeviceTables* __restrict__ tables,
+                                    const int32_t* __restrict__ salient_idx, int64_t n_salient,
+                                    const uint32_t* __restrict__ res_codes, const uint16_t* __restrict__ res_meta,
+                                    void* __restrict__ out, int out_aligned32) {
+  __shared__ uint4 fb_bf16[32];
+  fb4dev::fill_fb_bf16(fb_bf16, &tables->formatbook[0][0], threadIdx.x);
+  __syncthreads();
+  const bool wide = out_aligned32 != 0;
+  constexpr int kWordBytes = OUT_BF16 ? 16 : 32;
+  const int64_t total = n_salient * blocks_per_row;
+  for (int64_t rb = (int64_t)blockIdx.x * kDecodeThreads + threadIdx.x; rb < total;
+       rb += (int64_t)gridDim.x * kDecodeThreads) {
+    const int64_t srow = rb / blocks_per_row;
+    const int64_t b = (int64_t)__ldg(salient_idx + srow) * blocks_per_row + (rb - srow * blocks_per_row);
+    uint32_t cw[WPB], rcw[WPB];
+    load_block_codes<WPB>(codes + b * WPB, cw);
+    load_block_codes<WPB>(res_codes + rb * WPB, rcw);
+    const uint32_t m = (uint32_t)__ldg(meta + b), rm = (uint32_t)__ldg(res_meta + rb);
+    const uint4 dt = fb_bf16[(m >> 8) & 31u], rdt = fb_bf16[(rm >> 8) & 31u];
+    const uint32_t sc2 = scale_bf16x2(m), rsc2 = scale_bf16x2(rm);
+#pragma unroll
+    for (int k = 0; k < WPB; ++k) {
+      uint32_t pr[4], rr[4];
+      decode_word(cw[k], dt, sc2, pr);
+      decode_word(rcw[k], rdt, rsc2, rr);
+      uint32_t v[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        v[2 * j] = __float_as_uint(__fadd_rn(__uint_as_float(pr[j] << 16), __uint_as_float(rr[j] << 16)));
+        v[2 * j + 1] = __float_as_uint(
+            __fadd_rn(__uint_as_float(pr[j] & 0xffff0000u), __uint_as_float(rr[j] & 0xffff0000u)));
       }
-      if (RESID && srow >= 0) {
-        // Q(Act) + Q(Delta), rounded once to fp32 (Sec. 3.3)
-        uint32_t rcw[WPB], rr[WPB * 4];
-        load_block_codes<WPB>(res_codes + rb * WPB, rcw);
-        const uint32_t rm = (uint32_t)__ldg(res_meta + rb);
-        const uint4 rdt = fb_bf16[(rm >> 8) & 31u];
-        const uint32_t rsc2 = scale_bf16x2(rm);
-#pragma unroll
-        for (int k = 0; k < WPB; ++k) decode_word(rcw[k], rdt, rsc2, rr + 4 * k);
-        float v[WPB * 8];
-#pragma unroll
-        for (int j = 0; j < WPB * 4; ++j) {
-          v[2 * j] = __fadd_rn(__uint_as_float(pr[j] << 16), __uint_as_float(rr[j] << 16));
-          v[2 * j + 1] = __fadd_rn(__uint_as_float(pr[j] & 0xffff0000u), __uint_as_float(rr[j] & 0xffff0000u));
-        }
-        if (OUT_BF16) {
-          uint32_t o[WPB * 4];
-#pragma unroll
-          for (int j = 0; j < WPB * 4; ++j) o[j] = f32_to_bf16_rne(v[2 * j]) | (f32_to_bf16_rne(v[2 * j + 1]) << 16);
-          uint8_t* dst = reinterpret_cast<uint8_t*>(out) + b * (WPB * 16);
-#pragma unroll
-          for (int k = 0; k < WPB / 2; ++k) store_b32x8(dst + 32 * k, o + 8 * k, wide);
-        } else {
-          uint8_t* dst = reinterpret_cast<uint8_t*>(out) + b * (WPB * 32);
-#pragma unroll
-          for (int k = 0; k < WPB; ++k) store_b32x8(dst + 32 * k, reinterpret_cast<const uint32_t*>(v) + 8 * k, wide);
-        }
-      } else if (OUT_BF16) {
-        uint8_t* dst = reinterpret_cast<uint8_t*>(out) + b * (WPB * 16);
-#pragma unroll
-        for (int k = 0; k < WPB / 2; ++k) store_b32x8(dst + 32 * k, pr + 8 * k, wide);
+      uint8_t* dst = reinterpret_cast<uint8_t*>(out) + (b * WPB + k) * kWordBytes;
+      if (OUT_BF16) {
+        uint4 o;
+        o.x = f32_to_bf16_rne(__uint_as_float(v[0])) | (f32_to_bf16_rne(__uint_as_float(v[1])) << 16);
+        o.y = f32_to_bf16_rne(__uint_as_float(v[2])) | (f32_to_bf16_rne(__uint_as_float(v[3])) << 16);
+        o.z = f32_to_bf16_rne(__uint_as_float(v[4])) | (f32_to_bf16_rne(__uint_as_float(v[5])) << 16);
+        o.w = f32_to_bf16_rne(__uint_as_float(v[6])) | (f32_to_bf16_rne(__uint_as_float(v[7])) << 16);
+        *reinterpret_cast<uint4*>(dst) = o;
       } else {
-        uint8_t* dst = reinterpret_cast<uint8_t*>(out) + b * (WPB * 32);
-#pragma unroll
-        for (int k = 0; k < WPB; ++k) store_word<0>(dst + 32 * k, pr + 4 * k, wide);
+        store_b32x8(dst, v, wide);
       }
     }
   }
@@ -287,39 +244,50 @@ __global__ void fb4_select_salient_kernel(const float* __restrict__ score, int64
 cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T,
                                   int64_t C, const int32_t* salient_idx, int64_t n_salient,
                                   const uint8_t* res_codes, const uint16_t* res_meta, void* out, int out_dtype,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, int* launches) {
+  static_assert(kDecodeThreads == 256, "one thread per formatbook entry fills the shared table");
+  *launches = 0;
   if (T == 0 || C == 0) return cudaSuccess;
   const int B = (int)ctx->cfg.block_size;
   const int64_t blocks_per_row = C / B;
-  if (blocks_per_row > 0x7fffffffLL || n_salient > 0x7fffffffLL) return cudaErrorInvalidValue;
+  if (blocks_per_row > 0x7fffffffLL) return cudaErrorInvalidValue;
   const int64_t total = T * blocks_per_row;
   constexpr int64_t kStep = (int64_t)kDecodeThreads * kDecodeUnroll;
-  const int64_t want = (total + kStep - 1) / kStep;
   const int64_t cap = (int64_t)ctx->sm_count * 8;          // up to 8 CTAs of 256 threads per SM
+  const int64_t want = (total + kStep - 1) / kStep;
   const unsigned grid = (unsigned)(want < cap ? want : cap);
   const uint32_t* cw = reinterpret_cast<const uint32_t*>(codes);
   const uint32_t* rw = reinterpret_cast<const uint32_t*>(res_codes);
   const int a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
-#define FB4_DECODE(BF, RS, WPB)                                                                              \
-  fb4_dequantize_kernel<BF, RS, WPB><<<grid, kDecodeThreads, 0, stream>>>(                                   \
-      cw, meta, total, (uint32_t)blocks_per_row, ctx->d_tables, salient_idx, (int32_t)n_salient, rw, res_meta, out, a32)
-#define FB4_DECODE_B(BF, RS)                          \
-  do {                                                \
-    if (B == 32) FB4_DECODE(BF, RS, 4); else FB4_DECODE(BF, RS, 2); \
-  } while (0)
-  if (n_salient == 0 && B == 32) {
-    if (out_dtype == 1)
-      fb4_dequantize_b32_kernel<1><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, ctx->d_tables, out, a32);
-    else
-      fb4_dequantize_b32_kernel<0><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, ctx->d_tables, out, a32);
-  } else if (out_dtype == 1) {
-    if (n_salient > 0) FB4_DECODE_B(1, true); else FB4_DECODE_B(1, false);
+  const Fb4DeviceTables* tb = ctx->d_tables;
+  if (B == 32) {
+    if (out_dtype == 1) fb4_dequantize_b32_kernel<1><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
+    else fb4_dequantize_b32_kernel<0><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
   } else {
-    if (n_salient > 0) FB4_DECODE_B(0, true); else FB4_DECODE_B(0, false);
+    if (out_dtype == 1) fb4_dequantize_kernel<1, 2><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
+    else fb4_dequantize_kernel<0, 2><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
   }
-#undef FB4_DECODE_B
-#undef FB4_DECODE
-  return cudaGetLastError();
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  *launches = 1;
+  if (n_salient > 0) {
+    const int64_t rtotal = n_salient * blocks_per_row;
+    const int64_t rwant = (rtotal + kDecodeThreads - 1) / kDecodeThreads;
+    const unsigned rgrid = (unsigned)(rwant < cap ? rwant : cap);
+    const uint32_t bpr = (uint32_t)blocks_per_row;
+#define FB4_RESID(BF, WPB)                                                                 \
+  fb4_dequantize_residual_rows_kernel<BF, WPB><<<rgrid, kDecodeThreads, 0, stream>>>(      \
+      cw, meta, bpr, tb, salient_idx, n_salient, rw, res_meta, out, a32)
+    if (B == 32) {
+      if (out_dtype == 1) FB4_RESID(1, 4); else FB4_RESID(0, 4);
+    } else {
+      if (out_dtype == 1) FB4_RESID(1, 2); else FB4_RESID(0, 2);
+    }
+#undef FB4_RESID
+    e = cudaGetLastError();
+    if (e == cudaSuccess) *launches = 2;
+  }
+  return e;
 }
 
 cudaError_t fb4_launch_select_salient(const float* score, int64_t T, int32_t tile, int32_t* salient_idx,

@@ -22,9 +22,13 @@
 
 #include <cstring>
 
+#include "fb4_device.cuh"
 #include "fb4_internal.h"
 
 namespace {
+
+using fb4dev::pow2f;
+using fb4dev::prmt;
 
 constexpr int kWarps = 16;           // warps per CTA
 constexpr int kStages = 4;           // ring depth per warp
@@ -52,6 +56,7 @@ struct SmemTables {
   // 8-byte column, so the 64-bit loads of a warp never conflict
   uint64_t qerr_private[kMaxGroups][32][16];
   uint8_t pairlut[32 * kPairStride];     // [dialect][36*bin_hi + bin_lo] -> idx_lo | idx_hi<<4
+  uint4 fb_bf16[32];                     // [dialect] -> magnitudes as bf16, high bytes then low bytes (residual pass)
   FastTables c;
 };
 
@@ -60,6 +65,9 @@ struct FastParams {
   int64_t tiles_per_row, n_tiles;
   int64_t step_rows;    // gridDim.x*kWarps tiles ahead = step_rows rows + step_cols tile columns
   int32_t step_cols;
+  int32_t sal_tile;     // tokens per salient-token tile (a huge value when the salient set is a plain list)
+  int32_t step_slots;   // step_rows = step_slots * sal_tile + step_rem
+  int32_t step_rem;
   uint8_t* codes;
   uint16_t* meta;
   uint32_t* status;   // device word: bit 0 = a TMA wait ran out
@@ -102,18 +110,6 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
-}
-
-// prmt.b32 in its default mode: selector nibble bit 3 replicates the sign of the chosen byte
-// (the __byte_perm intrinsic only honours the low three bits).
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-  uint32_t d;
-  asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-  return d;
-}
-
-__device__ __forceinline__ float pow2f(int k) {   // 2^k, k in [-149,127]
-  return k >= -126 ? __int_as_float((k + 127) << 23) : __int_as_float(1 << (k + 149));
 }
 
 // Score an arbitrary candidate mask over 8 group bins with the byte table (SeDA masks that
@@ -179,25 +175,25 @@ template <bool SEDA>
 __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t* cw, int did, uint32_t Ec,
                                                uint32_t allowed, const SmemTables* tb, uint32_t qerr_lane,
                                                uint32_t pair_base, uint32_t* rcw, uint32_t* rmeta) {
-  const float sc = pow2f((int)Ec - 130);   // element scale 2^(e-3)
-  const uint2 fbd = *reinterpret_cast<const uint2*>(tb->c.fb[did]);
+  const uint4 dt = tb->fb_bf16[did];
+  const uint32_t sc2 = fb4dev::scale_bf16x2(Ec - 3u);   // element scale 2^(e-3) as two bf16
   uint32_t a[32];      // |Delta| bit patterns
   uint32_t sg[4];      // sign bits at bit 3 of every nibble
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
+    uint32_t xh[4];    // Q(x) of the word's 8 elements, two bf16 per register, signs included
+    fb4dev::decode_word(cw[q], dt, sc2, xh);
     uint32_t sq = 0;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const int k = q * 8 + i;
-      const uint32_t word = w[k >> 1];
-      const uint32_t xb = (k & 1) ? (word & 0xffff0000u) : (word << 16);
-      const uint32_t nib = cw[q] >> (4 * i);
-      const float mag = (float)(__byte_perm(fbd.x, fbd.y, nib & 7u) & 0xffu) * sc;
-      // Q(x) carries the sign of x
-      const float xhat = __uint_as_float(__float_as_uint(mag) | (xb & 0x80000000u));
-      const uint32_t db = __float_as_uint(__fsub_rn(__uint_as_float(xb), xhat));
-      a[k] = db & 0x7fffffffu;
-      sq |= (db >> 31) << (4 * i + 3);
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t xw = w[4 * q + j];
+      const uint32_t d0 = __float_as_uint(__fsub_rn(__uint_as_float(xw << 16), __uint_as_float(xh[j] << 16)));
+      const uint32_t d1 =
+          __float_as_uint(__fsub_rn(__uint_as_float(xw & 0xffff0000u), __uint_as_float(xh[j] & 0xffff0000u)));
+      a[8 * q + 2 * j] = d0 & 0x7fffffffu;
+      a[8 * q + 2 * j + 1] = d1 & 0x7fffffffu;
+      sq |= (d0 >> (28 - 8 * j)) & (0x8u << (8 * j));
+      sq |= (d1 >> (24 - 8 * j)) & (0x80u << (8 * j));
     }
     sg[q] = sq;
   }
@@ -231,14 +227,19 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
   *rmeta = (Er - 3u) | ((uint32_t)rdid << 8);
 }
 
-// Tile index -> (token row, tile column) without a division per tile: advance by a fixed step.
+// Tile index -> (token row, tile column, salient-token slot = row / sal_tile) without a division per
+// tile: advance by a fixed step.
 struct TilePos {
   int64_t row;
   int32_t col;
-  __device__ __forceinline__ void advance(int64_t step_rows, int32_t step_cols, int32_t tiles_per_row) {
-    row += step_rows;
-    col += step_cols;
-    if (col >= tiles_per_row) { col -= tiles_per_row; ++row; }
+  int32_t slot, rem;   // row = slot * sal_tile + rem
+  __device__ __forceinline__ void advance(const FastParams& p, int32_t tiles_per_row) {
+    row += p.step_rows;
+    col += p.step_cols;
+    slot += p.step_slots;
+    rem += p.step_rem;
+    if (col >= tiles_per_row) { col -= tiles_per_row; ++row; ++rem; }
+    if (rem >= p.sal_tile) { rem -= p.sal_tile; ++slot; }
   }
 };
 
@@ -268,19 +269,36 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
   TilePos cur, pre;   // tile being quantized; next tile to request
   cur.row = gwarp / tpr;
   cur.col = (int32_t)(gwarp - cur.row * tpr);
+  cur.slot = (int32_t)(cur.row / p.sal_tile);
+  cur.rem = (int32_t)(cur.row - (int64_t)cur.slot * p.sal_tile);
   pre = cur;
   int64_t g_pre = gwarp;
+  const bool use_seda = SEDA && ex.cluster_id != nullptr;
+  const bool use_tile = DECOMP && ex.tile > 0;
+  // Per-token extras travel in register queues, fetched as far ahead as the tile data: entry k
+  // belongs to the tile k steps ahead.  cidq = cluster id, salq = token stored in the row's
+  // salient slot; the cluster mask follows its id two steps behind.
+  int32_t cidq[kStages], salq[kStages];
   // prologue: fill the ring
-  if (lane == 0) {
 #pragma unroll
-    for (int s = 0; s < kStages; ++s) {
-      if (g_pre < p.n_tiles) {
+  for (int s = 0; s < kStages; ++s) {
+    cidq[s] = -1;
+    salq[s] = -1;
+    if (g_pre < p.n_tiles) {
+      if (lane == 0) {
         mbar_expect_tx(my_bars + 8 * s, kTileBytes);
         tma_load_tile(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, pre.col * 16, (int)pre.row);
       }
-      g_pre += wstride;
-      pre.advance(p.step_rows, p.step_cols, tpr);
+      if (use_seda) cidq[s] = ex.cluster_id[pre.row];
+      if (use_tile && pre.slot < ex.n_salient) salq[s] = ex.salient_idx[pre.slot];
     }
+    g_pre += wstride;
+    pre.advance(p, tpr);
+  }
+  uint32_t maskq[2] = {0xffffffffu, 0xffffffffu};
+  if (use_seda) {
+    if (cidq[0] >= 0) maskq[0] = ex.cluster_mask[cidq[0]];
+    if (cidq[1] >= 0) maskq[1] = ex.cluster_mask[cidq[1]];
   }
   // ---- expand the tables into shared memory (overlaps the first loads)
   {
@@ -291,6 +309,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     const uint64_t* q64 = reinterpret_cast<const uint64_t*>(g_tables->qerr64);
     uint64_t* qp = &tb->qerr_private[0][0][0];
     for (int i = threadIdx.x; i < kMaxGroups * 32 * 16; i += kWarps * 32) qp[i] = q64[i >> 4];
+    if (threadIdx.x < 256) fb4dev::fill_fb_bf16(tb->fb_bf16, &g_tables->fb[0][0], threadIdx.x);
     // pair tables, one 32-bit word (4 consecutive bin_lo) at a time
     for (int i = threadIdx.x; i < 32 * 32 * 8; i += kWarps * 32) {
       const int d = i >> 8, bh = (i >> 3) & 31, bl4 = (i & 7) * 4;
@@ -311,49 +330,21 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
 
   const int64_t nblk = p.C >> 5;
   const int64_t code_row_bytes = p.C >> 1;
-  const bool use_seda = SEDA && ex.cluster_id != nullptr;
-  const bool use_tile = DECOMP && ex.tile > 0;
-
-  // Per-token extras (cluster mask, salient slot) are fetched ahead of use so that their latency
-  // hides behind the tile being quantized: the cluster id two tiles ahead, the mask and the
-  // salient candidate one tile ahead.
-  TilePos n1 = cur, n2;
-  n1.advance(p.step_rows, p.step_cols, tpr);
-  n2 = n1;
-  n2.advance(p.step_rows, p.step_cols, tpr);
-  int32_t cid_n1 = -1;
-  uint32_t allowed_cur = 0xffffffffu;
-  if (use_seda) {
-    if (gwarp < p.n_tiles) {
-      const int32_t cid = ex.cluster_id[cur.row];
-      if (cid >= 0) allowed_cur = ex.cluster_mask[cid];
-    }
-    if (gwarp + wstride < p.n_tiles) cid_n1 = ex.cluster_id[n1.row];
-  }
-  int32_t sal_cur = -1;   // token id stored in the salient slot of the current row's tile
-  if (use_tile && gwarp < p.n_tiles) {
-    const uint32_t sidx = (uint32_t)cur.row / (uint32_t)ex.tile;
-    if ((int64_t)sidx < ex.n_salient) sal_cur = ex.salient_idx[sidx];
-  }
 
   int s = 0;
   uint32_t parity = 0;
   for (int64_t g = gwarp; g < p.n_tiles; g += wstride) {
-    // ---- prefetch the extras of the following tiles
-    uint32_t allowed_n1 = 0xffffffffu;
-    int32_t cid_n2 = -1;
-    int32_t sal_n1 = -1;
+    // ---- fetch the extras of the tiles ahead (pre = the tile kStages steps ahead)
+    int32_t cid_new = -1, sal_new = -1;
+    uint32_t mask_new = 0xffffffffu;
     if (SEDA) {
       if (use_seda) {
-        if (cid_n1 >= 0) allowed_n1 = ex.cluster_mask[cid_n1];
-        if (g + 2 * wstride < p.n_tiles) cid_n2 = ex.cluster_id[n2.row];
+        if (g_pre < p.n_tiles) cid_new = ex.cluster_id[pre.row];
+        if (cidq[2] >= 0) mask_new = ex.cluster_mask[cidq[2]];
       }
     }
     if (DECOMP) {
-      if (use_tile && g + wstride < p.n_tiles) {
-        const uint32_t sidx = (uint32_t)n1.row / (uint32_t)ex.tile;
-        if ((int64_t)sidx < ex.n_salient) sal_n1 = ex.salient_idx[sidx];
-      }
+      if (use_tile && g_pre < p.n_tiles && pre.slot < ex.n_salient) sal_new = ex.salient_idx[pre.slot];
     }
 
     const uint32_t bar = my_bars + 8 * s;
@@ -410,7 +401,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
 
     uint32_t allowed = 0xffffffffu;
     if (SEDA) {
-      allowed = allowed_cur;
+      allowed = maskq[0];
       if (allowed == 0) allowed = 1u;   // precondition violated: stay in bounds
     }
     // ---- dialect selection; the upper bf16 of a pair keeps the lower one as extra mantissa bits,
@@ -450,7 +441,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     if (DECOMP) {
       int64_t srow = -1;
       if (use_tile) {
-        if (sal_cur == (int32_t)row) srow = (int64_t)((uint32_t)row / (uint32_t)ex.tile);
+        if (salq[0] == (int32_t)row) srow = cur.slot;
       } else {
         int64_t lo = 0, hi = ex.n_salient - 1;
         while (lo <= hi) {
@@ -477,13 +468,17 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
       tma_load_tile(my_ring + s * kTileBytes, &tmap, bar, pre.col * 16, (int)pre.row);
     }
     g_pre += wstride;
-    pre.advance(p.step_rows, p.step_cols, tpr);
-    cur.advance(p.step_rows, p.step_cols, tpr);
-    n1.advance(p.step_rows, p.step_cols, tpr);
-    n2.advance(p.step_rows, p.step_cols, tpr);
-    allowed_cur = allowed_n1;
-    cid_n1 = cid_n2;
-    sal_cur = sal_n1;
+    pre.advance(p, tpr);
+    cur.advance(p, tpr);
+#pragma unroll
+    for (int k = 0; k + 1 < kStages; ++k) {
+      cidq[k] = cidq[k + 1];
+      salq[k] = salq[k + 1];
+    }
+    cidq[kStages - 1] = cid_new;
+    salq[kStages - 1] = sal_new;
+    maskq[0] = maskq[1];
+    maskq[1] = mask_new;
     if (++s == kStages) { s = 0; parity ^= 1u; }
   }
 }
@@ -619,6 +614,9 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   const int64_t wstride = (int64_t)grid * kWarps;
   p.step_rows = wstride / p.tiles_per_row;
   p.step_cols = (int32_t)(wstride % p.tiles_per_row);
+  p.sal_tile = ex.tile > 0 ? ex.tile : 0x7fffffff;
+  p.step_slots = (int32_t)(p.step_rows / p.sal_tile);
+  p.step_rem = (int32_t)(p.step_rows % p.sal_tile);
   const FastTables* tables = static_cast<const FastTables*>(ctx->d_fast_tables);
   const bool seda = ex.cluster_id != nullptr, decomp = ex.n_salient > 0;
   if (seda && decomp) return launch<true, true>(map, tables, p, ex, grid, stream);

@@ -58,6 +58,6 @@ cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int64
 cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T,
                                   int64_t C, const int32_t* salient_idx, int64_t n_salient,
                                   const uint8_t* res_codes, const uint16_t* res_meta, void* out, int out_dtype,
-                                  cudaStream_t stream);
+                                  cudaStream_t stream, int* launches);
 cudaError_t fb4_launch_select_salient(const float* score, int64_t T, int32_t tile, int32_t* salient_idx,
                                       cudaStream_t stream);
