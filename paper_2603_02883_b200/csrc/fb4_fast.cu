@@ -254,8 +254,23 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int64_t gwarp = (int64_t)blockIdx.x * kWarps + warp;
-  const int64_t wstride = (int64_t)gridDim.x * kWarps;
+  // Tile -> warp assignment.  Plain and SeDA calls: tile g goes to warp g mod (all warps of the grid),
+  // so the whole grid sweeps the tensor as one front.  Calls with a residual pass: every CTA takes a
+  // contiguous range of tiles and deals it round-robin to its own warps, which spreads the (much
+  // more expensive) tiles of a salient token over many warps and gives every CTA the same share
+  // of salient tokens.
+  int64_t gwarp, g_end, wstride;
+  if (DECOMP) {
+    const int64_t per = p.n_tiles / gridDim.x, extra = p.n_tiles % gridDim.x, b = blockIdx.x;
+    const int64_t t0 = b * per + (b < extra ? b : extra);
+    gwarp = t0 + warp;
+    g_end = t0 + per + (b < extra ? 1 : 0);
+    wstride = kWarps;
+  } else {
+    gwarp = (int64_t)blockIdx.x * kWarps + warp;
+    g_end = p.n_tiles;
+    wstride = (int64_t)gridDim.x * kWarps;
+  }
   const int32_t tpr = (int32_t)p.tiles_per_row;
 
   if (threadIdx.x == 0) {
@@ -284,7 +299,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
   for (int s = 0; s < kStages; ++s) {
     cidq[s] = -1;
     salq[s] = -1;
-    if (g_pre < p.n_tiles) {
+    if (g_pre < g_end) {
       if (lane == 0) {
         mbar_expect_tx(my_bars + 8 * s, kTileBytes);
         tma_load_tile(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, pre.col * 16, (int)pre.row);
@@ -333,18 +348,18 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
 
   int s = 0;
   uint32_t parity = 0;
-  for (int64_t g = gwarp; g < p.n_tiles; g += wstride) {
+  for (int64_t g = gwarp; g < g_end; g += wstride) {
     // ---- fetch the extras of the tiles ahead (pre = the tile kStages steps ahead)
     int32_t cid_new = -1, sal_new = -1;
     uint32_t mask_new = 0xffffffffu;
     if (SEDA) {
       if (use_seda) {
-        if (g_pre < p.n_tiles) cid_new = ex.cluster_id[pre.row];
+        if (g_pre < g_end) cid_new = ex.cluster_id[pre.row];
         if (cidq[2] >= 0) mask_new = ex.cluster_mask[cidq[2]];
       }
     }
     if (DECOMP) {
-      if (use_tile && g_pre < p.n_tiles && pre.slot < ex.n_salient) sal_new = ex.salient_idx[pre.slot];
+      if (use_tile && g_pre < g_end && pre.slot < ex.n_salient) sal_new = ex.salient_idx[pre.slot];
     }
 
     const uint32_t bar = my_bars + 8 * s;
@@ -358,7 +373,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
       int sj = s;
       uint32_t pj = parity;
       for (int j = 1; j < kStages; ++j) {
-        if (g + (int64_t)j * wstride >= p.n_tiles) break;
+        if (g + (int64_t)j * wstride >= g_end) break;
         if (++sj == kStages) { sj = 0; pj ^= 1u; }
         uint32_t tries = 0;
         while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
@@ -463,7 +478,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     }
     // ---- refill this stage (all lanes have consumed their registers from it)
     __syncwarp();
-    if (lane == 0 && g_pre < p.n_tiles) {
+    if (lane == 0 && g_pre < g_end) {
       mbar_expect_tx(bar, kTileBytes);
       tma_load_tile(my_ring + s * kTileBytes, &tmap, bar, pre.col * 16, (int)pre.row);
     }
@@ -611,14 +626,14 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   p.status = ctx->d_status;
   const int64_t want = (p.n_tiles + kWarps - 1) / kWarps;
   const int grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
-  const int64_t wstride = (int64_t)grid * kWarps;
+  const bool seda = ex.cluster_id != nullptr, decomp = ex.n_salient > 0;
+  const int64_t wstride = decomp ? kWarps : (int64_t)grid * kWarps;   // tiles between a warp's consecutive tiles
   p.step_rows = wstride / p.tiles_per_row;
   p.step_cols = (int32_t)(wstride % p.tiles_per_row);
   p.sal_tile = ex.tile > 0 ? ex.tile : 0x7fffffff;
   p.step_slots = (int32_t)(p.step_rows / p.sal_tile);
   p.step_rem = (int32_t)(p.step_rows % p.sal_tile);
   const FastTables* tables = static_cast<const FastTables*>(ctx->d_fast_tables);
-  const bool seda = ex.cluster_id != nullptr, decomp = ex.n_salient > 0;
   if (seda && decomp) return launch<true, true>(map, tables, p, ex, grid, stream);
   if (seda) return launch<true, false>(map, tables, p, ex, grid, stream);
   if (decomp) return launch<false, true>(map, tables, p, ex, grid, stream);
