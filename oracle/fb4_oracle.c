@@ -21,7 +21,10 @@
  *   Sec. 3.3  activation decomposition: residual Delta = Act - Q(Act) of the
  *             salient tokens is quantized again; one salient token per tile,
  *             the highest-scoring one.
- *   Sec. 3.4  SeDA: the candidate set of a token is its cluster's sub-formatbook.
+ *   Sec. 3.4  SeDA: the candidate set of a token is its cluster's sub-formatbook; a
+ *             sub-formatbook is built by counting, over a cluster's anchor tokens, how
+ *             often each dialect was chosen in each dynamic-range bucket and keeping
+ *             the most frequent dialect of every bucket.
  *
  * No lookup tables are used anywhere: each rounding searches the 8 magnitudes,
  * each error term is computed from the explicit bin midpoint.
@@ -39,13 +42,19 @@
  *     the SeDA mask falls back to the SeDA mask alone;
  *   - the residual is the fp32 value of x - xhat (exact for the default exponent
  *     range) and is quantized from that value, never rounded to bf16;
- *   - the scale byte is e + 124, i.e. the E8M0 code of the element scale 2^(e-3).
+ *   - the scale byte is e + 124, i.e. the E8M0 code of the element scale 2^(e-3);
+ *   - sub-formatbook construction: the dynamic-range buckets are the distinct entries
+ *     of the stage-1 table; frequency ties (and buckets no anchor block fell into)
+ *     go to the lowest dialect id; anchors with an id outside the tensor or a
+ *     cluster outside [0, n_clusters) are ignored.
  *
  * Pins (tests/test_oracle_*.py): every representable value of every dialect
  * round-trips; closed form for the uniform dialect; exact-rational brute force
  * on tiny blocks and on all 65536 bf16 patterns; |E_d - exact error| <= G/4;
  * argmin invariant; decomposition never increases any element's error; SeDA
- * choices lie in the mask; per-tile argmax by brute force.
+ * choices lie in the mask; per-tile argmax by brute force; sub-formatbooks on
+ * hand-counted cases, one dialect per bucket, and a constrained tensor giving
+ * back the sub-formatbook it was constrained to.
  * Parity unpinned: the formatbook VALUES (the paper's table is only in Fig. 2a)
  * and any worked numeric example (the paper prints none).
  */
@@ -358,5 +367,44 @@ int fb4o_quantize_block_f64(const double *x, const fb4o_config *cfg, const uint8
   quantize_block(x, sg, cfg, F, stage1, allowed, code, &d_, &e_, err_q4);
   *did = d_;
   *e = e_;
+  return 0;
+}
+
+/*
+ * Sub-formatbook construction, Sec. 3.4 ("bin-count profiling on anchor tokens ...
+ * selecting the most frequent dialect for each dynamic-range bucket").
+ * meta [T][nblk] holds the dialect chosen for every block (bits 8-12).  Anchor a is
+ * token anchor_token[a] and belongs to cluster anchor_cluster[a].  For every cluster:
+ * count how often each dialect occurs in the blocks of its anchor tokens; then, for
+ * every dynamic-range bucket (a distinct entry of the stage-1 table), keep the most
+ * frequent dialect among the bucket's members.  cluster_mask[c] = the kept dialects.
+ */
+int fb4o_build_subformatbook(const uint16_t *meta, int64_t T, int64_t nblk,
+                             const int32_t *anchor_token, const int32_t *anchor_cluster, int64_t n_anchor,
+                             int32_t n_clusters, const uint8_t *F, const uint32_t *stage1_in,
+                             uint32_t *cluster_mask) {
+  if (T < 0 || nblk <= 0 || n_anchor < 0 || n_clusters < 0 || !formatbook_ok(F)) return -1;
+  uint32_t stage1[32];
+  if (stage1_in) memcpy(stage1, stage1_in, sizeof stage1); else fb4o_default_stage1(F, stage1);
+  for (int32_t c = 0; c < n_clusters; ++c) {
+    int64_t count[32];
+    for (int d = 0; d < 32; ++d) count[d] = 0;
+    for (int64_t a = 0; a < n_anchor; ++a) {
+      if (anchor_cluster[a] != c) continue;
+      int64_t t = anchor_token[a];
+      if (t < 0 || t >= T) continue;
+      for (int64_t b = 0; b < nblk; ++b) count[(meta[t * nblk + b] >> 8) & 31] += 1;
+    }
+    uint32_t mask = 0;
+    for (int k = 0; k < 32; ++k) {            /* every bucket; repeated entries pick the same dialect again */
+      int best = -1;
+      for (int d = 0; d < 32; ++d) {
+        if (!((stage1[k] >> d) & 1u)) continue;
+        if (best < 0 || count[d] > count[best]) best = d;   /* ties keep the lowest id */
+      }
+      if (best >= 0) mask |= 1u << best;
+    }
+    cluster_mask[c] = mask;
+  }
   return 0;
 }

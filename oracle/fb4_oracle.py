@@ -76,6 +76,8 @@ def lib():
         L.fb4o_mse.restype = ctypes.c_double
         L.fb4o_quantize_block_f64.argtypes = [vp, ctypes.POINTER(_Cfg), vp, vp, u32, vp, vp, vp, vp]
         L.fb4o_quantize_block_f64.restype = ctypes.c_int
+        L.fb4o_build_subformatbook.argtypes = [vp, i64, i64, vp, vp, i64, i32, vp, vp, vp]
+        L.fb4o_build_subformatbook.restype = ctypes.c_int
         _libs[path] = L
     return _libs[path]
 
@@ -193,3 +195,18 @@ def quantize_block_f64(x, formatbook, cfg: Config = Config(), stage1=None, allow
     if r != 0:
         raise ValueError(f"fb4o_quantize_block_f64 failed: {r}")
     return code, int(did[0]), int(e[0]), err
+
+
+def build_subformatbook(meta, anchor_token, anchor_cluster, n_clusters: int, formatbook, stage1=None) -> np.ndarray:
+    """meta: uint16 [T][C/B]; anchors: int32 token ids and their clusters -> uint32 [n_clusters] masks."""
+    m = _c(meta, np.uint16)
+    T, nblk = m.shape
+    at = _c(anchor_token, np.int32)
+    ac = _c(anchor_cluster, np.int32)
+    assert at.shape == ac.shape
+    out = np.zeros(max(n_clusters, 1), dtype=np.uint32)
+    r = lib().fb4o_build_subformatbook(_p(m), T, nblk, _p(at), _p(ac), at.shape[0], n_clusters,
+                                       _p(_c(formatbook, np.uint8)), _p(_c(stage1, np.uint32)), _p(out))
+    if r != 0:
+        raise ValueError(f"fb4o_build_subformatbook failed: {r}")
+    return out[:n_clusters]

@@ -336,6 +336,72 @@ def pin_seda_choice_inside_mask(seed=4, n=120):
     assert np.array_equal(qa.codes, qb.codes) and np.array_equal(qa.meta, qb.meta)
 
 
+def _meta_with_dialects(rows):
+    """meta records (scale byte 124) for rows of dialect ids"""
+    return np.array([[124 | (d << 8) for d in r] for r in rows], dtype=np.uint16)
+
+
+def pin_subformatbook_hand_counted():
+    """Sec. 3.4 sub-formatbook construction on cases counted by hand.  Stand-in formatbook: buckets
+    (largest magnitude 8..15) hold dialects {0,1} {2,3} {4,5,6} {7,8,9} {10..13} {14..18} {19..24} {25..31}."""
+    assert [int(FB[d, 7]) for d in (0, 1, 2, 3, 4, 6, 7, 9, 10, 13, 14, 18, 19, 24, 25, 31)] == \
+        [8, 8, 9, 9, 10, 10, 11, 11, 12, 12, 13, 13, 14, 14, 15, 15]
+    meta = _meta_with_dialects([
+        [1, 1, 0, 5, 5, 6, 31, 30],      # token 0
+        [1, 3, 3, 2, 6, 6, 26, 30],      # token 1
+        [0, 0, 0, 0, 0, 0, 0, 0],        # token 2 (anchor of cluster 1)
+        [12, 12, 11, 11, 13, 17, 17, 20],  # token 3 (no anchor: must not count)
+    ])
+    # cluster 0 = tokens 0 and 1: bucket 8: d1 x3 vs d0 x1 -> 1; bucket 9: d3 x2 vs d2 x1 -> 3;
+    # bucket 10: d5 x2, d6 x3 -> 6; bucket 15: d30 x2, d31, d26 -> 30; buckets 11,12,13,14 empty -> 7,10,14,19
+    want0 = sum(1 << d for d in (1, 3, 6, 7, 10, 14, 19, 30))
+    # cluster 1 = token 2: only d0 occurs; every other bucket takes its lowest id
+    want1 = sum(1 << d for d in (0, 2, 4, 7, 10, 14, 19, 25))
+    # cluster 2 has no anchors at all: lowest id everywhere
+    got = orc.build_subformatbook(meta, [0, 2, 1], [0, 1, 0], 3, FB)
+    assert [int(m) for m in got] == [want0, want1, want1]
+    # an anchor listed twice counts twice: token 0 twice + token 1 -> bucket 10: d5 x4 vs d6 x4... d5=2*2=4, d6=1*2+2=4: tie -> 5
+    got = orc.build_subformatbook(meta, [0, 0, 1], [0, 0, 0], 1, FB)
+    assert int(got[0]) == sum(1 << d for d in (1, 3, 5, 7, 10, 14, 19, 30))
+    # anchors outside the tensor or outside the clusters are ignored
+    got = orc.build_subformatbook(meta, [0, 1, 7, -1, 3], [0, 0, 0, 0, 5], 1, FB)
+    assert int(got[0]) == want0
+    # a custom stage-1 table with two buckets {0..15} {16..31}: one pick per bucket
+    s1 = np.array([0x0000FFFF] * 16 + [0xFFFF0000] * 16, dtype=np.uint32)
+    got = orc.build_subformatbook(meta, [3], [0], 1, FB, stage1=s1)
+    assert int(got[0]) == (1 << 11) | (1 << 17)          # d11 x2 = d12 x2 -> lowest; d17 x2 vs d20 x1
+
+
+def pin_subformatbook_one_dialect_per_bucket_and_closed_loop(seed=8):
+    """An 8-dialect sub-formatbook has one dialect per dynamic range (Sec. 3.4); tokens that were
+    quantized under a sub-formatbook M give M back on every bucket their blocks fell into."""
+    w = synth.Workload("t", T=96, C=256, seed=seed, kind=1, n_outlier=2, outlier_gain=50.0,
+                       seda=True, n_clusters=3, cluster_seed=seed + 1)
+    bits = synth.activation(w)
+    cid, masks = synth.clusters(w)
+    free = orc.quantize(bits, FB)
+    tok = np.arange(w.T, dtype=np.int32)
+    built = orc.build_subformatbook(free.meta, tok, cid, 3, FB)
+    for m in built:
+        assert sorted(int(FB[d, 7]) for d in range(32) if (int(m) >> d) & 1) == list(range(8, 16))
+    # most frequent: no other member of the bucket was chosen more often
+    for c in range(3):
+        cnt = np.bincount(free.did[cid == c].ravel(), minlength=32)
+        for d in range(32):
+            if (int(built[c]) >> d) & 1:
+                rivals = [dd for dd in range(32) if int(FB[dd, 7]) == int(FB[d, 7])]
+                assert cnt[d] == max(cnt[dd] for dd in rivals)
+                assert d == min(dd for dd in rivals if cnt[dd] == cnt[d])
+    # closed loop
+    con = orc.quantize(bits, FB, cluster_id=cid, cluster_mask=masks)
+    again = orc.build_subformatbook(con.meta, tok, cid, 3, FB)
+    for c in range(3):
+        used_buckets = {int(FB[d, 7]) for d in np.unique(con.did[cid == c])}
+        for d in range(32):
+            if int(FB[d, 7]) in used_buckets:
+                assert ((int(again[c]) >> d) & 1) == ((int(masks[c]) >> d) & 1)
+
+
 # ---------------------------------------------------------------- decomposition (Sec. 3.3)
 
 def pin_salient_is_per_tile_argmax(seed=5):
@@ -417,5 +483,6 @@ ALL_PINS = [
     pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
     pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_decomposition,
-    pin_dequantize_formula, pin_mse,
+    pin_dequantize_formula, pin_mse, pin_subformatbook_hand_counted,
+    pin_subformatbook_one_dialect_per_bucket_and_closed_loop,
 ]

@@ -37,6 +37,15 @@ MUTANTS = {
     "zero_block_exponent": ("e = cfg->exp_min;\n  } else {", "e = 0;\n  } else {"),
     "stage1_bucket_shift": ("int bucket = k / 2 < 8 ? 8 : k / 2;", "int bucket = k / 2 < 9 ? 9 : k / 2;"),
     "mse_not_squared": ("row += d * d;", "row += fabs(d);"),
+    "subformatbook_ties_to_highest": ("if (best < 0 || count[d] > count[best]) best = d;",
+                                      "if (best < 0 || count[d] >= count[best]) best = d;"),
+    "subformatbook_least_frequent": ("if (best < 0 || count[d] > count[best]) best = d;",
+                                     "if (best < 0 || count[d] < count[best]) best = d;"),
+    "subformatbook_buckets_ignored": ("if (!((stage1[k] >> d) & 1u)) continue;\n        if (best < 0 || count[d] > count[best])",
+                                      "if (best < 0 || count[d] > count[best])"),
+    "subformatbook_all_anchors_one_cluster": ("if (anchor_cluster[a] != c) continue;", ";"),
+    "subformatbook_last_block_skipped": ("for (int64_t b = 0; b < nblk; ++b) count[", "for (int64_t b = 0; b + 1 < nblk; ++b) count["),
+    "subformatbook_counts_scale_byte": ("count[(meta[t * nblk + b] >> 8) & 31] += 1;", "count[meta[t * nblk + b] & 31] += 1;"),
 }
 
 
