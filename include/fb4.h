@@ -117,6 +117,26 @@ int fb4_quantize_seda(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, in
                       uint16_t* meta, void* stream);
 
 /*
+ * Sub-formatbook construction for SeDA (Sec. 3.4: "bin-count profiling on anchor tokens to
+ * measure how often each dialect is selected in each dynamic range ... selecting the most
+ * frequent dialect for each dynamic-range bucket").  `meta` is the metadata of a quantization of
+ * the layer's activation (normally unconstrained); anchor a is token anchor_token[a] and belongs
+ * to cluster anchor_cluster[a].  For every cluster the dialect ids of all blocks of its anchor
+ * tokens are counted; for every dynamic-range bucket (a distinct entry of the context's stage-1
+ * table) the most frequent member is kept, ties and buckets without any count going to the
+ * lowest dialect id.  cluster_mask[c] (the input of fb4_quantize_seda) = the kept dialects.
+ *   meta           : device uint16 [T][C/B]
+ *   anchor_token   : device int32 [n_anchor]; entries outside [0,T) are ignored
+ *   anchor_cluster : device int32 [n_anchor]; entries outside [0,n_clusters) are ignored
+ *   counts         : device uint32 [n_clusters][32], scratch provided by the caller; holds the
+ *                    per-cluster dialect counts on return (n_anchor * C/B must stay below 2^32)
+ *   cluster_mask   : device uint32 [n_clusters] (out)
+ */
+int fb4_build_subformatbook(fb4_ctx* ctx, const uint16_t* meta, int64_t T, int64_t C, const int32_t* anchor_token,
+                            const int32_t* anchor_cluster, int64_t n_anchor, int32_t n_clusters, uint32_t* counts,
+                            uint32_t* cluster_mask, void* stream);
+
+/*
  * Salient-token selection for activation decomposition (Sec. 3.3: "one salient
  * token per tile ... the highest-scoring token in each tile"): for every tile of
  * `tile` consecutive tokens, the index of the largest score (ties: lowest index).

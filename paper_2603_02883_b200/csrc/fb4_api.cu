@@ -305,6 +305,28 @@ int fb4_dequantize(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int
   return FB4_OK;
 }
 
+int fb4_build_subformatbook(fb4_ctx* ctx, const uint16_t* meta, int64_t T, int64_t C, const int32_t* anchor_token,
+                            const int32_t* anchor_cluster, int64_t n_anchor, int32_t n_clusters, uint32_t* counts,
+                            uint32_t* cluster_mask, void* stream) {
+  if (!ctx) return FB4_ERR_INVALID_ARG;
+  if (T < 0 || C <= 0 || C % ctx->cfg.block_size != 0 || T > 0x7fffffffLL) return FB4_ERR_SHAPE;
+  if (n_anchor < 0 || n_clusters < 0) return FB4_ERR_INVALID_ARG;
+  if (n_clusters == 0) return FB4_OK;
+  if (!counts || !cluster_mask) return FB4_ERR_INVALID_ARG;
+  if (n_anchor > 0 && (!meta || !anchor_token || !anchor_cluster)) return FB4_ERR_INVALID_ARG;
+  const int64_t nblk = C / ctx->cfg.block_size;
+  if (n_anchor > 0 && n_anchor > 0xffffffffLL / nblk) return FB4_ERR_SHAPE;   // counts are 32-bit
+  Fb4Stage1 s1;
+  std::memcpy(s1.m, ctx->host_tables.stage1, sizeof s1.m);
+  int launches = 0;
+  cudaError_t e = fb4_launch_subformatbook(meta, T, nblk, anchor_token, anchor_cluster, n_anchor, n_clusters, s1,
+                                           counts, cluster_mask, ctx->sm_count, static_cast<cudaStream_t>(stream),
+                                           &launches);
+  ctx->launches += launches;
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
+  return FB4_OK;
+}
+
 int fb4_quantize_host(fb4_ctx* ctx, const void* x_host, int64_t T, int64_t C, void* d_x, uint8_t* d_codes,
                       uint16_t* d_meta, uint8_t* codes_host, uint16_t* meta_host) {
   const int rc = check_quantize_args(ctx, d_x, T, C, C, d_codes, d_meta);

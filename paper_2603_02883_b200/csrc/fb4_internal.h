@@ -15,6 +15,11 @@ struct Fb4DeviceTables {
   uint32_t stage1[32];      // [bin of block maximum] -> candidate dialect mask
 };
 
+// Stage-1 table passed to a kernel by value.
+struct Fb4Stage1 {
+  uint32_t m[32];
+};
+
 // Per-row extras of one quantize launch (all pointers device, nullable).
 struct Fb4RowExtras {
   const int32_t* cluster_id;    // SeDA: token -> cluster, -1 = unconstrained
@@ -59,5 +64,9 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
                                   int64_t C, const int32_t* salient_idx, int64_t n_salient,
                                   const uint8_t* res_codes, const uint16_t* res_meta, void* out, int out_dtype,
                                   cudaStream_t stream, int* launches);
+cudaError_t fb4_launch_subformatbook(const uint16_t* meta, int64_t T, int64_t nblk, const int32_t* anchor_token,
+                                     const int32_t* anchor_cluster, int64_t n_anchor, int32_t n_clusters,
+                                     const Fb4Stage1& stage1, uint32_t* counts, uint32_t* cluster_mask, int sm_count,
+                                     cudaStream_t stream, int* launches);
 cudaError_t fb4_launch_select_salient(const float* score, int64_t T, int32_t tile, int32_t* salient_idx,
                                       cudaStream_t stream);

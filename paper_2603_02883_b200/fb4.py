@@ -20,7 +20,7 @@ ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_FORMATBOOK, ERR_CUDA, ERR_NO_DEVICE =
 
 EXPORTS = [
     "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_seda",
-    "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
+    "fb4_build_subformatbook", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
     "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
 
@@ -68,13 +68,15 @@ def lib() -> ctypes.CDLL:
     L.fb4_get_tables.argtypes = [vp, vp, vp, vp, vp]
     L.fb4_quantize.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.fb4_quantize_seda.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, vp, vp, vp]
+    L.fb4_build_subformatbook.argtypes = [vp, vp, i64, i64, vp, vp, i64, i32, vp, vp, vp]
+    L.fb4_build_subformatbook.restype = ci
     L.fb4_select_salient.argtypes = [vp, vp, i64, i32, vp, vp]
     L.fb4_quantize_decomposed.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.fb4_quantize_decomposed_idx.argtypes = [vp, vp, i64, i64, i64, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
     L.fb4_dequantize.argtypes = [vp, vp, vp, i64, i64, vp, i64, vp, vp, vp, ci, vp]
     L.fb4_quantize_host.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp]
     for name in ("fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_seda",
-                 "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx",
+                 "fb4_build_subformatbook", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx",
                  "fb4_dequantize", "fb4_quantize_host", "fb4_last_cuda_error"):
         getattr(L, name).restype = ci
     L.fb4_set_kernel_variant.argtypes = [vp, ci]
@@ -151,6 +153,13 @@ def fb4_quantize(ctx, x, T, C, ld_elems, codes, meta, stream=None) -> None:
 def fb4_quantize_seda(ctx, x, T, C, ld_elems, cluster_id, cluster_mask, n_clusters, codes, meta, stream=None) -> None:
     _check(lib().fb4_quantize_seda(ctx, _ptr(x), T, C, ld_elems, _ptr(cluster_id), _ptr(cluster_mask), n_clusters,
                                    _ptr(codes), _ptr(meta), _stream(stream)), "fb4_quantize_seda")
+
+
+def fb4_build_subformatbook(ctx, meta, T, C, anchor_token, anchor_cluster, n_anchor, n_clusters, counts, cluster_mask,
+                            stream=None) -> None:
+    _check(lib().fb4_build_subformatbook(ctx, _ptr(meta), T, C, _ptr(anchor_token), _ptr(anchor_cluster), n_anchor,
+                                         n_clusters, _ptr(counts), _ptr(cluster_mask), _stream(stream)),
+           "fb4_build_subformatbook")
 
 
 def fb4_select_salient(ctx, score, T, tile, salient_idx, stream=None) -> None:
@@ -276,6 +285,15 @@ class Fb4:
         fb4_quantize_decomposed_idx(self.ctx, x, T, C, ld, salient_idx, n, cluster_id, cluster_mask, ncl, codes, meta,
                                     rc, rm)
         return Quantized(codes, meta, salient_idx, rc[:n], rm[:n])
+
+    def build_subformatbook(self, meta, anchor_token, anchor_cluster, n_clusters: int):
+        """cluster masks (int32 tensor holding uint32 bit patterns) from the dialects chosen on anchor tokens"""
+        T, nblk = meta.shape
+        counts = torch.empty((max(n_clusters, 1), 32), dtype=torch.int32, device=meta.device)
+        masks = torch.empty(max(n_clusters, 1), dtype=torch.int32, device=meta.device)
+        fb4_build_subformatbook(self.ctx, meta, T, nblk * self.block_size, anchor_token, anchor_cluster,
+                                anchor_token.numel(), n_clusters, counts, masks)
+        return masks[:n_clusters], counts[:n_clusters]
 
     def select_salient(self, score, tile: int = 20):
         T = score.numel()

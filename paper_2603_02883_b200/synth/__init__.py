@@ -157,6 +157,23 @@ def clusters(w: Workload, formatbook: np.ndarray = STANDIN_FORMATBOOK):
     return cid, mask
 
 
+def anchors(cluster_id: np.ndarray, n_clusters: int, per_cluster: int = 8):
+    """Anchor tokens of a SeDA workload: up to `per_cluster` tokens spread evenly over every
+    cluster's token range (deterministic, no random draw).  Returns (anchor_token, anchor_cluster),
+    both int32, ordered by cluster."""
+    tok, clu = [], []
+    for c in range(n_clusters):
+        members = np.flatnonzero(cluster_id == c)
+        if members.size == 0:
+            continue
+        pick = np.unique(members[(np.arange(per_cluster) * members.size) // per_cluster])
+        tok.append(pick)
+        clu.append(np.full(pick.size, c))
+    if not tok:
+        return np.zeros(0, np.int32), np.zeros(0, np.int32)
+    return np.concatenate(tok).astype(np.int32), np.concatenate(clu).astype(np.int32)
+
+
 # ---- small helpers for hand-made test inputs (format conversion only) ----
 
 def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
