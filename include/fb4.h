@@ -54,6 +54,7 @@ extern "C" {
 #define FB4_ERR_FORMATBOOK (-4)  /* dialect not strictly ascending from 0 within 0..15 */
 #define FB4_ERR_CUDA (-5)        /* a CUDA runtime call failed; fb4_last_cuda_error() has the code */
 #define FB4_ERR_NO_DEVICE (-6)   /* no usable CUDA device / wrong architecture (needs sm_100) */
+#define FB4_ERR_STATIC_LIMIT (-7) /* more clusters than the built-in scratch of a *_static call holds */
 
 typedef struct fb4_ctx fb4_ctx;
 
@@ -135,6 +136,32 @@ int fb4_quantize_seda(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, in
 int fb4_build_subformatbook(fb4_ctx* ctx, const uint16_t* meta, int64_t T, int64_t C, const int32_t* anchor_token,
                             const int32_t* anchor_cluster, int64_t n_anchor, int32_t n_clusters, uint32_t* counts,
                             uint32_t* cluster_mask, void* stream);
+
+/*
+ * fb4_build_subformatbook without any device allocation (the paper has no counterpart; this is
+ * a packaging of the call above).  It is meant for code that holds a context from start-up but
+ * cannot obtain device memory at the point of the call: a plug-in that gets only the tensors
+ * its host runtime hands it, a serving loop whose memory plan is frozen, a caller whose
+ * allocator is off limits at that moment.  Such a caller has nowhere to get the `counts`
+ * scratch from, so this variant keeps the counts in an array built into the library image.
+ *   - Limit: n_clusters <= FB4_STATIC_MAX_CLUSTERS (1024); more returns FB4_ERR_STATIC_LIMIT and
+ *     launches nothing.  The array (128 KB) occupies every GPU the library is loaded on until
+ *     the process ends.
+ *   - The call itself allocates nothing and frees nothing, on the device or through any
+ *     library.  The first call on a device asks the CUDA runtime once for the array's address
+ *     on that device; make that first call outside any stream capture.
+ *   - All calls on a GPU share the one array, which still holds the previous call's counts:
+ *     each call clears the part it uses (on `stream`) before counting.  Two calls that may run
+ *     at the same time on one GPU (different streams, different contexts, different threads)
+ *     race on it and give wrong masks; order them, or use fb4_build_subformatbook with
+ *     separate scratch.
+ *   - The context's device must be the current device.  Arguments, ignored anchors, tie rules
+ *     and the result are those of fb4_build_subformatbook; the counts are not returned.
+ */
+#define FB4_STATIC_MAX_CLUSTERS 1024
+int fb4_build_subformatbook_static(fb4_ctx* ctx, const uint16_t* meta, int64_t T, int64_t C,
+                                   const int32_t* anchor_token, const int32_t* anchor_cluster, int64_t n_anchor,
+                                   int32_t n_clusters, uint32_t* cluster_mask, void* stream);
 
 /*
  * Salient-token selection for activation decomposition (Sec. 3.3: "one salient

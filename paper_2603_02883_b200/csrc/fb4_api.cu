@@ -399,6 +399,7 @@ const char* fb4_strerror(int code) {
     case FB4_ERR_FORMATBOOK: return "invalid formatbook";
     case FB4_ERR_CUDA: return "CUDA runtime error";
     case FB4_ERR_NO_DEVICE: return "no usable sm_100 CUDA device";
+    case FB4_ERR_STATIC_LIMIT: return "more clusters than the built-in scratch holds (FB4_STATIC_MAX_CLUSTERS)";
     default: return "unknown error";
   }
 }

@@ -17,10 +17,12 @@ from . import build as _build
 
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_ALIGN, ERR_FORMATBOOK, ERR_CUDA, ERR_NO_DEVICE = -1, -2, -3, -4, -5, -6
+ERR_STATIC_LIMIT = -7
+STATIC_MAX_CLUSTERS = 1024
 
 EXPORTS = [
     "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_seda",
-    "fb4_build_subformatbook", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
+    "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
     "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
 
@@ -70,13 +72,15 @@ def lib() -> ctypes.CDLL:
     L.fb4_quantize_seda.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, vp, vp, vp]
     L.fb4_build_subformatbook.argtypes = [vp, vp, i64, i64, vp, vp, i64, i32, vp, vp, vp]
     L.fb4_build_subformatbook.restype = ci
+    L.fb4_build_subformatbook_static.argtypes = [vp, vp, i64, i64, vp, vp, i64, i32, vp, vp]
+    L.fb4_build_subformatbook_static.restype = ci
     L.fb4_select_salient.argtypes = [vp, vp, i64, i32, vp, vp]
     L.fb4_quantize_decomposed.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.fb4_quantize_decomposed_idx.argtypes = [vp, vp, i64, i64, i64, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
     L.fb4_dequantize.argtypes = [vp, vp, vp, i64, i64, vp, i64, vp, vp, vp, ci, vp]
     L.fb4_quantize_host.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp]
     for name in ("fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_seda",
-                 "fb4_build_subformatbook", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx",
+                 "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx",
                  "fb4_dequantize", "fb4_quantize_host", "fb4_last_cuda_error"):
         getattr(L, name).restype = ci
     L.fb4_set_kernel_variant.argtypes = [vp, ci]
@@ -160,6 +164,15 @@ def fb4_build_subformatbook(ctx, meta, T, C, anchor_token, anchor_cluster, n_anc
     _check(lib().fb4_build_subformatbook(ctx, _ptr(meta), T, C, _ptr(anchor_token), _ptr(anchor_cluster), n_anchor,
                                          n_clusters, _ptr(counts), _ptr(cluster_mask), _stream(stream)),
            "fb4_build_subformatbook")
+
+
+def fb4_build_subformatbook_static(ctx, meta, T, C, anchor_token, anchor_cluster, n_anchor, n_clusters, cluster_mask,
+                                   stream=None) -> None:
+    """fb4_build_subformatbook for callers that cannot allocate: no `counts` argument, the library's
+    built-in array is used (at most STATIC_MAX_CLUSTERS clusters; calls on one GPU must not overlap)."""
+    _check(lib().fb4_build_subformatbook_static(ctx, _ptr(meta), T, C, _ptr(anchor_token), _ptr(anchor_cluster),
+                                                n_anchor, n_clusters, _ptr(cluster_mask), _stream(stream)),
+           "fb4_build_subformatbook_static")
 
 
 def fb4_select_salient(ctx, score, T, tile, salient_idx, stream=None) -> None:
