@@ -230,11 +230,11 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
 // Tile index -> (token row, tile column, salient-token slot = row / sal_tile) without a division per
 // tile: advance by a fixed step.
 struct TilePos {
-  int64_t row;
+  int32_t row;         // T < 2^31
   int32_t col;
   int32_t slot, rem;   // row = slot * sal_tile + rem
   __device__ __forceinline__ void advance(const FastParams& p, int32_t tiles_per_row) {
-    row += p.step_rows;
+    row += (int32_t)p.step_rows;
     col += p.step_cols;
     slot += p.step_slots;
     rem += p.step_rem;
@@ -282,12 +282,14 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
   const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytes);
   const uint32_t my_bars = smem_u32(bars + warp * kStages);
   TilePos cur, pre;   // tile being quantized; next tile to request
-  cur.row = gwarp / tpr;
-  cur.col = (int32_t)(gwarp - cur.row * tpr);
-  cur.slot = (int32_t)(cur.row / p.sal_tile);
-  cur.rem = (int32_t)(cur.row - (int64_t)cur.slot * p.sal_tile);
+  cur.row = (int32_t)(gwarp / tpr);
+  cur.col = (int32_t)(gwarp - (int64_t)cur.row * tpr);
+  cur.slot = cur.row / p.sal_tile;
+  cur.rem = cur.row - cur.slot * p.sal_tile;
   pre = cur;
-  int64_t g_pre = gwarp;
+  // this warp's tiles are gwarp, gwarp + wstride, ...: n_mine of them, counted in 32 bits
+  const int32_t n_mine = gwarp < g_end ? (int32_t)((g_end - gwarp + wstride - 1) / wstride) : 0;
+  int32_t it_pre = 0;   // iteration whose tile `pre` points at
   const bool use_seda = SEDA && ex.cluster_id != nullptr;
   const bool use_tile = DECOMP && ex.tile > 0;
   // Per-token extras travel in register queues, fetched as far ahead as the tile data: entry k
@@ -299,15 +301,15 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
   for (int s = 0; s < kStages; ++s) {
     cidq[s] = -1;
     salq[s] = -1;
-    if (g_pre < g_end) {
+    if (it_pre < n_mine) {
       if (lane == 0) {
         mbar_expect_tx(my_bars + 8 * s, kTileBytes);
-        tma_load_tile(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, pre.col * 16, (int)pre.row);
+        tma_load_tile(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, pre.col * 16, pre.row);
       }
       if (use_seda) cidq[s] = ex.cluster_id[pre.row];
-      if (use_tile && pre.slot < ex.n_salient) salq[s] = ex.salient_idx[pre.slot];
+      if (use_tile) salq[s] = ex.salient_idx[pre.slot];   // slot < ceil(T / tile) = n_salient
     }
-    g_pre += wstride;
+    ++it_pre;
     pre.advance(p, tpr);
   }
   uint32_t maskq[2] = {0xffffffffu, 0xffffffffu};
@@ -348,18 +350,18 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
 
   int s = 0;
   uint32_t parity = 0;
-  for (int64_t g = gwarp; g < g_end; g += wstride) {
+  for (int32_t it = 0; it < n_mine; ++it) {
     // ---- fetch the extras of the tiles ahead (pre = the tile kStages steps ahead)
     int32_t cid_new = -1, sal_new = -1;
     uint32_t mask_new = 0xffffffffu;
     if (SEDA) {
       if (use_seda) {
-        if (g_pre < g_end) cid_new = ex.cluster_id[pre.row];
+        if (it_pre < n_mine) cid_new = ex.cluster_id[pre.row];
         if (cidq[2] >= 0) mask_new = ex.cluster_mask[cidq[2]];
       }
     }
     if (DECOMP) {
-      if (use_tile && g_pre < g_end && pre.slot < ex.n_salient) sal_new = ex.salient_idx[pre.slot];
+      if (use_tile && it_pre < n_mine) sal_new = ex.salient_idx[pre.slot];
     }
 
     const uint32_t bar = my_bars + 8 * s;
@@ -373,14 +375,14 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
       int sj = s;
       uint32_t pj = parity;
       for (int j = 1; j < kStages; ++j) {
-        if (g + (int64_t)j * wstride >= g_end) break;
+        if (it + j >= n_mine) break;
         if (++sj == kStages) { sj = 0; pj ^= 1u; }
         uint32_t tries = 0;
         while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
       }
       break;
     }
-    const int64_t row = cur.row;
+    const int64_t row = cur.row;   // 64-bit for the output offsets
     const int64_t blk = (int64_t)cur.col * 32 + lane;
     const bool active = blk < nblk;
 
@@ -456,7 +458,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     if (DECOMP) {
       int64_t srow = -1;
       if (use_tile) {
-        if (salq[0] == (int32_t)row) srow = cur.slot;
+        if (salq[0] == cur.row) srow = cur.row / ex.tile;   // rare: one row in `tile`
       } else {
         int64_t lo = 0, hi = ex.n_salient - 1;
         while (lo <= hi) {
@@ -478,11 +480,11 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     }
     // ---- refill this stage (all lanes have consumed their registers from it)
     __syncwarp();
-    if (lane == 0 && g_pre < g_end) {
+    if (lane == 0 && it_pre < n_mine) {
       mbar_expect_tx(bar, kTileBytes);
-      tma_load_tile(my_ring + s * kTileBytes, &tmap, bar, pre.col * 16, (int)pre.row);
+      tma_load_tile(my_ring + s * kTileBytes, &tmap, bar, pre.col * 16, pre.row);
     }
-    g_pre += wstride;
+    ++it_pre;
     pre.advance(p, tpr);
     cur.advance(p, tpr);
 #pragma unroll
