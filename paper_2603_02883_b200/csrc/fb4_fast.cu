@@ -21,6 +21,7 @@
 #include <cuda.h>
 
 #include <cstring>
+#include <new>
 
 #include "fb4_device.cuh"
 #include "fb4_internal.h"
@@ -38,7 +39,7 @@ constexpr int kPairStride = 1148;    // 36*31 + 32 bytes per dialect; 287 words:
 constexpr int kMaxGroups = 8;        // distinct stage-1 groups the packed tables hold
 constexpr uint32_t kSpinLimit = 1u << 20;   // tries per wait before a warp gives up
 
-// Compact tables in global memory (built at init); the kernel expands them into shared memory.
+// Compact tables, built at init (the part of the shared-memory image that is read as is).
 struct FastTables {
   uint8_t qvalue[32][32];                // [dialect][bin] -> index of the nearest magnitude
   uint64_t qerr64[kMaxGroups][32];       // [group][bin] -> byte j = Qerror of candidate j (pad 31)
@@ -50,7 +51,8 @@ struct FastTables {
 };
 static_assert(sizeof(FastTables) % 16 == 0, "copied with 16-byte accesses");
 
-// Expanded tables in shared memory.
+// The tables as they sit in shared memory.  The image is built once on the host at init, kept in
+// global memory, and copied by every CTA with one bulk asynchronous copy.
 struct SmemTables {
   // [group][bin][lane & 15] -> the 8 candidate errors: each lane of a half-warp has its own
   // 8-byte column, so the 64-bit loads of a warp never conflict
@@ -95,6 +97,11 @@ __device__ __forceinline__ void tma_load_tile(uint32_t dst, const CUtensorMap* m
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(0), "r"(c_outer), "r"(row) : "memory");
+}
+// untiled bulk copy global -> shared, completing on an mbarrier (addresses and size multiples of 16)
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
   uint32_t v;
@@ -245,10 +252,11 @@ struct TilePos {
 
 template <bool SEDA, bool DECOMP>
 __global__ void __launch_bounds__(kWarps * 32, 1)
-fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTables* __restrict__ g_tables,
+fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
                          FastParams p, Fb4RowExtras ex) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  // [ring: kWarps*kStages*2048 B, 1 KB aligned for the 128-byte swizzle][tables][mbarriers]
+  // [ring: kWarps*kStages*2048 B, 1 KB aligned for the 128-byte swizzle][tables][mbarriers: one per
+  // stage of every warp, then one for the tables]
   uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
@@ -273,9 +281,12 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
   }
   const int32_t tpr = (int32_t)p.tiles_per_row;
 
+  const uint32_t table_bar = smem_u32(bars + kWarps * kStages);
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kWarps * kStages; ++i) mbar_init(smem_u32(bars + i), 1);
+    for (int i = 0; i <= kWarps * kStages; ++i) mbar_init(smem_u32(bars + i), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
+    bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
   }
   __syncthreads();
 
@@ -317,25 +328,21 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const FastTab
     if (cidq[0] >= 0) maskq[0] = ex.cluster_mask[cidq[0]];
     if (cidq[1] >= 0) maskq[1] = ex.cluster_mask[cidq[1]];
   }
-  // ---- expand the tables into shared memory (overlaps the first loads)
+  // ---- the tables arrive behind the first tile loads; bounded wait like every other wait here
   {
-    const uint4* src = reinterpret_cast<const uint4*>(g_tables);
-    uint4* dst = reinterpret_cast<uint4*>(&tb->c);
-    for (int i = threadIdx.x; i < (int)(sizeof(FastTables) / 16); i += kWarps * 32) dst[i] = src[i];
-    // every (group, bin) entry replicated into 16 lane-private columns
-    const uint64_t* q64 = reinterpret_cast<const uint64_t*>(g_tables->qerr64);
-    uint64_t* qp = &tb->qerr_private[0][0][0];
-    for (int i = threadIdx.x; i < kMaxGroups * 32 * 16; i += kWarps * 32) qp[i] = q64[i >> 4];
-    if (threadIdx.x < 256) fb4dev::fill_fb_bf16(tb->fb_bf16, &g_tables->fb[0][0], threadIdx.x);
-    // pair tables, one 32-bit word (4 consecutive bin_lo) at a time
-    for (int i = threadIdx.x; i < 32 * 32 * 8; i += kWarps * 32) {
-      const int d = i >> 8, bh = (i >> 3) & 31, bl4 = (i & 7) * 4;
-      const uint32_t lo4 = *reinterpret_cast<const uint32_t*>(&g_tables->qvalue[d][bl4]);
-      const uint32_t hi = g_tables->qvalue[d][bh];
-      *reinterpret_cast<uint32_t*>(&tb->pairlut[d * kPairStride + bh * kPairMul + bl4]) = lo4 | (hi * 0x10101010u);
+    uint32_t spins = 0;
+    bool ready = mbar_try_wait(table_bar, 0u);
+    while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(table_bar, 0u);
+    if (!__all_sync(0xffffffffu, ready)) {
+      if (lane == 0) atomicOr(p.status, 1u);
+      // give this warp's tile loads a bounded chance to land before the CTA's shared memory goes
+      for (int j = 0; j < kStages && j < n_mine; ++j) {
+        uint32_t tries = 0;
+        while (!mbar_try_wait(my_bars + 8 * j, 0u) && ++tries < kSpinLimit) {}
+      }
+      return;
     }
   }
-  __syncthreads();
 
   const uint32_t pair_base = smem_u32(tb->pairlut);
   const uint32_t qerr_base = smem_u32(tb->qerr_private) + ((uint32_t)lane & 15u) * 8u;
@@ -518,12 +525,13 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-constexpr size_t kSmemBytes = 1024 + (size_t)kWarps * kStages * kTileBytes + sizeof(SmemTables) + kWarps * kStages * 8;
+constexpr size_t kSmemBytes =
+    1024 + (size_t)kWarps * kStages * kTileBytes + sizeof(SmemTables) + (kWarps * kStages + 1) * 8;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
-static_assert(sizeof(SmemTables) % 16 == 0, "mbarriers behind the tables stay 8-byte aligned");
+static_assert(sizeof(SmemTables) % 16 == 0, "bulk copy size; mbarriers behind the tables stay 8-byte aligned");
 
 template <bool SEDA, bool DECOMP>
-cudaError_t launch(const CUtensorMap& map, const FastTables* tables, const FastParams& p, const Fb4RowExtras& ex,
+cudaError_t launch(const CUtensorMap& map, const SmemTables* tables, const FastParams& p, const Fb4RowExtras& ex,
                    int grid, cudaStream_t stream) {
   fb4_quantize_fast_kernel<SEDA, DECOMP><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
   return cudaGetLastError();
@@ -570,14 +578,38 @@ bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes
   std::memcpy(ft.qvalue, t.qvalue, sizeof ft.qvalue);
   std::memcpy(ft.qerror, t.qerror, sizeof ft.qerror);
   std::memcpy(ft.fb, t.formatbook, sizeof ft.fb);
-  void* d = nullptr;
-  if (cudaMalloc(&d, sizeof ft) != cudaSuccess) return false;
-  if (cudaMemcpy(d, &ft, sizeof ft, cudaMemcpyHostToDevice) != cudaSuccess) {
-    cudaFree(d);
-    return false;
+  // the image every CTA copies into its shared memory
+  SmemTables* img = new (std::nothrow) SmemTables;
+  if (!img) return false;
+  std::memset(img, 0, sizeof *img);
+  for (int g = 0; g < kMaxGroups; ++g)
+    for (int k = 0; k < 32; ++k)
+      for (int c = 0; c < 16; ++c) img->qerr_private[g][k][c] = ft.qerr64[g][k];
+  for (int d = 0; d < 32; ++d)
+    for (int bh = 0; bh < 32; ++bh)
+      for (int bl = 0; bl < 32; ++bl)
+        img->pairlut[d * kPairStride + bh * kPairMul + bl] = (uint8_t)(t.qvalue[d][bl] | (t.qvalue[d][bh] << 4));
+  for (int d = 0; d < 32; ++d) {
+    uint8_t* row = reinterpret_cast<uint8_t*>(&img->fb_bf16[d]);
+    for (int j = 0; j < 8; ++j) {
+      const float f = (float)t.formatbook[d][j];   // integers 0..15 are exact in bf16
+      uint32_t u;
+      std::memcpy(&u, &f, 4);
+      row[j] = (uint8_t)(u >> 24);
+      row[8 + j] = (uint8_t)(u >> 16);
+    }
   }
+  img->c = ft;
+  void* d = nullptr;
+  bool ok = cudaMalloc(&d, sizeof *img) == cudaSuccess;
+  if (ok && cudaMemcpy(d, img, sizeof *img, cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaFree(d);
+    ok = false;
+  }
+  delete img;
+  if (!ok) return false;
   *d_out = d;
-  *bytes = sizeof ft;
+  *bytes = sizeof(SmemTables);
   return true;
 }
 
@@ -635,7 +667,7 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   p.sal_tile = ex.tile > 0 ? ex.tile : 0x7fffffff;
   p.step_slots = (int32_t)(p.step_rows / p.sal_tile);
   p.step_rem = (int32_t)(p.step_rows % p.sal_tile);
-  const FastTables* tables = static_cast<const FastTables*>(ctx->d_fast_tables);
+  const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
   if (seda && decomp) return launch<true, true>(map, tables, p, ex, grid, stream);
   if (seda) return launch<true, false>(map, tables, p, ex, grid, stream);
   if (decomp) return launch<false, true>(map, tables, p, ex, grid, stream);
