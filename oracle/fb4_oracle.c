@@ -294,6 +294,37 @@ int fb4o_quantize(const uint16_t *x, int64_t T, int64_t C, int64_t ld,
   return 0;
 }
 
+/*
+ * The same quantization for float32 input (a producer handing over its fp32 result, App. D.2
+ * fusion with the preceding operation): every value is taken as it is, nothing is rounded to
+ * bf16 first.  Plain quantization only.
+ */
+int fb4o_quantize_f32(const float *x, int64_t T, int64_t C, int64_t ld, const fb4o_config *cfg,
+                      const uint8_t *F, const uint32_t *stage1_in, uint8_t *codes, uint16_t *meta) {
+  if (!config_ok(cfg, C) || T < 0 || ld < C) return -1;
+  if (!formatbook_ok(F)) return -2;
+  uint32_t stage1[32];
+  if (stage1_in) memcpy(stage1, stage1_in, sizeof stage1); else fb4o_default_stage1(F, stage1);
+  const int B = cfg->block_size;
+  const int64_t nblk = C / B;
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < T; ++t) {
+    for (int64_t blk = 0; blk < nblk; ++blk) {
+      double xv[FB4O_MAXB];
+      uint8_t sg[FB4O_MAXB], code[FB4O_MAXB];
+      for (int i = 0; i < B; ++i) {
+        float f = x[t * ld + blk * B + i];
+        xv[i] = (double)f;
+        sg[i] = (uint8_t)(signbit(f) ? 1 : 0);
+      }
+      int did, e;
+      quantize_block(xv, sg, cfg, F, stage1, 0xffffffffu, code, &did, &e, NULL);
+      store_block(code, B, did, e, codes + t * (C / 2), meta + t * nblk, blk);
+    }
+  }
+  return 0;
+}
+
 static uint16_t f32_to_bf16_rne(float f) {
   uint32_t u;
   memcpy(&u, &f, 4);

@@ -76,6 +76,8 @@ def lib():
         L.fb4o_mse.restype = ctypes.c_double
         L.fb4o_quantize_block_f64.argtypes = [vp, ctypes.POINTER(_Cfg), vp, vp, u32, vp, vp, vp, vp]
         L.fb4o_quantize_block_f64.restype = ctypes.c_int
+        L.fb4o_quantize_f32.argtypes = [vp, i64, i64, i64, ctypes.POINTER(_Cfg), vp, vp, vp, vp]
+        L.fb4o_quantize_f32.restype = ctypes.c_int
         L.fb4o_build_subformatbook.argtypes = [vp, i64, i64, vp, vp, i64, i32, vp, vp, vp]
         L.fb4o_build_subformatbook.restype = ctypes.c_int
         _libs[path] = L
@@ -210,3 +212,17 @@ def build_subformatbook(meta, anchor_token, anchor_cluster, n_clusters: int, for
     if r != 0:
         raise ValueError(f"fb4o_build_subformatbook failed: {r}")
     return out[:n_clusters]
+
+
+def quantize_f32(x, formatbook, cfg: Config = Config(), stage1=None) -> Quantized:
+    """x: float32 [T][C], quantized as it is (no rounding to bf16)."""
+    xv = np.ascontiguousarray(x, dtype=np.float32)
+    T, C = xv.shape
+    codes = np.zeros((T, C // 2), dtype=np.uint8)
+    meta = np.zeros((T, C // cfg.block_size), dtype=np.uint16)
+    ccfg = cfg.c()
+    r = lib().fb4o_quantize_f32(_p(xv), T, C, C, ctypes.byref(ccfg), _p(_c(formatbook, np.uint8)),
+                                _p(_c(stage1, np.uint32)), _p(codes), _p(meta))
+    if r != 0:
+        raise ValueError(f"fb4o_quantize_f32 failed: {r}")
+    return Quantized(codes, meta)

@@ -336,6 +336,38 @@ def pin_seda_choice_inside_mask(seed=4, n=120):
     assert np.array_equal(qa.codes, qb.codes) and np.array_equal(qa.meta, qb.meta)
 
 
+def pin_f32_input(seed=9, n=30):
+    """fp32 input: every block equals the block-wise definition on the exact values (pinned above
+    through quantize_block_f64), values that happen to be bf16 give the bf16 result, and a value
+    between two bf16 neighbours is NOT rounded to bf16 first (its bin comes from the fp32 mantissa)."""
+    rng = np.random.default_rng(seed)
+    for it in range(n):
+        x = (rng.standard_normal((3, 64)) * np.exp2(rng.integers(-30, 30, size=(3, 1)))).astype(np.float32)
+        x[0, 5] = -0.0
+        if it % 5 == 0:
+            x[1, :32] = 0.0
+        q = orc.quantize_f32(x, FB)
+        for t in range(3):
+            for blk in range(2):
+                code, did, e, _ = orc.quantize_block_f64(x[t, blk * 32:blk * 32 + 32].astype(np.float64), FB)
+                assert np.array_equal(unpack_codes(q.codes[t, blk * 16:(blk + 1) * 16]), code)
+                assert int(q.meta[t, blk]) == (e + 124) | (did << 8)
+        bits = synth.f32_to_bf16_bits(x)
+        xb = synth.bf16_bits_to_f32(bits)
+        qa, qb = orc.quantize_f32(xb, FB), orc.quantize(bits, FB)
+        assert np.array_equal(qa.codes, qb.codes) and np.array_equal(qa.meta, qb.meta)
+    # 8.0 sets the scale (e = 3, v = x); 2.4990234375 = 2.5 - 2^-10 lies below the 2|3 boundary of
+    # dialect d0..: as fp32 its bin is floor(4.998) = 4, while its bf16 rounding 2.5 has bin 5
+    x = np.zeros((1, 32), np.float32)
+    x[0, 0], x[0, 1] = 8.0, 2.4990234375
+    q = orc.quantize_f32(x, FB)
+    did = int(q.meta[0, 0]) >> 8
+    codes = unpack_codes(q.codes[0])
+    assert int(FB[did, codes[1] & 7]) == 2
+    qb = orc.quantize(synth.f32_to_bf16_bits(x), FB)
+    assert int(FB[int(qb.meta[0, 0]) >> 8, unpack_codes(qb.codes[0])[1] & 7]) == 3
+
+
 def _meta_with_dialects(rows):
     """meta records (scale byte 124) for rows of dialect ids"""
     return np.array([[124 | (d << 8) for d in r] for r in rows], dtype=np.uint16)
@@ -483,6 +515,6 @@ ALL_PINS = [
     pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
     pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_decomposition,
-    pin_dequantize_formula, pin_mse, pin_subformatbook_hand_counted,
+    pin_dequantize_formula, pin_mse, pin_f32_input, pin_subformatbook_hand_counted,
     pin_subformatbook_one_dialect_per_bucket_and_closed_loop,
 ]

@@ -37,6 +37,10 @@ MUTANTS = {
     "zero_block_exponent": ("e = cfg->exp_min;\n  } else {", "e = 0;\n  } else {"),
     "stage1_bucket_shift": ("int bucket = k / 2 < 8 ? 8 : k / 2;", "int bucket = k / 2 < 9 ? 9 : k / 2;"),
     "mse_not_squared": ("row += d * d;", "row += fabs(d);"),
+    "f32_sign_dropped": ("sg[i] = (uint8_t)(signbit(f) ? 1 : 0);", "sg[i] = 0;"),
+    "f32_rounded_to_bf16_first": ("xv[i] = (double)f;",
+                                  "{ uint32_t u_; memcpy(&u_, &f, 4); u_ = (u_ + 0x7fffu + ((u_ >> 16) & 1u)) & 0xffff0000u; "
+                                  "float g_; memcpy(&g_, &u_, 4); xv[i] = (double)g_; }"),
     "subformatbook_ties_to_highest": ("if (best < 0 || count[d] > count[best]) best = d;",
                                       "if (best < 0 || count[d] >= count[best]) best = d;"),
     "subformatbook_least_frequent": ("if (best < 0 || count[d] > count[best]) best = d;",
