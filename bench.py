@@ -200,6 +200,10 @@ class Ops:
         meta = self.buf("meta", (T, C // B), torch.int16)
         if name == "plain":
             return (lambda: fb4.fb4_quantize(q.ctx, x, T, C, C, codes, meta)), algorithmic_bytes(T, C)
+        if name == "plain_f32":
+            xf = self.buf("x32", (T, C), torch.float32)
+            xf.copy_(x)
+            return (lambda: fb4.fb4_quantize_f32(q.ctx, xf, T, C, C, codes, meta)), T * C * 4.5 + T * (C // B) * 2
         ex = self.extras()
         n_sal, tile, cid, cmask, score = ex["n_sal"], ex["tile"], ex["cid"], ex["cmask"], ex["score"]
         rc = self.buf("rc", (n_sal, C // 2), torch.uint8)
@@ -239,7 +243,7 @@ class Ops:
         raise KeyError(name)
 
 
-OP_NAMES = ["plain", "seda", "decomposed", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
+OP_NAMES = ["plain", "plain_f32", "seda", "decomposed", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
             "dequantize_bf16_plain", "dequantize_bf16_decomposed"]
 
 
@@ -363,6 +367,8 @@ def run_variants(ops, args, torch, fb4, synth, peak):
                      "kernel_variant": q.last_variant if not name.startswith("dequantize") else "decode"}
         if name == "dequantize_f32_decomposed":
             ops.drop("out32")
+        if name == "plain_f32":
+            ops.drop("x32")
     ops.drop("out16")
     if w.name != "c2":
         w2 = synth.workloads()["c2"]

@@ -105,6 +105,16 @@ int fb4_quantize(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t
                  uint16_t* meta, void* stream);
 
 /*
+ * fb4_quantize for float32 input (App. D.2: "Quantization is fused with the preceding operation
+ * (e.g., GeLU, LayerNorm) where possible" -- a producer that still holds its result in fp32 hands
+ * it over without rounding it to bf16 first).  The values are quantized as they are: the block
+ * exponent is the fp32 exponent of the largest magnitude, bins come from the full fp32 mantissa.
+ *   x : device float32 [T][ld_elems], finite; 16-byte aligned, ld_elems a multiple of 4
+ */
+int fb4_quantize_f32(fb4_ctx* ctx, const float* x, int64_t T, int64_t C, int64_t ld_elems, uint8_t* codes,
+                     uint16_t* meta, void* stream);
+
+/*
  * SeDA-constrained quantization (Sec. 3.4): token t may only use the dialects in
  * cluster_mask[cluster_id[t]] (its cluster's sub-formatbook); cluster_id[t] == -1
  * means unconstrained.  Stage 1 is intersected with the mask; if the intersection

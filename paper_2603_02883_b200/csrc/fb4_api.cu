@@ -97,7 +97,7 @@ int run_quantize(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, 
     e = fb4_launch_quantize_fast(ctx, x, T, C, ld, ex, codes, meta, stream);
     ctx->last_variant = "fast";
   } else {
-    e = fb4_launch_quantize_generic(ctx, x, T, C, ld, ex, codes, meta, stream);
+    e = fb4_launch_quantize_generic(ctx, x, 0, T, C, ld, ex, codes, meta, stream);
     ctx->last_variant = "generic";
   }
   if (e != cudaSuccess) return fb4_set_cuda_error(e);
@@ -213,6 +213,29 @@ int fb4_quantize(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, 
   if (rc != FB4_OK) return rc;
   Fb4RowExtras ex{};
   return run_quantize(ctx, x, T, C, ld, ex, codes, meta, static_cast<cudaStream_t>(stream));
+}
+
+int fb4_quantize_f32(fb4_ctx* ctx, const float* x, int64_t T, int64_t C, int64_t ld, uint8_t* codes, uint16_t* meta,
+                     void* stream) {
+  if (!ctx) return FB4_ERR_INVALID_ARG;
+  if (T < 0 || C <= 0 || C % ctx->cfg.block_size != 0 || ld < C) return FB4_ERR_SHAPE;
+  if (T == 0) return FB4_OK;
+  if (!x || !codes || !meta) return FB4_ERR_INVALID_ARG;
+  if (T > 0x7fffffffLL) return FB4_ERR_SHAPE;
+  if (!aligned16(x) || !aligned16(codes) || !aligned16(meta) || (ld & 3)) return FB4_ERR_ALIGN;
+  cudaError_t e;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!ctx->force_generic && fb4_fast_f32_eligible(ctx, x, T, C, ld)) {
+    e = fb4_launch_quantize_fast_f32(ctx, x, T, C, ld, codes, meta, st);
+    ctx->last_variant = "fast";
+  } else {
+    Fb4RowExtras ex{};
+    e = fb4_launch_quantize_generic(ctx, x, 1, T, C, ld, ex, codes, meta, st);
+    ctx->last_variant = "generic";
+  }
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
+  ctx->launches += 1;
+  return FB4_OK;
 }
 
 int fb4_quantize_seda(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const int32_t* cluster_id,

@@ -175,6 +175,43 @@ __device__ __forceinline__ int choose_dialect(const float (&gm)[8], float sG, ui
   return select_general(cand, gb, tb);
 }
 
+// One block given as 32 fp32 magnitudes (bit patterns, sign cleared) plus the sign bits already at
+// bit 3 of every nibble of the four code words: scale, group maxima, dialect selection and LUT
+// quantization with the same tables as the bf16 path.  Writes the code words and the metadata record.
+template <bool SEDA>
+__device__ __forceinline__ void quantize_f32_block(const uint32_t (&a)[32], const uint32_t (&sg)[4], uint32_t allowed,
+                                                   const SmemTables* tb, uint32_t qerr_lane, uint32_t pair_base,
+                                                   uint32_t* rcw, uint32_t* rmeta) {
+  uint32_t gmx[8];
+  uint32_t amax = 0;
+#pragma unroll
+  for (int g = 0; g < 8; ++g) {
+    gmx[g] = max(max(a[4 * g], a[4 * g + 1]), max(a[4 * g + 2], a[4 * g + 3]));
+    amax = max(amax, gmx[g]);
+  }
+  const uint32_t Er = max(amax >> 23, 3u);
+  const float s2 = __uint_as_float((257u - Er) << 23);   // 2^(3-e)
+  const float sG = s2 * 0x1p-21f, sH = s2 * 0x1p-25f, sL = s2 * 0x1p-5f;
+  const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax), sG, 2.0f)) & 31u;
+  float gm[8];
+#pragma unroll
+  for (int g = 0; g < 8; ++g) gm[g] = __uint_as_float(gmx[g]);
+  const int rdid = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
+  const float magic_lo = __uint_as_float(0x48000000u + pair_base + (uint32_t)rdid * kPairStride);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    uint32_t idx = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j + 1]), sH, 0.125f));
+      const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j]), sL, magic_lo));
+      idx |= lds_u8(th * (uint32_t)kPairMul + tl) << (8 * j);
+    }
+    rcw[q] = idx | sg[q];
+  }
+  *rmeta = (Er - 3u) | ((uint32_t)rdid << 8);
+}
+
 // Residual pass of one block (Sec. 3.3): Delta = x - Q(x) in fp32 (exact), quantized again with
 // the same tables as the main pass; the fp32 magnitudes take the place of the bf16 ones.
 // w = the 16 input registers (2 bf16 each), cw = the block's 4 code words, Ec = biased exponent.
@@ -204,34 +241,7 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
     }
     sg[q] = sq;
   }
-  uint32_t gmx[8];
-  uint32_t amax = 0;
-#pragma unroll
-  for (int g = 0; g < 8; ++g) {
-    gmx[g] = max(max(a[4 * g], a[4 * g + 1]), max(a[4 * g + 2], a[4 * g + 3]));
-    amax = max(amax, gmx[g]);
-  }
-  const uint32_t Er = max(amax >> 23, 3u);
-  const float s2 = __uint_as_float((257u - Er) << 23);   // 2^(3-e)
-  const float sG = s2 * 0x1p-21f, sH = s2 * 0x1p-25f, sL = s2 * 0x1p-5f;
-  const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax), sG, 2.0f)) & 31u;
-  float gm[8];
-#pragma unroll
-  for (int g = 0; g < 8; ++g) gm[g] = __uint_as_float(gmx[g]);
-  const int rdid = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
-  const float magic_lo = __uint_as_float(0x48000000u + pair_base + (uint32_t)rdid * kPairStride);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    uint32_t idx = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j + 1]), sH, 0.125f));
-      const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j]), sL, magic_lo));
-      idx |= lds_u8(th * (uint32_t)kPairMul + tl) << (8 * j);
-    }
-    rcw[q] = idx | sg[q];
-  }
-  *rmeta = (Er - 3u) | ((uint32_t)rdid << 8);
+  quantize_f32_block<SEDA>(a, sg, allowed, tb, qerr_lane, pair_base, rcw, rmeta);
 }
 
 // Tile index -> (token row, tile column, salient-token slot = row / sal_tile) without a division per
@@ -507,6 +517,134 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// fp32 input (the hook for a producer that still holds its result in fp32): same ring and tables,
+// 8 warps per CTA, tiles of 1024 channels = 4 KB (view [T][C/32][32 floats], box 1 x 32 x 32,
+// 128-byte swizzle: row r of a stage is block r).  Lane i reads its block with eight conflict-free
+// 16-byte shared loads and quantizes it with quantize_f32_block.
+constexpr int kWarpsF32 = 8;
+constexpr int kTileBytesF32 = 4096;
+
+__global__ void __launch_bounds__(kWarpsF32 * 32, 1)
+fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
+                        FastParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarpsF32 * kStages * kTileBytesF32);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t gwarp = (int64_t)blockIdx.x * kWarpsF32 + warp;
+  const int64_t wstride = (int64_t)gridDim.x * kWarpsF32;
+  const int32_t tpr = (int32_t)p.tiles_per_row;
+
+  const uint32_t table_bar = smem_u32(bars + kWarpsF32 * kStages);
+  if (threadIdx.x == 0) {
+    for (int i = 0; i <= kWarpsF32 * kStages; ++i) mbar_init(smem_u32(bars + i), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
+    bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+  }
+  __syncthreads();
+
+  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytesF32);
+  const uint32_t my_bars = smem_u32(bars + warp * kStages);
+  TilePos cur, pre;
+  cur.row = (int32_t)(gwarp / tpr);
+  cur.col = (int32_t)(gwarp - (int64_t)cur.row * tpr);
+  cur.slot = cur.rem = 0;
+  pre = cur;
+  const int32_t n_mine = gwarp < p.n_tiles ? (int32_t)((p.n_tiles - gwarp + wstride - 1) / wstride) : 0;
+  int32_t it_pre = 0;
+#pragma unroll
+  for (int s = 0; s < kStages; ++s) {
+    if (it_pre < n_mine && lane == 0) {
+      mbar_expect_tx(my_bars + 8 * s, kTileBytesF32);
+      tma_load_tile(my_ring + s * kTileBytesF32, &tmap, my_bars + 8 * s, pre.col * 32, pre.row);
+    }
+    ++it_pre;
+    pre.advance(p, tpr);
+  }
+  {
+    uint32_t spins = 0;
+    bool ready = mbar_try_wait(table_bar, 0u);
+    while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(table_bar, 0u);
+    if (!__all_sync(0xffffffffu, ready)) {
+      if (lane == 0) atomicOr(p.status, 1u);
+      for (int j = 0; j < kStages && j < n_mine; ++j) {
+        uint32_t tries = 0;
+        while (!mbar_try_wait(my_bars + 8 * j, 0u) && ++tries < kSpinLimit) {}
+      }
+      return;
+    }
+  }
+  const uint32_t pair_base = smem_u32(tb->pairlut);
+  const uint32_t qerr_base = smem_u32(tb->qerr_private) + ((uint32_t)lane & 15u) * 8u;
+  uint32_t chunk_off[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) chunk_off[j] = (uint32_t)lane * 128u + ((((uint32_t)j) ^ ((uint32_t)lane & 7u)) << 4);
+  const int64_t nblk = p.C >> 5;
+  const int64_t code_row_bytes = p.C >> 1;
+
+  int s = 0;
+  uint32_t parity = 0;
+  for (int32_t it = 0; it < n_mine; ++it) {
+    const uint32_t bar = my_bars + 8 * s;
+    uint32_t spins = 0;
+    bool ready = mbar_try_wait(bar, parity);
+    while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(bar, parity);
+    if (!__all_sync(0xffffffffu, ready)) {
+      if (lane == 0) atomicOr(p.status, 1u);
+      int sj = s;
+      uint32_t pj = parity;
+      for (int j = 1; j < kStages; ++j) {
+        if (it + j >= n_mine) break;
+        if (++sj == kStages) { sj = 0; pj ^= 1u; }
+        uint32_t tries = 0;
+        while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
+      }
+      break;
+    }
+    const int64_t row = cur.row;
+    const int64_t blk = (int64_t)cur.col * 32 + lane;
+    uint32_t a[32], sg[4];
+    {
+      const uint32_t base = my_ring + s * kTileBytesF32;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 v0 = lds_v4(base + chunk_off[2 * q]), v1 = lds_v4(base + chunk_off[2 * q + 1]);
+        const uint32_t x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+        uint32_t sq = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          a[8 * q + i] = x[i] & 0x7fffffffu;
+          // sign bit 31 -> bit 4i+3 of the code word
+          sq |= (4 * i + 3 == 31) ? (x[i] & 0x80000000u) : ((x[i] >> (28 - 4 * i)) & (8u << (4 * i)));
+        }
+        sg[q] = sq;
+      }
+    }
+    uint32_t cw[4], m;
+    quantize_f32_block<false>(a, sg, 0xffffffffu, tb, qerr_base, pair_base, cw, &m);
+    if (blk < nblk) {
+      *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      p.meta[row * nblk + blk] = (uint16_t)m;
+    }
+    __syncwarp();
+    if (lane == 0 && it_pre < n_mine) {
+      mbar_expect_tx(bar, kTileBytesF32);
+      tma_load_tile(my_ring + s * kTileBytesF32, &tmap, bar, pre.col * 32, pre.row);
+    }
+    ++it_pre;
+    pre.advance(p, tpr);
+    cur.advance(p, tpr);
+    if (++s == kStages) { s = 0; parity ^= 1u; }
+  }
+}
+
+constexpr size_t kSmemBytesF32 =
+    1024 + (size_t)kWarpsF32 * kStages * kTileBytesF32 + sizeof(SmemTables) + (kWarpsF32 * kStages + 1) * 8;
+static_assert(kSmemBytesF32 <= 227 * 1024, "shared memory budget of one CTA");
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -626,6 +764,9 @@ cudaError_t fb4_fast_prepare_device() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kSmemBytes);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kSmemBytesF32);
   return e;
 }
 
@@ -672,4 +813,46 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   if (seda) return launch<true, false>(map, tables, p, ex, grid, stream);
   if (decomp) return launch<false, true>(map, tables, p, ex, grid, stream);
   return launch<false, false>(map, tables, p, ex, grid, stream);
+}
+
+bool fb4_fast_f32_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {
+  const fb4_config& c = ctx->cfg;
+  if (!ctx->fast_ok || !ctx->d_fast_tables) return false;
+  if (c.block_size != 32 || c.num_groups != 8 || c.select_mode != 0 || c.exp_min != -124 || c.exp_max != 127)
+    return false;
+  if (C % 32 != 0 || (ld & 3) || (reinterpret_cast<uintptr_t>(x) & 15)) return false;
+  if (T > 0x7fffffffLL || C / 32 > 0x7fffffffLL) return false;
+  return encode_tiled_fn() != nullptr;
+}
+
+cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
+                                         uint8_t* codes, uint16_t* meta, cudaStream_t stream) {
+  CUtensorMap map;
+  const cuuint64_t dims[3] = {32, (cuuint64_t)(C / 32), (cuuint64_t)T};
+  const cuuint64_t strides[2] = {128, (cuuint64_t)ld * 4};
+  const cuuint32_t box[3] = {32, 32, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  const CUresult r = encode_tiled_fn()(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(x), dims, strides,
+                                       box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  FastParams p{};
+  p.T = T;
+  p.C = C;
+  p.tiles_per_row = (C + 1023) / 1024;
+  p.n_tiles = T * p.tiles_per_row;
+  p.codes = codes;
+  p.meta = meta;
+  p.status = ctx->d_status;
+  const int64_t want = (p.n_tiles + kWarpsF32 - 1) / kWarpsF32;
+  const int grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
+  const int64_t wstride = (int64_t)grid * kWarpsF32;
+  p.step_rows = wstride / p.tiles_per_row;
+  p.step_cols = (int32_t)(wstride % p.tiles_per_row);
+  p.sal_tile = 0x7fffffff;
+  p.step_slots = 0;
+  p.step_rem = 0;
+  fb4_quantize_f32_kernel<<<grid, kWarpsF32 * 32, kSmemBytesF32, stream>>>(
+      map, static_cast<const SmemTables*>(ctx->d_fast_tables), p);
+  return cudaGetLastError();
 }

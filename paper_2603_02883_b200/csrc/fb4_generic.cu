@@ -114,9 +114,9 @@ __device__ __forceinline__ int64_t salient_row(const Fb4RowExtras& ex, int64_t t
   return -1;
 }
 
-template <int B, int GS>
+template <int B, int GS, bool F32>
 __global__ void __launch_bounds__(128)
-fb4_quantize_generic_kernel(const uint16_t* __restrict__ x, int64_t T, int64_t C, int64_t ld,
+fb4_quantize_generic_kernel(const void* __restrict__ xin, int64_t T, int64_t C, int64_t ld,
                             const Fb4DeviceTables* __restrict__ tables, GenericParams p, Fb4RowExtras ex,
                             uint8_t* __restrict__ codes, uint16_t* __restrict__ meta) {
   __shared__ SmemTables tb;
@@ -132,11 +132,24 @@ fb4_quantize_generic_kernel(const uint16_t* __restrict__ x, int64_t T, int64_t C
   for (int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; id < total; id += stride) {
     const int64_t t = id / nblk;
     const int64_t blk = id - t * nblk;
-    const uint4* src = reinterpret_cast<const uint4*>(x + t * ld + blk * B);
     float xs[B], ax[B];
     uint32_t sgn = 0;
+    if (F32) {   // fp32 input: the values as they are
+      const uint4* src = reinterpret_cast<const uint4*>(static_cast<const float*>(xin) + t * ld + blk * B);
 #pragma unroll
-    for (int q = 0; q < B / 8; ++q) {
+      for (int q = 0; q < B / 4; ++q) {
+        const uint4 v = src[q];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          xs[q * 4 + j] = __uint_as_float(w[j]);
+          sgn |= (w[j] >> 31) << (q * 4 + j);
+        }
+      }
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(xin) + t * ld + blk * B);
+#pragma unroll
+    for (int q = 0; q < (F32 ? 0 : B / 8); ++q) {
       const uint4 v = src[q];
       const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -184,8 +197,8 @@ fb4_quantize_generic_kernel(const uint16_t* __restrict__ x, int64_t T, int64_t C
 
 }  // namespace
 
-cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
-                                        const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
+cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x_is_f32, int64_t T, int64_t C,
+                                        int64_t ld, const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
                                         cudaStream_t stream) {
   const int B = (int)ctx->cfg.block_size, G = (int)ctx->cfg.num_groups;
   const int64_t total = T * (C / B);
@@ -195,9 +208,15 @@ cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int64
   int64_t want = (total + threads - 1) / threads;
   const int64_t cap = (int64_t)ctx->sm_count * 16;
   const int grid = (int)(want < cap ? want : cap);
-  const uint16_t* xp = static_cast<const uint16_t*>(x);
-#define FB4_LAUNCH(BB, GSZ) \
-  fb4_quantize_generic_kernel<BB, GSZ><<<grid, threads, 0, stream>>>(xp, T, C, ld, ctx->d_tables, p, ex, codes, meta)
+#define FB4_LAUNCH(BB, GSZ)                                                                                          \
+  do {                                                                                                               \
+    if (x_is_f32)                                                                                                    \
+      fb4_quantize_generic_kernel<BB, GSZ, true><<<grid, threads, 0, stream>>>(x, T, C, ld, ctx->d_tables, p, ex,    \
+                                                                               codes, meta);                         \
+    else                                                                                                             \
+      fb4_quantize_generic_kernel<BB, GSZ, false><<<grid, threads, 0, stream>>>(x, T, C, ld, ctx->d_tables, p, ex,   \
+                                                                                codes, meta);                        \
+  } while (0)
   if (B == 32 && G == 8) FB4_LAUNCH(32, 4);
   else if (B == 32 && G == 32) FB4_LAUNCH(32, 1);
   else if (B == 16 && G == 8) FB4_LAUNCH(16, 2);

@@ -56,9 +56,13 @@ bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, 
 cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
                                      const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta, cudaStream_t stream);
 
+bool fb4_fast_f32_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld);
+cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
+                                         uint8_t* codes, uint16_t* meta, cudaStream_t stream);
+
 // generic kernels (any supported config)
-cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
-                                        const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
+cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x_is_f32, int64_t T, int64_t C,
+                                        int64_t ld, const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
                                         cudaStream_t stream);
 cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T,
                                   int64_t C, const int32_t* salient_idx, int64_t n_salient,

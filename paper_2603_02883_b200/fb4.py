@@ -21,7 +21,7 @@ ERR_STATIC_LIMIT = -7
 STATIC_MAX_CLUSTERS = 1024
 
 EXPORTS = [
-    "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_seda",
+    "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
     "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
     "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
     L.fb4_destroy.argtypes = [vp]
     L.fb4_get_tables.argtypes = [vp, vp, vp, vp, vp]
     L.fb4_quantize.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
+    L.fb4_quantize_f32.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
+    L.fb4_quantize_f32.restype = ci
     L.fb4_quantize_seda.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, vp, vp, vp]
     L.fb4_build_subformatbook.argtypes = [vp, vp, i64, i64, vp, vp, i64, i32, vp, vp, vp]
     L.fb4_build_subformatbook.restype = ci
@@ -79,7 +81,7 @@ def lib() -> ctypes.CDLL:
     L.fb4_quantize_decomposed_idx.argtypes = [vp, vp, i64, i64, i64, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
     L.fb4_dequantize.argtypes = [vp, vp, vp, i64, i64, vp, i64, vp, vp, vp, ci, vp]
     L.fb4_quantize_host.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp]
-    for name in ("fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_seda",
+    for name in ("fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
                  "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx",
                  "fb4_dequantize", "fb4_quantize_host", "fb4_last_cuda_error"):
         getattr(L, name).restype = ci
@@ -152,6 +154,11 @@ def fb4_get_tables(ctx):
 
 def fb4_quantize(ctx, x, T, C, ld_elems, codes, meta, stream=None) -> None:
     _check(lib().fb4_quantize(ctx, _ptr(x), T, C, ld_elems, _ptr(codes), _ptr(meta), _stream(stream)), "fb4_quantize")
+
+
+def fb4_quantize_f32(ctx, x, T, C, ld_elems, codes, meta, stream=None) -> None:
+    _check(lib().fb4_quantize_f32(ctx, _ptr(x), T, C, ld_elems, _ptr(codes), _ptr(meta), _stream(stream)),
+           "fb4_quantize_f32")
 
 
 def fb4_quantize_seda(ctx, x, T, C, ld_elems, cluster_id, cluster_mask, n_clusters, codes, meta, stream=None) -> None:
@@ -270,13 +277,16 @@ class Fb4:
 
     @staticmethod
     def _shape(x):
-        assert x.dtype == torch.bfloat16 and x.dim() == 2 and x.stride(1) == 1 and x.is_cuda
+        assert x.dtype in (torch.bfloat16, torch.float32) and x.dim() == 2 and x.stride(1) == 1 and x.is_cuda
         return x.shape[0], x.shape[1], (x.stride(0) if x.shape[0] > 1 else x.shape[1])
 
     def quantize(self, x, cluster_id=None, cluster_mask=None) -> Quantized:
         T, C, ld = self._shape(x)
         codes, meta = self._outs(T, C)
-        if cluster_id is None:
+        if x.dtype == torch.float32:
+            assert cluster_id is None, "fp32 input: plain quantization only"
+            fb4_quantize_f32(self.ctx, x, T, C, ld, codes, meta)
+        elif cluster_id is None:
             fb4_quantize(self.ctx, x, T, C, ld, codes, meta)
         else:
             fb4_quantize_seda(self.ctx, x, T, C, ld, cluster_id, cluster_mask, cluster_mask.numel(), codes, meta)
@@ -284,6 +294,7 @@ class Fb4:
 
     def quantize_decomposed(self, x, score=None, tile: int = 20, salient_idx=None, cluster_id=None,
                             cluster_mask=None) -> Quantized:
+        assert x.dtype == torch.bfloat16
         T, C, ld = self._shape(x)
         ncl = 0 if cluster_mask is None else cluster_mask.numel()
         if salient_idx is None:

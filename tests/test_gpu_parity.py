@@ -208,3 +208,39 @@ def test_host_buffer_entry_point(q32):
     dm = torch.empty((w.T, w.C // 32), dtype=torch.int16, device="cuda")
     fb4.fb4_quantize_host(q32.ctx, xh, w.T, w.C, dx, dc, dm, ch, mh)
     assert np.array_equal(ch.numpy(), ref.codes) and np.array_equal(mh.numpy().view(np.uint16), ref.meta)
+
+
+def f32_inputs():
+    rng = np.random.default_rng(23)
+    yield "edge", synth.bf16_bits_to_f32(edge_blocks())           # bf16-valued fp32, all the edge cases
+    x = (rng.standard_normal((67, 1024 + 96)) * np.exp2(rng.integers(-40, 40, size=(67, 1)))).astype(np.float32)
+    x[3, 40:80] = 0.0
+    x[5, :] = np.float32(1e-41)                                    # fp32 subnormals
+    x[6, 7] = np.float32(3.4e38)
+    x[7, :64] = np.nextafter(np.float32(2.5), np.float32(0), dtype=np.float32)   # just below a rounding boundary
+    x[7, 0] = 8.0
+    yield "random", x
+    yield "student-t", synth.bf16_bits_to_f32(heavy(130, 2048, 31)) * np.float32(1.0009765625)   # not bf16 values
+
+
+@pytest.mark.parametrize("cfg", [dict(), dict(block_size=16), dict(select_mode=1), dict(exp_min=-15, exp_max=16)],
+                         ids=["default", "b16", "select-all", "exp5"])
+def test_f32_input(cfg):
+    q = fb4.Fb4(**cfg)
+    ocfg = orc.Config(**cfg)
+    for name, x in f32_inputs():
+        ref = orc.quantize_f32(x, FB, ocfg)
+        xd = torch.from_numpy(x).cuda()
+        for variant in (0, 1):
+            q.set_kernel_variant(variant)
+            got = q.quantize(xd)
+            assert_same_quantized(got, ref, f"f32 {name} {cfg} variant {variant}")
+        if not cfg:
+            q.set_kernel_variant(0)
+            q.quantize(xd)
+            assert q.last_variant == "fast"
+            # strided rows
+            view = xd[:, :64]
+            assert_same_quantized(q.quantize(view), orc.quantize_f32(np.ascontiguousarray(x[:, :64]), FB), "f32 strided")
+    assert q.device_status == 0
+    q.close()
