@@ -21,6 +21,9 @@
  *   Sec. 3.3  activation decomposition: residual Delta = Act - Q(Act) of the
  *             salient tokens is quantized again; one salient token per tile,
  *             the highest-scoring one.
+ *   App. D.2  MXFP8 view: the integer magnitudes 0..15 are exact in FP8 e4m3 and the
+ *             power-of-two block scale is an E8M0 scale, so a quantized tensor can be
+ *             re-expressed as an MXFP8 operand without any rounding.
  *   Sec. 3.4  SeDA: the candidate set of a token is its cluster's sub-formatbook; a
  *             sub-formatbook is built by counting, over a cluster's anchor tokens, how
  *             often each dialect was chosen in each dynamic-range bucket and keeping
@@ -436,6 +439,61 @@ int fb4o_build_subformatbook(const uint16_t *meta, int64_t T, int64_t nblk,
       if (best >= 0) mask |= 1u << best;
     }
     cluster_mask[c] = mask;
+  }
+  return 0;
+}
+
+/*
+ * MXFP8 view of a quantized tensor (App. D.2: FB4's "normalized integer values (0-15) are exactly
+ * representable in FP8 e4m3" and its scaling is power-of-two, hence "directly compatible with
+ * MXFP8 GEMM").  Every element becomes the e4m3 byte of its signed integer magnitude
+ * (sign, 4-bit exponent with bias 7, 3-bit mantissa), every 32-element block gets the E8M0 byte
+ * of its element scale 2^(e-3), which is the block's scale byte itself (E8M0 of 2^k is k+127).
+ *
+ * Scale layouts: 0 = row-major [T][C/32].  1 = tiles of 128 rows x 4 scale columns, 512 bytes
+ * each, the tiles of a row band stored one after the other (column tiles contiguous); inside a
+ * tile the scale of (row r, column c) sits at (r mod 32)*16 + (r div 32)*4 + c.  This is the
+ * arrangement block-scaled tensor-core GEMMs on Blackwell read their scale factors in; rows are
+ * padded to a multiple of 128 and scale columns to a multiple of 4, padding entries hold 0x7f
+ * (scale 1).
+ */
+int64_t fb4o_mxfp8_scale_offset(int64_t row, int64_t col, int64_t n_col, int layout) {
+  if (layout == 0) return row * n_col + col;
+  int64_t col_tiles = (n_col + 3) / 4;
+  int64_t tile = (row / 128) * col_tiles + col / 4;
+  int64_t r = row % 128;
+  return tile * 512 + (r % 32) * 16 + (r / 32) * 4 + col % 4;
+}
+
+int64_t fb4o_mxfp8_scale_bytes(int64_t T, int64_t C, int layout) {
+  int64_t n_col = C / 32;
+  if (layout == 0) return T * n_col;
+  return ((T + 127) / 128) * ((n_col + 3) / 4) * 512;
+}
+
+static uint8_t e4m3_of_small_int(int m) {   /* m in 0..15, exact */
+  if (m == 0) return 0;
+  int ex = 0;
+  while ((m >> (ex + 1)) != 0) ++ex;               /* floor(log2 m) */
+  int frac = m - (1 << ex);                          /* m = 2^ex * (1 + frac / 2^ex) */
+  int mant = ex <= 3 ? frac << (3 - ex) : frac >> (ex - 3);
+  return (uint8_t)(((ex + 7) << 3) | mant);
+}
+
+int fb4o_to_mxfp8(const uint8_t *codes, const uint16_t *meta, int64_t T, int64_t C, const uint8_t *F,
+                  uint8_t *e4m3, uint8_t *scales, int layout) {
+  if (C <= 0 || C % 32 || T < 0 || !formatbook_ok(F) || (layout != 0 && layout != 1)) return -1;
+  const int64_t nblk = C / 32;
+  memset(scales, 0x7f, (size_t)fb4o_mxfp8_scale_bytes(T, C, layout));
+  for (int64_t t = 0; t < T; ++t) {
+    for (int64_t c = 0; c < C; ++c) {
+      uint16_t m = meta[t * nblk + c / 32];
+      uint8_t byte = codes[t * (C / 2) + c / 2];
+      uint8_t code = (c & 1) ? (byte >> 4) : (byte & 15);
+      e4m3[t * C + c] = (uint8_t)(e4m3_of_small_int(F[(m >> 8) * 8 + (code & 7)]) | ((code & 8) << 4));
+    }
+    for (int64_t b = 0; b < nblk; ++b)
+      scales[fb4o_mxfp8_scale_offset(t, b, nblk, layout)] = (uint8_t)(meta[t * nblk + b] & 0xff);
   }
   return 0;
 }

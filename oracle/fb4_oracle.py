@@ -78,6 +78,12 @@ def lib():
         L.fb4o_quantize_block_f64.restype = ctypes.c_int
         L.fb4o_quantize_f32.argtypes = [vp, i64, i64, i64, ctypes.POINTER(_Cfg), vp, vp, vp, vp]
         L.fb4o_quantize_f32.restype = ctypes.c_int
+        L.fb4o_to_mxfp8.argtypes = [vp, vp, i64, i64, vp, vp, vp, ctypes.c_int]
+        L.fb4o_to_mxfp8.restype = ctypes.c_int
+        L.fb4o_mxfp8_scale_offset.argtypes = [i64, i64, i64, ctypes.c_int]
+        L.fb4o_mxfp8_scale_offset.restype = i64
+        L.fb4o_mxfp8_scale_bytes.argtypes = [i64, i64, ctypes.c_int]
+        L.fb4o_mxfp8_scale_bytes.restype = i64
         L.fb4o_build_subformatbook.argtypes = [vp, i64, i64, vp, vp, i64, i32, vp, vp, vp]
         L.fb4o_build_subformatbook.restype = ctypes.c_int
         _libs[path] = L
@@ -226,3 +232,21 @@ def quantize_f32(x, formatbook, cfg: Config = Config(), stage1=None) -> Quantize
     if r != 0:
         raise ValueError(f"fb4o_quantize_f32 failed: {r}")
     return Quantized(codes, meta)
+
+
+def mxfp8_scale_offset(row: int, col: int, n_col: int, layout: int) -> int:
+    return int(lib().fb4o_mxfp8_scale_offset(row, col, n_col, layout))
+
+
+def to_mxfp8(q: Quantized, formatbook, layout: int = 0):
+    """(e4m3 bytes uint8 [T][C], E8M0 scale bytes in the given layout) of a block-32 quantized tensor."""
+    T, C2 = q.codes.shape
+    C = C2 * 2
+    out = np.zeros((T, C), dtype=np.uint8)
+    n = int(lib().fb4o_mxfp8_scale_bytes(T, C, layout))
+    sc = np.zeros(max(n, 1), dtype=np.uint8)
+    r = lib().fb4o_to_mxfp8(_p(_c(q.codes, np.uint8)), _p(_c(q.meta, np.uint16)), T, C, _p(_c(formatbook, np.uint8)),
+                            _p(out), _p(sc), layout)
+    if r != 0:
+        raise ValueError(f"fb4o_to_mxfp8 failed: {r}")
+    return out, sc[:n]

@@ -368,6 +368,61 @@ def pin_f32_input(seed=9, n=30):
     assert int(FB[int(qb.meta[0, 0]) >> 8, unpack_codes(qb.codes[0])[1] & 7]) == 3
 
 
+def _e4m3_value(b: int) -> Fraction:
+    """FP8 e4m3 from its definition: 1 sign, 4 exponent bits (bias 7), 3 mantissa bits; exponent 0 = subnormal."""
+    s, ex, mant = b >> 7, (b >> 3) & 15, b & 7
+    v = Fraction(mant, 8) * Fraction(2) ** -6 if ex == 0 else (1 + Fraction(mant, 8)) * Fraction(2) ** (ex - 7)
+    return -v if s else v
+
+
+def pin_mxfp8_view(seed=10):
+    """App. D.2: the e4m3 byte times the E8M0 block scale is exactly the decoded FB4 value, for every
+    dialect, index, sign and scale; the scale byte is the E8M0 code of 2^(e-3)."""
+    rng = np.random.default_rng(seed)
+    codes = rng.integers(0, 256, size=(40, 32), dtype=np.uint8)        # 40 x 64 elements: every nibble value
+    did = np.arange(80).reshape(40, 2) % 32
+    sb = rng.integers(0, 252, size=(40, 2))
+    sb[0], sb[1] = [0, 1], [250, 251]
+    meta = (sb | (did << 8)).astype(np.uint16)
+    q = orc.Quantized(codes, meta)
+    y = orc.dequantize(q, FB)
+    for layout in (0, 1):
+        e, sc = orc.to_mxfp8(q, FB, layout)
+        for t in range(40):
+            for c in range(64):
+                k = int(sc[orc.mxfp8_scale_offset(t, c // 32, 2, layout)])
+                assert k == int(sb[t, c // 32])                          # E8M0 code = scale byte
+                want = f32_value(y[t, c])
+                got = _e4m3_value(int(e[t, c])) * Fraction(2) ** (k - 127)
+                assert got == want
+                assert (int(e[t, c]) >> 7) == int(np.signbit(y[t, c]))   # signed zeros keep their sign
+                assert (int(e[t, c]) & 0x7F) != 0x7F                     # never the NaN pattern
+
+
+def pin_mxfp8_scale_layout():
+    """The tiled scale layout: 512-byte tiles of 128 rows x 4 columns, column tiles of a row band
+    contiguous; inside a tile rows 32 apart are 4 bytes apart, neighbouring rows 16 bytes, neighbouring
+    columns 1 byte; every scale has its own byte; padding holds 0x7f."""
+    off = orc.mxfp8_scale_offset
+    n_col = 10                                               # 3 column tiles (padded to 12)
+    assert off(0, 0, n_col, 1) == 0 and off(0, 4, n_col, 1) == 512 and off(0, 8, n_col, 1) == 1024
+    assert off(128, 0, n_col, 1) == 3 * 512
+    assert off(1, 0, n_col, 1) - off(0, 0, n_col, 1) == 16
+    assert off(32, 0, n_col, 1) - off(0, 0, n_col, 1) == 4 and off(96, 0, n_col, 1) == 12
+    assert off(0, 3, n_col, 1) == 3 and off(31, 3, n_col, 1) == 31 * 16 + 3 and off(127, 3, n_col, 1) == 511
+    T = 300
+    seen = {off(r, c, n_col, 1) for r in range(T) for c in range(n_col)}
+    assert len(seen) == T * n_col and max(seen) < 3 * 3 * 512
+    assert [off(r, c, n_col, 0) for r in (0, 1) for c in (0, 9)] == [0, 9, 10, 19]
+    meta = np.full((T, n_col), 130 | (3 << 8), dtype=np.uint16)
+    q = orc.Quantized(np.zeros((T, n_col * 16), np.uint8), meta)
+    _, sc = orc.to_mxfp8(q, FB, 1)
+    assert len(sc) == 3 * 3 * 512
+    real = np.zeros(len(sc), bool)
+    real[list(seen)] = True
+    assert np.all(sc[real] == 130) and np.all(sc[~real] == 0x7F)
+
+
 def _meta_with_dialects(rows):
     """meta records (scale byte 124) for rows of dialect ids"""
     return np.array([[124 | (d << 8) for d in r] for r in rows], dtype=np.uint16)
@@ -515,6 +570,7 @@ ALL_PINS = [
     pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
     pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_decomposition,
-    pin_dequantize_formula, pin_mse, pin_f32_input, pin_subformatbook_hand_counted,
+    pin_dequantize_formula, pin_mse, pin_f32_input, pin_mxfp8_view, pin_mxfp8_scale_layout,
+    pin_subformatbook_hand_counted,
     pin_subformatbook_one_dialect_per_bucket_and_closed_loop,
 ]

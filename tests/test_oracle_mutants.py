@@ -41,6 +41,14 @@ MUTANTS = {
     "f32_rounded_to_bf16_first": ("xv[i] = (double)f;",
                                   "{ uint32_t u_; memcpy(&u_, &f, 4); u_ = (u_ + 0x7fffu + ((u_ >> 16) & 1u)) & 0xffff0000u; "
                                   "float g_; memcpy(&g_, &u_, 4); xv[i] = (double)g_; }"),
+    "mxfp8_exponent_bias": ("return (uint8_t)(((ex + 7) << 3) | mant);", "return (uint8_t)(((ex + 8) << 3) | mant);"),
+    "mxfp8_mantissa_shift": ("int mant = ex <= 3 ? frac << (3 - ex) : frac >> (ex - 3);", "int mant = frac;"),
+    "mxfp8_sign_lost": ("| ((code & 8) << 4));", "| ((code & 8) << 3));"),
+    "mxfp8_scale_plus_3": ("(uint8_t)(meta[t * nblk + b] & 0xff);", "(uint8_t)((meta[t * nblk + b] & 0xff) + 3);"),
+    "mxfp8_tile_rows_swapped": ("return tile * 512 + (r % 32) * 16 + (r / 32) * 4 + col % 4;",
+                                "return tile * 512 + (r / 4) * 16 + (r % 4) * 4 + col % 4;"),
+    "mxfp8_row_tiles_fastest": ("int64_t tile = (row / 128) * col_tiles + col / 4;",
+                                "int64_t tile = (col / 4) * 3 + row / 128;"),
     "subformatbook_ties_to_highest": ("if (best < 0 || count[d] > count[best]) best = d;",
                                       "if (best < 0 || count[d] >= count[best]) best = d;"),
     "subformatbook_least_frequent": ("if (best < 0 || count[d] > count[best]) best = d;",
