@@ -224,6 +224,11 @@ class Ops:
         fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, tile, None, None, 0, codes, meta, sal, rc, rm)
         plain_bytes = T * C * 0.5 + T * (C // B) * 2
         res_bytes = n_sal * (C * 0.5 + (C // B) * 2) + 4 * n_sal
+        if name == "to_mxfp8_tiled_scales":
+            e8 = self.buf("e4m3", (T, C), torch.uint8)
+            sc = self.buf("sf", (fb4.fb4_mxfp8_scale_bytes(T, C, 1),), torch.uint8)
+            return (lambda: fb4.fb4_to_mxfp8(q.ctx, codes, meta, T, C, e8, sc, 1)), \
+                plain_bytes + T * C + T * (C // B)
         if name == "dequantize_f32_decomposed":
             out = self.buf("out32", (T, C), torch.float32)
             return (lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, sal, n_sal, rc, rm, out, 0)), \
@@ -244,7 +249,7 @@ class Ops:
 
 
 OP_NAMES = ["plain", "plain_f32", "seda", "decomposed", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
-            "dequantize_bf16_plain", "dequantize_bf16_decomposed"]
+            "dequantize_bf16_plain", "dequantize_bf16_decomposed", "to_mxfp8_tiled_scales"]
 
 
 def main():
@@ -364,7 +369,8 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         total, per = time_steps(fn, steps, warm, torch)
         ms = total / steps
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
-                     "kernel_variant": q.last_variant if not name.startswith("dequantize") else "decode"}
+                     "kernel_variant": q.last_variant if name in ("plain", "plain_f32", "seda", "decomposed",
+                                                                         "decomposed_seda") else "decode"}
         if name == "dequantize_f32_decomposed":
             ops.drop("out32")
         if name == "plain_f32":

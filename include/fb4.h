@@ -225,6 +225,27 @@ int fb4_dequantize(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int
                    const uint16_t* res_meta, void* out, int out_dtype, void* stream);
 
 /*
+ * MXFP8 view of a quantized tensor (App. D.2: FB4's integer magnitudes 0..15 "are exactly
+ * representable in FP8 e4m3" and its scaling is power-of-two, so it is "directly compatible with
+ * MXFP8 GEMM").  Element -> the e4m3 byte of its signed magnitude; block -> the E8M0 byte of its
+ * element scale 2^(e-3), which is the scale byte of `meta`.  Exact: e4m3 * scale equals the value
+ * fb4_dequantize gives.  Block size 32 only (FB4_ERR_INVALID_ARG otherwise); residual tensors
+ * (res_codes / res_meta) are converted by a second call.
+ *   e4m3         : device uint8 [T][C] (out), 16-byte aligned
+ *   scales       : device uint8 (out), fb4_mxfp8_scale_bytes(T, C, scale_layout) bytes
+ *   scale_layout : 0 = row-major [T][C/32];
+ *                  1 = tiles of 128 rows x 4 scale columns (512 bytes each; the column tiles of a
+ *                      band of 128 rows follow one another), scale (r, c) of a tile at byte
+ *                      (r mod 32)*16 + (r div 32)*4 + c: the order block-scaled tensor-core GEMMs
+ *                      read scale factors in.  Rows are padded to a multiple of 128 and scale
+ *                      columns to a multiple of 4; padding bytes are written as 0x7f (scale 1).
+ */
+int fb4_to_mxfp8(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T, int64_t C, uint8_t* e4m3,
+                 uint8_t* scales, int scale_layout, void* stream);
+/* Size in bytes of the scale buffer of fb4_to_mxfp8 (-1 for invalid arguments).  Host only. */
+int64_t fb4_mxfp8_scale_bytes(int64_t T, int64_t C, int scale_layout);
+
+/*
  * Host-buffer form of fb4_quantize for callers whose tensors live in host memory:
  * copies x from the host, quantizes, and copies codes and meta back, in row
  * chunks pipelined over the context's own streams, then waits for completion.

@@ -350,6 +350,27 @@ int fb4_build_subformatbook(fb4_ctx* ctx, const uint16_t* meta, int64_t T, int64
   return FB4_OK;
 }
 
+int64_t fb4_mxfp8_scale_bytes(int64_t T, int64_t C, int layout) {
+  if (T < 0 || C <= 0 || C % 32 != 0 || (layout != 0 && layout != 1)) return -1;
+  const int64_t n_col = C / 32;
+  return layout == 0 ? T * n_col : ((T + 127) / 128) * ((n_col + 3) / 4) * 512;
+}
+
+int fb4_to_mxfp8(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T, int64_t C, uint8_t* e4m3,
+                 uint8_t* scales, int scale_layout, void* stream) {
+  if (!ctx || ctx->cfg.block_size != 32) return FB4_ERR_INVALID_ARG;   // an MX block is 32 elements
+  if (scale_layout != 0 && scale_layout != 1) return FB4_ERR_INVALID_ARG;
+  if (T < 0 || C <= 0 || C % 32 != 0 || T > 0x7fffffffLL) return FB4_ERR_SHAPE;
+  if (T == 0) return FB4_OK;
+  if (!codes || !meta || !e4m3 || !scales) return FB4_ERR_INVALID_ARG;
+  if (!aligned16(codes) || !aligned16(meta) || !aligned16(e4m3)) return FB4_ERR_ALIGN;
+  cudaError_t e = fb4_launch_to_mxfp8(ctx, codes, meta, T, C, e4m3, scales, scale_layout,
+                                      static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
+  ctx->launches += 1;
+  return FB4_OK;
+}
+
 int fb4_quantize_host(fb4_ctx* ctx, const void* x_host, int64_t T, int64_t C, void* d_x, uint8_t* d_codes,
                       uint16_t* d_meta, uint8_t* codes_host, uint16_t* meta_host) {
   const int rc = check_quantize_args(ctx, d_x, T, C, C, d_codes, d_meta);

@@ -1,0 +1,119 @@
+// MXFP8 view of an FB4 tensor (App. D.2: the integer magnitudes 0..15 are exact in FP8 e4m3 and the
+// block scale is a power of two, so FB4 feeds an MXFP8 GEMM without rounding): 4-bit codes ->
+// e4m3 bytes, scale bytes -> E8M0 scale factors in row-major or 128x4-tiled order.
+//
+// Thread <-> block of 32 elements: one 128-bit load of the codes, one 16-bit load of the metadata,
+// one 256-bit store of the 32 e4m3 bytes (a warp writes 1 KB contiguous), one byte store of the scale.
+// The dialect's 8 magnitudes sit in two registers as e4m3 bytes; a byte permute with four 3-bit
+// indices as selector looks up four elements at once, sign bits come from sign-replicating permutes.
+#include "fb4_device.cuh"
+#include "fb4_internal.h"
+
+namespace {
+
+using fb4dev::prmt;
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 2;
+
+// e4m3 byte of an integer 0..15: 1.mmm * 2^(E-7)
+__device__ __forceinline__ uint32_t e4m3_of_small_int(uint32_t m) {
+  if (m == 0) return 0u;
+  const int ex = 31 - __clz((int)m);
+  const uint32_t frac = m - (1u << ex);
+  return ((uint32_t)(ex + 7) << 3) | (frac << 3 >> ex);   // ex <= 3
+}
+
+__device__ __forceinline__ int64_t scale_offset(int64_t row, int64_t col, int64_t n_col, int64_t col_tiles, int tiled) {
+  if (!tiled) return row * n_col + col;
+  const int64_t r = row & 127;
+  return ((row >> 7) * col_tiles + (col >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (col & 3);
+}
+
+// 8 codes -> 8 e4m3 bytes (two registers)
+__device__ __forceinline__ void convert_word(uint32_t cw, uint2 fb, uint32_t& lo, uint32_t& hi) {
+  const uint32_t sel = cw & 0x77777777u;
+  const uint32_t s_odd = prmt(cw, 0u, 0xba98u), s_even = prmt(cw << 4, 0u, 0xba98u);   // 0xff where negative
+  lo = prmt(fb.x, fb.y, sel) | (__byte_perm(s_even, s_odd, 0x5140) & 0x80808080u);
+  hi = prmt(fb.x, fb.y, sel >> 16) | (__byte_perm(s_even, s_odd, 0x7362) & 0x80808080u);
+}
+
+__global__ void __launch_bounds__(kThreads)
+fb4_to_mxfp8_kernel(const uint4* __restrict__ codes, const uint16_t* __restrict__ meta, int64_t T, int64_t n_col,
+                    const Fb4DeviceTables* __restrict__ tables, uint8_t* __restrict__ e4m3,
+                    uint8_t* __restrict__ scales, int tiled, int out_aligned32) {
+  __shared__ uint2 fb8[32];   // per dialect: its 8 magnitudes as e4m3 bytes
+  reinterpret_cast<uint8_t*>(fb8)[threadIdx.x] =
+      (uint8_t)e4m3_of_small_int(tables->formatbook[threadIdx.x >> 3][threadIdx.x & 7]);
+  __syncthreads();
+  const int64_t total = T * n_col;
+  const int64_t col_tiles = (n_col + 3) >> 2;
+  constexpr int64_t kStep = (int64_t)kThreads * kUnroll;
+  for (int64_t base = (int64_t)blockIdx.x * kStep; base < total; base += (int64_t)gridDim.x * kStep) {
+    uint4 cw[kUnroll];
+    uint32_t m[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int64_t b = base + u * kThreads + threadIdx.x;
+      if (b < total) {
+        cw[u] = __ldg(codes + b);
+        m[u] = (uint32_t)__ldg(meta + b);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int64_t b = base + u * kThreads + threadIdx.x;
+      if (b >= total) continue;
+      const uint2 fb = fb8[(m[u] >> 8) & 31u];
+      uint32_t o[8];
+      convert_word(cw[u].x, fb, o[0], o[1]);
+      convert_word(cw[u].y, fb, o[2], o[3]);
+      convert_word(cw[u].z, fb, o[4], o[5]);
+      convert_word(cw[u].w, fb, o[6], o[7]);
+      uint8_t* dst = e4m3 + b * 32;
+      if (out_aligned32) {
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(o[0]), "r"(o[1]),
+                     "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+      } else {
+        reinterpret_cast<uint4*>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
+        reinterpret_cast<uint4*>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
+      }
+      const int64_t row = b / n_col;
+      scales[scale_offset(row, b - row * n_col, n_col, col_tiles, tiled)] = (uint8_t)m[u];   // E8M0 of 2^(e-3)
+    }
+  }
+  if (tiled) {
+    // padding of the tiled layout holds scale 1: rows [T, Tp) x all padded columns, then rows [0, T)
+    // x columns [n_col, n_col_p)
+    const int64_t Tp = (T + 127) & ~127ll, n_col_p = col_tiles * 4;
+    const int64_t pad_a = (Tp - T) * n_col_p, pad_b = T * (n_col_p - n_col);
+    for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < pad_a + pad_b;
+         i += (int64_t)gridDim.x * kThreads) {
+      int64_t row, col;
+      if (i < pad_a) {
+        row = T + i / n_col_p;
+        col = i % n_col_p;
+      } else {
+        const int64_t j = i - pad_a, w = n_col_p - n_col;
+        row = j / w;
+        col = n_col + j % w;
+      }
+      scales[scale_offset(row, col, n_col, col_tiles, 1)] = 0x7f;
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t fb4_launch_to_mxfp8(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T, int64_t C,
+                                uint8_t* e4m3, uint8_t* scales, int layout, cudaStream_t stream) {
+  static_assert(kThreads == 256, "one thread per formatbook entry fills the shared table");
+  const int64_t n_col = C / 32, total = T * n_col;
+  if (total == 0) return cudaSuccess;
+  constexpr int64_t kStep = (int64_t)kThreads * kUnroll;
+  const int64_t want = (total + kStep - 1) / kStep, cap = (int64_t)ctx->sm_count * 8;
+  const int a32 = (reinterpret_cast<uintptr_t>(e4m3) & 31u) == 0 ? 1 : 0;
+  fb4_to_mxfp8_kernel<<<(unsigned)(want < cap ? want : cap), kThreads, 0, stream>>>(
+      reinterpret_cast<const uint4*>(codes), meta, T, n_col, ctx->d_tables, e4m3, scales, layout, a32);
+  return cudaGetLastError();
+}

@@ -23,7 +23,7 @@ STATIC_MAX_CLUSTERS = 1024
 EXPORTS = [
     "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
     "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
-    "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
+    "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
 
 
@@ -80,6 +80,10 @@ def lib() -> ctypes.CDLL:
     L.fb4_quantize_decomposed.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.fb4_quantize_decomposed_idx.argtypes = [vp, vp, i64, i64, i64, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
     L.fb4_dequantize.argtypes = [vp, vp, vp, i64, i64, vp, i64, vp, vp, vp, ci, vp]
+    L.fb4_to_mxfp8.argtypes = [vp, vp, vp, i64, i64, vp, vp, ci, vp]
+    L.fb4_to_mxfp8.restype = ci
+    L.fb4_mxfp8_scale_bytes.argtypes = [i64, i64, ci]
+    L.fb4_mxfp8_scale_bytes.restype = i64
     L.fb4_quantize_host.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp]
     for name in ("fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
                  "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx",
@@ -208,6 +212,15 @@ def fb4_dequantize(ctx, codes, meta, T, C, salient_idx, n_salient, res_codes, re
                                 _ptr(res_meta), _ptr(out), out_dtype, _stream(stream)), "fb4_dequantize")
 
 
+def fb4_to_mxfp8(ctx, codes, meta, T, C, e4m3, scales, scale_layout, stream=None) -> None:
+    _check(lib().fb4_to_mxfp8(ctx, _ptr(codes), _ptr(meta), T, C, _ptr(e4m3), _ptr(scales), scale_layout,
+                              _stream(stream)), "fb4_to_mxfp8")
+
+
+def fb4_mxfp8_scale_bytes(T, C, scale_layout) -> int:
+    return int(lib().fb4_mxfp8_scale_bytes(T, C, scale_layout))
+
+
 def fb4_quantize_host(ctx, x_host, T, C, d_x, d_codes, d_meta, codes_host, meta_host) -> None:
     _check(lib().fb4_quantize_host(ctx, _ptr(x_host), T, C, _ptr(d_x), _ptr(d_codes), _ptr(d_meta),
                                    _ptr(codes_host), _ptr(meta_host)), "fb4_quantize_host")
@@ -333,6 +346,15 @@ class Fb4:
                        q.res_codes if n else None, q.res_meta if n else None, out,
                        0 if dtype == torch.float32 else 1)
         return out
+
+    def to_mxfp8(self, q: Quantized, scale_layout: int = 0):
+        """(e4m3 bytes [T][C], E8M0 scale bytes) of the main tensor of q."""
+        T, C = q.codes.shape[0], q.codes.shape[1] * 2
+        e4m3 = torch.empty((T, C), dtype=torch.uint8, device=q.codes.device)
+        scales = torch.empty(max(fb4_mxfp8_scale_bytes(T, C, scale_layout), 1), dtype=torch.uint8,
+                             device=q.codes.device)
+        fb4_to_mxfp8(self.ctx, q.codes, q.meta, T, C, e4m3, scales, scale_layout)
+        return e4m3, scales[:fb4_mxfp8_scale_bytes(T, C, scale_layout)]
 
     def set_kernel_variant(self, variant: int) -> None:
         fb4_set_kernel_variant(self.ctx, variant)

@@ -1,0 +1,70 @@
+"""GPU parity of the MXFP8 view (e4m3 bytes + E8M0 scale bytes, both scale layouts) against the CPU
+oracle, byte for byte, padding of the tiled layout included."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import FB, to_dev_bf16
+from oracle import fb4_oracle as orc
+from paper_2603_02883_b200 import fb4, synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q32():
+    q = fb4.Fb4()
+    yield q
+    assert q.device_status == 0
+    q.close()
+
+
+@pytest.mark.parametrize("T,C", [(1, 32), (130, 96), (300, 320), (257, 1024 + 64), (128, 128)])
+def test_random_codes_every_dialect(q32, T, C):
+    rng = np.random.default_rng(T + C)
+    codes = rng.integers(0, 256, size=(T, C // 2), dtype=np.uint8)
+    meta = (rng.integers(0, 252, size=(T, C // 32)) | (rng.integers(0, 32, size=(T, C // 32)) << 8)).astype(np.uint16)
+    ref = orc.Quantized(codes, meta)
+    got = fb4.Quantized(torch.from_numpy(codes).cuda(), torch.from_numpy(meta.view(np.int16)).cuda())
+    for layout in (0, 1):
+        e_ref, s_ref = orc.to_mxfp8(ref, FB, layout)
+        e4m3, scales = q32.to_mxfp8(got, layout)
+        scales_before = scales.clone()
+        assert np.array_equal(e4m3.cpu().numpy(), e_ref), f"e4m3 bytes, layout {layout}"
+        assert np.array_equal(scales.cpu().numpy(), s_ref), f"scale bytes, layout {layout}"
+        assert scales.numel() == fb4.fb4_mxfp8_scale_bytes(T, C, layout) == len(s_ref)
+        del scales_before
+
+
+def test_c2_workload_and_decoded_value(q32):
+    w = synth.workloads()["c2"]
+    bits = synth.activation(w)
+    q = q32.quantize(to_dev_bf16(bits))
+    ref = orc.quantize(bits, FB)
+    e_ref, s_ref = orc.to_mxfp8(ref, FB, 1)
+    e4m3, scales = q32.to_mxfp8(q, 1)
+    assert np.array_equal(e4m3.cpu().numpy(), e_ref) and np.array_equal(scales.cpu().numpy(), s_ref)
+    # e4m3 * 2^(scale-127) is the decoded value (torch's own e4m3 decoder on a slab of rows)
+    rows = slice(1000, 1256)
+    vals = e4m3[rows].view(torch.float8_e4m3fn).float().view(256, w.C // 32, 32)
+    e0, s0 = q32.to_mxfp8(fb4.Quantized(q.codes[rows].contiguous(), q.meta[rows].contiguous()), 0)
+    sc = torch.exp2(s0.view(256, w.C // 32, 1).float() - 127.0)
+    want = q32.dequantize(fb4.Quantized(q.codes[rows].contiguous(), q.meta[rows].contiguous()))
+    assert torch.equal((vals * sc).view(256, w.C), want)
+
+
+def test_argument_checks(q32):
+    L = fb4.lib()
+    t = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    p = ctypes.c_void_p(t.data_ptr())
+    assert L.fb4_to_mxfp8(q32.ctx, p, p, 4, 48, p, p, 0, None) == fb4.ERR_SHAPE
+    assert L.fb4_to_mxfp8(q32.ctx, p, p, 4, 64, p, p, 2, None) == fb4.ERR_INVALID_ARG
+    assert L.fb4_to_mxfp8(q32.ctx, p, p, 4, 64, None, p, 0, None) == fb4.ERR_INVALID_ARG
+    assert L.fb4_to_mxfp8(q32.ctx, None, None, 0, 64, None, None, 0, None) == fb4.OK
+    assert L.fb4_mxfp8_scale_bytes(300, 320, 1) == 3 * 3 * 512 and L.fb4_mxfp8_scale_bytes(300, 320, 0) == 3000
+    assert L.fb4_mxfp8_scale_bytes(300, 330, 0) == -1
+    q16 = fb4.Fb4(block_size=16)
+    assert L.fb4_to_mxfp8(q16.ctx, p, p, 4, 64, p, p, 0, None) == fb4.ERR_INVALID_ARG
+    q16.close()
