@@ -21,6 +21,8 @@
  *   Sec. 3.3  activation decomposition: residual Delta = Act - Q(Act) of the
  *             salient tokens is quantized again; one salient token per tile,
  *             the highest-scoring one.
+ *   Sec. 3.3 / App. C  weights are quantized offline with exhaustive selection: the
+ *             squared error of every dialect over all elements of the block, minimum wins.
  *   App. D.2  MXFP8 view: the integer magnitudes 0..15 are exact in FP8 e4m3 and the
  *             power-of-two block scale is an E8M0 scale, so a quantized tensor can be
  *             re-expressed as an MXFP8 operand without any rounding.
@@ -121,6 +123,24 @@ void fb4o_default_stage1(const uint8_t *F, uint32_t *stage1 /*32*/) {
   }
 }
 
+/* Sec. 3.1: normalised magnitude v = |x| * 2^(3-e), in [0,16) unless the exponent was clamped from above */
+static double normalised(double x, int e) { return ldexp(fabs(x), 3 - e); }
+
+/* Sec. 3.1: block exponent e = floor(log2(amax)), clamped; an all-zero block gets exp_min. */
+static int block_exponent(double amax, const fb4o_config *cfg) {
+  int e;
+  if (amax == 0.0) {
+    e = cfg->exp_min;
+  } else {
+    int ex;
+    (void)frexp(amax, &ex);          /* amax = m * 2^ex, m in [0.5,1)  =>  floor(log2) = ex-1 */
+    e = ex - 1;
+    if (e < cfg->exp_min) e = cfg->exp_min;
+    if (e > cfg->exp_max) e = cfg->exp_max;
+  }
+  return e;
+}
+
 /*
  * One block.  x[B] are the real input values, sgn[B] their sign bits.
  * allowed = SeDA mask (all ones when unconstrained).
@@ -135,19 +155,10 @@ static void quantize_block(const double *x, const uint8_t *sgn, const fb4o_confi
   /* Sec. 3.1: shared power-of-two scale from floor(log2(max magnitude)) */
   double amax = 0.0;
   for (int i = 0; i < B; ++i) if (fabs(x[i]) > amax) amax = fabs(x[i]);
-  int e;
-  if (amax == 0.0) {
-    e = cfg->exp_min;
-  } else {
-    int ex;
-    (void)frexp(amax, &ex);          /* amax = m * 2^ex, m in [0.5,1)  =>  floor(log2) = ex-1 */
-    e = ex - 1;
-    if (e < cfg->exp_min) e = cfg->exp_min;
-    if (e > cfg->exp_max) e = cfg->exp_max;
-  }
+  const int e = block_exponent(amax, cfg);
   /* normalise: v = |x| * 2^(3-e), in [0,16) unless the exponent was clamped from above */
   double v[FB4O_MAXB];
-  for (int i = 0; i < B; ++i) v[i] = ldexp(fabs(x[i]), 3 - e);
+  for (int i = 0; i < B; ++i) v[i] = normalised(x[i], e);
   /* Sec. 3.2: group-wise maxima */
   double gmax[FB4O_MAXB];
   double vmax = 0.0;
@@ -494,6 +505,55 @@ int fb4o_to_mxfp8(const uint8_t *codes, const uint16_t *meta, int64_t T, int64_t
     }
     for (int64_t b = 0; b < nblk; ++b)
       scales[fb4o_mxfp8_scale_offset(t, b, nblk, layout)] = (uint8_t)(meta[t * nblk + b] & 0xff);
+  }
+  return 0;
+}
+
+/*
+ * Offline weight quantization (Sec. 3.3: weights "can be quantized offline, allowing exhaustive
+ * dialect selection without runtime approximations"; App. C: "weight dialect selection and
+ * quantization follow an MSE-based criterion").  Per block: the same power-of-two scale as for
+ * activations; then for EVERY dialect the squared error of rounding every element to its nearest
+ * magnitude, summed over the block's elements in index order in double precision (each term
+ * (v - m)^2 is exact in double; only the running sum rounds); the dialect with the smallest sum
+ * wins, ties to the lowest id; the elements are rounded with it.  No groups, no stage 1, no tables.
+ * sse (optional, [N*K/B][32]) receives the sums.
+ */
+int fb4o_quantize_weights(const uint16_t *w, int64_t N, int64_t K, int64_t ld, const fb4o_config *cfg,
+                          const uint8_t *F, uint8_t *codes, uint16_t *meta, double *sse) {
+  if (!config_ok(cfg, K) || N < 0 || ld < K) return -1;
+  if (!formatbook_ok(F)) return -2;
+  const int B = cfg->block_size;
+  const int64_t nblk = K / B;
+#pragma omp parallel for schedule(static)
+  for (int64_t n = 0; n < N; ++n) {
+    for (int64_t blk = 0; blk < nblk; ++blk) {
+      double x[FB4O_MAXB], v[FB4O_MAXB];
+      uint8_t sg[FB4O_MAXB], code[FB4O_MAXB];
+      double amax = 0.0;
+      for (int i = 0; i < B; ++i) {
+        uint16_t b = w[n * ld + blk * B + i];
+        x[i] = bf16_to_double(b);
+        sg[i] = (uint8_t)(b >> 15);
+        if (fabs(x[i]) > amax) amax = fabs(x[i]);
+      }
+      const int e = block_exponent(amax, cfg);
+      for (int i = 0; i < B; ++i) v[i] = normalised(x[i], e);
+      int best = 0;
+      double best_err = 0.0;
+      for (int d = 0; d < 32; ++d) {
+        double err = 0.0;
+        for (int i = 0; i < B; ++i) {
+          double diff = v[i] - (double)F[d * 8 + nearest_index(F + d * 8, v[i])];
+          err += diff * diff;
+        }
+        if (sse) sse[(n * nblk + blk) * 32 + d] = err;
+        if (d == 0 || err < best_err) { best = d; best_err = err; }
+      }
+      for (int i = 0; i < B; ++i)
+        code[i] = (uint8_t)((sg[i] << 3) | nearest_index(F + best * 8, v[i]));
+      store_block(code, B, best, e, codes + n * (K / 2), meta + n * nblk, blk);
+    }
   }
   return 0;
 }

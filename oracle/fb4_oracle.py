@@ -84,6 +84,8 @@ def lib():
         L.fb4o_mxfp8_scale_offset.restype = i64
         L.fb4o_mxfp8_scale_bytes.argtypes = [i64, i64, ctypes.c_int]
         L.fb4o_mxfp8_scale_bytes.restype = i64
+        L.fb4o_quantize_weights.argtypes = [vp, i64, i64, i64, ctypes.POINTER(_Cfg), vp, vp, vp, vp]
+        L.fb4o_quantize_weights.restype = ctypes.c_int
         L.fb4o_build_subformatbook.argtypes = [vp, i64, i64, vp, vp, i64, i32, vp, vp, vp]
         L.fb4o_build_subformatbook.restype = ctypes.c_int
         _libs[path] = L
@@ -250,3 +252,20 @@ def to_mxfp8(q: Quantized, formatbook, layout: int = 0):
     if r != 0:
         raise ValueError(f"fb4o_to_mxfp8 failed: {r}")
     return out, sc[:n]
+
+
+def quantize_weights(w_bits, formatbook, cfg: Config = Config(), want_sse: bool = False):
+    """w_bits: uint16 [N][K] bf16 bit patterns; exhaustive exact-squared-error dialect selection."""
+    w = np.ascontiguousarray(w_bits, dtype=np.uint16)
+    N, K = w.shape
+    B = cfg.block_size
+    codes = np.zeros((N, K // 2), dtype=np.uint8)
+    meta = np.zeros((N, K // B), dtype=np.uint16)
+    sse = np.zeros((N, K // B, 32), dtype=np.float64) if want_sse else None
+    ccfg = cfg.c()
+    r = lib().fb4o_quantize_weights(_p(w), N, K, K, ctypes.byref(ccfg), _p(_c(formatbook, np.uint8)), _p(codes),
+                                    _p(meta), _p(sse))
+    if r != 0:
+        raise ValueError(f"fb4o_quantize_weights failed: {r}")
+    q = Quantized(codes, meta)
+    return (q, sse) if want_sse else q

@@ -423,6 +423,37 @@ def pin_mxfp8_scale_layout():
     assert np.all(sc[real] == 130) and np.all(sc[~real] == 0x7F)
 
 
+def pin_weight_quantization(seed=11, n=25):
+    """Exhaustive selection (Sec. 3.3 / App. C): the chosen dialect attains the minimum of the exact
+    (rational) squared error over all 32 dialects, lowest id among exact ties; its elements are rounded
+    to the nearest magnitude; its error never exceeds that of the online (LUT, two-stage) choice."""
+    rng = np.random.default_rng(seed)
+    for it in range(n):
+        B = 32 if it % 3 else 16
+        cfg = orc.Config(block_size=B, num_groups=8)
+        bits = rand_block_bits(rng, B, (-6, 6) if it % 2 else (-20, 20))
+        if it == 4:
+            bits[:] = 0
+        q, sse = orc.quantize_weights(bits.reshape(1, B), FB, cfg, want_sse=True)
+        did, e = int(q.did[0, 0]), int(q.exponent[0, 0])
+        vals = [abs(bf16_value(int(b))) * Fraction(2) ** (3 - e) for b in bits]
+        exact = []
+        for d in range(32):
+            mags = [int(m) for m in FB[d]]
+            exact.append(sum(min((v - m) ** 2 for m in mags) for v in vals))
+        assert exact[did] == min(exact) and did == exact.index(min(exact))
+        for d in range(32):
+            assert abs(float(exact[d]) - sse[0, 0, d]) <= 1e-12 * max(1.0, float(exact[d]))
+        codes = unpack_codes(q.codes[0])
+        for i, v in enumerate(vals):
+            m = int(FB[did, codes[i] & 7])
+            assert all(abs(v - m) <= abs(v - int(mm)) for mm in FB[did])
+            assert (codes[i] >> 3) == (int(bits[i]) >> 15)
+        qa = orc.quantize(bits.reshape(1, B), FB, cfg)
+        assert int(qa.exponent[0, 0]) == e
+        assert exact[did] <= exact[int(qa.did[0, 0])]
+
+
 def _meta_with_dialects(rows):
     """meta records (scale byte 124) for rows of dialect ids"""
     return np.array([[124 | (d << 8) for d in r] for r in rows], dtype=np.uint16)
@@ -570,7 +601,7 @@ ALL_PINS = [
     pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
     pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_decomposition,
-    pin_dequantize_formula, pin_mse, pin_f32_input, pin_mxfp8_view, pin_mxfp8_scale_layout,
+    pin_dequantize_formula, pin_mse, pin_f32_input, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
     pin_subformatbook_hand_counted,
     pin_subformatbook_one_dialect_per_bucket_and_closed_loop,
 ]

@@ -14,7 +14,7 @@ SRC = os.path.join(os.path.dirname(orc.__file__), "fb4_oracle.c")
 MUTANTS = {
     "round_ties_down": ("if (dj <= bestd) { bestd = dj; best = j; }", "if (dj < bestd) { bestd = dj; best = j; }"),
     "dialect_ties_to_highest": ("if (best < 0 || err < best_err)", "if (best < 0 || err <= best_err)"),
-    "exponent_offset_2": ("v[i] = ldexp(fabs(x[i]), 3 - e);", "v[i] = ldexp(fabs(x[i]), 2 - e);"),
+    "exponent_offset_2": ("return ldexp(fabs(x), 3 - e);", "return ldexp(fabs(x), 2 - e);"),
     "floor_log2_off_by_one": ("e = ex - 1;", "e = ex;"),
     "midpoint_dropped": ("+ 0.25;", "+ 0.0;"),
     "squared_error": ("err += fabs(mid - (double)F[d * 8 + nearest_index(F + d * 8, mid)]);",
@@ -49,6 +49,11 @@ MUTANTS = {
                                 "return tile * 512 + (r / 4) * 16 + (r % 4) * 4 + col % 4;"),
     "mxfp8_row_tiles_fastest": ("int64_t tile = (row / 128) * col_tiles + col / 4;",
                                 "int64_t tile = (col / 4) * 3 + row / 128;"),
+    "weights_absolute_error": ("err += diff * diff;", "err += fabs(diff);"),
+    "weights_last_element_skipped": ("for (int i = 0; i < B; ++i) {\n          double diff", "for (int i = 0; i + 1 < B; ++i) {\n          double diff"),
+    "weights_ties_to_highest": ("if (d == 0 || err < best_err) { best = d; best_err = err; }",
+                                "if (d == 0 || err <= best_err) { best = d; best_err = err; }"),
+    "weights_half_the_formatbook": ("for (int d = 0; d < 32; ++d) {\n        double err = 0.0;", "for (int d = 0; d < 16; ++d) {\n        double err = 0.0;"),
     "subformatbook_ties_to_highest": ("if (best < 0 || count[d] > count[best]) best = d;",
                                       "if (best < 0 || count[d] >= count[best]) best = d;"),
     "subformatbook_least_frequent": ("if (best < 0 || count[d] > count[best]) best = d;",
