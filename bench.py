@@ -394,6 +394,21 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         torch.cuda.synchronize()
         ms = float(np.mean([a.elapsed_time(b) for a, b in evs[warm:]]))
         alg = algorithmic_bytes(w2.T, w2.C)
+        # offline weight quantizer on the same tensor, and how often the online (LUT, two-stage)
+        # choice differs from the exhaustive exact-error choice (the paper's Table 2 comparison)
+        cw2, mw2 = torch.empty_like(c2), torch.empty_like(m2)
+        tot, _ = time_steps(lambda: fb4.fb4_quantize_weights(q.ctx, x2, w2.T, w2.C, w2.C, cw2, mw2), 3, 1, torch)
+        dis = float(((m2.view(torch.int16).to(torch.int32) >> 8) != (mw2.view(torch.int16).to(torch.int32) >> 8))
+                    .float().mean())
+        o_a = torch.empty((w2.T, w2.C), dtype=torch.float32, device="cuda")
+        fb4.fb4_dequantize(q.ctx, c2, m2, w2.T, w2.C, None, 0, None, None, o_a, 0)
+        mse_lut = float(((o_a - x2.float()).double() ** 2).mean())
+        fb4.fb4_dequantize(q.ctx, cw2, mw2, w2.T, w2.C, None, 0, None, None, o_a, 0)
+        mse_exh = float(((o_a - x2.float()).double() ** 2).mean())
+        del o_a
+        res["c2_weights_exhaustive"] = {"ms": tot / 3, "Gelem/s": w2.T * w2.C / (tot / 3 * 1e-3) / 1e9,
+                                        "dialect_disagreement_vs_online": dis,
+                                        "mse_online_over_mse_exhaustive": mse_lut / mse_exh}
         res["c2_plain_32760x3072_l2_flushed"] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9,
                                                  "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
                                                  "kernel_variant": q.last_variant}

@@ -225,6 +225,18 @@ int fb4_dequantize(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int
                    const uint16_t* res_meta, void* out, int out_dtype, void* stream);
 
 /*
+ * Offline weight quantization (Sec. 3.3: weights are "quantized offline, allowing exhaustive
+ * dialect selection without runtime approximations"; App. C: "an MSE-based criterion").  Same
+ * format and scale as fb4_quantize, but the dialect of a block is the one with the smallest
+ * squared error over ALL its elements among ALL 32 dialects (no groups, no stage 1, no error
+ * table), ties to the lowest id.  The errors are summed in double precision in element order.
+ * Uses the context's block size and exponent clamp.  Not a bandwidth path.
+ *   w : device bfloat16 [N][ld_elems]; blocks run along the K (contiguous) axis
+ */
+int fb4_quantize_weights(fb4_ctx* ctx, const void* w_bf16, int64_t N, int64_t K, int64_t ld_elems, uint8_t* codes,
+                         uint16_t* meta, void* stream);
+
+/*
  * MXFP8 view of a quantized tensor (App. D.2: FB4's integer magnitudes 0..15 "are exactly
  * representable in FP8 e4m3" and its scaling is power-of-two, so it is "directly compatible with
  * MXFP8 GEMM").  Element -> the e4m3 byte of its signed magnitude; block -> the E8M0 byte of its

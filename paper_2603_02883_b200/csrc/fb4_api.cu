@@ -350,6 +350,17 @@ int fb4_build_subformatbook(fb4_ctx* ctx, const uint16_t* meta, int64_t T, int64
   return FB4_OK;
 }
 
+int fb4_quantize_weights(fb4_ctx* ctx, const void* w, int64_t N, int64_t K, int64_t ld, uint8_t* codes, uint16_t* meta,
+                         void* stream) {
+  const int rc = check_quantize_args(ctx, w, N, K, ld, codes, meta);
+  if (rc != FB4_OK) return rc;
+  if (N == 0) return FB4_OK;
+  cudaError_t e = fb4_launch_quantize_weights(ctx, w, N, K, ld, codes, meta, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
+  ctx->launches += 1;
+  return FB4_OK;
+}
+
 int64_t fb4_mxfp8_scale_bytes(int64_t T, int64_t C, int layout) {
   if (T < 0 || C <= 0 || C % 32 != 0 || (layout != 0 && layout != 1)) return -1;
   const int64_t n_col = C / 32;

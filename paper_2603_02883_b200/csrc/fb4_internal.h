@@ -72,6 +72,8 @@ cudaError_t fb4_launch_subformatbook(const uint16_t* meta, int64_t T, int64_t nb
                                      const int32_t* anchor_cluster, int64_t n_anchor, int32_t n_clusters,
                                      const Fb4Stage1& stage1, uint32_t* counts, uint32_t* cluster_mask, int sm_count,
                                      cudaStream_t stream, int* launches);
+cudaError_t fb4_launch_quantize_weights(const fb4_ctx* ctx, const void* w, int64_t N, int64_t K, int64_t ld,
+                                        uint8_t* codes, uint16_t* meta, cudaStream_t stream);
 cudaError_t fb4_launch_to_mxfp8(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T, int64_t C,
                                 uint8_t* e4m3, uint8_t* scales, int layout, cudaStream_t stream);
 cudaError_t fb4_launch_select_salient(const float* score, int64_t T, int32_t tile, int32_t* salient_idx,

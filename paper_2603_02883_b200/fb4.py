@@ -23,7 +23,7 @@ STATIC_MAX_CLUSTERS = 1024
 EXPORTS = [
     "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
     "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
-    "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
+    "fb4_quantize_weights", "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
 
 
@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
     L.fb4_quantize_decomposed.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.fb4_quantize_decomposed_idx.argtypes = [vp, vp, i64, i64, i64, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
     L.fb4_dequantize.argtypes = [vp, vp, vp, i64, i64, vp, i64, vp, vp, vp, ci, vp]
+    L.fb4_quantize_weights.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
+    L.fb4_quantize_weights.restype = ci
     L.fb4_to_mxfp8.argtypes = [vp, vp, vp, i64, i64, vp, vp, ci, vp]
     L.fb4_to_mxfp8.restype = ci
     L.fb4_mxfp8_scale_bytes.argtypes = [i64, i64, ci]
@@ -210,6 +212,11 @@ def fb4_dequantize(ctx, codes, meta, T, C, salient_idx, n_salient, res_codes, re
                    stream=None) -> None:
     _check(lib().fb4_dequantize(ctx, _ptr(codes), _ptr(meta), T, C, _ptr(salient_idx), n_salient, _ptr(res_codes),
                                 _ptr(res_meta), _ptr(out), out_dtype, _stream(stream)), "fb4_dequantize")
+
+
+def fb4_quantize_weights(ctx, w, N, K, ld_elems, codes, meta, stream=None) -> None:
+    _check(lib().fb4_quantize_weights(ctx, _ptr(w), N, K, ld_elems, _ptr(codes), _ptr(meta), _stream(stream)),
+           "fb4_quantize_weights")
 
 
 def fb4_to_mxfp8(ctx, codes, meta, T, C, e4m3, scales, scale_layout, stream=None) -> None:
@@ -346,6 +353,14 @@ class Fb4:
                        q.res_codes if n else None, q.res_meta if n else None, out,
                        0 if dtype == torch.float32 else 1)
         return out
+
+    def quantize_weights(self, w) -> Quantized:
+        """offline weight quantization: exhaustive squared-error dialect selection"""
+        assert w.dtype == torch.bfloat16
+        N, K, ld = self._shape(w)
+        codes, meta = self._outs(N, K)
+        fb4_quantize_weights(self.ctx, w, N, K, ld, codes, meta)
+        return Quantized(codes, meta)
 
     def to_mxfp8(self, q: Quantized, scale_layout: int = 0):
         """(e4m3 bytes [T][C], E8M0 scale bytes) of the main tensor of q."""
