@@ -255,8 +255,8 @@ OP_NAMES = ["plain", "plain_f32", "seda", "decomposed", "decomposed_seda", "dequ
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5_plain", help="c5_plain (default) or c2 (smaller tensor, for profiling)")
     ap.add_argument("--op", default="plain", choices=OP_NAMES,
@@ -361,7 +361,7 @@ def run_variants(ops, args, torch, fb4, synth, peak):
     """The other library paths on the same device, each timed like the headline step."""
     q, w, B = ops.q, ops.w, 32
     res = {}
-    steps, warm = max(3, args.steps // 2), 3
+    steps, warm = max(3, min(args.steps // 2, 20)), 3
     for name in OP_NAMES:
         if name == args.op:
             continue
