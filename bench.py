@@ -200,6 +200,12 @@ class Ops:
         meta = self.buf("meta", (T, C // B), torch.int16)
         if name == "plain":
             return (lambda: fb4.fb4_quantize(q.ctx, x, T, C, C, codes, meta)), algorithmic_bytes(T, C)
+        if name == "plain_block16":
+            if "q16" not in self._buf:
+                self._buf["q16"] = fb4.Fb4(device=torch.cuda.current_device(), block_size=16)
+            q16 = self._buf["q16"]
+            meta16 = self.buf("meta16", (T, C // 16), torch.int16)
+            return (lambda: fb4.fb4_quantize(q16.ctx, x, T, C, C, codes, meta16)), T * C * 2.5 + T * (C // 16) * 2
         if name == "plain_f32":
             xf = self.buf("x32", (T, C), torch.float32)
             xf.copy_(x)
@@ -248,7 +254,7 @@ class Ops:
         raise KeyError(name)
 
 
-OP_NAMES = ["plain", "plain_f32", "seda", "decomposed", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
+OP_NAMES = ["plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
             "dequantize_bf16_plain", "dequantize_bf16_decomposed", "to_mxfp8_tiled_scales"]
 
 
@@ -369,10 +375,16 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         total, per = time_steps(fn, steps, warm, torch)
         ms = total / steps
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
-                     "kernel_variant": q.last_variant if name in ("plain", "plain_f32", "seda", "decomposed",
+                     "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "seda", "decomposed",
                                                                          "decomposed_seda") else "decode"}
         if name == "dequantize_f32_decomposed":
             ops.drop("out32")
+        if name == "plain_block16":
+            if "q16" not in self._buf:
+                self._buf["q16"] = fb4.Fb4(device=torch.cuda.current_device(), block_size=16)
+            q16 = self._buf["q16"]
+            meta16 = self.buf("meta16", (T, C // 16), torch.int16)
+            return (lambda: fb4.fb4_quantize(q16.ctx, x, T, C, C, codes, meta16)), T * C * 2.5 + T * (C // 16) * 2
         if name == "plain_f32":
             ops.drop("x32")
     ops.drop("out16")

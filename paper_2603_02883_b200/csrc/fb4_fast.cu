@@ -260,7 +260,7 @@ struct TilePos {
   }
 };
 
-template <bool SEDA, bool DECOMP>
+template <bool SEDA, bool DECOMP, bool B16>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
                          FastParams p, Fb4RowExtras ex) {
@@ -416,49 +416,80 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
     uint32_t a[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) a[i] = w[i] & 0x7fff7fffu;
-    uint32_t g2[4];   // (group 2q+1 max << 16) | group 2q max
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint32_t m0 = __vmaxu2(a[4 * q], a[4 * q + 1]);
-      const uint32_t m1 = __vmaxu2(a[4 * q + 2], a[4 * q + 3]);
-      g2[q] = __vmaxu2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));
-    }
-    const uint32_t mm = __vmaxu2(__vmaxu2(g2[0], g2[1]), __vmaxu2(g2[2], g2[3]));
-    const uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
-    // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
-    const uint32_t Ec = max(amax16 >> 7, 3u);
-    const float s2 = __uint_as_float((257u - Ec) << 23);   // 2^(3-e)
-    const float sG = s2 * 0x1p-21f;                        // bin in the mantissa of 2.0 + x
-    const float sH = s2 * 0x1p-25f;                        // bin in the mantissa of 0.125 + x
-    const float sL = s2 * 0x1p-5f;                         // bin in the mantissa of 2^17 + x
-    const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax16 << 16), sG, 2.0f)) & 31u;
-
     uint32_t allowed = 0xffffffffu;
     if (SEDA) {
       allowed = maskq[0];
       if (allowed == 0) allowed = 1u;   // precondition violated: stay in bounds
     }
-    // ---- dialect selection; the upper bf16 of a pair keeps the lower one as extra mantissa bits,
-    // which truncation discards
-    float gm[8];
+    // per half of the lane's 32 elements (block size 32: both halves belong to one block):
+    // biased exponent, the two bin scales of the Qvalue lookup, the chosen dialect's table address
+    uint32_t Ech[2];
+    float sHh[2], sLh[2], magich[2];
+    int didh[2];
+    if (!B16) {
+      uint32_t g2[4];   // (group 2q+1 max << 16) | group 2q max
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      gm[2 * q] = __uint_as_float(g2[q] << 16);
-      gm[2 * q + 1] = __uint_as_float(g2[q]);
+      for (int q = 0; q < 4; ++q) {
+        const uint32_t m0 = __vmaxu2(a[4 * q], a[4 * q + 1]);
+        const uint32_t m1 = __vmaxu2(a[4 * q + 2], a[4 * q + 3]);
+        g2[q] = __vmaxu2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));
+      }
+      const uint32_t mm = __vmaxu2(__vmaxu2(g2[0], g2[1]), __vmaxu2(g2[2], g2[3]));
+      const uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
+      // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
+      const uint32_t Ec = max(amax16 >> 7, 3u);
+      const float s2 = __uint_as_float((257u - Ec) << 23);   // 2^(3-e)
+      const float sG = s2 * 0x1p-21f;                        // bin in the mantissa of 2.0 + x
+      const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax16 << 16), sG, 2.0f)) & 31u;
+      // ---- dialect selection; the upper bf16 of a pair keeps the lower one as extra mantissa bits,
+      // which truncation discards
+      float gm[8];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        gm[2 * q] = __uint_as_float(g2[q] << 16);
+        gm[2 * q + 1] = __uint_as_float(g2[q]);
+      }
+      const int did = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_base);
+      Ech[0] = Ech[1] = Ec;
+      sHh[0] = sHh[1] = s2 * 0x1p-25f;                       // bin in the mantissa of 0.125 + x
+      sLh[0] = sLh[1] = s2 * 0x1p-5f;                        // bin in the mantissa of 2^17 + x
+      didh[0] = didh[1] = did;
+    } else {
+      // block size 16: the lane's two halves are two blocks; a group is the two elements of one register
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        uint32_t gx[8];   // group maximum in both halves of the register
+#pragma unroll
+        for (int k = 0; k < 8; ++k) gx[k] = __vmaxu2(a[8 * h + k], __byte_perm(a[8 * h + k], 0u, 0x1032));
+        const uint32_t mm = __vmaxu2(__vmaxu2(__vmaxu2(gx[0], gx[1]), __vmaxu2(gx[2], gx[3])),
+                                     __vmaxu2(__vmaxu2(gx[4], gx[5]), __vmaxu2(gx[6], gx[7])));
+        const uint32_t Ec = max((mm & 0xffffu) >> 7, 3u);
+        const float s2 = __uint_as_float((257u - Ec) << 23);
+        const float sG = s2 * 0x1p-21f;
+        const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(mm), sG, 2.0f)) & 31u;
+        float gm[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) gm[k] = __uint_as_float(gx[k]);   // the low copy is truncated away
+        Ech[h] = Ec;
+        sHh[h] = s2 * 0x1p-25f;
+        sLh[h] = s2 * 0x1p-5f;
+        didh[h] = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_base);
+      }
     }
-    const int did = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_base);
     // ---- Qvalue: one lookup per element pair.  124*36 + 144 = 9*512, so the exponent fields of
     // 36*bits(0.125 + ..) + bits(2^17 + ..) cancel mod 2^32 and leave table + 36*bin_hi + bin_lo.
-    const float magic_lo = __uint_as_float(0x48000000u + pair_base + (uint32_t)did * kPairStride);
+    magich[0] = __uint_as_float(0x48000000u + pair_base + (uint32_t)didh[0] * kPairStride);
+    magich[1] = B16 ? __uint_as_float(0x48000000u + pair_base + (uint32_t)didh[1] * kPairStride) : magich[0];
     uint32_t cw[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
+      const int h = B16 ? (q >> 1) : 0;
       uint32_t b[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const uint32_t av = a[4 * q + j];
-        const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sH, 0.125f));
-        const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sL, magic_lo));
+        const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sHh[h], 0.125f));
+        const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sLh[h], magich[h]));
         b[j] = lds_u8(th * (uint32_t)kPairMul + tl);
       }
       const uint32_t idx = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
@@ -470,7 +501,11 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
     }
     if (active) {
       *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-      p.meta[row * nblk + blk] = (uint16_t)((Ec - 3u) | ((uint32_t)did << 8));
+      if (B16)   // two records
+        *reinterpret_cast<uint32_t*>(p.meta + (row * nblk + blk) * 2) =
+            ((Ech[0] - 3u) | ((uint32_t)didh[0] << 8)) | (((Ech[1] - 3u) | ((uint32_t)didh[1] << 8)) << 16);
+      else
+        p.meta[row * nblk + blk] = (uint16_t)((Ech[0] - 3u) | ((uint32_t)didh[0] << 8));
     }
     if (DECOMP) {
       int64_t srow = -1;
@@ -487,7 +522,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
       }
       if (srow >= 0) {   // warp-uniform: a tile lies inside one token
         uint32_t rcw[4], rmeta;
-        residual_block<SEDA>(w, cw, did, Ec, allowed, tb, qerr_base, pair_base, rcw, &rmeta);
+        residual_block<SEDA>(w, cw, didh[0], Ech[0], allowed, tb, qerr_base, pair_base, rcw, &rmeta);
         if (active) {
           *reinterpret_cast<uint4*>(ex.res_codes + srow * code_row_bytes + blk * 16) =
               make_uint4(rcw[0], rcw[1], rcw[2], rcw[3]);
@@ -668,10 +703,10 @@ constexpr size_t kSmemBytes =
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
 static_assert(sizeof(SmemTables) % 16 == 0, "bulk copy size; mbarriers behind the tables stay 8-byte aligned");
 
-template <bool SEDA, bool DECOMP>
+template <bool SEDA, bool DECOMP, bool B16>
 cudaError_t launch(const CUtensorMap& map, const SmemTables* tables, const FastParams& p, const Fb4RowExtras& ex,
                    int grid, cudaStream_t stream) {
-  fb4_quantize_fast_kernel<SEDA, DECOMP><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
+  fb4_quantize_fast_kernel<SEDA, DECOMP, B16><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
   return cudaGetLastError();
 }
 
@@ -753,28 +788,25 @@ bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes
 
 // Opt in to the kernel's dynamic shared memory on the current device (once per context).
 cudaError_t fb4_fast_prepare_device() {
-  cudaError_t e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, false>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kSmemBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kSmemBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kSmemBytes);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kSmemBytesF32);
+  const int bytes = (int)kSmemBytes;
+  const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  cudaError_t e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, false, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, false, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, true, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, true, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, false, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, false, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
   return e;
 }
 
-bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {
+// Block size 32 with every extension; block size 16 for plain and SeDA calls (a residual pass on
+// 16-element blocks takes the generic kernel).
+bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, bool residual_pass) {
   const fb4_config& c = ctx->cfg;
   if (!ctx->fast_ok || !ctx->d_fast_tables) return false;
-  if (c.block_size != 32 || c.num_groups != 8 || c.select_mode != 0 || c.exp_min != -124 || c.exp_max != 127)
-    return false;
+  if (c.num_groups != 8 || c.select_mode != 0 || c.exp_min != -124 || c.exp_max != 127) return false;
+  if (c.block_size != 32 && (c.block_size != 16 || residual_pass)) return false;
   if (C % 64 != 0 || (ld & 7) || (reinterpret_cast<uintptr_t>(x) & 15)) return false;
   if (T > 0x7fffffffLL || C / 64 > 0x7fffffffLL) return false;
   return encode_tiled_fn() != nullptr;
@@ -809,10 +841,14 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   p.step_slots = (int32_t)(p.step_rows / p.sal_tile);
   p.step_rem = (int32_t)(p.step_rows % p.sal_tile);
   const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
-  if (seda && decomp) return launch<true, true>(map, tables, p, ex, grid, stream);
-  if (seda) return launch<true, false>(map, tables, p, ex, grid, stream);
-  if (decomp) return launch<false, true>(map, tables, p, ex, grid, stream);
-  return launch<false, false>(map, tables, p, ex, grid, stream);
+  if (ctx->cfg.block_size == 16) {
+    if (seda) return launch<true, false, true>(map, tables, p, ex, grid, stream);
+    return launch<false, false, true>(map, tables, p, ex, grid, stream);
+  }
+  if (seda && decomp) return launch<true, true, false>(map, tables, p, ex, grid, stream);
+  if (seda) return launch<true, false, false>(map, tables, p, ex, grid, stream);
+  if (decomp) return launch<false, true, false>(map, tables, p, ex, grid, stream);
+  return launch<false, false, false>(map, tables, p, ex, grid, stream);
 }
 
 bool fb4_fast_f32_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {

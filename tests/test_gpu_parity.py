@@ -244,3 +244,37 @@ def test_f32_input(cfg):
             assert_same_quantized(q.quantize(view), orc.quantize_f32(np.ascontiguousarray(x[:, :64]), FB), "f32 strided")
     assert q.device_status == 0
     q.close()
+
+
+def test_block16_fast_kernel_plain_and_seda():
+    """Block size 16 takes the TMA-staged kernel for plain and SeDA calls (two blocks per lane) and
+    the generic kernel when a residual pass is asked for; both equal the oracle."""
+    q = fb4.Fb4(block_size=16)
+    ocfg = orc.Config(block_size=16)
+    w = synth.Workload("t", T=300, C=3072, seed=51, kind=1, n_outlier=15, outlier_gain=50.0, seda=True, n_clusters=9,
+                       cluster_seed=52, score_seed=53)
+    bits = synth.activation(w)
+    cid, masks = synth.clusters(w)
+    masks = masks.copy()
+    masks[2] = 0x0000F0F3                      # cuts stage-1 groups
+    masks[5] = 1 << 30
+    cid = cid.copy()
+    cid[10:20] = -1
+    x = to_dev_bf16(bits)
+    dcid, dmask = torch.from_numpy(cid).cuda(), torch.from_numpy(masks.view(np.int32)).cuda()
+    ref_plain = orc.quantize(bits, FB, ocfg)
+    ref_seda = orc.quantize(bits, FB, ocfg, cluster_id=cid, cluster_mask=masks)
+    for variant, name in ((0, "fast"), (1, "generic")):
+        q.set_kernel_variant(variant)
+        assert_same_quantized(q.quantize(x), ref_plain, f"b16 plain {name}")
+        assert q.last_variant == name
+        assert_same_quantized(q.quantize(x, dcid, dmask), ref_seda, f"b16 seda {name}")
+        assert q.last_variant == name
+    q.set_kernel_variant(0)
+    sal = orc.select_salient(synth.scores(w), 20)
+    got = q.quantize_decomposed(x, torch.from_numpy(synth.scores(w)).cuda(), 20)
+    assert q.last_variant == "generic"
+    assert_same_quantized(got, orc.quantize(bits, FB, ocfg, salient_idx=sal), "b16 decomposed")
+    assert_same_bits_f32(q.dequantize(q.quantize(x)), orc.dequantize(ref_plain, FB, 16), "b16 dequant")
+    assert q.device_status == 0
+    q.close()
