@@ -159,8 +159,9 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "gelem_per_s": rows * w.C / dt / 1e9,
-        "config": {"workload": "plain FB4 quantize, 75600x12288 bf16 (config-5 tensor), block 32, full formatbook",
-                   "sample": sample},
+        "config": {"workload": f"plain FB4 quantize, {w.T}x{w.C} bf16 (config-5 tensor), block 32, "
+                               "full formatbook, two-stage selection",
+                   "per_gpu_tokens": w.T, "channels": w.C, "block_size": 32, "sample": sample},
         "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
