@@ -344,6 +344,8 @@ def main():
                      "launch_ms_mean": kernel_ms, "launch_ms_min": float(np.min(per))},
     }
 
+    if rank == 0 and args.op == "plain":
+        out["quality"] = quality_report(ops, torch, fb4)
     if rank == 0 and not args.no_variants:
         out["variants"] = run_variants(ops, args, torch, fb4, synth, peak)
     del ops
@@ -364,6 +366,24 @@ def main():
         dist.destroy_process_group()
 
 
+def quality_report(ops, torch, fb4):
+    """What the plain step produced: mean squared error of the decoded tensor (fp64 accumulation,
+    over the first 8192 tokens) and how often each dialect was chosen."""
+    q, x, T, C, B = ops.q, ops.x, ops.T, ops.C, ops.B
+    codes, meta = ops.buf("codes", (T, C // 2), torch.uint8), ops.buf("meta", (T, C // B), torch.int16)
+    fb4.fb4_quantize(q.ctx, x, T, C, C, codes, meta)
+    n = min(T, 8192)
+    dec = torch.empty((n, C), dtype=torch.float32, device="cuda")
+    fb4.fb4_dequantize(q.ctx, codes[:n], meta[:n], n, C, None, 0, None, None, dec, 0)
+    xs = x[:n].double()
+    mse = float(((dec.double() - xs) ** 2).mean())
+    power = float((xs ** 2).mean())
+    did = (meta.to(torch.int32) >> 8) & 31
+    hist = torch.bincount(did.flatten(), minlength=32).double()
+    return {"mse_first_8192_tokens": mse, "signal_power": power, "sqnr_db": 10 * float(np.log10(power / mse)),
+            "dialect_share": [round(float(v), 5) for v in (hist / hist.sum()).tolist()]}
+
+
 def run_variants(ops, args, torch, fb4, synth, peak):
     """The other library paths on the same device, each timed like the headline step."""
     q, w, B = ops.q, ops.w, 32
@@ -380,12 +400,6 @@ def run_variants(ops, args, torch, fb4, synth, peak):
                                                                          "decomposed_seda") else "decode"}
         if name == "dequantize_f32_decomposed":
             ops.drop("out32")
-        if name == "plain_block16":
-            if "q16" not in self._buf:
-                self._buf["q16"] = fb4.Fb4(device=torch.cuda.current_device(), block_size=16)
-            q16 = self._buf["q16"]
-            meta16 = self.buf("meta16", (T, C // 16), torch.int16)
-            return (lambda: fb4.fb4_quantize(q16.ctx, x, T, C, C, codes, meta16)), T * C * 2.5 + T * (C // 16) * 2
         if name == "plain_f32":
             ops.drop("x32")
     ops.drop("out16")
