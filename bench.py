@@ -31,8 +31,8 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this
 # workload, from the ncu capture summarised in profiles/fb4_quantize_fast_c5_plain_dram_bytes.md
-# (1 858 100 736 B read + 502 537 216 B written; set back to None whenever that kernel changes).
-NCU_TRAFFIC_BYTES = 2360637952
+# (1 858 055 936 B read + 502 568 448 B written; set back to None whenever that kernel changes).
+NCU_TRAFFIC_BYTES = 2360624384
 
 
 def algorithmic_bytes(T: int, C: int, B: int = 32, n_res_rows: int = 0, seda: bool = False,
@@ -344,7 +344,7 @@ def main():
                      "launch_ms_mean": kernel_ms, "launch_ms_min": float(np.min(per))},
     }
 
-    if rank == 0 and args.op == "plain":
+    if rank == 0 and args.op == "plain" and not args.no_variants:
         out["quality"] = quality_report(ops, torch, fb4)
     if rank == 0 and not args.no_variants:
         out["variants"] = run_variants(ops, args, torch, fb4, synth, peak)

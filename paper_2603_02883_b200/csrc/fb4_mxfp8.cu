@@ -48,10 +48,12 @@ fb4_to_mxfp8_kernel(const uint4* __restrict__ codes, const uint16_t* __restrict_
   __syncthreads();
   const int64_t total = T * n_col;
   const int64_t col_tiles = (n_col + 3) >> 2;
+  const bool small = total < 0xffffffffLL;   // block indices fit 32 bits: row/column by 32-bit division
   constexpr int64_t kStep = (int64_t)kThreads * kUnroll;
-  for (int64_t base = (int64_t)blockIdx.x * kStep; base < total; base += (int64_t)gridDim.x * kStep) {
-    uint4 cw[kUnroll];
-    uint32_t m[kUnroll];
+  const int64_t stride = (int64_t)gridDim.x * kStep;
+  uint4 cw[kUnroll];
+  uint32_t m[kUnroll];
+  auto load = [&](int64_t base) {
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const int64_t b = base + u * kThreads + threadIdx.x;
@@ -60,16 +62,28 @@ fb4_to_mxfp8_kernel(const uint4* __restrict__ codes, const uint16_t* __restrict_
         m[u] = (uint32_t)__ldg(meta + b);
       }
     }
+  };
+  int64_t base = (int64_t)blockIdx.x * kStep;
+  if (base < total) load(base);
+  for (; base < total; base += stride) {
+    uint4 c[kUnroll];
+    uint32_t mm[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      c[u] = cw[u];
+      mm[u] = m[u];
+    }
+    if (base + stride < total) load(base + stride);   // the next step's loads fly while this one is converted
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const int64_t b = base + u * kThreads + threadIdx.x;
       if (b >= total) continue;
-      const uint2 fb = fb8[(m[u] >> 8) & 31u];
+      const uint2 fb = fb8[(mm[u] >> 8) & 31u];
       uint32_t o[8];
-      convert_word(cw[u].x, fb, o[0], o[1]);
-      convert_word(cw[u].y, fb, o[2], o[3]);
-      convert_word(cw[u].z, fb, o[4], o[5]);
-      convert_word(cw[u].w, fb, o[6], o[7]);
+      convert_word(c[u].x, fb, o[0], o[1]);
+      convert_word(c[u].y, fb, o[2], o[3]);
+      convert_word(c[u].z, fb, o[4], o[5]);
+      convert_word(c[u].w, fb, o[6], o[7]);
       uint8_t* dst = e4m3 + b * 32;
       if (out_aligned32) {
         asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(o[0]), "r"(o[1]),
@@ -78,8 +92,20 @@ fb4_to_mxfp8_kernel(const uint4* __restrict__ codes, const uint16_t* __restrict_
         reinterpret_cast<uint4*>(dst)[0] = make_uint4(o[0], o[1], o[2], o[3]);
         reinterpret_cast<uint4*>(dst)[1] = make_uint4(o[4], o[5], o[6], o[7]);
       }
-      const int64_t row = b / n_col;
-      scales[scale_offset(row, b - row * n_col, n_col, col_tiles, tiled)] = (uint8_t)m[u];   // E8M0 of 2^(e-3)
+      int64_t off = b;   // row-major: the block index itself
+      if (tiled) {
+        int64_t row, col;
+        if (small) {
+          const uint32_t r32 = (uint32_t)b / (uint32_t)n_col;
+          row = r32;
+          col = (uint32_t)b - r32 * (uint32_t)n_col;
+        } else {
+          row = b / n_col;
+          col = b - row * n_col;
+        }
+        off = scale_offset(row, col, n_col, col_tiles, 1);
+      }
+      scales[off] = (uint8_t)mm[u];   // E8M0 of 2^(e-3)
     }
   }
   if (tiled) {
