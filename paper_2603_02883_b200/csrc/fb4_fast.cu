@@ -73,6 +73,7 @@ struct FastParams {
   uint8_t* codes;
   uint16_t* meta;
   uint32_t* status;   // device word: bit 0 = a TMA wait ran out
+  uint32_t ec_lo, ec_hi;   // clamp of the biased block exponent (CLAMP kernels): exp_min + 127, exp_max + 127
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -260,7 +261,7 @@ struct TilePos {
   }
 };
 
-template <bool SEDA, bool DECOMP, bool B16>
+template <bool SEDA, bool DECOMP, bool B16, bool CLAMP>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
                          FastParams p, Fb4RowExtras ex) {
@@ -435,9 +436,20 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
         g2[q] = __vmaxu2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));
       }
       const uint32_t mm = __vmaxu2(__vmaxu2(g2[0], g2[1]), __vmaxu2(g2[2], g2[3]));
-      const uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
+      uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
       // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
-      const uint32_t Ec = max(amax16 >> 7, 3u);
+      uint32_t Ec = max(amax16 >> 7, 3u);
+      if (CLAMP) {
+        // clamped exponent range: magnitudes that would normalise to 16 or more saturate at the
+        // largest value of bin 31 (biased exponent Ec, mantissa all ones)
+        Ec = min(max(amax16 >> 7, p.ec_lo), p.ec_hi);
+        const uint32_t bound = ((Ec << 7) | 0x7fu) * 0x10001u;
+        amax16 = min(amax16, bound & 0xffffu);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) a[i] = __vminu2(a[i], bound);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) g2[q] = __vminu2(g2[q], bound);
+      }
       const float s2 = __uint_as_float((257u - Ec) << 23);   // 2^(3-e)
       const float sG = s2 * 0x1p-21f;                        // bin in the mantissa of 2.0 + x
       const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax16 << 16), sG, 2.0f)) & 31u;
@@ -461,9 +473,19 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
         uint32_t gx[8];   // group maximum in both halves of the register
 #pragma unroll
         for (int k = 0; k < 8; ++k) gx[k] = __vmaxu2(a[8 * h + k], __byte_perm(a[8 * h + k], 0u, 0x1032));
-        const uint32_t mm = __vmaxu2(__vmaxu2(__vmaxu2(gx[0], gx[1]), __vmaxu2(gx[2], gx[3])),
-                                     __vmaxu2(__vmaxu2(gx[4], gx[5]), __vmaxu2(gx[6], gx[7])));
-        const uint32_t Ec = max((mm & 0xffffu) >> 7, 3u);
+        uint32_t mm = __vmaxu2(__vmaxu2(__vmaxu2(gx[0], gx[1]), __vmaxu2(gx[2], gx[3])),
+                               __vmaxu2(__vmaxu2(gx[4], gx[5]), __vmaxu2(gx[6], gx[7])));
+        uint32_t Ec = max((mm & 0xffffu) >> 7, 3u);
+        if (CLAMP) {
+          Ec = min(max((mm & 0xffffu) >> 7, p.ec_lo), p.ec_hi);
+          const uint32_t bound = ((Ec << 7) | 0x7fu) * 0x10001u;
+          mm = __vminu2(mm, bound);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            a[8 * h + k] = __vminu2(a[8 * h + k], bound);
+            gx[k] = __vminu2(gx[k], bound);
+          }
+        }
         const float s2 = __uint_as_float((257u - Ec) << 23);
         const float sG = s2 * 0x1p-21f;
         const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(mm), sG, 2.0f)) & 31u;
@@ -703,10 +725,10 @@ constexpr size_t kSmemBytes =
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
 static_assert(sizeof(SmemTables) % 16 == 0, "bulk copy size; mbarriers behind the tables stay 8-byte aligned");
 
-template <bool SEDA, bool DECOMP, bool B16>
+template <bool SEDA, bool DECOMP, bool B16, bool CLAMP>
 cudaError_t launch(const CUtensorMap& map, const SmemTables* tables, const FastParams& p, const Fb4RowExtras& ex,
                    int grid, cudaStream_t stream) {
-  fb4_quantize_fast_kernel<SEDA, DECOMP, B16><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
+  fb4_quantize_fast_kernel<SEDA, DECOMP, B16, CLAMP><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
   return cudaGetLastError();
 }
 
@@ -790,23 +812,33 @@ bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes
 cudaError_t fb4_fast_prepare_device() {
   const int bytes = (int)kSmemBytes;
   const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-  cudaError_t e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, false, false>, attr, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, false, false>, attr, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, true, false>, attr, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, true, false>, attr, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<false, false, true>, attr, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<true, false, true>, attr, bytes);
+  cudaError_t e = cudaSuccess;
+#define FB4_OPT_IN(...) \
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_fast_kernel<__VA_ARGS__>, attr, bytes)
+  FB4_OPT_IN(false, false, false, false);
+  FB4_OPT_IN(true, false, false, false);
+  FB4_OPT_IN(false, true, false, false);
+  FB4_OPT_IN(true, true, false, false);
+  FB4_OPT_IN(false, false, true, false);
+  FB4_OPT_IN(true, false, true, false);
+  FB4_OPT_IN(false, false, false, true);
+  FB4_OPT_IN(true, false, false, true);
+  FB4_OPT_IN(false, false, true, true);
+  FB4_OPT_IN(true, false, true, true);
+#undef FB4_OPT_IN
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
   return e;
 }
 
-// Block size 32 with every extension; block size 16 for plain and SeDA calls (a residual pass on
-// 16-element blocks takes the generic kernel).
+// Block size 32 with every extension; block size 16 and clamped exponent ranges (the 5-bit exponent
+// of Sec. 3.1) for plain and SeDA calls: their residual pass takes the generic kernel.
 bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, bool residual_pass) {
   const fb4_config& c = ctx->cfg;
   if (!ctx->fast_ok || !ctx->d_fast_tables) return false;
-  if (c.num_groups != 8 || c.select_mode != 0 || c.exp_min != -124 || c.exp_max != 127) return false;
-  if (c.block_size != 32 && (c.block_size != 16 || residual_pass)) return false;
+  if (c.num_groups != 8 || c.select_mode != 0) return false;
+  const bool clamp = c.exp_min != -124 || c.exp_max != 127;
+  if (c.block_size != 32 && c.block_size != 16) return false;
+  if ((c.block_size == 16 || clamp) && residual_pass) return false;
   if (C % 64 != 0 || (ld & 7) || (reinterpret_cast<uintptr_t>(x) & 15)) return false;
   if (T > 0x7fffffffLL || C / 64 > 0x7fffffffLL) return false;
   return encode_tiled_fn() != nullptr;
@@ -841,14 +873,22 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   p.step_slots = (int32_t)(p.step_rows / p.sal_tile);
   p.step_rem = (int32_t)(p.step_rows % p.sal_tile);
   const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
-  if (ctx->cfg.block_size == 16) {
-    if (seda) return launch<true, false, true>(map, tables, p, ex, grid, stream);
-    return launch<false, false, true>(map, tables, p, ex, grid, stream);
+  p.ec_lo = (uint32_t)(ctx->cfg.exp_min + 127);
+  p.ec_hi = (uint32_t)(ctx->cfg.exp_max + 127);
+  const bool b16 = ctx->cfg.block_size == 16;
+  const bool clamp = ctx->cfg.exp_min != -124 || ctx->cfg.exp_max != 127;
+  if (clamp) {
+    if (b16) return seda ? launch<true, false, true, true>(map, tables, p, ex, grid, stream)
+                         : launch<false, false, true, true>(map, tables, p, ex, grid, stream);
+    return seda ? launch<true, false, false, true>(map, tables, p, ex, grid, stream)
+                : launch<false, false, false, true>(map, tables, p, ex, grid, stream);
   }
-  if (seda && decomp) return launch<true, true, false>(map, tables, p, ex, grid, stream);
-  if (seda) return launch<true, false, false>(map, tables, p, ex, grid, stream);
-  if (decomp) return launch<false, true, false>(map, tables, p, ex, grid, stream);
-  return launch<false, false, false>(map, tables, p, ex, grid, stream);
+  if (b16) return seda ? launch<true, false, true, false>(map, tables, p, ex, grid, stream)
+                       : launch<false, false, true, false>(map, tables, p, ex, grid, stream);
+  if (seda && decomp) return launch<true, true, false, false>(map, tables, p, ex, grid, stream);
+  if (seda) return launch<true, false, false, false>(map, tables, p, ex, grid, stream);
+  if (decomp) return launch<false, true, false, false>(map, tables, p, ex, grid, stream);
+  return launch<false, false, false, false>(map, tables, p, ex, grid, stream);
 }
 
 bool fb4_fast_f32_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {

@@ -278,3 +278,30 @@ def test_block16_fast_kernel_plain_and_seda():
     assert_same_bits_f32(q.dequantize(q.quantize(x)), orc.dequantize(ref_plain, FB, 16), "b16 dequant")
     assert q.device_status == 0
     q.close()
+
+
+@pytest.mark.parametrize("cfg", [dict(exp_min=-15, exp_max=16), dict(block_size=16, exp_min=-15, exp_max=16),
+                                 dict(exp_min=-3, exp_max=2), dict(block_size=16, exp_min=0, exp_max=0)],
+                         ids=["exp5", "b16-exp5", "narrow", "b16-single-exponent"])
+def test_clamped_exponent_fast_kernel(cfg):
+    """The paper's 5-bit shared exponent (and narrower clamps, which saturate many elements) in the
+    TMA-staged kernel, plain and SeDA, against the oracle and the generic kernel."""
+    q = fb4.Fb4(**cfg)
+    ocfg = orc.Config(**cfg)
+    w = synth.Workload("t", T=200, C=1024 + 128, seed=61, kind=1, n_outlier=6, outlier_gain=50.0, seda=True,
+                       n_clusters=4, cluster_seed=62)
+    cid, masks = synth.clusters(w)
+    for bits in (synth.activation(w), np.tile(edge_blocks(), (5, 18))[:200]):
+        x = to_dev_bf16(bits)
+        ref = orc.quantize(bits, FB, ocfg)
+        ref_seda = orc.quantize(bits, FB, ocfg, cluster_id=cid, cluster_mask=masks)
+        for variant, name in ((0, "fast"), (1, "generic")):
+            q.set_kernel_variant(variant)
+            got = q.quantize(x)
+            assert q.last_variant == name
+            assert_same_quantized(got, ref, f"clamped {cfg} {name}")
+            got = q.quantize(x, torch.from_numpy(cid).cuda(), torch.from_numpy(masks.view(np.int32)).cuda())
+            assert_same_quantized(got, ref_seda, f"clamped seda {cfg} {name}")
+        assert_same_bits_f32(q.dequantize(got), orc.dequantize(ref_seda, FB, cfg.get("block_size", 32)), "clamped dequant")
+    assert q.device_status == 0
+    q.close()
