@@ -90,23 +90,33 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
   constexpr int64_t kStep = (int64_t)kDecodeThreads * kDecodeUnroll;
   const int64_t stride = (int64_t)gridDim.x * kStep;
 
-  uint32_t cw[kDecodeUnroll][4], m[kDecodeUnroll];
+  // m = the metadata records of the lane's whole quad (4 x 16 bits): after the transpose a lane
+  // decodes one word of each of the quad's blocks and needs all four records
+  uint32_t cw[kDecodeUnroll][4];
+  uint2 m[kDecodeUnroll];
   auto load = [&](int64_t base) {
 #pragma unroll
     for (int u = 0; u < kDecodeUnroll; ++u) {
       const int64_t b = base + u * kDecodeThreads + threadIdx.x;
+      const int64_t qb = b & ~3ll;
       cw[u][0] = cw[u][1] = cw[u][2] = cw[u][3] = 0u;
-      m[u] = 0u;
-      if (b < total_blocks) {
-        load_block_codes<4>(codes + b * 4, cw[u]);
-        m[u] = (uint32_t)__ldg(meta + b);
+      m[u] = make_uint2(0u, 0u);
+      if (b < total_blocks) load_block_codes<4>(codes + b * 4, cw[u]);
+      if (qb + 4 <= total_blocks) {
+        m[u] = __ldg(reinterpret_cast<const uint2*>(meta + qb));   // 8-byte aligned: qb is a multiple of 4
+      } else if (qb < total_blocks) {                               // ragged last quad
+        uint32_t r[4] = {0u, 0u, 0u, 0u};
+        for (int i = 0; i < 4; ++i)
+          if (qb + i < total_blocks) r[i] = (uint32_t)__ldg(meta + qb + i);
+        m[u] = make_uint2(r[0] | (r[1] << 16), r[2] | (r[3] << 16));
       }
     }
   };
   int64_t base = (int64_t)blockIdx.x * kStep;
   if (base < total_blocks) load(base);
   for (; base < total_blocks; base += stride) {
-    uint32_t c[kDecodeUnroll][4], mm[kDecodeUnroll];
+    uint32_t c[kDecodeUnroll][4];
+    uint2 mm[kDecodeUnroll];
 #pragma unroll
     for (int u = 0; u < kDecodeUnroll; ++u) {
       mm[u] = m[u];
@@ -120,7 +130,7 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
       const int64_t qb = base + u * kDecodeThreads + (threadIdx.x & ~3);   // first block of this quad
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint32_t mi = __shfl_sync(0xffffffffu, mm[u], (lane & ~3) + i);
+        const uint32_t mi = ((i & 2) ? mm[u].y : mm[u].x) >> (16 * (i & 1)) & 0xffffu;
         if (qb + i < total_blocks) {
           uint32_t pr[4];
           decode_word(c[u][i], fb_bf16[(mi >> 8) & 31u], scale_bf16x2(mi), pr);
