@@ -60,8 +60,10 @@
  * choices lie in the mask; per-tile argmax by brute force; sub-formatbooks on
  * hand-counted cases, one dialect per bucket, and a constrained tensor giving
  * back the sub-formatbook it was constrained to.
- * Parity unpinned: the formatbook VALUES (the paper's table is only in Fig. 2a)
- * and any worked numeric example (the paper prints none).
+ * Parity unpinned: the formatbook VALUES (the paper's table is only in Fig. 2a),
+ * any worked numeric example (the paper prints none), and the tiled order of the
+ * MXFP8 scale bytes against a GEMM that consumes it (pinned only by its stated
+ * properties).
  */
 #include <math.h>
 #include <stdint.h>
