@@ -236,6 +236,25 @@ int64_t fb4o_select_salient(const float *score, int64_t T, int32_t tile, int32_t
   return n;
 }
 
+/* The other reading of "salient tokens = the top 5 % by score": the k highest-scoring tokens of the
+ * whole sequence (ties -> lowest index), listed in ascending token order.  Plain selection sort of
+ * the candidates, k rounds. */
+int64_t fb4o_select_salient_topk(const float *score, int64_t T, int64_t k, int32_t *salient_idx) {
+  if (T < 0 || k < 0 || k > T) return -1;
+  uint8_t *taken = (uint8_t *)calloc((size_t)(T > 0 ? T : 1), 1);
+  if (!taken) return -1;
+  for (int64_t r = 0; r < k; ++r) {
+    int64_t arg = -1;
+    for (int64_t t = 0; t < T; ++t)
+      if (!taken[t] && (arg < 0 || score[t] > score[arg])) arg = t;   /* first maximum = lowest index */
+    taken[arg] = 1;
+  }
+  int64_t n = 0;
+  for (int64_t t = 0; t < T; ++t) if (taken[t]) salient_idx[n++] = (int32_t)t;
+  free(taken);
+  return n;
+}
+
 /*
  * Quantize a T x C bf16 tensor (bit patterns, `ld` elements between rows).
  * Optional SeDA tables (cluster_id NULL => unconstrained).  Optional residual

@@ -67,6 +67,8 @@ def lib():
         L.fb4o_default_stage1.restype = None
         L.fb4o_select_salient.argtypes = [vp, i64, i32, vp]
         L.fb4o_select_salient.restype = i64
+        L.fb4o_select_salient_topk.argtypes = [vp, i64, i64, vp]
+        L.fb4o_select_salient_topk.restype = i64
         L.fb4o_quantize.argtypes = [vp, i64, i64, i64, ctypes.POINTER(_Cfg), vp, vp,
                                     vp, vp, i32, vp, i64, vp, vp, vp, vp, vp]
         L.fb4o_quantize.restype = ctypes.c_int
@@ -116,6 +118,15 @@ def select_salient(score, tile: int) -> np.ndarray:
     n = lib().fb4o_select_salient(_p(s), T, tile, _p(out))
     assert n >= 0
     return out[:n].copy()
+
+
+def select_salient_topk(score, k: int) -> np.ndarray:
+    """the k highest-scoring tokens of the whole sequence (ties -> lowest index), ascending"""
+    s = _c(score, np.float32)
+    out = np.zeros(max(1, k), dtype=np.int32)
+    n = lib().fb4o_select_salient_topk(_p(s), s.shape[0], k, _p(out))
+    assert n == k
+    return out[:k].copy()
 
 
 @dataclass

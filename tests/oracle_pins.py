@@ -534,6 +534,24 @@ def pin_salient_is_per_tile_argmax(seed=5):
         assert np.all(np.diff(idx) > 0)
 
 
+def pin_salient_topk(seed=12):
+    """Global reading of the salient set: the k largest scores, ties to the lowest index, ascending."""
+    rng = np.random.default_rng(seed)
+    s = np.array([0.5, 0.9, 0.1, 0.9, 0.9, 0.2, 0.5], dtype=np.float32)
+    assert list(orc.select_salient_topk(s, 0)) == []
+    assert list(orc.select_salient_topk(s, 1)) == [1]
+    assert list(orc.select_salient_topk(s, 2)) == [1, 3]                 # tie at 0.9: lowest indices first
+    assert list(orc.select_salient_topk(s, 4)) == [0, 1, 3, 4]           # tie at 0.5: index 0 before 6
+    assert list(orc.select_salient_topk(s, 7)) == list(range(7))
+    for T, k in [(50, 3), (333, 17), (1000, 50), (64, 64)]:
+        s = rng.random(T).astype(np.float32)
+        s[rng.integers(0, T, size=T // 4)] = s[1]                         # many ties
+        got = orc.select_salient_topk(s, k)
+        order = np.argsort(-s.astype(np.float64), kind="stable")          # stable: ties keep index order
+        assert np.array_equal(got, np.sort(order[:k]))
+        assert np.all(np.diff(got) > 0)
+
+
 def pin_decomposition(seed=6, n=40):
     """Act = Q(Act) + Delta exactly; Q(Act) + Q(Delta) is never farther from Act than Q(Act)
     in any element; the residual codes decode to the sign of Delta."""
@@ -600,7 +618,7 @@ def pin_mse():
 ALL_PINS = [
     pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
-    pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_decomposition,
+    pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_salient_topk, pin_decomposition,
     pin_dequantize_formula, pin_mse, pin_f32_input, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
     pin_subformatbook_hand_counted,
     pin_subformatbook_one_dialect_per_bucket_and_closed_loop,

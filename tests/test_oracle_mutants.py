@@ -33,6 +33,10 @@ MUTANTS = {
     "residual_not_added": ("val = (float)((double)val + r);", "val = (float)((double)val + 0.0 * r);"),
     "salient_last_on_tie": ("if (score[t] > score[arg]) arg = t;", "if (score[t] >= score[arg]) arg = t;"),
     "salient_min": ("if (score[t] > score[arg]) arg = t;", "if (score[t] < score[arg]) arg = t;"),
+    "topk_ties_to_highest": ("if (!taken[t] && (arg < 0 || score[t] > score[arg])) arg = t;",
+                             "if (!taken[t] && (arg < 0 || score[t] >= score[arg])) arg = t;"),
+    "topk_smallest": ("if (!taken[t] && (arg < 0 || score[t] > score[arg])) arg = t;",
+                      "if (!taken[t] && (arg < 0 || score[t] < score[arg])) arg = t;"),
     "clamp_min_ignored": ("if (e < cfg->exp_min) e = cfg->exp_min;", ";"),
     "zero_block_exponent": ("e = cfg->exp_min;\n  } else {", "e = 0;\n  } else {"),
     "stage1_bucket_shift": ("int bucket = k / 2 < 8 ? 8 : k / 2;", "int bucket = k / 2 < 9 ? 9 : k / 2;"),
