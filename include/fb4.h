@@ -184,6 +184,19 @@ int fb4_select_salient(fb4_ctx* ctx, const float* score, int64_t T, int32_t tile
                        void* stream);
 
 /*
+ * The global alternative to the per-tile selection: the k highest-scoring tokens of the whole
+ * sequence, ties to the lowest index, written in ascending token order (the input format of
+ * fb4_quantize_decomposed_idx).  Sec. 3.3 selects per tile and App. F argues against a global
+ * top-k; this call exists for workloads stated as "the top p % of the tokens by score".
+ * One thread block does the work (a few passes over `score`): meant for sequence lengths, not
+ * for large arrays.
+ *   score       : device float [T] (finite; -0 counts as +0)
+ *   salient_idx : device int32 [k] (out), 0 <= k <= T
+ */
+int fb4_select_salient_topk(fb4_ctx* ctx, const float* score, int64_t T, int64_t k, int32_t* salient_idx,
+                            void* stream);
+
+/*
  * Quantization with activation decomposition (Sec. 3.3): every token is quantized
  * as in fb4_quantize[_seda]; for the salient tokens the residual
  * Delta = x - dequant(Q(x)) is formed in registers (exactly, in fp32), quantized

@@ -262,6 +262,19 @@ int fb4_select_salient(fb4_ctx* ctx, const float* score, int64_t T, int32_t tile
   return FB4_OK;
 }
 
+int fb4_select_salient_topk(fb4_ctx* ctx, const float* score, int64_t T, int64_t k, int32_t* salient_idx,
+                            void* stream) {
+  if (!ctx) return FB4_ERR_INVALID_ARG;
+  if (T < 0 || T > 0x7fffffffLL) return FB4_ERR_SHAPE;
+  if (k < 0 || k > T) return FB4_ERR_INVALID_ARG;
+  if (T == 0 || k == 0) return FB4_OK;
+  if (!score || !salient_idx) return FB4_ERR_INVALID_ARG;
+  cudaError_t e = fb4_launch_select_salient_topk(score, T, k, salient_idx, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
+  ctx->launches += 1;
+  return FB4_OK;
+}
+
 int fb4_quantize_decomposed(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const float* score,
                             int32_t tile, const int32_t* cluster_id, const uint32_t* cluster_mask,
                             int32_t n_clusters, uint8_t* codes, uint16_t* meta, int32_t* salient_idx,

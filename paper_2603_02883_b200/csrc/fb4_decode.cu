@@ -249,6 +249,81 @@ __global__ void fb4_select_salient_kernel(const float* __restrict__ score, int64
   salient_idx[k] = (int32_t)arg;
 }
 
+// The k highest scores of the whole sequence (ties to the lowest index), indices in ascending order:
+// the global reading of "top 5 % of the tokens".  One CTA: a 4-pass radix select finds the k-th
+// largest key, then one ordered pass writes the indices above it and the first few equal to it.
+constexpr int kTopkThreads = 1024;
+
+__device__ __forceinline__ uint32_t score_key(float f) {   // order-preserving; -0 counts as +0
+  uint32_t u = __float_as_uint(f);
+  if (u == 0x80000000u) u = 0u;
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(kTopkThreads)
+fb4_select_salient_topk_kernel(const float* __restrict__ score, int64_t T, int64_t k,
+                               int32_t* __restrict__ salient_idx) {
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t s_prefix, s_remaining;
+  __shared__ uint32_t warp_sums[kTopkThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) { s_prefix = 0u; s_remaining = (uint32_t)k; }
+  for (int pass = 3; pass >= 0; --pass) {
+    if (tid < 256) hist[tid] = 0u;
+    __syncthreads();
+    const uint32_t prefix = s_prefix;
+    const uint32_t high_mask = pass == 3 ? 0u : (0xffffffffu << (8 * (pass + 1)));
+    for (int64_t t = tid; t < T; t += kTopkThreads) {
+      const uint32_t key = score_key(score[t]);
+      if ((key & high_mask) == prefix) atomicAdd(&hist[(key >> (8 * pass)) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid == 0) {   // walk the bins from the top until the k-th largest key falls into one
+      uint32_t remaining = s_remaining;
+      int bin = 255;
+      for (; bin > 0; --bin) {
+        if (hist[bin] >= remaining) break;
+        remaining -= hist[bin];
+      }
+      s_remaining = remaining;
+      s_prefix = prefix | ((uint32_t)bin << (8 * pass));
+    }
+    __syncthreads();
+  }
+  const uint32_t kth = s_prefix;          // key of the k-th largest score
+  const uint32_t quota = s_remaining;     // how many scores equal to it are taken (lowest indices first)
+  uint32_t written = 0, ties_seen = 0;    // uniform across the CTA
+  for (int64_t base = 0; base < T; base += kTopkThreads) {
+    const int64_t t = base + tid;
+    uint32_t g = 0, e = 0;
+    if (t < T) {
+      const uint32_t key = score_key(score[t]);
+      g = key > kth;
+      e = key == kth;
+    }
+    // exclusive counts of greater / equal elements before this thread within the chunk
+    const uint32_t bg = __ballot_sync(0xffffffffu, g), be = __ballot_sync(0xffffffffu, e);
+    const uint32_t lower = (1u << lane) - 1u;
+    uint32_t gb = __popc(bg & lower), eb = __popc(be & lower);
+    if (lane == 0) warp_sums[warp] = (__popc(bg) << 16) | __popc(be);
+    __syncthreads();
+    uint32_t before = 0, total = 0;
+    for (int w = 0; w < kTopkThreads / 32; ++w) {
+      const uint32_t v = warp_sums[w];
+      if (w < warp) before += v;
+      total += v;
+    }
+    __syncthreads();
+    gb += before >> 16;
+    eb += before & 0xffffu;
+    const uint32_t quota_left = quota > ties_seen ? quota - ties_seen : 0u;
+    if (g) salient_idx[written + gb + min(eb, quota_left)] = (int32_t)t;
+    else if (e && eb < quota_left) salient_idx[written + gb + eb] = (int32_t)t;
+    written += (total >> 16) + min(total & 0xffffu, quota_left);
+    ties_seen += total & 0xffffu;
+  }
+}
+
 }  // namespace
 
 cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T,
@@ -307,5 +382,12 @@ cudaError_t fb4_launch_select_salient(const float* score, int64_t T, int32_t til
   const int threads = 128;
   fb4_select_salient_kernel<<<(unsigned)((n_tiles + threads - 1) / threads), threads, 0, stream>>>(
       score, T, tile, salient_idx, n_tiles);
+  return cudaGetLastError();
+}
+
+cudaError_t fb4_launch_select_salient_topk(const float* score, int64_t T, int64_t k, int32_t* salient_idx,
+                                           cudaStream_t stream) {
+  if (T == 0 || k == 0) return cudaSuccess;
+  fb4_select_salient_topk_kernel<<<1, kTopkThreads, 0, stream>>>(score, T, k, salient_idx);
   return cudaGetLastError();
 }

@@ -76,5 +76,7 @@ cudaError_t fb4_launch_quantize_weights(const fb4_ctx* ctx, const void* w, int64
                                         uint8_t* codes, uint16_t* meta, cudaStream_t stream);
 cudaError_t fb4_launch_to_mxfp8(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T, int64_t C,
                                 uint8_t* e4m3, uint8_t* scales, int layout, cudaStream_t stream);
+cudaError_t fb4_launch_select_salient_topk(const float* score, int64_t T, int64_t k, int32_t* salient_idx,
+                                           cudaStream_t stream);
 cudaError_t fb4_launch_select_salient(const float* score, int64_t T, int32_t tile, int32_t* salient_idx,
                                       cudaStream_t stream);

@@ -22,7 +22,7 @@ STATIC_MAX_CLUSTERS = 1024
 
 EXPORTS = [
     "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
-    "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
+    "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_select_salient_topk", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
     "fb4_quantize_weights", "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
 
@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
     L.fb4_build_subformatbook_static.argtypes = [vp, vp, i64, i64, vp, vp, i64, i32, vp, vp]
     L.fb4_build_subformatbook_static.restype = ci
     L.fb4_select_salient.argtypes = [vp, vp, i64, i32, vp, vp]
+    L.fb4_select_salient_topk.argtypes = [vp, vp, i64, i64, vp, vp]
+    L.fb4_select_salient_topk.restype = ci
     L.fb4_quantize_decomposed.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
     L.fb4_quantize_decomposed_idx.argtypes = [vp, vp, i64, i64, i64, vp, i64, vp, vp, i32, vp, vp, vp, vp, vp]
     L.fb4_dequantize.argtypes = [vp, vp, vp, i64, i64, vp, i64, vp, vp, vp, ci, vp]
@@ -88,7 +90,7 @@ def lib() -> ctypes.CDLL:
     L.fb4_mxfp8_scale_bytes.restype = i64
     L.fb4_quantize_host.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp]
     for name in ("fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
-                 "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx",
+                 "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_select_salient_topk", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx",
                  "fb4_dequantize", "fb4_quantize_host", "fb4_last_cuda_error"):
         getattr(L, name).restype = ci
     L.fb4_set_kernel_variant.argtypes = [vp, ci]
@@ -191,6 +193,11 @@ def fb4_build_subformatbook_static(ctx, meta, T, C, anchor_token, anchor_cluster
 def fb4_select_salient(ctx, score, T, tile, salient_idx, stream=None) -> None:
     _check(lib().fb4_select_salient(ctx, _ptr(score), T, tile, _ptr(salient_idx), _stream(stream)),
            "fb4_select_salient")
+
+
+def fb4_select_salient_topk(ctx, score, T, k, salient_idx, stream=None) -> None:
+    _check(lib().fb4_select_salient_topk(ctx, _ptr(score), T, k, _ptr(salient_idx), _stream(stream)),
+           "fb4_select_salient_topk")
 
 
 def fb4_quantize_decomposed(ctx, x, T, C, ld_elems, score, tile, cluster_id, cluster_mask, n_clusters, codes, meta,
@@ -344,6 +351,11 @@ class Fb4:
         out = torch.empty(max(-(-T // tile), 1), dtype=torch.int32, device=score.device)
         fb4_select_salient(self.ctx, score, T, tile, out)
         return out[:-(-T // tile)]
+
+    def select_salient_topk(self, score, k: int):
+        out = torch.empty(max(k, 1), dtype=torch.int32, device=score.device)
+        fb4_select_salient_topk(self.ctx, score, score.numel(), k, out)
+        return out[:k]
 
     def dequantize(self, q: Quantized, dtype=torch.float32):
         T, C = q.codes.shape[0], q.codes.shape[1] * 2

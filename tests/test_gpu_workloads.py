@@ -130,3 +130,33 @@ def test_c5_decomposed_seda_and_plain_sampled_rows(q32):
     e = torch.floor(torch.log2(amax.clamp_min(2.0 ** -124))).to(torch.int32)
     sb = plain.meta.view(torch.int16).to(torch.int32) & 0xFF
     assert bool((sb == e + 124).all())
+
+
+def test_c3_global_top5_percent_reading(q32, c2_bits):
+    """Config 3 read literally ("top 5 % by score" over the whole sequence instead of one token per
+    tile of 20): global top-k selection feeding the decomposition with a given salient set."""
+    w = synth.workloads()["c3"]
+    score = synth.scores(w)
+    k = -(-w.T * 5 // 100)
+    assert k == 1638
+    sal = orc.select_salient_topk(score, k)
+    got_sal = q32.select_salient_topk(torch.from_numpy(score).cuda(), k)
+    assert np.array_equal(got_sal.cpu().numpy(), sal)
+    ref = orc.quantize(c2_bits, FB, salient_idx=sal)
+    got = q32.quantize_decomposed(to_dev_bf16(c2_bits), salient_idx=got_sal)
+    assert_same_quantized(got, ref, "c3 global")
+    assert_same_bits_f32(q32.dequantize(got), orc.dequantize(ref, FB), "c3 global dequant")
+
+
+@pytest.mark.parametrize("T,k", [(1, 1), (7, 0), (7, 7), (1000, 50), (1024, 1), (5000, 4999), (75600, 3780)])
+def test_topk_selection_with_ties(q32, T, k):
+    rng = np.random.default_rng(T + k)
+    s = rng.random(T).astype(np.float32)
+    if T > 4:
+        s[rng.integers(0, T, size=T // 3)] = s[T // 2]           # a large tie group, likely at the threshold
+        s[rng.integers(0, T, size=3)] = -0.0
+        s[rng.integers(0, T, size=3)] = 0.0
+        s[rng.integers(0, T, size=T // 10)] *= -1                 # negative scores
+    want = orc.select_salient_topk(s, k) if T <= 5000 else np.sort(np.argsort(-s.astype(np.float64), kind="stable")[:k])
+    got = q32.select_salient_topk(torch.from_numpy(s).cuda(), k)
+    assert np.array_equal(got.cpu().numpy(), want)
