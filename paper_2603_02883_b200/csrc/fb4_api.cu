@@ -93,7 +93,7 @@ int run_quantize(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, 
                  uint8_t* codes, uint16_t* meta, cudaStream_t stream) {
   if (T == 0) return FB4_OK;
   cudaError_t e;
-  if (!ctx->force_generic && fb4_fast_eligible(ctx, x, T, C, ld, ex.n_salient > 0)) {
+  if (!ctx->force_generic && fb4_fast_eligible(ctx, x, T, C, ld)) {
     e = fb4_launch_quantize_fast(ctx, x, T, C, ld, ex, codes, meta, stream);
     ctx->last_variant = "fast";
   } else {

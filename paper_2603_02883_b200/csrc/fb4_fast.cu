@@ -176,56 +176,83 @@ __device__ __forceinline__ int choose_dialect(const float (&gm)[8], float sG, ui
   return select_general(cand, gb, tb);
 }
 
-// One block given as 32 fp32 magnitudes (bit patterns, sign cleared) plus the sign bits already at
-// bit 3 of every nibble of the four code words: scale, group maxima, dialect selection and LUT
-// quantization with the same tables as the bf16 path.  Writes the code words and the metadata record.
-template <bool SEDA>
-__device__ __forceinline__ void quantize_f32_block(const uint32_t (&a)[32], const uint32_t (&sg)[4], uint32_t allowed,
+// The lane's 32 elements given as fp32 magnitudes (bit patterns, sign cleared) plus their sign bits
+// already at bit 3 of every nibble of the four code words: scale, group maxima, dialect selection
+// and LUT quantization with the same tables as the bf16 path.  One block of 32, or (B16) two blocks
+// of 16 with a scale, a selection and a metadata record each; CLAMP: clamped exponent range,
+// magnitudes saturate at the largest value of bin 31.  Writes the code words and the metadata
+// (one record, or two records in one 32-bit word).
+template <bool SEDA, bool B16, bool CLAMP>
+__device__ __forceinline__ void quantize_f32_block(uint32_t (&a)[32], const uint32_t (&sg)[4], uint32_t allowed,
                                                    const SmemTables* tb, uint32_t qerr_lane, uint32_t pair_base,
-                                                   uint32_t* rcw, uint32_t* rmeta) {
-  uint32_t gmx[8];
-  uint32_t amax = 0;
+                                                   uint32_t ec_lo, uint32_t ec_hi, uint32_t* rcw, uint32_t* rmeta) {
+  constexpr int NH = B16 ? 2 : 1;      // blocks in the lane's 32 elements
+  constexpr int NE = 32 / NH;          // elements per block
+  constexpr int GS = NE / 8;           // elements per group
+  uint32_t meta = 0;
 #pragma unroll
-  for (int g = 0; g < 8; ++g) {
-    gmx[g] = max(max(a[4 * g], a[4 * g + 1]), max(a[4 * g + 2], a[4 * g + 3]));
-    amax = max(amax, gmx[g]);
-  }
-  const uint32_t Er = max(amax >> 23, 3u);
-  const float s2 = __uint_as_float((257u - Er) << 23);   // 2^(3-e)
-  const float sG = s2 * 0x1p-21f, sH = s2 * 0x1p-25f, sL = s2 * 0x1p-5f;
-  const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax), sG, 2.0f)) & 31u;
-  float gm[8];
+  for (int h = 0; h < NH; ++h) {
+    uint32_t gmx[8];
+    uint32_t amax = 0;
 #pragma unroll
-  for (int g = 0; g < 8; ++g) gm[g] = __uint_as_float(gmx[g]);
-  const int rdid = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
-  const float magic_lo = __uint_as_float(0x48000000u + pair_base + (uint32_t)rdid * kPairStride);
+    for (int g = 0; g < 8; ++g) {
+      uint32_t m = a[NE * h + GS * g];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    uint32_t idx = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j + 1]), sH, 0.125f));
-      const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j]), sL, magic_lo));
-      idx |= lds_u8(th * (uint32_t)kPairMul + tl) << (8 * j);
+      for (int i = 1; i < GS; ++i) m = max(m, a[NE * h + GS * g + i]);
+      gmx[g] = m;
+      amax = max(amax, m);
     }
-    rcw[q] = idx | sg[q];
+    uint32_t Er = max(amax >> 23, 3u);
+    if (CLAMP) {
+      Er = min(max(amax >> 23, ec_lo), ec_hi);
+      const uint32_t bound = (Er << 23) | 0x7fffffu;
+      amax = min(amax, bound);
+#pragma unroll
+      for (int g = 0; g < 8; ++g) gmx[g] = min(gmx[g], bound);
+#pragma unroll
+      for (int i = 0; i < NE; ++i) a[NE * h + i] = min(a[NE * h + i], bound);
+    }
+    const float s2 = __uint_as_float((257u - Er) << 23);   // 2^(3-e)
+    const float sG = s2 * 0x1p-21f, sH = s2 * 0x1p-25f, sL = s2 * 0x1p-5f;
+    const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax), sG, 2.0f)) & 31u;
+    float gm[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) gm[g] = __uint_as_float(gmx[g]);
+    const int rdid = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
+    const float magic_lo = __uint_as_float(0x48000000u + pair_base + (uint32_t)rdid * kPairStride);
+#pragma unroll
+    for (int q = (4 / NH) * h; q < (4 / NH) * (h + 1); ++q) {
+      uint32_t idx = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j + 1]), sH, 0.125f));
+        const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j]), sL, magic_lo));
+        idx |= lds_u8(th * (uint32_t)kPairMul + tl) << (8 * j);
+      }
+      rcw[q] = idx | sg[q];
+    }
+    meta |= ((Er - 3u) | ((uint32_t)rdid << 8)) << (16 * h);
   }
-  *rmeta = (Er - 3u) | ((uint32_t)rdid << 8);
+  *rmeta = meta;
 }
 
-// Residual pass of one block (Sec. 3.3): Delta = x - Q(x) in fp32 (exact), quantized again with
-// the same tables as the main pass; the fp32 magnitudes take the place of the bf16 ones.
-// w = the 16 input registers (2 bf16 each), cw = the block's 4 code words, Ec = biased exponent.
-template <bool SEDA>
-__device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t* cw, int did, uint32_t Ec,
-                                               uint32_t allowed, const SmemTables* tb, uint32_t qerr_lane,
-                                               uint32_t pair_base, uint32_t* rcw, uint32_t* rmeta) {
-  const uint4 dt = tb->fb_bf16[did];
-  const uint32_t sc2 = fb4dev::scale_bf16x2(Ec - 3u);   // element scale 2^(e-3) as two bf16
+// Residual pass of the lane's block(s) (Sec. 3.3): Delta = x - Q(x) in fp32 (exact for the full
+// exponent range, the correctly rounded difference otherwise), quantized again with the same tables
+// as the main pass; the fp32 magnitudes take the place of the bf16 ones.
+// w = the 16 input registers (2 bf16 each), cw = the 4 code words, didh / Ech = dialect and biased
+// exponent per half (equal halves for block size 32).
+template <bool SEDA, bool B16, bool CLAMP>
+__device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t* cw, const int* didh,
+                                               const uint32_t* Ech, uint32_t allowed, const SmemTables* tb,
+                                               uint32_t qerr_lane, uint32_t pair_base, uint32_t ec_lo, uint32_t ec_hi,
+                                               uint32_t* rcw, uint32_t* rmeta) {
   uint32_t a[32];      // |Delta| bit patterns
   uint32_t sg[4];      // sign bits at bit 3 of every nibble
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
+    const int h = B16 ? (q >> 1) : 0;
+    const uint4 dt = tb->fb_bf16[didh[h]];
+    const uint32_t sc2 = fb4dev::scale_bf16x2(Ech[h] - 3u);   // element scale 2^(e-3) as two bf16
     uint32_t xh[4];    // Q(x) of the word's 8 elements, two bf16 per register, signs included
     fb4dev::decode_word(cw[q], dt, sc2, xh);
     uint32_t sq = 0;
@@ -242,7 +269,7 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
     }
     sg[q] = sq;
   }
-  quantize_f32_block<SEDA>(a, sg, allowed, tb, qerr_lane, pair_base, rcw, rmeta);
+  quantize_f32_block<SEDA, B16, CLAMP>(a, sg, allowed, tb, qerr_lane, pair_base, ec_lo, ec_hi, rcw, rmeta);
 }
 
 // Tile index -> (token row, tile column, salient-token slot = row / sal_tile) without a division per
@@ -544,11 +571,13 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
       }
       if (srow >= 0) {   // warp-uniform: a tile lies inside one token
         uint32_t rcw[4], rmeta;
-        residual_block<SEDA>(w, cw, didh[0], Ech[0], allowed, tb, qerr_base, pair_base, rcw, &rmeta);
+        residual_block<SEDA, B16, CLAMP>(w, cw, didh, Ech, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, rcw,
+                                         &rmeta);
         if (active) {
           *reinterpret_cast<uint4*>(ex.res_codes + srow * code_row_bytes + blk * 16) =
               make_uint4(rcw[0], rcw[1], rcw[2], rcw[3]);
-          ex.res_meta[srow * nblk + blk] = (uint16_t)rmeta;
+          if (B16) *reinterpret_cast<uint32_t*>(ex.res_meta + (srow * nblk + blk) * 2) = rmeta;
+          else ex.res_meta[srow * nblk + blk] = (uint16_t)rmeta;
         }
       }
     }
@@ -681,7 +710,7 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
       }
     }
     uint32_t cw[4], m;
-    quantize_f32_block<false>(a, sg, 0xffffffffu, tb, qerr_base, pair_base, cw, &m);
+    quantize_f32_block<false, false, false>(a, sg, 0xffffffffu, tb, qerr_base, pair_base, 3u, 254u, cw, &m);
     if (blk < nblk) {
       *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
       p.meta[row * nblk + blk] = (uint16_t)m;
@@ -821,24 +850,28 @@ cudaError_t fb4_fast_prepare_device() {
   FB4_OPT_IN(true, true, false, false);
   FB4_OPT_IN(false, false, true, false);
   FB4_OPT_IN(true, false, true, false);
+  FB4_OPT_IN(false, true, true, false);
+  FB4_OPT_IN(true, true, true, false);
   FB4_OPT_IN(false, false, false, true);
   FB4_OPT_IN(true, false, false, true);
+  FB4_OPT_IN(false, true, false, true);
+  FB4_OPT_IN(true, true, false, true);
   FB4_OPT_IN(false, false, true, true);
   FB4_OPT_IN(true, false, true, true);
+  FB4_OPT_IN(false, true, true, true);
+  FB4_OPT_IN(true, true, true, true);
 #undef FB4_OPT_IN
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
   return e;
 }
 
-// Block size 32 with every extension; block size 16 and clamped exponent ranges (the 5-bit exponent
-// of Sec. 3.1) for plain and SeDA calls: their residual pass takes the generic kernel.
-bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, bool residual_pass) {
+// Block sizes 32 and 16, any exponent clamp (the 5-bit exponent of Sec. 3.1 included), every
+// extension; num_groups 8 and two-stage selection only.
+bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {
   const fb4_config& c = ctx->cfg;
   if (!ctx->fast_ok || !ctx->d_fast_tables) return false;
   if (c.num_groups != 8 || c.select_mode != 0) return false;
-  const bool clamp = c.exp_min != -124 || c.exp_max != 127;
   if (c.block_size != 32 && c.block_size != 16) return false;
-  if ((c.block_size == 16 || clamp) && residual_pass) return false;
   if (C % 64 != 0 || (ld & 7) || (reinterpret_cast<uintptr_t>(x) & 15)) return false;
   if (T > 0x7fffffffLL || C / 64 > 0x7fffffffLL) return false;
   return encode_tiled_fn() != nullptr;
@@ -877,18 +910,29 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   p.ec_hi = (uint32_t)(ctx->cfg.exp_max + 127);
   const bool b16 = ctx->cfg.block_size == 16;
   const bool clamp = ctx->cfg.exp_min != -124 || ctx->cfg.exp_max != 127;
-  if (clamp) {
-    if (b16) return seda ? launch<true, false, true, true>(map, tables, p, ex, grid, stream)
-                         : launch<false, false, true, true>(map, tables, p, ex, grid, stream);
-    return seda ? launch<true, false, false, true>(map, tables, p, ex, grid, stream)
-                : launch<false, false, false, true>(map, tables, p, ex, grid, stream);
+  const int variant = (seda ? 1 : 0) | (decomp ? 2 : 0) | (b16 ? 4 : 0) | (clamp ? 8 : 0);
+  switch (variant) {
+#define FB4_CASE(V, S, D, B, K) \
+  case V: return launch<S, D, B, K>(map, tables, p, ex, grid, stream)
+    FB4_CASE(0, false, false, false, false);
+    FB4_CASE(1, true, false, false, false);
+    FB4_CASE(2, false, true, false, false);
+    FB4_CASE(3, true, true, false, false);
+    FB4_CASE(4, false, false, true, false);
+    FB4_CASE(5, true, false, true, false);
+    FB4_CASE(6, false, true, true, false);
+    FB4_CASE(7, true, true, true, false);
+    FB4_CASE(8, false, false, false, true);
+    FB4_CASE(9, true, false, false, true);
+    FB4_CASE(10, false, true, false, true);
+    FB4_CASE(11, true, true, false, true);
+    FB4_CASE(12, false, false, true, true);
+    FB4_CASE(13, true, false, true, true);
+    FB4_CASE(14, false, true, true, true);
+    FB4_CASE(15, true, true, true, true);
+#undef FB4_CASE
   }
-  if (b16) return seda ? launch<true, false, true, false>(map, tables, p, ex, grid, stream)
-                       : launch<false, false, true, false>(map, tables, p, ex, grid, stream);
-  if (seda && decomp) return launch<true, true, false, false>(map, tables, p, ex, grid, stream);
-  if (seda) return launch<true, false, false, false>(map, tables, p, ex, grid, stream);
-  if (decomp) return launch<false, true, false, false>(map, tables, p, ex, grid, stream);
-  return launch<false, false, false, false>(map, tables, p, ex, grid, stream);
+  return cudaErrorInvalidValue;
 }
 
 bool fb4_fast_f32_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {

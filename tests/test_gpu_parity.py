@@ -247,8 +247,8 @@ def test_f32_input(cfg):
 
 
 def test_block16_fast_kernel_plain_and_seda():
-    """Block size 16 takes the TMA-staged kernel for plain and SeDA calls (two blocks per lane) and
-    the generic kernel when a residual pass is asked for; both equal the oracle."""
+    """Block size 16 in the TMA-staged kernel (two blocks per lane), plain, SeDA and with a residual
+    pass, against the oracle and the generic kernel."""
     q = fb4.Fb4(block_size=16)
     ocfg = orc.Config(block_size=16)
     w = synth.Workload("t", T=300, C=3072, seed=51, kind=1, n_outlier=15, outlier_gain=50.0, seda=True, n_clusters=9,
@@ -270,11 +270,18 @@ def test_block16_fast_kernel_plain_and_seda():
         assert q.last_variant == name
         assert_same_quantized(q.quantize(x, dcid, dmask), ref_seda, f"b16 seda {name}")
         assert q.last_variant == name
-    q.set_kernel_variant(0)
     sal = orc.select_salient(synth.scores(w), 20)
-    got = q.quantize_decomposed(x, torch.from_numpy(synth.scores(w)).cuda(), 20)
-    assert q.last_variant == "generic"
-    assert_same_quantized(got, orc.quantize(bits, FB, ocfg, salient_idx=sal), "b16 decomposed")
+    ref_dec = orc.quantize(bits, FB, ocfg, salient_idx=sal)
+    ref_dec_seda = orc.quantize(bits, FB, ocfg, cluster_id=cid, cluster_mask=masks, salient_idx=sal)
+    for variant, name in ((0, "fast"), (1, "generic")):
+        q.set_kernel_variant(variant)
+        got = q.quantize_decomposed(x, torch.from_numpy(synth.scores(w)).cuda(), 20)
+        assert q.last_variant == name
+        assert_same_quantized(got, ref_dec, f"b16 decomposed {name}")
+        got = q.quantize_decomposed(x, torch.from_numpy(synth.scores(w)).cuda(), 20, cluster_id=dcid, cluster_mask=dmask)
+        assert_same_quantized(got, ref_dec_seda, f"b16 decomposed seda {name}")
+        assert_same_bits_f32(q.dequantize(got), orc.dequantize(ref_dec_seda, FB, 16), "b16 decomposed dequant")
+    q.set_kernel_variant(0)
     assert_same_bits_f32(q.dequantize(q.quantize(x)), orc.dequantize(ref_plain, FB, 16), "b16 dequant")
     assert q.device_status == 0
     q.close()
@@ -285,7 +292,7 @@ def test_block16_fast_kernel_plain_and_seda():
                          ids=["exp5", "b16-exp5", "narrow", "b16-single-exponent"])
 def test_clamped_exponent_fast_kernel(cfg):
     """The paper's 5-bit shared exponent (and narrower clamps, which saturate many elements) in the
-    TMA-staged kernel, plain and SeDA, against the oracle and the generic kernel."""
+    TMA-staged kernel, plain, SeDA and with a residual pass, against the oracle and the generic kernel."""
     q = fb4.Fb4(**cfg)
     ocfg = orc.Config(**cfg)
     w = synth.Workload("t", T=200, C=1024 + 128, seed=61, kind=1, n_outlier=6, outlier_gain=50.0, seda=True,
@@ -295,8 +302,16 @@ def test_clamped_exponent_fast_kernel(cfg):
         x = to_dev_bf16(bits)
         ref = orc.quantize(bits, FB, ocfg)
         ref_seda = orc.quantize(bits, FB, ocfg, cluster_id=cid, cluster_mask=masks)
+        sal = np.arange(3, 200, 7, dtype=np.int32)
+        ref_dec = orc.quantize(bits, FB, ocfg, cluster_id=cid, cluster_mask=masks, salient_idx=sal)
         for variant, name in ((0, "fast"), (1, "generic")):
             q.set_kernel_variant(variant)
+            got = q.quantize_decomposed(x, salient_idx=torch.from_numpy(sal).cuda(), cluster_id=torch.from_numpy(cid).cuda(),
+                                        cluster_mask=torch.from_numpy(masks.view(np.int32)).cuda())
+            assert q.last_variant == name
+            assert_same_quantized(got, ref_dec, f"clamped decomposed {cfg} {name}")
+            assert_same_bits_f32(q.dequantize(got), orc.dequantize(ref_dec, FB, cfg.get("block_size", 32)),
+                                 "clamped decomposed dequant")
             got = q.quantize(x)
             assert q.last_variant == name
             assert_same_quantized(got, ref, f"clamped {cfg} {name}")
