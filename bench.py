@@ -223,6 +223,12 @@ class Ops:
             return (lambda: fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, tile, None, None, 0, codes, meta,
                                                         sal, rc, rm)), \
                 algorithmic_bytes(T, C, n_res_rows=n_sal, decomposed=True)
+        if name == "decomposed_given_set":
+            # salient set given by the caller (reused from an earlier step / global top-k reading)
+            fb4.fb4_select_salient_topk(q.ctx, score, T, n_sal, sal)
+            return (lambda: fb4.fb4_quantize_decomposed_idx(q.ctx, x, T, C, C, sal, n_sal, None, None, 0, codes, meta,
+                                                            rc, rm)), \
+                algorithmic_bytes(T, C, n_res_rows=n_sal, decomposed=True) - 4 * T
         if name == "decomposed_seda":
             return (lambda: fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, tile, cid, cmask, cmask.numel(),
                                                         codes, meta, sal, rc, rm)), \
@@ -255,7 +261,7 @@ class Ops:
         raise KeyError(name)
 
 
-OP_NAMES = ["plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
+OP_NAMES = ["plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
             "dequantize_bf16_plain", "dequantize_bf16_decomposed", "to_mxfp8_tiled_scales"]
 
 
@@ -396,7 +402,7 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         total, per = time_steps(fn, steps, warm, torch)
         ms = total / steps
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
-                     "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "seda", "decomposed",
+                     "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_given_set",
                                                                          "decomposed_seda") else "decode"}
         if name == "dequantize_f32_decomposed":
             ops.drop("out32")

@@ -361,6 +361,18 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
     ++it_pre;
     pre.advance(p, tpr);
   }
+  // caller-given salient list (no tile structure): position of the first entry >= this warp's first row
+  int64_t list_pos = 0;
+  int32_t list_next = 0x7fffffff;
+  if (DECOMP && !use_tile && n_mine > 0) {
+    int64_t lo = 0, hi = ex.n_salient;
+    while (lo < hi) {
+      const int64_t mid = (lo + hi) >> 1;
+      if (ex.salient_idx[mid] < cur.row) lo = mid + 1; else hi = mid;
+    }
+    list_pos = lo;
+    if (lo < ex.n_salient) list_next = ex.salient_idx[lo];
+  }
   uint32_t maskq[2] = {0xffffffffu, 0xffffffffu};
   if (use_seda) {
     if (cidq[0] >= 0) maskq[0] = ex.cluster_mask[cidq[0]];
@@ -561,13 +573,12 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
       if (use_tile) {
         if (salq[0] == cur.row) srow = cur.row / ex.tile;   // rare: one row in `tile`
       } else {
-        int64_t lo = 0, hi = ex.n_salient - 1;
-        while (lo <= hi) {
-          const int64_t mid = (lo + hi) >> 1;
-          const int32_t v = ex.salient_idx[mid];
-          if (v == (int32_t)row) { srow = mid; break; }
-          if (v < (int32_t)row) lo = mid + 1; else hi = mid - 1;
+        // caller-given ascending list: this warp's rows never decrease, so a cursor walks the list
+        while (list_next < cur.row) {
+          ++list_pos;
+          list_next = list_pos < ex.n_salient ? ex.salient_idx[list_pos] : 0x7fffffff;
         }
+        if (list_next == cur.row) srow = list_pos;
       }
       if (srow >= 0) {   // warp-uniform: a tile lies inside one token
         uint32_t rcw[4], rmeta;
