@@ -71,14 +71,14 @@ __device__ __forceinline__ void store_word(uint8_t* dst, const uint32_t* pr, boo
   }
 }
 
-// Flat decode for 32-element blocks without residuals.  A lane loads the 16 code bytes and the
-// metadata of one block (one 128-bit and one 16-bit load); the quad transposes the code words so
-// that lane p decodes word p of the quad's four blocks and the quad stores contiguous lines.
-// kDecodeUnroll blocks per thread are in flight; the loads of the next step are issued before the
-// current step is decoded.
-template <int OUT_BF16>
+// Flat decode without residuals, in units of 32 elements (one block of 32, or two blocks of 16).
+// A lane loads the 16 code bytes of one unit (one 128-bit load) and the metadata records of its
+// whole quad (one 64- or 128-bit load); the quad transposes the code words so that lane p decodes
+// word p of the quad's four units and the quad stores contiguous lines.  kDecodeUnroll units per
+// thread are in flight; the loads of the next step are issued before the current step is decoded.
+template <int OUT_BF16, bool B16>
 __global__ void __launch_bounds__(kDecodeThreads)
-fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restrict__ meta, int64_t total_blocks,
+fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restrict__ meta, int64_t total_units,
                           const Fb4DeviceTables* __restrict__ tables, void* __restrict__ out, int out_aligned32) {
   __shared__ uint4 fb_bf16[32];   // per dialect: high bytes (8) then low bytes (8) of its magnitudes as bf16
   fb4dev::fill_fb_bf16(fb_bf16, &tables->formatbook[0][0], threadIdx.x);
@@ -86,52 +86,61 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
   const bool wide = out_aligned32 != 0;
   const int lane = threadIdx.x & 31;
   const int qp = lane & 3;
+  constexpr int RPU = B16 ? 2 : 1;   // metadata records per unit
   constexpr int kWordBytes = OUT_BF16 ? 16 : 32;
   constexpr int64_t kStep = (int64_t)kDecodeThreads * kDecodeUnroll;
   const int64_t stride = (int64_t)gridDim.x * kStep;
 
-  // m = the metadata records of the lane's whole quad (4 x 16 bits): after the transpose a lane
-  // decodes one word of each of the quad's blocks and needs all four records
+  // m = the metadata records of the lane's whole quad (4 units): after the transpose a lane decodes
+  // one word of each of the quad's units and needs the record that covers it
   uint32_t cw[kDecodeUnroll][4];
-  uint2 m[kDecodeUnroll];
+  uint32_t m[kDecodeUnroll][2 * RPU];
   auto load = [&](int64_t base) {
 #pragma unroll
     for (int u = 0; u < kDecodeUnroll; ++u) {
       const int64_t b = base + u * kDecodeThreads + threadIdx.x;
       const int64_t qb = b & ~3ll;
       cw[u][0] = cw[u][1] = cw[u][2] = cw[u][3] = 0u;
-      m[u] = make_uint2(0u, 0u);
-      if (b < total_blocks) load_block_codes<4>(codes + b * 4, cw[u]);
-      if (qb + 4 <= total_blocks) {
-        m[u] = __ldg(reinterpret_cast<const uint2*>(meta + qb));   // 8-byte aligned: qb is a multiple of 4
-      } else if (qb < total_blocks) {                               // ragged last quad
-        uint32_t r[4] = {0u, 0u, 0u, 0u};
-        for (int i = 0; i < 4; ++i)
-          if (qb + i < total_blocks) r[i] = (uint32_t)__ldg(meta + qb + i);
-        m[u] = make_uint2(r[0] | (r[1] << 16), r[2] | (r[3] << 16));
+#pragma unroll
+      for (int k = 0; k < 2 * RPU; ++k) m[u][k] = 0u;
+      if (b < total_units) load_block_codes<4>(codes + b * 4, cw[u]);
+      if (qb + 4 <= total_units) {   // aligned: qb is a multiple of 4
+        if (B16) {
+          const uint4 v = __ldg(reinterpret_cast<const uint4*>(meta + qb * 2));
+          m[u][0] = v.x; m[u][1] = v.y; m[u][2 % (2 * RPU)] = v.z; m[u][3 % (2 * RPU)] = v.w;
+        } else {
+          const uint2 v = __ldg(reinterpret_cast<const uint2*>(meta + qb));
+          m[u][0] = v.x; m[u][1] = v.y;
+        }
+      } else if (qb < total_units) {   // ragged last quad
+        for (int i = 0; i < 4 * RPU; ++i)
+          if (qb * RPU + i < total_units * RPU)
+            m[u][i >> 1] |= (uint32_t)__ldg(meta + qb * RPU + i) << (16 * (i & 1));
       }
     }
   };
   int64_t base = (int64_t)blockIdx.x * kStep;
-  if (base < total_blocks) load(base);
-  for (; base < total_blocks; base += stride) {
-    uint32_t c[kDecodeUnroll][4];
-    uint2 mm[kDecodeUnroll];
+  if (base < total_units) load(base);
+  for (; base < total_units; base += stride) {
+    uint32_t c[kDecodeUnroll][4], mm[kDecodeUnroll][2 * RPU];
 #pragma unroll
     for (int u = 0; u < kDecodeUnroll; ++u) {
-      mm[u] = m[u];
+#pragma unroll
+      for (int k = 0; k < 2 * RPU; ++k) mm[u][k] = m[u][k];
 #pragma unroll
       for (int k = 0; k < 4; ++k) c[u][k] = cw[u][k];
     }
-    if (base + stride < total_blocks) load(base + stride);
+    if (base + stride < total_units) load(base + stride);
 #pragma unroll
     for (int u = 0; u < kDecodeUnroll; ++u) {
       quad_transpose(c[u], lane);
-      const int64_t qb = base + u * kDecodeThreads + (threadIdx.x & ~3);   // first block of this quad
+      const int64_t qb = base + u * kDecodeThreads + (threadIdx.x & ~3);   // first unit of this quad
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const uint32_t mi = ((i & 2) ? mm[u].y : mm[u].x) >> (16 * (i & 1)) & 0xffffu;
-        if (qb + i < total_blocks) {
+        // record of unit i (block 32), or of the half of unit i that holds word qp (block 16)
+        const uint32_t mi = B16 ? (mm[u][i] >> (16 * (qp >> 1))) & 0xffffu
+                                : (mm[u][i >> 1] >> (16 * (i & 1))) & 0xffffu;
+        if (qb + i < total_units) {
           uint32_t pr[4];
           decode_word(c[u][i], fb_bf16[(mi >> 8) & 31u], scale_bf16x2(mi), pr);
           store_word<OUT_BF16>(reinterpret_cast<uint8_t*>(out) + ((qb + i) * 4 + qp) * kWordBytes, pr, wide);
@@ -346,8 +355,14 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
   const int a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
   const Fb4DeviceTables* tb = ctx->d_tables;
   if (B == 32) {
-    if (out_dtype == 1) fb4_dequantize_b32_kernel<1><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
-    else fb4_dequantize_b32_kernel<0><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
+    if (out_dtype == 1) fb4_dequantize_b32_kernel<1, false><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
+    else fb4_dequantize_b32_kernel<0, false><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
+  } else if (C % 32 == 0) {   // block 16 in units of two blocks
+    const int64_t units = total / 2;
+    const int64_t uwant = (units + kStep - 1) / kStep;
+    const unsigned ugrid = (unsigned)(uwant < cap ? uwant : cap);
+    if (out_dtype == 1) fb4_dequantize_b32_kernel<1, true><<<ugrid, kDecodeThreads, 0, stream>>>(cw, meta, units, tb, out, a32);
+    else fb4_dequantize_b32_kernel<0, true><<<ugrid, kDecodeThreads, 0, stream>>>(cw, meta, units, tb, out, a32);
   } else {
     if (out_dtype == 1) fb4_dequantize_kernel<1, 2><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
     else fb4_dequantize_kernel<0, 2><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
