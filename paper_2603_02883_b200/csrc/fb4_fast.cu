@@ -67,9 +67,6 @@ struct FastParams {
   int64_t tiles_per_row, n_tiles;
   int64_t step_rows;    // gridDim.x*kWarps tiles ahead = step_rows rows + step_cols tile columns
   int32_t step_cols;
-  int32_t sal_tile;     // tokens per salient-token tile (a huge value when the salient set is a plain list)
-  int32_t step_slots;   // step_rows = step_slots * sal_tile + step_rem
-  int32_t step_rem;
   uint8_t* codes;
   uint16_t* meta;
   uint32_t* status;   // device word: bit 0 = a TMA wait ran out
@@ -272,19 +269,14 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
   quantize_f32_block<SEDA, B16, CLAMP>(a, sg, allowed, tb, qerr_lane, pair_base, ec_lo, ec_hi, rcw, rmeta);
 }
 
-// Tile index -> (token row, tile column, salient-token slot = row / sal_tile) without a division per
-// tile: advance by a fixed step.
+// Tile index -> (token row, tile column) without a division per tile: advance by a fixed step.
 struct TilePos {
   int32_t row;         // T < 2^31
   int32_t col;
-  int32_t slot, rem;   // row = slot * sal_tile + rem
   __device__ __forceinline__ void advance(const FastParams& p, int32_t tiles_per_row) {
     row += (int32_t)p.step_rows;
     col += p.step_cols;
-    slot += p.step_slots;
-    rem += p.step_rem;
-    if (col >= tiles_per_row) { col -= tiles_per_row; ++row; ++rem; }
-    if (rem >= p.sal_tile) { rem -= p.sal_tile; ++slot; }
+    if (col >= tiles_per_row) { col -= tiles_per_row; ++row; }
   }
 };
 
@@ -333,38 +325,34 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
   TilePos cur, pre;   // tile being quantized; next tile to request
   cur.row = (int32_t)(gwarp / tpr);
   cur.col = (int32_t)(gwarp - (int64_t)cur.row * tpr);
-  cur.slot = cur.row / p.sal_tile;
-  cur.rem = cur.row - cur.slot * p.sal_tile;
   pre = cur;
   // this warp's tiles are gwarp, gwarp + wstride, ...: n_mine of them, counted in 32 bits
   const int32_t n_mine = gwarp < g_end ? (int32_t)((g_end - gwarp + wstride - 1) / wstride) : 0;
   int32_t it_pre = 0;   // iteration whose tile `pre` points at
   const bool use_seda = SEDA && ex.cluster_id != nullptr;
-  const bool use_tile = DECOMP && ex.tile > 0;
   // Per-token extras travel in register queues, fetched as far ahead as the tile data: entry k
-  // belongs to the tile k steps ahead.  cidq = cluster id, salq = token stored in the row's
-  // salient slot; the cluster mask follows its id two steps behind.
-  int32_t cidq[kStages], salq[kStages];
+  // belongs to the tile k steps ahead.  cidq = cluster id; the cluster mask follows its id two steps
+  // behind.
+  int32_t cidq[kStages];
   // prologue: fill the ring
 #pragma unroll
   for (int s = 0; s < kStages; ++s) {
     cidq[s] = -1;
-    salq[s] = -1;
     if (it_pre < n_mine) {
       if (lane == 0) {
         mbar_expect_tx(my_bars + 8 * s, kTileBytes);
         tma_load_tile(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, pre.col * 16, pre.row);
       }
       if (use_seda) cidq[s] = ex.cluster_id[pre.row];
-      if (use_tile) salq[s] = ex.salient_idx[pre.slot];   // slot < ceil(T / tile) = n_salient
     }
     ++it_pre;
     pre.advance(p, tpr);
   }
-  // caller-given salient list (no tile structure): position of the first entry >= this warp's first row
+  // salient tokens: an ascending list (one per tile, or given by the caller); this warp's rows never
+  // decrease, so a cursor walks it.  Position of the first entry >= this warp's first row:
   int64_t list_pos = 0;
   int32_t list_next = 0x7fffffff;
-  if (DECOMP && !use_tile && n_mine > 0) {
+  if (DECOMP && n_mine > 0) {
     int64_t lo = 0, hi = ex.n_salient;
     while (lo < hi) {
       const int64_t mid = (lo + hi) >> 1;
@@ -409,16 +397,13 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
   uint32_t parity = 0;
   for (int32_t it = 0; it < n_mine; ++it) {
     // ---- fetch the extras of the tiles ahead (pre = the tile kStages steps ahead)
-    int32_t cid_new = -1, sal_new = -1;
+    int32_t cid_new = -1;
     uint32_t mask_new = 0xffffffffu;
     if (SEDA) {
       if (use_seda) {
         if (it_pre < n_mine) cid_new = ex.cluster_id[pre.row];
         if (cidq[2] >= 0) mask_new = ex.cluster_mask[cidq[2]];
       }
-    }
-    if (DECOMP) {
-      if (use_tile && it_pre < n_mine) sal_new = ex.salient_idx[pre.slot];
     }
 
     const uint32_t bar = my_bars + 8 * s;
@@ -570,16 +555,11 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
     }
     if (DECOMP) {
       int64_t srow = -1;
-      if (use_tile) {
-        if (salq[0] == cur.row) srow = cur.row / ex.tile;   // rare: one row in `tile`
-      } else {
-        // caller-given ascending list: this warp's rows never decrease, so a cursor walks the list
-        while (list_next < cur.row) {
-          ++list_pos;
-          list_next = list_pos < ex.n_salient ? ex.salient_idx[list_pos] : 0x7fffffff;
-        }
-        if (list_next == cur.row) srow = list_pos;
+      while (list_next < cur.row) {
+        ++list_pos;
+        list_next = list_pos < ex.n_salient ? ex.salient_idx[list_pos] : 0x7fffffff;
       }
+      if (list_next == cur.row) srow = list_pos;
       if (srow >= 0) {   // warp-uniform: a tile lies inside one token
         uint32_t rcw[4], rmeta;
         residual_block<SEDA, B16, CLAMP>(w, cw, didh, Ech, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, rcw,
@@ -604,10 +584,8 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
 #pragma unroll
     for (int k = 0; k + 1 < kStages; ++k) {
       cidq[k] = cidq[k + 1];
-      salq[k] = salq[k + 1];
     }
     cidq[kStages - 1] = cid_new;
-    salq[kStages - 1] = sal_new;
     maskq[0] = maskq[1];
     maskq[1] = mask_new;
     if (++s == kStages) { s = 0; parity ^= 1u; }
@@ -648,7 +626,6 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
   TilePos cur, pre;
   cur.row = (int32_t)(gwarp / tpr);
   cur.col = (int32_t)(gwarp - (int64_t)cur.row * tpr);
-  cur.slot = cur.rem = 0;
   pre = cur;
   const int32_t n_mine = gwarp < p.n_tiles ? (int32_t)((p.n_tiles - gwarp + wstride - 1) / wstride) : 0;
   int32_t it_pre = 0;
@@ -913,9 +890,6 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   const int64_t wstride = decomp ? kWarps : (int64_t)grid * kWarps;   // tiles between a warp's consecutive tiles
   p.step_rows = wstride / p.tiles_per_row;
   p.step_cols = (int32_t)(wstride % p.tiles_per_row);
-  p.sal_tile = ex.tile > 0 ? ex.tile : 0x7fffffff;
-  p.step_slots = (int32_t)(p.step_rows / p.sal_tile);
-  p.step_rem = (int32_t)(p.step_rows % p.sal_tile);
   const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
   p.ec_lo = (uint32_t)(ctx->cfg.exp_min + 127);
   p.ec_hi = (uint32_t)(ctx->cfg.exp_max + 127);
@@ -980,9 +954,6 @@ cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int6
   const int64_t wstride = (int64_t)grid * kWarpsF32;
   p.step_rows = wstride / p.tiles_per_row;
   p.step_cols = (int32_t)(wstride % p.tiles_per_row);
-  p.sal_tile = 0x7fffffff;
-  p.step_slots = 0;
-  p.step_rem = 0;
   fb4_quantize_f32_kernel<<<grid, kWarpsF32 * 32, kSmemBytesF32, stream>>>(
       map, static_cast<const SmemTables*>(ctx->d_fast_tables), p);
   return cudaGetLastError();
