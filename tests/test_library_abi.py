@@ -72,3 +72,22 @@ def test_no_device_is_an_error_not_a_fallback():
     assert fb4.lib().fb4_init(ctypes.byref(h), 0, None, None, None) == fb4.ERR_NO_DEVICE
     with pytest.raises(RuntimeError):
         fb4.Fb4()
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/fb4.h is a C header: it must compile as C99 on its own, and a C caller must link."""
+    import subprocess
+    src = tmp_path / "use_fb4.c"
+    src.write_text('#include "fb4.h"\n'
+                   "int main(void) {\n"
+                   "  fb4_config cfg;\n"
+                   "  fb4_default_config(&cfg);\n"
+                   "  return (cfg.block_size == 32 && fb4_mxfp8_scale_bytes(128, 128, 1) == 512 &&\n"
+                   "          fb4_quantize(0, 0, 1, 32, 32, 0, 0, 0) == FB4_ERR_INVALID_ARG) ? 0 : 1;\n"
+                   "}\n")
+    exe = tmp_path / "use_fb4"
+    libdir = os.path.dirname(fb4.library_path())
+    fb4.lib()
+    subprocess.check_call(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           str(src), "-o", str(exe), "-L", libdir, "-lfb4", f"-Wl,-rpath,{libdir}"])
+    assert subprocess.call([str(exe)]) == 0
