@@ -320,3 +320,52 @@ def test_clamped_exponent_fast_kernel(cfg):
         assert_same_bits_f32(q.dequantize(got), orc.dequantize(ref_seda, FB, cfg.get("block_size", 32)), "clamped dequant")
     assert q.device_status == 0
     q.close()
+
+
+def _random_formatbook(rng, tops):
+    """32 dialects, strictly ascending from 0, largest magnitude as listed"""
+    fb = np.zeros((32, 8), dtype=np.uint8)
+    seen = set()
+    for d, top in enumerate(tops):
+        while True:
+            inner = np.sort(rng.choice(np.arange(1, top), size=6, replace=False))
+            row = (0, *inner.tolist(), top)
+            if row not in seen:
+                seen.add(row)
+                fb[d] = row
+                break
+    return fb
+
+
+def test_custom_formatbooks():
+    """The formatbook is init-time data: another table whose dynamic-range groups fit the packed
+    tables runs in the TMA-staged kernel, one with a group of 12 dialects falls back to the generic
+    kernel; both match the oracle run with the same table (quantize, SeDA, residual, decode, MXFP8)."""
+    rng = np.random.default_rng(99)
+    fits = _random_formatbook(rng, [8] * 3 + [9] * 3 + [10] * 4 + [11] * 4 + [12] * 4 + [13] * 4 + [14] * 5 + [15] * 5)
+    wide = _random_formatbook(rng, [8] * 2 + [9] * 2 + [10] * 2 + [11] * 2 + [12] * 4 + [13] * 4 + [14] * 4 + [15] * 12)
+    w = synth.Workload("t", T=160, C=1024, seed=81, kind=1, n_outlier=5, outlier_gain=50.0, seda=True, n_clusters=5,
+                       cluster_seed=82, score_seed=83)
+    bits = synth.activation(w)
+    x = to_dev_bf16(bits)
+    score = synth.scores(w)
+    sal = orc.select_salient(score, 20)
+    for fbk, want in ((fits, "fast"), (wide, "generic")):
+        cid, masks = synth.clusters(w, fbk)
+        q = fb4.Fb4(formatbook=fbk)
+        got = q.quantize(x)
+        assert q.last_variant == want
+        ref = orc.quantize(bits, fbk)
+        assert_same_quantized(got, ref, f"custom formatbook plain ({want})")
+        got = q.quantize_decomposed(x, torch.from_numpy(score).cuda(), 20, cluster_id=torch.from_numpy(cid).cuda(),
+                                    cluster_mask=torch.from_numpy(masks.view(np.int32)).cuda())
+        ref = orc.quantize(bits, fbk, cluster_id=cid, cluster_mask=masks, salient_idx=sal)
+        assert_same_quantized(got, ref, f"custom formatbook decomposed+seda ({want})")
+        assert np.array_equal(q.dequantize(got).cpu().numpy().view(np.uint32), orc.dequantize(ref, fbk).view(np.uint32))
+        e4m3, sc = q.to_mxfp8(got, 1)
+        e_ref, s_ref = orc.to_mxfp8(orc.Quantized(ref.codes, ref.meta), fbk, 1)
+        assert np.array_equal(e4m3.cpu().numpy(), e_ref) and np.array_equal(sc.cpu().numpy(), s_ref)
+        qw = q.quantize_weights(x)
+        assert_same_quantized(qw, orc.quantize_weights(bits, fbk), f"custom formatbook weights ({want})")
+        assert q.device_status == 0
+        q.close()
