@@ -274,6 +274,8 @@ def main():
     ap.add_argument("--workload", default="c5_plain", help="c5_plain (default) or c2 (smaller tensor, for profiling)")
     ap.add_argument("--op", default="plain", choices=OP_NAMES,
                     help="library path timed as the step (default: plain fb4_quantize, the headline metric)")
+    ap.add_argument("--generic-kernel", action="store_true",
+                    help="force the generic quantize kernel (what the packed, TMA-staged kernel is compared with)")
     ap.add_argument("--no-variants", action="store_true", help="time only the step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -305,6 +307,8 @@ def main():
     bits = synth.activation(w)
     x = torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
     q = fb4.Fb4(device=local_rank)
+    if args.generic_kernel:
+        q.set_kernel_variant(1)
     T, C, B = w.T, w.C, 32
     ops = Ops(q, x, w, torch, fb4, synth)
     step, alg = ops.get(args.op)

@@ -40,14 +40,16 @@ __device__ __forceinline__ void quantize_block(const float (&ax)[B], uint32_t sg
   // floor(log2(amax)) is the exponent field; zero and subnormal maxima clamp to exp_min (>= -124)
   int e = amax == 0.f ? p.exp_min : (int)((__float_as_uint(amax) >> 23) & 0xff) - 127;
   e = max(p.exp_min, min(p.exp_max, e));
-  const float s = pow2f(3 - e);   // 3-e in [-124,127]
+  // bin = floor(2 * |x| * 2^(3-e)), saturated at 31.  Magnitudes that would normalise to 16 or more
+  // (possible only when the exponent was clamped from above) are first cut to the largest fp32 below
+  // 2^(e+1); then 2v < 32 and the bin is read from the low mantissa bits of 2.0 + 2v * 2^-22, formed
+  // by one round-toward-zero FMA (exact: no conversion instruction, no intermediate rounding).
+  const float cut = __uint_as_float(((uint32_t)(e + 128) << 23) - 1u);
+  const float sG = pow2f(3 - e) * 0x1p-21f;   // 3-e-21 in [-145,106]
   uint8_t bin[B];
 #pragma unroll
-  for (int i = 0; i < B; ++i) {
-    // |x| * 2^(3-e) is exact (or irrelevant: underflow stays in bin 0, overflow saturates)
-    const float v2 = 2.0f * (ax[i] * s);
-    bin[i] = (uint8_t)min(31, __float2int_rd(v2));
-  }
+  for (int i = 0; i < B; ++i)
+    bin[i] = (uint8_t)(__float_as_uint(__fmaf_rz(fminf(ax[i], cut), sG, 2.0f)) & 31u);
   uint8_t gb[G];
   int bmax = 0;
 #pragma unroll
@@ -114,7 +116,7 @@ __device__ __forceinline__ int64_t salient_row(const Fb4RowExtras& ex, int64_t t
   return -1;
 }
 
-template <int B, int GS, bool F32>
+template <int B, int GS, bool F32, bool RESID>
 __global__ void __launch_bounds__(128)
 fb4_quantize_generic_kernel(const void* __restrict__ xin, int64_t T, int64_t C, int64_t ld,
                             const Fb4DeviceTables* __restrict__ tables, GenericParams p, Fb4RowExtras ex,
@@ -174,8 +176,8 @@ fb4_quantize_generic_kernel(const void* __restrict__ xin, int64_t T, int64_t C, 
     quantize_block<B, GS>(ax, sgn, tb, p, allowed, packed, did, e);
     store_block<B>(packed, did, e, codes + t * (C / 2), meta + t * nblk, blk);
 
-    const int64_t srow = salient_row(ex, t);
-    if (srow >= 0) {
+    const int64_t srow = RESID ? salient_row(ex, t) : -1;
+    if (RESID && srow >= 0) {
       // Sec. 3.3: Delta = x - Q(x), exact in fp32 for the default exponent range; quantized again
       const float sc = pow2f(e - 3);
       uint32_t dsgn = 0;
@@ -208,14 +210,14 @@ cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x
   int64_t want = (total + threads - 1) / threads;
   const int64_t cap = (int64_t)ctx->sm_count * 16;
   const int grid = (int)(want < cap ? want : cap);
-#define FB4_LAUNCH(BB, GSZ)                                                                                          \
-  do {                                                                                                               \
-    if (x_is_f32)                                                                                                    \
-      fb4_quantize_generic_kernel<BB, GSZ, true><<<grid, threads, 0, stream>>>(x, T, C, ld, ctx->d_tables, p, ex,    \
-                                                                               codes, meta);                         \
-    else                                                                                                             \
-      fb4_quantize_generic_kernel<BB, GSZ, false><<<grid, threads, 0, stream>>>(x, T, C, ld, ctx->d_tables, p, ex,   \
-                                                                                codes, meta);                        \
+  const bool resid = ex.n_salient > 0;
+#define FB4_LAUNCH_K(BB, GSZ, F, R) \
+  fb4_quantize_generic_kernel<BB, GSZ, F, R><<<grid, threads, 0, stream>>>(x, T, C, ld, ctx->d_tables, p, ex, codes, meta)
+#define FB4_LAUNCH(BB, GSZ)                                  \
+  do {                                                       \
+    if (x_is_f32) FB4_LAUNCH_K(BB, GSZ, true, false);        \
+    else if (resid) FB4_LAUNCH_K(BB, GSZ, false, true);      \
+    else FB4_LAUNCH_K(BB, GSZ, false, false);                \
   } while (0)
   if (B == 32 && G == 8) FB4_LAUNCH(32, 4);
   else if (B == 32 && G == 32) FB4_LAUNCH(32, 1);
@@ -223,5 +225,6 @@ cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x
   else if (B == 16 && G == 16) FB4_LAUNCH(16, 1);
   else return cudaErrorInvalidValue;
 #undef FB4_LAUNCH
+#undef FB4_LAUNCH_K
   return cudaGetLastError();
 }
