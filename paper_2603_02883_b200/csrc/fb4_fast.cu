@@ -1,12 +1,16 @@
-// TMA-staged FB4 quantize kernel for sm_100a (default configuration: block 32, 8 groups,
-// two-stage selection, exponent range [-124,127]).
+// TMA-staged FB4 quantize kernels for sm_100a: num_groups 8, two-stage selection, block size 32
+// or 16, any exponent clamp, with the SeDA restriction and the residual pass of salient tokens
+// fused in (template parameters), plus a variant for fp32 input.
 //
 // Work unit: a tile of 1024 consecutive channels of one token (2 KB of bf16 = 32 blocks).
 // Every warp owns a ring of shared-memory stages; lane 0 keeps the ring full with 3-D TMA
 // loads (tensor view [T][C/64][64], box 1 x 16 x 64, 128-byte swizzle) that complete on
 // per-stage mbarriers.  Lane i then quantizes block i of the tile entirely in registers:
 // it reads its 64 bytes with four conflict-free 16-byte shared loads, and the warp writes
-// 512 B of codes and 64 B of metadata with one coalesced store each.
+// 512 B of codes and 64 B of metadata with one coalesced store each.  With block size 16 a
+// lane's 64 bytes are two blocks.  The lookup tables (75 KB, built on the host at init) arrive by
+// one bulk asynchronous copy per CTA.  Every wait on an mbarrier is bounded and raises a status
+// bit when it runs out.
 //
 // Arithmetic (all exact):
 //  * magnitudes are compared as 15-bit integers (bf16 patterns are monotone), two per register;
