@@ -31,8 +31,8 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this
 # workload, from the ncu capture summarised in profiles/fb4_quantize_fast_c5_plain_dram_bytes.md
-# (1 858 055 936 B read + 502 568 448 B written; set back to None whenever that kernel changes).
-NCU_TRAFFIC_BYTES = 2360624384
+# (1 858 067 712 B read + 502 677 760 B written; set back to None whenever that kernel changes).
+NCU_TRAFFIC_BYTES = 2360745472
 
 
 def algorithmic_bytes(T: int, C: int, B: int = 32, n_res_rows: int = 0, seda: bool = False,
