@@ -207,6 +207,11 @@ class Ops:
             q16 = self._buf["q16"]
             meta16 = self.buf("meta16", (T, C // 16), torch.int16)
             return (lambda: fb4.fb4_quantize(q16.ctx, x, T, C, C, codes, meta16)), T * C * 2.5 + T * (C // 16) * 2
+        if name == "quantize_mxfp8_tiled_scales":
+            e8 = self.buf("e4m3", (T, C), torch.uint8)
+            sc = self.buf("sf", (fb4.fb4_mxfp8_scale_bytes(T, C, 1),), torch.uint8)
+            return (lambda: fb4.fb4_quantize_mxfp8(q.ctx, x, T, C, C, None, None, 0, e8, sc, 1)), \
+                T * C * 3.0 + T * (C // B)
         if name == "plain_f32":
             xf = self.buf("x32", (T, C), torch.float32)
             xf.copy_(x)
@@ -262,7 +267,8 @@ class Ops:
 
 
 OP_NAMES = ["plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
-            "dequantize_bf16_plain", "dequantize_bf16_decomposed", "to_mxfp8_tiled_scales"]
+            "dequantize_bf16_plain", "dequantize_bf16_decomposed", "to_mxfp8_tiled_scales",
+            "quantize_mxfp8_tiled_scales"]
 
 
 def main():
@@ -407,7 +413,8 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         ms = total / steps
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
                      "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_given_set",
-                                                                         "decomposed_seda") else "decode"}
+                                                                         "decomposed_seda", "quantize_mxfp8_tiled_scales")
+                     else "decode"}
         if name == "dequantize_f32_decomposed":
             ops.drop("out32")
         if name == "plain_f32":

@@ -267,6 +267,25 @@ int fb4_quantize_weights(fb4_ctx* ctx, const void* w_bf16, int64_t N, int64_t K,
  */
 int fb4_to_mxfp8(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T, int64_t C, uint8_t* e4m3,
                  uint8_t* scales, int scale_layout, void* stream);
+/*
+ * fb4_quantize[_seda] and fb4_to_mxfp8 in one pass (App. D.2 names an MXFP8 GEMM on Blackwell as
+ * the consumer of FB4): x is quantized as in fb4_quantize / fb4_quantize_seda, and the result is
+ * written directly as e4m3 bytes and E8M0 scales; the 4-bit codes and the dialect ids are not
+ * stored (3.03 instead of 2.56 + 1.59 bytes per element of traffic).  The output equals
+ * fb4_to_mxfp8 applied to the output of fb4_quantize[_seda], byte for byte.
+ * Default configuration only (block size 32, num_groups 8, two-stage selection, full exponent
+ * range, a formatbook that fits the packed tables) and C a multiple of 64: otherwise
+ * FB4_ERR_INVALID_ARG / FB4_ERR_SHAPE, and the two calls are used instead.
+ *   cluster_id : NULL = no SeDA restriction (then cluster_mask is ignored)
+ *   e4m3       : device uint8 [T][C] (out), 32-byte aligned
+ *   scales     : device uint8 (out), fb4_mxfp8_scale_bytes(T, C, scale_layout) bytes; with the
+ *                tiled layout and T or C/32 not a multiple of 128 / 4 the whole buffer is first
+ *                filled with 0x7f (scale 1) on the stream
+ */
+int fb4_quantize_mxfp8(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems,
+                       const int32_t* cluster_id, const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* e4m3,
+                       uint8_t* scales, int scale_layout, void* stream);
+
 /* Size in bytes of the scale buffer of fb4_to_mxfp8 (-1 for invalid arguments).  Host only. */
 int64_t fb4_mxfp8_scale_bytes(int64_t T, int64_t C, int scale_layout);
 

@@ -374,6 +374,28 @@ int fb4_quantize_weights(fb4_ctx* ctx, const void* w, int64_t N, int64_t K, int6
   return FB4_OK;
 }
 
+int fb4_quantize_mxfp8(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const int32_t* cluster_id,
+                       const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* e4m3, uint8_t* scales,
+                       int scale_layout, void* stream) {
+  if (!ctx) return FB4_ERR_INVALID_ARG;
+  if (scale_layout != 0 && scale_layout != 1) return FB4_ERR_INVALID_ARG;
+  if (T < 0 || C <= 0 || C % 64 != 0 || ld < C || T > 0x7fffffffLL) return FB4_ERR_SHAPE;
+  if (T == 0) return FB4_OK;
+  if (!x || !e4m3 || !scales) return FB4_ERR_INVALID_ARG;
+  if (cluster_id && (!cluster_mask || n_clusters <= 0)) return FB4_ERR_INVALID_ARG;
+  if (!aligned16(x) || (ld & 7) || (reinterpret_cast<uintptr_t>(e4m3) & 31u)) return FB4_ERR_ALIGN;
+  if (!fb4_fast_mx_eligible(ctx, x, T, C, ld)) return FB4_ERR_INVALID_ARG;   // default configuration only
+  Fb4RowExtras ex{};
+  ex.cluster_id = cluster_id;
+  ex.cluster_mask = cluster_id ? cluster_mask : nullptr;
+  cudaError_t e = fb4_launch_quantize_fast_mx(ctx, x, T, C, ld, ex, e4m3, scales, scale_layout,
+                                              static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
+  ctx->launches += 1;
+  ctx->last_variant = "fast";
+  return FB4_OK;
+}
+
 int64_t fb4_mxfp8_scale_bytes(int64_t T, int64_t C, int layout) {
   if (T < 0 || C <= 0 || C % 32 != 0 || (layout != 0 && layout != 1)) return -1;
   const int64_t n_col = C / 32;

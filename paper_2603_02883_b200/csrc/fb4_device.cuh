@@ -60,4 +60,32 @@ __device__ __forceinline__ void decode_word(uint32_t cw, const uint4& dt, uint32
   for (int j = 0; j < 4; ++j) pr[j] = mul_bf16x2(mag[j], sc2) | (sgn[j] & 0x80008000u);
 }
 
+// e4m3 byte (1 sign, 4 exponent bits with bias 7, 3 mantissa bits) of an integer 0..15: exact
+__host__ __device__ inline uint32_t e4m3_of_small_int(uint32_t m) {
+  if (m == 0) return 0u;
+  int ex = 0;
+  while ((m >> (ex + 1)) != 0) ++ex;   // floor(log2 m) <= 3
+  const uint32_t frac = m - (1u << ex);
+  return ((uint32_t)(ex + 7) << 3) | (frac << 3 >> ex);
+}
+
+// 8 codes (one 32-bit code word) -> 8 e4m3 bytes (two registers).  fb = the dialect's 8 magnitudes as
+// e4m3 bytes: a byte permute with four 3-bit indices as selector looks up four elements at once;
+// sign bits come from sign-replicating permutes.
+__device__ __forceinline__ void codes_to_e4m3(uint32_t cw, uint2 fb, uint32_t& lo, uint32_t& hi) {
+  const uint32_t sel = cw & 0x77777777u;
+  const uint32_t s_odd = prmt(cw, 0u, 0xba98u), s_even = prmt(cw << 4, 0u, 0xba98u);   // 0xff where negative
+  lo = prmt(fb.x, fb.y, sel) | (__byte_perm(s_even, s_odd, 0x5140) & 0x80808080u);
+  hi = prmt(fb.x, fb.y, sel >> 16) | (__byte_perm(s_even, s_odd, 0x7362) & 0x80808080u);
+}
+
+// Byte offset of the E8M0 scale of (row, 32-element block col): row-major, or tiles of 128 rows x 4
+// columns (512 bytes, column tiles contiguous, (r mod 32)*16 + (r div 32)*4 + c inside a tile).
+__host__ __device__ inline int64_t mx_scale_offset(int64_t row, int64_t col, int64_t n_col, int64_t col_tiles,
+                                                   int tiled) {
+  if (!tiled) return row * n_col + col;
+  const int64_t r = row & 127;
+  return ((row >> 7) * col_tiles + (col >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (col & 3);
+}
+
 }  // namespace fb4dev

@@ -63,6 +63,7 @@ struct SmemTables {
   uint64_t qerr_private[kMaxGroups][32][16];
   uint8_t pairlut[32 * kPairStride];     // [dialect][36*bin_hi + bin_lo] -> idx_lo | idx_hi<<4
   uint4 fb_bf16[32];                     // [dialect] -> magnitudes as bf16, high bytes then low bytes (residual pass)
+  uint2 fb_e4m3[32];                     // [dialect] -> magnitudes as e4m3 bytes (MXFP8 output)
   FastTables c;
 };
 
@@ -75,6 +76,10 @@ struct FastParams {
   uint16_t* meta;
   uint32_t* status;   // device word: bit 0 = a TMA wait ran out
   uint32_t ec_lo, ec_hi;   // clamp of the biased block exponent (CLAMP kernels): exp_min + 127, exp_max + 127
+  uint8_t* e4m3;           // MX kernels: e4m3 bytes [T][C] and E8M0 scale bytes instead of codes / meta
+  uint8_t* scales;
+  int64_t scale_col_tiles;
+  int32_t scale_tiled;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -284,7 +289,7 @@ struct TilePos {
   }
 };
 
-template <bool SEDA, bool DECOMP, bool B16, bool CLAMP>
+template <bool SEDA, bool DECOMP, bool B16, bool CLAMP, bool MX = false>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
                          FastParams p, Fb4RowExtras ex) {
@@ -549,7 +554,19 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
       const uint32_t ev = __byte_perm(sa, sb, 0x6420), od = __byte_perm(sa, sb, 0x7531);
       cw[q] = idx | (((ev & 0x0f0f0f0fu) | (od & 0xf0f0f0f0u)) & 0x88888888u);
     }
-    if (active) {
+    if (MX) {
+      // MXFP8 output (block size 32): the codes become e4m3 bytes in registers, the scale byte is the
+      // E8M0 scale; 32 contiguous bytes per lane, 1 KB per warp
+      if (active) {
+        const uint2 fb = tb->fb_e4m3[didh[0]];
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) fb4dev::codes_to_e4m3(cw[q], fb, o[2 * q], o[2 * q + 1]);
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p.e4m3 + row * p.C + blk * 32),
+                     "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+        p.scales[fb4dev::mx_scale_offset(row, blk, nblk, p.scale_col_tiles, p.scale_tiled)] = (uint8_t)(Ech[0] - 3u);
+      }
+    } else if (active) {
       *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
       if (B16)   // two records
         *reinterpret_cast<uint32_t*>(p.meta + (row * nblk + blk) * 2) =
@@ -815,6 +832,9 @@ bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes
       row[8 + j] = (uint8_t)(u >> 16);
     }
   }
+  for (int d = 0; d < 32; ++d)
+    for (int j = 0; j < 8; ++j)
+      reinterpret_cast<uint8_t*>(&img->fb_e4m3[d])[j] = (uint8_t)fb4dev::e4m3_of_small_int(t.formatbook[d][j]);
   img->c = ft;
   void* d = nullptr;
   bool ok = cudaMalloc(&d, sizeof *img) == cudaSuccess;
@@ -852,6 +872,8 @@ cudaError_t fb4_fast_prepare_device() {
   FB4_OPT_IN(true, false, true, true);
   FB4_OPT_IN(false, true, true, true);
   FB4_OPT_IN(true, true, true, true);
+  FB4_OPT_IN(false, false, false, false, true);
+  FB4_OPT_IN(true, false, false, false, true);
 #undef FB4_OPT_IN
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
   return e;
@@ -869,34 +891,45 @@ bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, 
   return encode_tiled_fn() != nullptr;
 }
 
-cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
-                                     const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta, cudaStream_t stream) {
-  CUtensorMap map;
+// Tensor map, grid and tile-walk parameters of one launch of the bf16-input kernels.
+static cudaError_t fast_setup(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, bool chunked,
+                              CUtensorMap* map, FastParams* p, int* grid_out) {
   const cuuint64_t dims[3] = {64, (cuuint64_t)(C / 64), (cuuint64_t)T};
   const cuuint64_t strides[2] = {128, (cuuint64_t)ld * 2};
   const cuuint32_t box[3] = {64, 16, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = encode_tiled_fn()(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides,
+  const CUresult r = encode_tiled_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides,
                                        box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  *p = FastParams{};
+  p->T = T;
+  p->C = C;
+  p->tiles_per_row = (C + 1023) / 1024;
+  p->n_tiles = T * p->tiles_per_row;
+  p->status = ctx->d_status;
+  const int64_t want = (p->n_tiles + kWarps - 1) / kWarps;
+  const int grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
+  const int64_t wstride = chunked ? kWarps : (int64_t)grid * kWarps;   // tiles between a warp's consecutive tiles
+  p->step_rows = wstride / p->tiles_per_row;
+  p->step_cols = (int32_t)(wstride % p->tiles_per_row);
+  p->ec_lo = (uint32_t)(ctx->cfg.exp_min + 127);
+  p->ec_hi = (uint32_t)(ctx->cfg.exp_max + 127);
+  *grid_out = grid;
+  return cudaSuccess;
+}
+
+cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
+                                     const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta, cudaStream_t stream) {
+  const bool seda = ex.cluster_id != nullptr, decomp = ex.n_salient > 0;
+  CUtensorMap map;
   FastParams p;
-  p.T = T;
-  p.C = C;
-  p.tiles_per_row = (C + 1023) / 1024;
-  p.n_tiles = T * p.tiles_per_row;
+  int grid = 0;
+  const cudaError_t e = fast_setup(ctx, x, T, C, ld, decomp, &map, &p, &grid);
+  if (e != cudaSuccess) return e;
   p.codes = codes;
   p.meta = meta;
-  p.status = ctx->d_status;
-  const int64_t want = (p.n_tiles + kWarps - 1) / kWarps;
-  const int grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
-  const bool seda = ex.cluster_id != nullptr, decomp = ex.n_salient > 0;
-  const int64_t wstride = decomp ? kWarps : (int64_t)grid * kWarps;   // tiles between a warp's consecutive tiles
-  p.step_rows = wstride / p.tiles_per_row;
-  p.step_cols = (int32_t)(wstride % p.tiles_per_row);
   const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
-  p.ec_lo = (uint32_t)(ctx->cfg.exp_min + 127);
-  p.ec_hi = (uint32_t)(ctx->cfg.exp_max + 127);
   const bool b16 = ctx->cfg.block_size == 16;
   const bool clamp = ctx->cfg.exp_min != -124 || ctx->cfg.exp_max != 127;
   const int variant = (seda ? 1 : 0) | (decomp ? 2 : 0) | (b16 ? 4 : 0) | (clamp ? 8 : 0);
@@ -960,5 +993,36 @@ cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int6
   p.step_cols = (int32_t)(wstride % p.tiles_per_row);
   fb4_quantize_f32_kernel<<<grid, kWarpsF32 * 32, kSmemBytesF32, stream>>>(
       map, static_cast<const SmemTables*>(ctx->d_fast_tables), p);
+  return cudaGetLastError();
+}
+
+// Quantize straight to an MXFP8 operand (e4m3 bytes + E8M0 scales): default configuration only.
+bool fb4_fast_mx_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {
+  const fb4_config& c = ctx->cfg;
+  return c.block_size == 32 && c.exp_min == -124 && c.exp_max == 127 && fb4_fast_eligible(ctx, x, T, C, ld);
+}
+
+cudaError_t fb4_launch_quantize_fast_mx(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
+                                        const Fb4RowExtras& ex, uint8_t* e4m3, uint8_t* scales, int tiled,
+                                        cudaStream_t stream) {
+  CUtensorMap map;
+  FastParams p;
+  int grid = 0;
+  cudaError_t e = fast_setup(ctx, x, T, C, ld, false, &map, &p, &grid);
+  if (e != cudaSuccess) return e;
+  p.e4m3 = e4m3;
+  p.scales = scales;
+  p.scale_tiled = tiled;
+  const int64_t n_col = C / 32;
+  p.scale_col_tiles = (n_col + 3) / 4;
+  if (tiled && ((T & 127) || (n_col & 3))) {   // the kernel writes real entries only: padding = scale 1
+    e = cudaMemsetAsync(scales, 0x7f, (size_t)(((T + 127) / 128) * p.scale_col_tiles * 512), stream);
+    if (e != cudaSuccess) return e;
+  }
+  const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
+  if (ex.cluster_id)
+    fb4_quantize_fast_kernel<true, false, false, false, true><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
+  else
+    fb4_quantize_fast_kernel<false, false, false, false, true><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
   return cudaGetLastError();
 }

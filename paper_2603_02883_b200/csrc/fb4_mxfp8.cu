@@ -11,32 +11,10 @@
 
 namespace {
 
-using fb4dev::prmt;
+using fb4dev::e4m3_of_small_int;
 
 constexpr int kThreads = 256;
 constexpr int kUnroll = 2;
-
-// e4m3 byte of an integer 0..15: 1.mmm * 2^(E-7)
-__device__ __forceinline__ uint32_t e4m3_of_small_int(uint32_t m) {
-  if (m == 0) return 0u;
-  const int ex = 31 - __clz((int)m);
-  const uint32_t frac = m - (1u << ex);
-  return ((uint32_t)(ex + 7) << 3) | (frac << 3 >> ex);   // ex <= 3
-}
-
-__device__ __forceinline__ int64_t scale_offset(int64_t row, int64_t col, int64_t n_col, int64_t col_tiles, int tiled) {
-  if (!tiled) return row * n_col + col;
-  const int64_t r = row & 127;
-  return ((row >> 7) * col_tiles + (col >> 2)) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (col & 3);
-}
-
-// 8 codes -> 8 e4m3 bytes (two registers)
-__device__ __forceinline__ void convert_word(uint32_t cw, uint2 fb, uint32_t& lo, uint32_t& hi) {
-  const uint32_t sel = cw & 0x77777777u;
-  const uint32_t s_odd = prmt(cw, 0u, 0xba98u), s_even = prmt(cw << 4, 0u, 0xba98u);   // 0xff where negative
-  lo = prmt(fb.x, fb.y, sel) | (__byte_perm(s_even, s_odd, 0x5140) & 0x80808080u);
-  hi = prmt(fb.x, fb.y, sel >> 16) | (__byte_perm(s_even, s_odd, 0x7362) & 0x80808080u);
-}
 
 __global__ void __launch_bounds__(kThreads)
 fb4_to_mxfp8_kernel(const uint4* __restrict__ codes, const uint16_t* __restrict__ meta, int64_t T, int64_t n_col,
@@ -80,10 +58,10 @@ fb4_to_mxfp8_kernel(const uint4* __restrict__ codes, const uint16_t* __restrict_
       if (b >= total) continue;
       const uint2 fb = fb8[(mm[u] >> 8) & 31u];
       uint32_t o[8];
-      convert_word(c[u].x, fb, o[0], o[1]);
-      convert_word(c[u].y, fb, o[2], o[3]);
-      convert_word(c[u].z, fb, o[4], o[5]);
-      convert_word(c[u].w, fb, o[6], o[7]);
+      fb4dev::codes_to_e4m3(c[u].x, fb, o[0], o[1]);
+      fb4dev::codes_to_e4m3(c[u].y, fb, o[2], o[3]);
+      fb4dev::codes_to_e4m3(c[u].z, fb, o[4], o[5]);
+      fb4dev::codes_to_e4m3(c[u].w, fb, o[6], o[7]);
       uint8_t* dst = e4m3 + b * 32;
       if (out_aligned32) {
         asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(o[0]), "r"(o[1]),
@@ -103,7 +81,7 @@ fb4_to_mxfp8_kernel(const uint4* __restrict__ codes, const uint16_t* __restrict_
           row = b / n_col;
           col = b - row * n_col;
         }
-        off = scale_offset(row, col, n_col, col_tiles, 1);
+        off = fb4dev::mx_scale_offset(row, col, n_col, col_tiles, 1);
       }
       scales[off] = (uint8_t)mm[u];   // E8M0 of 2^(e-3)
     }
@@ -124,7 +102,7 @@ fb4_to_mxfp8_kernel(const uint4* __restrict__ codes, const uint16_t* __restrict_
         row = j / w;
         col = n_col + j % w;
       }
-      scales[scale_offset(row, col, n_col, col_tiles, 1)] = 0x7f;
+      scales[fb4dev::mx_scale_offset(row, col, n_col, col_tiles, 1)] = 0x7f;
     }
   }
 }

@@ -23,7 +23,7 @@ STATIC_MAX_CLUSTERS = 1024
 EXPORTS = [
     "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
     "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_select_salient_topk", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
-    "fb4_quantize_weights", "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
+    "fb4_quantize_weights", "fb4_quantize_mxfp8", "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
 
 
@@ -84,6 +84,8 @@ def lib() -> ctypes.CDLL:
     L.fb4_dequantize.argtypes = [vp, vp, vp, i64, i64, vp, i64, vp, vp, vp, ci, vp]
     L.fb4_quantize_weights.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.fb4_quantize_weights.restype = ci
+    L.fb4_quantize_mxfp8.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, vp, vp, ci, vp]
+    L.fb4_quantize_mxfp8.restype = ci
     L.fb4_to_mxfp8.argtypes = [vp, vp, vp, i64, i64, vp, vp, ci, vp]
     L.fb4_to_mxfp8.restype = ci
     L.fb4_mxfp8_scale_bytes.argtypes = [i64, i64, ci]
@@ -224,6 +226,12 @@ def fb4_dequantize(ctx, codes, meta, T, C, salient_idx, n_salient, res_codes, re
 def fb4_quantize_weights(ctx, w, N, K, ld_elems, codes, meta, stream=None) -> None:
     _check(lib().fb4_quantize_weights(ctx, _ptr(w), N, K, ld_elems, _ptr(codes), _ptr(meta), _stream(stream)),
            "fb4_quantize_weights")
+
+
+def fb4_quantize_mxfp8(ctx, x, T, C, ld_elems, cluster_id, cluster_mask, n_clusters, e4m3, scales, scale_layout,
+                       stream=None) -> None:
+    _check(lib().fb4_quantize_mxfp8(ctx, _ptr(x), T, C, ld_elems, _ptr(cluster_id), _ptr(cluster_mask), n_clusters,
+                                    _ptr(e4m3), _ptr(scales), scale_layout, _stream(stream)), "fb4_quantize_mxfp8")
 
 
 def fb4_to_mxfp8(ctx, codes, meta, T, C, e4m3, scales, scale_layout, stream=None) -> None:
@@ -373,6 +381,17 @@ class Fb4:
         codes, meta = self._outs(N, K)
         fb4_quantize_weights(self.ctx, w, N, K, ld, codes, meta)
         return Quantized(codes, meta)
+
+    def quantize_mxfp8(self, x, scale_layout: int = 1, cluster_id=None, cluster_mask=None):
+        """quantize straight to (e4m3 bytes [T][C], E8M0 scale bytes)"""
+        assert x.dtype == torch.bfloat16
+        T, C, ld = self._shape(x)
+        e4m3 = torch.empty((T, C), dtype=torch.uint8, device=x.device)
+        n = fb4_mxfp8_scale_bytes(T, C, scale_layout)
+        scales = torch.empty(max(n, 1), dtype=torch.uint8, device=x.device)
+        fb4_quantize_mxfp8(self.ctx, x, T, C, ld, cluster_id, cluster_mask,
+                           0 if cluster_mask is None else cluster_mask.numel(), e4m3, scales, scale_layout)
+        return e4m3, scales[:n]
 
     def to_mxfp8(self, q: Quantized, scale_layout: int = 0):
         """(e4m3 bytes [T][C], E8M0 scale bytes) of the main tensor of q."""

@@ -68,3 +68,40 @@ def test_argument_checks(q32):
     q16 = fb4.Fb4(block_size=16)
     assert L.fb4_to_mxfp8(q16.ctx, p, p, 4, 64, p, p, 0, None) == fb4.ERR_INVALID_ARG
     q16.close()
+
+
+@pytest.mark.parametrize("T,C", [(1, 64), (130, 3072), (300, 1024 + 64), (257, 128), (2368, 64)])
+def test_fused_quantize_to_mxfp8(q32, T, C):
+    """fb4_quantize_mxfp8 equals quantize followed by the MXFP8 view (oracle), plain and SeDA, both layouts."""
+    w = synth.Workload("m", T=T, C=C, seed=T + C, kind=1, n_outlier=2, outlier_gain=50.0, seda=True,
+                       n_clusters=min(4, T), cluster_seed=5)
+    bits = synth.activation(w)
+    cid, masks = synth.clusters(w)
+    x = to_dev_bf16(bits)
+    ref_plain = orc.quantize(bits, FB)
+    ref_seda = orc.quantize(bits, FB, cluster_id=cid, cluster_mask=masks)
+    for layout in (0, 1):
+        e4m3, scales = q32.quantize_mxfp8(x, layout)
+        e_ref, s_ref = orc.to_mxfp8(ref_plain, FB, layout)
+        assert np.array_equal(e4m3.cpu().numpy(), e_ref) and np.array_equal(scales.cpu().numpy(), s_ref)
+        e4m3, scales = q32.quantize_mxfp8(x, layout, torch.from_numpy(cid).cuda(),
+                                          torch.from_numpy(masks.view(np.int32)).cuda())
+        e_ref, s_ref = orc.to_mxfp8(ref_seda, FB, layout)
+        assert np.array_equal(e4m3.cpu().numpy(), e_ref) and np.array_equal(scales.cpu().numpy(), s_ref)
+
+
+def test_fused_quantize_to_mxfp8_rejects_other_configurations():
+    import ctypes
+    q16 = fb4.Fb4(block_size=16)
+    x = torch.zeros((4, 64), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    L = fb4.lib()
+    assert L.fb4_quantize_mxfp8(q16.ctx, p(x), 4, 64, 64, None, None, 0, p(out), p(out), 0, None) == fb4.ERR_INVALID_ARG
+    q16.close()
+    q = fb4.Fb4()
+    assert L.fb4_quantize_mxfp8(q.ctx, p(x), 4, 32, 64, None, None, 0, p(out), p(out), 0, None) == fb4.ERR_SHAPE
+    assert L.fb4_quantize_mxfp8(q.ctx, p(x), 4, 64, 64, None, None, 0, ctypes.c_void_p(out.data_ptr() + 16), p(out), 0,
+                                None) == fb4.ERR_ALIGN
+    assert L.fb4_quantize_mxfp8(q.ctx, p(x), 4, 64, 64, None, None, 0, p(out), p(out), 3, None) == fb4.ERR_INVALID_ARG
+    q.close()
