@@ -354,7 +354,8 @@ def main():
         "gpu_launches": launches,
         "clocks": clk.summary(),
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_TRAFFIC_BYTES if (args.op == "plain" and args.workload == "c5_plain") else None,
+                     "traffic": NCU_TRAFFIC_BYTES if (args.op == "plain" and args.workload == "c5_plain"
+                                                      and not args.generic_kernel) else None,
                      "peak_kind": f"{peak_kind} copy bandwidth",
                      "kernel": f"fb4 {args.op} ({variant})", "algorithmic_bytes_per_launch": alg,
                      "launch_ms_mean": kernel_ms, "launch_ms_min": float(np.min(per))},
