@@ -454,6 +454,31 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         res["c2_weights_exhaustive"] = {"ms": tot / 3, "Gelem/s": w2.T * w2.C / (tot / 3 * 1e-3) / 1e9,
                                         "dialect_disagreement_vs_online": dis,
                                         "mse_online_over_mse_exhaustive": mse_lut / mse_exh}
+        # the small tensor (256 x 3072): launch-latency-bound; quantize + decode as a pair, launched
+        # one by one and replayed from a CUDA graph of 20 pairs
+        w1 = synth.workloads()["c1"]
+        x1 = torch.from_numpy(synth.activation(w1).view(np.int16)).cuda().view(torch.bfloat16)
+        c1 = torch.empty((w1.T, w1.C // 2), dtype=torch.uint8, device="cuda")
+        m1 = torch.empty((w1.T, w1.C // B), dtype=torch.int16, device="cuda")
+        o1 = torch.empty((w1.T, w1.C), dtype=torch.float32, device="cuda")
+
+        def pair():
+            fb4.fb4_quantize(q.ctx, x1, w1.T, w1.C, w1.C, c1, m1)
+            fb4.fb4_dequantize(q.ctx, c1, m1, w1.T, w1.C, None, 0, None, None, o1, 0)
+
+        tot, _ = time_steps(pair, 200, 20, torch)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            pair()
+        torch.cuda.current_stream().wait_stream(side)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(20):
+                pair()
+        tot_g, _ = time_steps(graph.replay, 20, 3, torch)
+        res["c1_256x3072_quantize_plus_decode"] = {"us_per_pair_launched_one_by_one": tot / 200 * 1e3,
+                                                   "us_per_pair_in_a_cuda_graph": tot_g / (20 * 20) * 1e3}
         res["c2_plain_32760x3072_l2_flushed"] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9,
                                                  "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
                                                  "kernel_variant": q.last_variant}
