@@ -371,7 +371,9 @@ static uint16_t f32_to_bf16_rne(float f) {
 /*
  * Decode: xhat = (-1)^s * F[did][idx] * 2^(e-3); salient rows add the decoded
  * residual, the sum being rounded once to fp32.  out_dtype 0: float32 out,
- * 1: bf16 bit patterns (round-to-nearest-even of the fp32 result).
+ * 1: bf16 bit patterns (round-to-nearest-even of the fp32 result),
+ * 2: IEEE half bit patterns (the compiler's float -> _Float16 conversion: round to
+ *    nearest even, overflow to infinity), the type the paper's H100 pipeline decodes to (App. D.2).
  */
 int fb4o_dequantize(const uint8_t *codes, const uint16_t *meta, int64_t T, int64_t C, int block_size,
                     const uint8_t *F, const int32_t *salient_idx, int64_t n_salient,
@@ -396,8 +398,14 @@ int fb4o_dequantize(const uint8_t *codes, const uint16_t *meta, int64_t T, int64
         double r = dequant_value(F, rm >> 8, (int)(rm & 0xff) - 124, rc);
         val = (float)((double)val + r);
       }
-      if (out_dtype == 0) ((float *)out)[t * C + c] = val;
-      else ((uint16_t *)out)[t * C + c] = f32_to_bf16_rne(val);
+      if (out_dtype == 0) {
+        ((float *)out)[t * C + c] = val;
+      } else if (out_dtype == 1) {
+        ((uint16_t *)out)[t * C + c] = f32_to_bf16_rne(val);
+      } else {
+        _Float16 h = (_Float16)val;
+        memcpy((uint16_t *)out + t * C + c, &h, 2);
+      }
     }
   }
   return 0;

@@ -183,11 +183,12 @@ def dequantize(q: Quantized, formatbook, block_size: int = 32, out_dtype: str = 
     C = C2 * 2
     F = _c(formatbook, np.uint8)
     ns = 0 if q.salient_idx is None else q.salient_idx.shape[0]
-    out = np.zeros((T, C), dtype=np.float32 if out_dtype == "f32" else np.uint16)
+    code = {"f32": 0, "bf16": 1, "f16": 2}[out_dtype]
+    out = np.zeros((T, C), dtype=np.float32 if code == 0 else np.uint16)
     r = lib().fb4o_dequantize(_p(_c(q.codes, np.uint8)), _p(_c(q.meta, np.uint16)), T, C, block_size, _p(F),
                               _p(_c(q.salient_idx, np.int32)), ns,
                               _p(_c(q.res_codes, np.uint8)), _p(_c(q.res_meta, np.uint16)),
-                              _p(out), 0 if out_dtype == "f32" else 1)
+                              _p(out), code)
     if r != 0:
         raise ValueError(f"fb4o_dequantize failed: {r}")
     return out

@@ -609,6 +609,26 @@ def pin_dequantize_formula(seed=7):
             assert float(synth.bf16_bits_to_f32(yb[t:t + 1, c])[0]) == want   # 4-bit magnitudes are exact in bf16
 
 
+def pin_dequantize_f16(seed=13):
+    """Half-precision decode = the fp32 decode rounded to IEEE half (numpy's conversion as the independent
+    rounding: nearest even, overflow to infinity, gradual underflow), residual rows included."""
+    rng = np.random.default_rng(seed)
+    codes = rng.integers(0, 256, size=(6, 32), dtype=np.uint8)
+    did = rng.integers(0, 32, size=(6, 2))
+    sb = np.array([[0, 90], [100, 103], [110, 121], [124, 130], [139, 140], [141, 251]])   # under- and overflow
+    meta = (sb | (did << 8)).astype(np.uint16)
+    q = orc.Quantized(codes, meta, salient_idx=np.array([2, 3], np.int32),
+                      res_codes=rng.integers(0, 256, size=(2, 32), dtype=np.uint8),
+                      res_meta=(np.array([[103, 113], [118, 123]]) | (did[:2] << 8)).astype(np.uint16))
+    y32 = orc.dequantize(q, FB)
+    assert np.count_nonzero(y32.view(np.uint32) & 0xFFFF) > 20      # sums that are not bf16 values
+    with np.errstate(over="ignore"):
+        want = y32.astype(np.float16).view(np.uint16)
+    got = orc.dequantize(q, FB, out_dtype="f16")
+    assert np.array_equal(got, want)
+    assert np.isinf(want.view(np.float16)).any() and (want.view(np.float16) == 0).any()
+
+
 def pin_mse():
     x = synth.f32_to_bf16_bits(np.array([[1.0, 2.0, -3.0, 0.5]], np.float32))
     r = np.array([[1.5, 2.0, -1.0, 0.5]], np.float32)
@@ -619,7 +639,7 @@ ALL_PINS = [
     pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
     pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_salient_topk, pin_decomposition,
-    pin_dequantize_formula, pin_mse, pin_f32_input, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
+    pin_dequantize_formula, pin_dequantize_f16, pin_mse, pin_f32_input, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
     pin_subformatbook_hand_counted,
     pin_subformatbook_one_dialect_per_bucket_and_closed_loop,
 ]

@@ -37,6 +37,7 @@ MUTANTS = {
                              "if (!taken[t] && (arg < 0 || score[t] >= score[arg])) arg = t;"),
     "topk_smallest": ("if (!taken[t] && (arg < 0 || score[t] > score[arg])) arg = t;",
                       "if (!taken[t] && (arg < 0 || score[t] < score[arg])) arg = t;"),
+    "f16_through_bf16": ("_Float16 h = (_Float16)val;", "_Float16 h = (_Float16)bf16_to_double(f32_to_bf16_rne(val));"),
     "clamp_min_ignored": ("if (e < cfg->exp_min) e = cfg->exp_min;", ";"),
     "zero_block_exponent": ("e = cfg->exp_min;\n  } else {", "e = 0;\n  } else {"),
     "stage1_bucket_shift": ("int bucket = k / 2 < 8 ? 8 : k / 2;", "int bucket = k / 2 < 9 ? 9 : k / 2;"),
