@@ -259,6 +259,10 @@ class Ops:
             out = self.buf("out16", (T, C), torch.bfloat16)
             return (lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, None, 0, None, None, out, 1)), \
                 plain_bytes + T * C * 2
+        if name == "dequantize_f16_plain":
+            out = self.buf("out16", (T, C), torch.bfloat16)
+            return (lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, None, 0, None, None, out, 2)), \
+                plain_bytes + T * C * 2
         if name == "dequantize_bf16_decomposed":
             out = self.buf("out16", (T, C), torch.bfloat16)
             return (lambda: fb4.fb4_dequantize(q.ctx, codes, meta, T, C, sal, n_sal, rc, rm, out, 1)), \
@@ -267,7 +271,7 @@ class Ops:
 
 
 OP_NAMES = ["plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
-            "dequantize_bf16_plain", "dequantize_bf16_decomposed", "to_mxfp8_tiled_scales",
+            "dequantize_bf16_plain", "dequantize_bf16_decomposed", "dequantize_f16_plain", "to_mxfp8_tiled_scales",
             "quantize_mxfp8_tiled_scales"]
 
 

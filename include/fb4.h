@@ -230,8 +230,9 @@ int fb4_quantize_decomposed_idx(fb4_ctx* ctx, const void* x_bf16, int64_t T, int
  * residual is added, the sum rounded once to fp32 (Sec. 3.3: Q(Act)+Q(Delta)).
  *   salient_idx : NULL / n_salient = 0 for plain tensors; else device int32
  *                 [n_salient], strictly ascending
- *   out         : device, [T][C] contiguous; out_dtype 0 = float32, 1 = bfloat16
- *                 (round-to-nearest-even of the fp32 result)
+ *   out         : device, [T][C] contiguous; out_dtype 0 = float32, 1 = bfloat16, 2 = IEEE half
+ *                 (the type App. D.2 decodes to); 1 and 2 are the round-to-nearest-even of the
+ *                 fp32 result (half: overflow to infinity, gradual underflow)
  */
 int fb4_dequantize(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T, int64_t C,
                    const int32_t* salient_idx, int64_t n_salient, const uint8_t* res_codes,

@@ -326,7 +326,7 @@ int fb4_dequantize(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int
                    const uint16_t* res_meta, void* out, int out_dtype, void* stream) {
   if (!ctx) return FB4_ERR_INVALID_ARG;
   if (T < 0 || C <= 0 || C % ctx->cfg.block_size != 0 || T > 0x7fffffffLL) return FB4_ERR_SHAPE;
-  if (out_dtype != 0 && out_dtype != 1) return FB4_ERR_INVALID_ARG;
+  if (out_dtype < 0 || out_dtype > 2) return FB4_ERR_INVALID_ARG;
   if (n_salient < 0) return FB4_ERR_INVALID_ARG;
   if (T == 0) return FB4_OK;
   if (!codes || !meta || !out) return FB4_ERR_INVALID_ARG;

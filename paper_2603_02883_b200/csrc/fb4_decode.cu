@@ -16,6 +16,13 @@ __device__ __forceinline__ uint32_t f32_to_bf16_rne(float f) {
 constexpr int kDecodeThreads = 256;
 constexpr int kDecodeUnroll = 2;          // blocks in flight per thread
 
+// two fp32 -> two IEEE halves (round to nearest even, overflow to infinity), low half = a
+__device__ __forceinline__ uint32_t f32x2_to_f16x2(float a, float b) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(b), "f"(a));
+  return d;
+}
+
 // 32 bytes per store: a lane writes whole 32-byte sectors.  p must be 32-byte aligned when wide.
 __device__ __forceinline__ void store_b32x8(void* p, const uint32_t* v, bool wide) {
   if (wide) {
@@ -55,11 +62,17 @@ __device__ __forceinline__ void quad_transpose(uint32_t (&c)[4], int lane) {
   }
 }
 
-// word (8 elements as 4 x bf16x2) -> 32 bytes of fp32 or 16 bytes of bf16 at dst
-template <int OUT_BF16>
+// word (8 elements as 4 x bf16x2) -> 32 bytes of fp32 (OUT 0), 16 bytes of bf16 (1) or of IEEE half (2) at dst
+template <int OUT>
 __device__ __forceinline__ void store_word(uint8_t* dst, const uint32_t* pr, bool wide) {
-  if (OUT_BF16) {
+  if (OUT == 1) {
     *reinterpret_cast<uint4*>(dst) = make_uint4(pr[0], pr[1], pr[2], pr[3]);
+  } else if (OUT == 2) {
+    uint32_t h[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      h[j] = f32x2_to_f16x2(__uint_as_float(pr[j] << 16), __uint_as_float(pr[j] & 0xffff0000u));
+    *reinterpret_cast<uint4*>(dst) = make_uint4(h[0], h[1], h[2], h[3]);
   } else {
     uint32_t v[8];
 #pragma unroll
@@ -228,12 +241,19 @@ fb4_dequantize_residual_rows_kernel(const uint32_t* __restrict__ codes, const ui
             __fadd_rn(__uint_as_float(pr[j] & 0xffff0000u), __uint_as_float(rr[j] & 0xffff0000u)));
       }
       uint8_t* dst = reinterpret_cast<uint8_t*>(out) + (b * WPB + k) * kWordBytes;
-      if (OUT_BF16) {
+      if (OUT_BF16 == 1) {
         uint4 o;
         o.x = f32_to_bf16_rne(__uint_as_float(v[0])) | (f32_to_bf16_rne(__uint_as_float(v[1])) << 16);
         o.y = f32_to_bf16_rne(__uint_as_float(v[2])) | (f32_to_bf16_rne(__uint_as_float(v[3])) << 16);
         o.z = f32_to_bf16_rne(__uint_as_float(v[4])) | (f32_to_bf16_rne(__uint_as_float(v[5])) << 16);
         o.w = f32_to_bf16_rne(__uint_as_float(v[6])) | (f32_to_bf16_rne(__uint_as_float(v[7])) << 16);
+        *reinterpret_cast<uint4*>(dst) = o;
+      } else if (OUT_BF16 == 2) {
+        uint4 o;
+        o.x = f32x2_to_f16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
+        o.y = f32x2_to_f16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
+        o.z = f32x2_to_f16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
+        o.w = f32x2_to_f16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
         *reinterpret_cast<uint4*>(dst) = o;
       } else {
         store_b32x8(dst, v, wide);
@@ -354,18 +374,27 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
   const uint32_t* rw = reinterpret_cast<const uint32_t*>(res_codes);
   const int a32 = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
   const Fb4DeviceTables* tb = ctx->d_tables;
+#define FB4_BY_DTYPE(CALL)          \
+  do {                              \
+    if (out_dtype == 1) { CALL(1); } \
+    else if (out_dtype == 2) { CALL(2); } \
+    else { CALL(0); }               \
+  } while (0)
   if (B == 32) {
-    if (out_dtype == 1) fb4_dequantize_b32_kernel<1, false><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
-    else fb4_dequantize_b32_kernel<0, false><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
+#define FB4_CALL(O) fb4_dequantize_b32_kernel<O, false><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32)
+    FB4_BY_DTYPE(FB4_CALL);
+#undef FB4_CALL
   } else if (C % 32 == 0) {   // block 16 in units of two blocks
     const int64_t units = total / 2;
     const int64_t uwant = (units + kStep - 1) / kStep;
     const unsigned ugrid = (unsigned)(uwant < cap ? uwant : cap);
-    if (out_dtype == 1) fb4_dequantize_b32_kernel<1, true><<<ugrid, kDecodeThreads, 0, stream>>>(cw, meta, units, tb, out, a32);
-    else fb4_dequantize_b32_kernel<0, true><<<ugrid, kDecodeThreads, 0, stream>>>(cw, meta, units, tb, out, a32);
+#define FB4_CALL(O) fb4_dequantize_b32_kernel<O, true><<<ugrid, kDecodeThreads, 0, stream>>>(cw, meta, units, tb, out, a32)
+    FB4_BY_DTYPE(FB4_CALL);
+#undef FB4_CALL
   } else {
-    if (out_dtype == 1) fb4_dequantize_kernel<1, 2><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
-    else fb4_dequantize_kernel<0, 2><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32);
+#define FB4_CALL(O) fb4_dequantize_kernel<O, 2><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32)
+    FB4_BY_DTYPE(FB4_CALL);
+#undef FB4_CALL
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -379,14 +408,19 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
   fb4_dequantize_residual_rows_kernel<BF, WPB><<<rgrid, kDecodeThreads, 0, stream>>>(      \
       cw, meta, bpr, tb, salient_idx, n_salient, rw, res_meta, out, a32)
     if (B == 32) {
-      if (out_dtype == 1) FB4_RESID(1, 4); else FB4_RESID(0, 4);
+#define FB4_CALL(O) FB4_RESID(O, 4)
+      FB4_BY_DTYPE(FB4_CALL);
+#undef FB4_CALL
     } else {
-      if (out_dtype == 1) FB4_RESID(1, 2); else FB4_RESID(0, 2);
+#define FB4_CALL(O) FB4_RESID(O, 2)
+      FB4_BY_DTYPE(FB4_CALL);
+#undef FB4_CALL
     }
 #undef FB4_RESID
     e = cudaGetLastError();
     if (e == cudaSuccess) *launches = 2;
   }
+#undef FB4_BY_DTYPE
   return e;
 }
 

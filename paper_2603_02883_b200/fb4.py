@@ -371,7 +371,7 @@ class Fb4:
         n = 0 if q.salient_idx is None else q.salient_idx.numel()
         fb4_dequantize(self.ctx, q.codes, q.meta, T, C, q.salient_idx if n else None, n,
                        q.res_codes if n else None, q.res_meta if n else None, out,
-                       0 if dtype == torch.float32 else 1)
+                       {torch.float32: 0, torch.bfloat16: 1, torch.float16: 2}[dtype])
         return out
 
     def quantize_weights(self, w) -> Quantized:

@@ -88,6 +88,9 @@ def test_edge_blocks_and_random_small(cfg):
         outb = q.dequantize(got, torch.bfloat16)
         refb = orc.dequantize(ref, FB, cfg["block_size"], out_dtype="bf16")
         assert np.array_equal(outb.view(torch.int16).cpu().numpy().view(np.uint16), refb)
+        outh = q.dequantize(got, torch.float16)                      # IEEE half: overflow to inf, gradual underflow
+        refh = orc.dequantize(ref, FB, cfg["block_size"], out_dtype="f16")
+        assert np.array_equal(outh.view(torch.int16).cpu().numpy().view(np.uint16), refh)
     q.close()
 
 
@@ -151,6 +154,9 @@ def test_decomposed_small(q32, T, tile):
     assert_same_quantized(got, ref, "decomposed")
     assert np.array_equal(q32.select_salient(torch.from_numpy(score).cuda(), tile).cpu().numpy(), sal)
     assert_same_bits_f32(q32.dequantize(got), orc.dequantize(ref, FB), "decomposed dequant")
+    for dt, name in ((torch.bfloat16, "bf16"), (torch.float16, "f16")):
+        o = q32.dequantize(got, dt)
+        assert np.array_equal(o.view(torch.int16).cpu().numpy().view(np.uint16), orc.dequantize(ref, FB, out_dtype=name))
     # caller-given salient set (reused from an earlier step): arbitrary ascending list
     mine = np.unique(np.random.default_rng(T).integers(0, T, size=max(1, T // 3))).astype(np.int32)
     ref2 = orc.quantize(bits, FB, salient_idx=mine)
