@@ -591,6 +591,31 @@ def pin_decomposition(seed=6, n=40):
                 assert rq == 0 or (rq > 0) == (dl > 0)
 
 
+def pin_residual_uses_the_seda_mask(seed=14):
+    """App. C: with SeDA and decomposition together, the residual is constrained to the cluster's
+    sub-formatbook like the original values; its block equals the block-wise definition under that mask."""
+    rng = np.random.default_rng(seed)
+    w = synth.Workload("t", T=6, C=128, seed=15, kind=1, n_outlier=1, outlier_gain=50.0, seda=True, n_clusters=2,
+                       cluster_seed=16)
+    bits = synth.activation(w)
+    cid, masks = synth.clusters(w)
+    masks = masks.copy()
+    masks[1] = 0x00F00F03                     # an arbitrary mask as well
+    sal = np.array([0, 2, 5], dtype=np.int32)
+    q = orc.quantize(bits, FB, cluster_id=cid, cluster_mask=masks, salient_idx=sal)
+    main = orc.dequantize(orc.Quantized(q.codes, q.meta), FB)
+    for s_, t in enumerate(sal):
+        allowed = int(masks[cid[t]])
+        for blk in range(4):
+            rdid = int(q.res_meta[s_, blk]) >> 8
+            assert (allowed >> rdid) & 1
+            sl = slice(blk * 32, blk * 32 + 32)
+            delta = np.array([float(bf16_value(int(b)) - f32_value(m)) for b, m in zip(bits[t, sl], main[t, sl])])
+            code, did, e, _ = orc.quantize_block_f64(delta, FB, allowed=allowed)
+            assert did == rdid and int(q.res_meta[s_, blk]) & 0xFF == e + 124
+            assert np.array_equal(unpack_codes(q.res_codes[s_, blk * 16:(blk + 1) * 16]), code)
+
+
 def pin_dequantize_formula(seed=7):
     rng = np.random.default_rng(seed)
     codes = rng.integers(0, 256, size=(3, 32), dtype=np.uint8)
@@ -638,7 +663,7 @@ def pin_mse():
 ALL_PINS = [
     pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
-    pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_salient_topk, pin_decomposition,
+    pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_salient_topk, pin_decomposition, pin_residual_uses_the_seda_mask,
     pin_dequantize_formula, pin_dequantize_f16, pin_mse, pin_f32_input, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
     pin_subformatbook_hand_counted,
     pin_subformatbook_one_dialect_per_bucket_and_closed_loop,

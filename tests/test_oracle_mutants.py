@@ -38,6 +38,8 @@ MUTANTS = {
     "topk_smallest": ("if (!taken[t] && (arg < 0 || score[t] > score[arg])) arg = t;",
                       "if (!taken[t] && (arg < 0 || score[t] < score[arg])) arg = t;"),
     "f16_through_bf16": ("_Float16 h = (_Float16)val;", "_Float16 h = (_Float16)bf16_to_double(f32_to_bf16_rne(val));"),
+    "residual_ignores_seda_mask": ("quantize_block(dv, dsg, cfg, F, stage1, allowed, dcode, &rdid, &re, NULL);",
+                                   "quantize_block(dv, dsg, cfg, F, stage1, 0xffffffffu, dcode, &rdid, &re, NULL);"),
     "clamp_min_ignored": ("if (e < cfg->exp_min) e = cfg->exp_min;", ";"),
     "zero_block_exponent": ("e = cfg->exp_min;\n  } else {", "e = 0;\n  } else {"),
     "stage1_bucket_shift": ("int bucket = k / 2 < 8 ? 8 : k / 2;", "int bucket = k / 2 < 9 ? 9 : k / 2;"),
