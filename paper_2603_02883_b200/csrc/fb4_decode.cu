@@ -14,7 +14,7 @@ __device__ __forceinline__ uint32_t f32_to_bf16_rne(float f) {
 }
 
 constexpr int kDecodeThreads = 256;
-constexpr int kDecodeUnroll = 2;          // blocks in flight per thread
+constexpr int kDecodeUnroll = 4;          // blocks in flight per thread
 
 // two fp32 -> two IEEE halves (round to nearest even, overflow to infinity), low half = a
 __device__ __forceinline__ uint32_t f32x2_to_f16x2(float a, float b) {
