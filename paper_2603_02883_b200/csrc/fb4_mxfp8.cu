@@ -14,7 +14,7 @@ namespace {
 using fb4dev::e4m3_of_small_int;
 
 constexpr int kThreads = 256;
-constexpr int kUnroll = 2;
+constexpr int kUnroll = 4;
 
 __global__ void __launch_bounds__(kThreads)
 fb4_to_mxfp8_kernel(const uint4* __restrict__ codes, const uint16_t* __restrict__ meta, int64_t T, int64_t n_col,
