@@ -105,3 +105,33 @@ def test_fused_quantize_to_mxfp8_rejects_other_configurations():
                                 None) == fb4.ERR_ALIGN
     assert L.fb4_quantize_mxfp8(q.ctx, p(x), 4, 64, 64, None, None, 0, p(out), p(out), 3, None) == fb4.ERR_INVALID_ARG
     q.close()
+
+
+@pytest.mark.parametrize("T,N,K", [(256, 256, 3072), (300, 144, 1088), (130, 16, 96)])
+def test_library_block_scaled_gemm_consumes_the_view(q32, T, N, K):
+    """External pin of the tiled scale layout (Sec. 4.1: FB4 mapped to MXFP8): the library's block-scaled
+    e4m3 GEMM, given FB4 activations and FB4 weights in the MXFP8 view, reproduces the product of the two
+    dequantized matrices to bf16 rounding; with the scales in the other (row-major) order it does not."""
+    if not hasattr(torch, "_scaled_mm") or not hasattr(torch, "float8_e8m0fnu"):
+        pytest.skip("this torch build has no block-scaled GEMM")
+    a_bits = synth.activation(synth.Workload("a", T=T, C=K, seed=T + K, kind=1, n_outlier=2, outlier_gain=50.0))
+    w_bits = synth.activation(synth.Workload("w", T=N, C=K, seed=N + K + 1, kind=1, n_outlier=0, outlier_gain=1.0))
+    qa = q32.quantize(to_dev_bf16(a_bits))
+    qw = q32.quantize_weights(to_dev_bf16(w_bits))
+    ea, sa = q32.to_mxfp8(qa, 1)
+    ew, sw = q32.to_mxfp8(qw, 1)
+    da, dw = q32.dequantize(qa).double(), q32.dequantize(qw).double()
+    want, bound = da @ dw.T, da.abs() @ dw.abs().T
+
+    def gemm(scale_a, scale_w):
+        return torch._scaled_mm(ea.view(torch.float8_e4m3fn), ew.view(torch.float8_e4m3fn).t(),
+                                scale_a=scale_a.view(torch.float8_e8m0fnu), scale_b=scale_w.view(torch.float8_e8m0fnu),
+                                out_dtype=torch.bfloat16).double()
+
+    tol = want.abs() * 2.0 ** -8 + bound * 1e-5      # one bf16 rounding + fp32 accumulation
+    assert bool(((gemm(sa, sw) - want).abs() <= tol).all())
+    # negative control: the same scale bytes, row-major, zero-padded to the tiled size
+    sa_rm = torch.zeros_like(sa)
+    sa_rm[: T * (K // 32)] = q32.to_mxfp8(qa, 0)[1]
+    if not torch.equal(sa_rm, sa):
+        assert not bool(((gemm(sa_rm, sw) - want).abs() <= tol).all())
