@@ -202,9 +202,42 @@ fb4_dequantize_kernel(const uint32_t* __restrict__ codes, const uint16_t* __rest
   }
 }
 
+// Sum of a decoded word and a decoded residual word (8 elements each as 4 x bf16x2), rounded once to
+// fp32, then stored as fp32 / bf16 / half at dst.
+template <int OUT_BF16>
+__device__ __forceinline__ void store_sum_word(uint8_t* dst, const uint32_t* pr, const uint32_t* rr, bool wide) {
+  uint32_t v[8];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    v[2 * j] = __float_as_uint(__fadd_rn(__uint_as_float(pr[j] << 16), __uint_as_float(rr[j] << 16)));
+    v[2 * j + 1] = __float_as_uint(
+        __fadd_rn(__uint_as_float(pr[j] & 0xffff0000u), __uint_as_float(rr[j] & 0xffff0000u)));
+  }
+  if (OUT_BF16 == 1) {
+    uint4 o;
+    o.x = f32_to_bf16_rne(__uint_as_float(v[0])) | (f32_to_bf16_rne(__uint_as_float(v[1])) << 16);
+    o.y = f32_to_bf16_rne(__uint_as_float(v[2])) | (f32_to_bf16_rne(__uint_as_float(v[3])) << 16);
+    o.z = f32_to_bf16_rne(__uint_as_float(v[4])) | (f32_to_bf16_rne(__uint_as_float(v[5])) << 16);
+    o.w = f32_to_bf16_rne(__uint_as_float(v[6])) | (f32_to_bf16_rne(__uint_as_float(v[7])) << 16);
+    *reinterpret_cast<uint4*>(dst) = o;
+  } else if (OUT_BF16 == 2) {
+    uint4 o;
+    o.x = f32x2_to_f16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
+    o.y = f32x2_to_f16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
+    o.z = f32x2_to_f16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
+    o.w = f32x2_to_f16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
+    *reinterpret_cast<uint4*>(dst) = o;
+  } else {
+    store_b32x8(dst, v, wide);
+  }
+}
+
 // Rows with a residual (Sec. 3.3: Q(Act) + Q(Delta), the sum rounded once to fp32): thread <-> one
 // block of one salient row; decodes the main and the residual codes and writes the row of `out`
-// again.  Runs after the flat decode on the same stream.
+// again.  Runs after the flat decode on the same stream.  With 32-element blocks (WPB 4) the code
+// words are transposed inside each quad of lanes, as in the flat kernel, so that a quad stores
+// whole lines; block index and metadata of the quad's other blocks come by shuffle (a quad may
+// straddle two salient rows, so each block keeps its own destination).
 template <int OUT_BF16, int WPB>
 __global__ void __launch_bounds__(kDecodeThreads)
 fb4_dequantize_residual_rows_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restrict__ meta,
@@ -218,45 +251,48 @@ fb4_dequantize_residual_rows_kernel(const uint32_t* __restrict__ codes, const ui
   const bool wide = out_aligned32 != 0;
   constexpr int kWordBytes = OUT_BF16 ? 16 : 32;
   const int64_t total = n_salient * blocks_per_row;
-  for (int64_t rb = (int64_t)blockIdx.x * kDecodeThreads + threadIdx.x; rb < total;
+  const int lane = threadIdx.x & 31, qp = lane & 3;
+  // the loop bound is warp-uniform (first lane's block), so that the shuffles below are convergent
+  for (int64_t rb = (int64_t)blockIdx.x * kDecodeThreads + threadIdx.x; rb - lane < total;
        rb += (int64_t)gridDim.x * kDecodeThreads) {
-    const int64_t srow = rb / blocks_per_row;
-    const int64_t b = (int64_t)__ldg(salient_idx + srow) * blocks_per_row + (rb - srow * blocks_per_row);
-    uint32_t cw[WPB], rcw[WPB];
-    load_block_codes<WPB>(codes + b * WPB, cw);
-    load_block_codes<WPB>(res_codes + rb * WPB, rcw);
-    const uint32_t m = (uint32_t)__ldg(meta + b), rm = (uint32_t)__ldg(res_meta + rb);
-    const uint4 dt = fb_bf16[(m >> 8) & 31u], rdt = fb_bf16[(rm >> 8) & 31u];
-    const uint32_t sc2 = scale_bf16x2(m), rsc2 = scale_bf16x2(rm);
+    uint32_t cw[WPB], rcw[WPB], m = 0u, rm = 0u;
 #pragma unroll
-    for (int k = 0; k < WPB; ++k) {
-      uint32_t pr[4], rr[4];
-      decode_word(cw[k], dt, sc2, pr);
-      decode_word(rcw[k], rdt, rsc2, rr);
-      uint32_t v[8];
+    for (int k = 0; k < WPB; ++k) cw[k] = rcw[k] = 0u;
+    int64_t b = -1;   // destination block; -1 = past the end
+    if (rb < total) {
+      const int64_t srow = rb / blocks_per_row;
+      b = (int64_t)__ldg(salient_idx + srow) * blocks_per_row + (rb - srow * blocks_per_row);
+      load_block_codes<WPB>(codes + b * WPB, cw);
+      load_block_codes<WPB>(res_codes + rb * WPB, rcw);
+      m = (uint32_t)__ldg(meta + b);
+      rm = (uint32_t)__ldg(res_meta + rb);
+    }
+    if (WPB == 4) {
+      uint32_t c4[4] = {cw[0], cw[1], cw[2 % WPB], cw[3 % WPB]};
+      uint32_t r4[4] = {rcw[0], rcw[1], rcw[2 % WPB], rcw[3 % WPB]};
+      quad_transpose(c4, lane);
+      quad_transpose(r4, lane);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        v[2 * j] = __float_as_uint(__fadd_rn(__uint_as_float(pr[j] << 16), __uint_as_float(rr[j] << 16)));
-        v[2 * j + 1] = __float_as_uint(
-            __fadd_rn(__uint_as_float(pr[j] & 0xffff0000u), __uint_as_float(rr[j] & 0xffff0000u)));
+      for (int i = 0; i < 4; ++i) {
+        const int src = (lane & ~3) + i;
+        const uint32_t mi = __shfl_sync(0xffffffffu, m, src), rmi = __shfl_sync(0xffffffffu, rm, src);
+        const int64_t bi = __shfl_sync(0xffffffffu, b, src);
+        if (bi < 0) continue;
+        uint32_t pr[4], rr[4];
+        decode_word(c4[i], fb_bf16[(mi >> 8) & 31u], scale_bf16x2(mi), pr);
+        decode_word(r4[i], fb_bf16[(rmi >> 8) & 31u], scale_bf16x2(rmi), rr);
+        store_sum_word<OUT_BF16>(reinterpret_cast<uint8_t*>(out) + (bi * 4 + qp) * kWordBytes, pr, rr, wide);
       }
-      uint8_t* dst = reinterpret_cast<uint8_t*>(out) + (b * WPB + k) * kWordBytes;
-      if (OUT_BF16 == 1) {
-        uint4 o;
-        o.x = f32_to_bf16_rne(__uint_as_float(v[0])) | (f32_to_bf16_rne(__uint_as_float(v[1])) << 16);
-        o.y = f32_to_bf16_rne(__uint_as_float(v[2])) | (f32_to_bf16_rne(__uint_as_float(v[3])) << 16);
-        o.z = f32_to_bf16_rne(__uint_as_float(v[4])) | (f32_to_bf16_rne(__uint_as_float(v[5])) << 16);
-        o.w = f32_to_bf16_rne(__uint_as_float(v[6])) | (f32_to_bf16_rne(__uint_as_float(v[7])) << 16);
-        *reinterpret_cast<uint4*>(dst) = o;
-      } else if (OUT_BF16 == 2) {
-        uint4 o;
-        o.x = f32x2_to_f16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
-        o.y = f32x2_to_f16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
-        o.z = f32x2_to_f16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
-        o.w = f32x2_to_f16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
-        *reinterpret_cast<uint4*>(dst) = o;
-      } else {
-        store_b32x8(dst, v, wide);
+    } else {
+      if (b < 0) continue;
+      const uint4 dt = fb_bf16[(m >> 8) & 31u], rdt = fb_bf16[(rm >> 8) & 31u];
+      const uint32_t sc2 = scale_bf16x2(m), rsc2 = scale_bf16x2(rm);
+#pragma unroll
+      for (int k = 0; k < WPB; ++k) {
+        uint32_t pr[4], rr[4];
+        decode_word(cw[k], dt, sc2, pr);
+        decode_word(rcw[k], rdt, rsc2, rr);
+        store_sum_word<OUT_BF16>(reinterpret_cast<uint8_t*>(out) + (b * WPB + k) * kWordBytes, pr, rr, wide);
       }
     }
   }
