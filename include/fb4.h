@@ -119,7 +119,9 @@ int fb4_quantize_f32(fb4_ctx* ctx, const float* x, int64_t T, int64_t C, int64_t
  * cluster_mask[cluster_id[t]] (its cluster's sub-formatbook); cluster_id[t] == -1
  * means unconstrained.  Stage 1 is intersected with the mask; if the intersection
  * is empty the whole mask is scored.
- *   cluster_id   : device int32 [T], values in [-1, n_clusters)
+ *   cluster_id   : device int32 [T], values in [-1, n_clusters).  The kernels check the range: any
+ *                  other value is treated as -1 and raises bit 1 of the status word
+ *                  (fb4_device_status); the mask table is never read out of bounds
  *   cluster_mask : device uint32 [n_clusters], every entry non-zero (precondition;
  *                  a zero mask yields dialect 0 for the affected tokens)
  */
@@ -229,7 +231,8 @@ int fb4_quantize_decomposed_idx(fb4_ctx* ctx, const void* x_bf16, int64_t T, int
  * out[t][c] = value(codes, meta); for tokens listed in salient_idx the decoded
  * residual is added, the sum rounded once to fp32 (Sec. 3.3: Q(Act)+Q(Delta)).
  *   salient_idx : NULL / n_salient = 0 for plain tensors; else device int32
- *                 [n_salient], strictly ascending
+ *                 [n_salient], strictly ascending.  An entry outside [0, T) is skipped (its
+ *                 residual row is not added anywhere) and raises bit 1 of the status word
  *   out         : device, [T][C] contiguous; out_dtype 0 = float32, 1 = bfloat16, 2 = IEEE half
  *                 (the type App. D.2 decodes to); 1 and 2 are the round-to-nearest-even of the
  *                 fp32 result (half: overflow to infinity, gradual underflow)
@@ -310,7 +313,9 @@ int fb4_set_kernel_variant(fb4_ctx* ctx, int variant);
 
 /* Device-side status word of the context, read back with a blocking copy: 0 = fine; bit 0 =
  * a bounded wait on an asynchronous (TMA) load inside a kernel ran out of tries, in which case
- * the affected warp stopped early and the outputs of that call are incomplete. */
+ * the affected warp stopped early and the outputs of that call are incomplete; bit 1 = an index
+ * argument on the device (a cluster id, a salient token index on decode) was outside its table
+ * and was handled as documented at the call.  Bits stay set for the life of the context. */
 int fb4_device_status(fb4_ctx* ctx, uint32_t* status);
 
 /* Number of kernel launches this context has enqueued so far (diagnostic counter). */

@@ -247,6 +247,7 @@ int fb4_quantize_seda(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t
   Fb4RowExtras ex{};
   ex.cluster_id = cluster_id;
   ex.cluster_mask = cluster_mask;
+  ex.n_clusters = n_clusters;
   return run_quantize(ctx, x, T, C, ld, ex, codes, meta, static_cast<cudaStream_t>(stream));
 }
 
@@ -291,6 +292,7 @@ int fb4_quantize_decomposed(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, i
   Fb4RowExtras ex{};
   ex.cluster_id = cluster_id;
   ex.cluster_mask = cluster_id ? cluster_mask : nullptr;
+  ex.n_clusters = cluster_id ? n_clusters : 0;
   ex.salient_idx = salient_idx;
   ex.n_salient = (T + tile - 1) / tile;
   ex.tile = tile;
@@ -313,6 +315,7 @@ int fb4_quantize_decomposed_idx(fb4_ctx* ctx, const void* x, int64_t T, int64_t 
   Fb4RowExtras ex{};
   ex.cluster_id = cluster_id;
   ex.cluster_mask = cluster_id ? cluster_mask : nullptr;
+  ex.n_clusters = cluster_id ? n_clusters : 0;
   ex.salient_idx = salient_idx;
   ex.n_salient = n_salient;
   ex.tile = 0;
@@ -388,6 +391,7 @@ int fb4_quantize_mxfp8(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_
   Fb4RowExtras ex{};
   ex.cluster_id = cluster_id;
   ex.cluster_mask = cluster_id ? cluster_mask : nullptr;
+  ex.n_clusters = cluster_id ? n_clusters : 0;
   cudaError_t e = fb4_launch_quantize_fast_mx(ctx, x, T, C, ld, ex, e4m3, scales, scale_layout,
                                               static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return fb4_set_cuda_error(e);

@@ -234,7 +234,8 @@ __device__ __forceinline__ void store_sum_word(uint8_t* dst, const uint32_t* pr,
 
 // Rows with a residual (Sec. 3.3: Q(Act) + Q(Delta), the sum rounded once to fp32): thread <-> one
 // block of one salient row; decodes the main and the residual codes and writes the row of `out`
-// again.  Runs after the flat decode on the same stream.  With 32-element blocks (WPB 4) the code
+// again.  Runs after the flat decode on the same stream.  An entry of salient_idx outside [0, T) is
+// skipped and raises bit 1 of the status word.  With 32-element blocks (WPB 4) the code
 // words are transposed inside each quad of lanes, as in the flat kernel, so that a quad stores
 // whole lines; block index and metadata of the quad's other blocks come by shuffle (a quad may
 // straddle two salient rows, so each block keeps its own destination).
@@ -244,7 +245,8 @@ fb4_dequantize_residual_rows_kernel(const uint32_t* __restrict__ codes, const ui
                                     uint32_t blocks_per_row, const Fb4DeviceTables* __restrict__ tables,
                                     const int32_t* __restrict__ salient_idx, int64_t n_salient,
                                     const uint32_t* __restrict__ res_codes, const uint16_t* __restrict__ res_meta,
-                                    void* __restrict__ out, int out_aligned32) {
+                                    void* __restrict__ out, int out_aligned32, int64_t T,
+                                    uint32_t* __restrict__ status) {
   __shared__ uint4 fb_bf16[32];
   fb4dev::fill_fb_bf16(fb_bf16, &tables->formatbook[0][0], threadIdx.x);
   __syncthreads();
@@ -261,11 +263,16 @@ fb4_dequantize_residual_rows_kernel(const uint32_t* __restrict__ codes, const ui
     int64_t b = -1;   // destination block; -1 = past the end
     if (rb < total) {
       const int64_t srow = rb / blocks_per_row;
-      b = (int64_t)__ldg(salient_idx + srow) * blocks_per_row + (rb - srow * blocks_per_row);
-      load_block_codes<WPB>(codes + b * WPB, cw);
-      load_block_codes<WPB>(res_codes + rb * WPB, rcw);
-      m = (uint32_t)__ldg(meta + b);
-      rm = (uint32_t)__ldg(res_meta + rb);
+      const int64_t row = (int64_t)__ldg(salient_idx + srow);
+      if (row >= 0 && row < T) {
+        b = row * blocks_per_row + (rb - srow * blocks_per_row);
+        load_block_codes<WPB>(codes + b * WPB, cw);
+        load_block_codes<WPB>(res_codes + rb * WPB, rcw);
+        m = (uint32_t)__ldg(meta + b);
+        rm = (uint32_t)__ldg(res_meta + rb);
+      } else {
+        atomicOr(status, 2u);   // a token index outside the tensor: the entry is skipped and reported
+      }
     }
     if (WPB == 4) {
       uint32_t c4[4] = {cw[0], cw[1], cw[2 % WPB], cw[3 % WPB]};
@@ -442,7 +449,7 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
     const uint32_t bpr = (uint32_t)blocks_per_row;
 #define FB4_RESID(BF, WPB)                                                                 \
   fb4_dequantize_residual_rows_kernel<BF, WPB><<<rgrid, kDecodeThreads, 0, stream>>>(      \
-      cw, meta, bpr, tb, salient_idx, n_salient, rw, res_meta, out, a32)
+      cw, meta, bpr, tb, salient_idx, n_salient, rw, res_meta, out, a32, T, ctx->d_status)
     if (B == 32) {
 #define FB4_CALL(O) FB4_RESID(O, 4)
       FB4_BY_DTYPE(FB4_CALL);

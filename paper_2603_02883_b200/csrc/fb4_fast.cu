@@ -370,10 +370,17 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
     list_pos = lo;
     if (lo < ex.n_salient) list_next = ex.salient_idx[lo];
   }
+  // a cluster id outside [-1, n_clusters) is treated as -1 (unconstrained) and reported in bit 1 of
+  // the status word when the warp is done: the mask table is never read out of bounds
+  const uint32_t n_cl = (uint32_t)ex.n_clusters;
+  bool bad_cid = false;
   uint32_t maskq[2] = {0xffffffffu, 0xffffffffu};
   if (use_seda) {
-    if (cidq[0] >= 0) maskq[0] = ex.cluster_mask[cidq[0]];
-    if (cidq[1] >= 0) maskq[1] = ex.cluster_mask[cidq[1]];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      if ((uint32_t)cidq[k] < n_cl) maskq[k] = ex.cluster_mask[cidq[k]];
+      else if (cidq[k] != -1) bad_cid = true;
+    }
   }
   // ---- the tables arrive behind the first tile loads; bounded wait like every other wait here
   {
@@ -411,7 +418,8 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
     if (SEDA) {
       if (use_seda) {
         if (it_pre < n_mine) cid_new = ex.cluster_id[pre.row];
-        if (cidq[2] >= 0) mask_new = ex.cluster_mask[cidq[2]];
+        if ((uint32_t)cidq[2] < n_cl) mask_new = ex.cluster_mask[cidq[2]];
+        else if (cidq[2] != -1) bad_cid = true;
       }
     }
 
@@ -611,6 +619,7 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
     maskq[1] = mask_new;
     if (++s == kStages) { s = 0; parity ^= 1u; }
   }
+  if (SEDA && bad_cid && lane == 0) atomicOr(p.status, 2u);
 }
 
 // ---------------------------------------------------------------------------------------------

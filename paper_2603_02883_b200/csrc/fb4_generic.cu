@@ -120,7 +120,7 @@ template <int B, int GS, bool F32, bool RESID>
 __global__ void __launch_bounds__(128)
 fb4_quantize_generic_kernel(const void* __restrict__ xin, int64_t T, int64_t C, int64_t ld,
                             const Fb4DeviceTables* __restrict__ tables, GenericParams p, Fb4RowExtras ex,
-                            uint8_t* __restrict__ codes, uint16_t* __restrict__ meta) {
+                            uint8_t* __restrict__ codes, uint16_t* __restrict__ meta, uint32_t* __restrict__ status) {
   __shared__ SmemTables tb;
   {
     const uint32_t* src = reinterpret_cast<const uint32_t*>(tables);
@@ -168,7 +168,8 @@ fb4_quantize_generic_kernel(const void* __restrict__ xin, int64_t T, int64_t C, 
     uint32_t allowed = 0xffffffffu;
     if (ex.cluster_id) {
       const int32_t cid = ex.cluster_id[t];
-      if (cid >= 0) allowed = ex.cluster_mask[cid];
+      if ((uint32_t)cid < (uint32_t)ex.n_clusters) allowed = ex.cluster_mask[cid];
+      else if (cid != -1) atomicOr(status, 2u);   // out of range: unconstrained, reported in the status word
       if (allowed == 0) allowed = 1u;   // precondition violated: stay in bounds
     }
     uint32_t packed[B / 8];
@@ -212,7 +213,8 @@ cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x
   const int grid = (int)(want < cap ? want : cap);
   const bool resid = ex.n_salient > 0;
 #define FB4_LAUNCH_K(BB, GSZ, F, R) \
-  fb4_quantize_generic_kernel<BB, GSZ, F, R><<<grid, threads, 0, stream>>>(x, T, C, ld, ctx->d_tables, p, ex, codes, meta)
+  fb4_quantize_generic_kernel<BB, GSZ, F, R><<<grid, threads, 0, stream>>>(x, T, C, ld, ctx->d_tables, p, ex, codes, meta, \
+                                                                           ctx->d_status)
 #define FB4_LAUNCH(BB, GSZ)                                  \
   do {                                                       \
     if (x_is_f32) FB4_LAUNCH_K(BB, GSZ, true, false);        \

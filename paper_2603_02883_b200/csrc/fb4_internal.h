@@ -24,6 +24,7 @@ struct Fb4Stage1 {
 struct Fb4RowExtras {
   const int32_t* cluster_id;    // SeDA: token -> cluster, -1 = unconstrained
   const uint32_t* cluster_mask; // SeDA: cluster -> allowed dialect mask
+  int32_t n_clusters;           // entries of cluster_mask; ids outside [-1, n_clusters) count as -1 and raise status bit 1
   const int32_t* salient_idx;   // ascending token ids whose residual is quantized too
   int64_t n_salient;
   int32_t tile;                 // > 0: salient_idx[t / tile] is the only possible match for token t
@@ -40,7 +41,7 @@ struct fb4_ctx {
   int force_generic;             // fb4_set_kernel_variant(ctx, 1): always take the generic kernel
   int fast_ok;                   // formatbook/stage-1 table fit the fast kernel's packed layout
   int sm_count;
-  uint32_t* d_status;            // device status word (bit 0: a TMA wait ran out of tries)
+  uint32_t* d_status;            // device status word (bit 0: a TMA wait ran out of tries; bit 1: an index argument out of range)
   int64_t launches;
   const char* last_variant;
   cudaStream_t pipe_stream[3];   // fb4_quantize_host pipeline
