@@ -135,3 +135,23 @@ def test_library_block_scaled_gemm_consumes_the_view(q32, T, N, K):
     sa_rm[: T * (K // 32)] = q32.to_mxfp8(qa, 0)[1]
     if not torch.equal(sa_rm, sa):
         assert not bool(((gemm(sa_rm, sw) - want).abs() <= tol).all())
+
+
+@pytest.mark.parametrize("T,C", [(130, 96), (300, 320), (257, 1024 + 64), (129, 32 * 33)])
+def test_tiled_scales_at_an_odd_address(q32, T, C):
+    """The tiled scale order goes through a CTA-staged kernel when the scale buffer is 16-byte aligned and
+    through the byte-store kernel otherwise: both give the oracle's bytes."""
+    rng = np.random.default_rng(T * C)
+    codes = rng.integers(0, 256, size=(T, C // 2), dtype=np.uint8)
+    meta = (rng.integers(0, 252, size=(T, C // 32)) | (rng.integers(0, 32, size=(T, C // 32)) << 8)).astype(np.uint16)
+    e_ref, s_ref = orc.to_mxfp8(orc.Quantized(codes, meta), FB, 1)
+    d_codes, d_meta = torch.from_numpy(codes).cuda(), torch.from_numpy(meta.view(np.int16)).cuda()
+    n = fb4.fb4_mxfp8_scale_bytes(T, C, 1)
+    for shift in (0, 1, 8):
+        e4m3 = torch.zeros((T, C), dtype=torch.uint8, device="cuda")
+        buf = torch.full((n + 64,), 0xEE, dtype=torch.uint8, device="cuda")
+        fb4.fb4_to_mxfp8(q32.ctx, d_codes, d_meta, T, C, e4m3, buf[shift:], 1)
+        assert np.array_equal(e4m3.cpu().numpy(), e_ref), f"e4m3 bytes, shift {shift}"
+        got = buf.cpu().numpy()
+        assert np.array_equal(got[shift:shift + n], s_ref), f"scale bytes, shift {shift}"
+        assert (got[:shift] == 0xEE).all() and (got[shift + n:] == 0xEE).all(), "bytes outside the scale array"
