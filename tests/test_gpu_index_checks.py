@@ -69,9 +69,9 @@ def test_decode_skips_salient_rows_outside_the_tensor(block_size, C):
     try:
         got = q.quantize_decomposed(to_dev_bf16(bits), salient_idx=torch.from_numpy(keep).cuda())
         assert_same_quantized(got, ref, "given set")
-        # the same residual rows, with entries that point outside [0, T) put in between
-        idx = np.array([3, -1, 50, T, 51, np.iinfo(np.int32).max, 199, np.iinfo(np.int32).min], dtype=np.int32)
-        pos = [0, 2, 4, 6]
+        # the same residual rows in a list (still ascending) that also has entries outside [0, T)
+        idx = np.array([np.iinfo(np.int32).min, -1, 3, 50, 51, 199, T, np.iinfo(np.int32).max], dtype=np.int32)
+        pos = [2, 3, 4, 5]
         nblk = C // block_size
         rc = torch.zeros((len(idx), C // 2), dtype=torch.uint8, device="cuda")
         rm = torch.zeros((len(idx), nblk), dtype=torch.int16, device="cuda")
