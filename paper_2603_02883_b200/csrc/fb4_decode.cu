@@ -84,15 +84,63 @@ __device__ __forceinline__ void store_word(uint8_t* dst, const uint32_t* pr, boo
   }
 }
 
+// Sum of a decoded word and a decoded residual word (8 elements each as 4 x bf16x2), rounded once to
+// fp32, then stored as fp32 / bf16 / half at dst.
+template <int OUT_BF16>
+__device__ __forceinline__ void store_sum_word(uint8_t* dst, const uint32_t* pr, const uint32_t* rr, bool wide) {
+  uint32_t v[8];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    v[2 * j] = __float_as_uint(__fadd_rn(__uint_as_float(pr[j] << 16), __uint_as_float(rr[j] << 16)));
+    v[2 * j + 1] = __float_as_uint(
+        __fadd_rn(__uint_as_float(pr[j] & 0xffff0000u), __uint_as_float(rr[j] & 0xffff0000u)));
+  }
+  if (OUT_BF16 == 1) {
+    uint4 o;
+    o.x = f32_to_bf16_rne(__uint_as_float(v[0])) | (f32_to_bf16_rne(__uint_as_float(v[1])) << 16);
+    o.y = f32_to_bf16_rne(__uint_as_float(v[2])) | (f32_to_bf16_rne(__uint_as_float(v[3])) << 16);
+    o.z = f32_to_bf16_rne(__uint_as_float(v[4])) | (f32_to_bf16_rne(__uint_as_float(v[5])) << 16);
+    o.w = f32_to_bf16_rne(__uint_as_float(v[6])) | (f32_to_bf16_rne(__uint_as_float(v[7])) << 16);
+    *reinterpret_cast<uint4*>(dst) = o;
+  } else if (OUT_BF16 == 2) {
+    uint4 o;
+    o.x = f32x2_to_f16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
+    o.y = f32x2_to_f16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
+    o.z = f32x2_to_f16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
+    o.w = f32x2_to_f16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
+    *reinterpret_cast<uint4*>(dst) = o;
+  } else {
+    store_b32x8(dst, v, wide);
+  }
+}
+
+// The residual tensor of salient rows, for the flat decode that adds it in the same pass
+struct ResidualRows {
+  const int32_t* salient_idx;   // ascending token ids
+  int64_t n_salient;
+  const uint32_t* res_codes;    // [n_salient][units_per_row * 4 words]
+  const uint16_t* res_meta;     // [n_salient][units_per_row]
+  uint32_t units_per_row;
+  float guess_scale;            // n_salient / T: list position of a row, to first order
+  int64_t T;
+  uint32_t* status;
+};
+
 // Flat decode without residuals, in units of 32 elements (one block of 32, or two blocks of 16).
 // A lane loads the 16 code bytes of one unit (one 128-bit load) and the metadata records of its
 // whole quad (one 64- or 128-bit load); the quad transposes the code words so that lane p decodes
 // word p of the quad's four units and the quad stores contiguous lines.  kDecodeUnroll units per
 // thread are in flight; the loads of the next step are issued before the current step is decoded.
-template <int OUT_BF16, bool B16>
-__global__ void __launch_bounds__(kDecodeThreads)
+// RESID (block size 32, fewer than 2^32 units): rows listed in rr.salient_idx also get their decoded
+// residual added (Sec. 3.3: Q(Act) + Q(Delta), rounded once to fp32) in the same pass.  Per step the
+// CTA finds the first list entry at or after the step's first row; a step whose rows hold no
+// salient token (most of them) runs the plain code, the others look up each unit's row, load the
+// residual codes of salient rows and add.
+template <int OUT_BF16, bool B16, bool RESID>
+__global__ void __launch_bounds__(kDecodeThreads, 3)
 fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restrict__ meta, int64_t total_units,
-                          const Fb4DeviceTables* __restrict__ tables, void* __restrict__ out, int out_aligned32) {
+                          const Fb4DeviceTables* __restrict__ tables, void* __restrict__ out, int out_aligned32,
+                          ResidualRows rr) {
   __shared__ uint4 fb_bf16[32];   // per dialect: high bytes (8) then low bytes (8) of its magnitudes as bf16
   fb4dev::fill_fb_bf16(fb_bf16, &tables->formatbook[0][0], threadIdx.x);
   __syncthreads();
@@ -102,7 +150,16 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
   constexpr int RPU = B16 ? 2 : 1;   // metadata records per unit
   constexpr int kWordBytes = OUT_BF16 ? 16 : 32;
   constexpr int64_t kStep = (int64_t)kDecodeThreads * kDecodeUnroll;
-  const int64_t stride = (int64_t)gridDim.x * kStep;
+  int64_t base = (int64_t)blockIdx.x * kStep, end = total_units, stride = (int64_t)gridDim.x * kStep;
+  int64_t pos = 0;   // RESID: first list entry at or after the current step's first row
+  if (RESID && blockIdx.x == 0) {   // entries outside the tensor match no row; they are reported
+    bool bad = false;
+    for (int64_t i = threadIdx.x; i < rr.n_salient; i += kDecodeThreads) {
+      const int32_t r = __ldg(rr.salient_idx + i);
+      bad |= r < 0 || r >= rr.T;
+    }
+    if (bad) atomicOr(rr.status, 2u);
+  }
 
   // m = the metadata records of the lane's whole quad (4 units): after the transpose a lane decodes
   // one word of each of the quad's units and needs the record that covers it
@@ -132,9 +189,8 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
       }
     }
   };
-  int64_t base = (int64_t)blockIdx.x * kStep;
-  if (base < total_units) load(base);
-  for (; base < total_units; base += stride) {
+  if (base < end) load(base);
+  for (; base < end; base += stride) {
     uint32_t c[kDecodeUnroll][4], mm[kDecodeUnroll][2 * RPU];
 #pragma unroll
     for (int u = 0; u < kDecodeUnroll; ++u) {
@@ -143,7 +199,100 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
 #pragma unroll
       for (int k = 0; k < 4; ++k) c[u][k] = cw[u][k];
     }
-    if (base + stride < total_units) load(base + stride);
+    if (base + stride < end) load(base + stride);
+    if (RESID) {
+      // rows of this step: [row_first, row_last]; uniform over the CTA
+      const uint32_t last_unit = (uint32_t)(base + kStep < total_units ? base + kStep : total_units) - 1u;
+      const int64_t row_first = (uint32_t)base / rr.units_per_row, row_last = last_unit / rr.units_per_row;
+      {
+        // lower bound of row_first in the ascending list.  Salient tokens are spread over the sequence
+        // (one per tile of tokens), so the entry sits next to the proportional guess: a few probes
+        // around it, else a binary search.
+        int64_t g = (int64_t)((float)row_first * rr.guess_scale);
+        g = g < 0 ? 0 : (g > rr.n_salient ? rr.n_salient : g);
+        int tries = 0;
+        while (g > 0 && (int64_t)__ldg(rr.salient_idx + g - 1) >= row_first && tries < 8) { --g; ++tries; }
+        while (g < rr.n_salient && (int64_t)__ldg(rr.salient_idx + g) < row_first && tries < 8) { ++g; ++tries; }
+        if (tries == 8) {
+          int64_t lo = 0, hi = rr.n_salient;
+          while (lo < hi) {
+            const int64_t mid = (lo + hi) >> 1;
+            if ((int64_t)__ldg(rr.salient_idx + mid) < row_first) lo = mid + 1; else hi = mid;
+          }
+          g = lo;
+        }
+        pos = g;
+      }
+      const int64_t r0 = pos < rr.n_salient ? (int64_t)__ldg(rr.salient_idx + pos) : row_last + 1;
+      if (r0 <= row_last) {
+        // a salient row in this step.  Per warp and unit slot: the lanes look up their unit's row; if
+        // none of the 32 units lies in a salient row the plain code runs, else the lanes of salient
+        // rows load their residual codes and the quad adds the decoded residual.
+        const bool more = pos + 1 < rr.n_salient && (int64_t)__ldg(rr.salient_idx + pos + 1) <= row_last;
+#pragma unroll
+        for (int u = 0; u < kDecodeUnroll; ++u) {
+          const int64_t b = base + u * kDecodeThreads + threadIdx.x;
+          int64_t s = -1;              // residual row of this lane's unit
+          uint32_t col = 0;
+          if (b < total_units) {
+            const uint32_t row = (uint32_t)b / rr.units_per_row;
+            col = (uint32_t)b - row * rr.units_per_row;
+            if ((int64_t)row == r0) {
+              s = pos;
+            } else if (more && (int64_t)row > r0) {
+              for (int64_t k = pos + 1; k < rr.n_salient; ++k) {
+                const int64_t r = (int64_t)__ldg(rr.salient_idx + k);
+                if (r >= (int64_t)row) {
+                  if (r == (int64_t)row) s = k;
+                  break;
+                }
+              }
+            }
+          }
+          const bool any_res = __any_sync(0xffffffffu, s >= 0);
+          quad_transpose(c[u], lane);
+          const int64_t qb = base + u * kDecodeThreads + (threadIdx.x & ~3);
+          if (!any_res) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t mi = (mm[u][i >> 1] >> (16 * (i & 1))) & 0xffffu;
+              if (qb + i < total_units) {
+                uint32_t pr[4];
+                decode_word(c[u][i], fb_bf16[(mi >> 8) & 31u], scale_bf16x2(mi), pr);
+                store_word<OUT_BF16>(reinterpret_cast<uint8_t*>(out) + ((qb + i) * 4 + qp) * kWordBytes, pr, wide);
+              }
+            }
+            continue;
+          }
+          uint32_t rcw[4] = {0u, 0u, 0u, 0u}, rm = 0u;
+          if (s >= 0) {
+            load_block_codes<4>(rr.res_codes + (s * rr.units_per_row + col) * 4, rcw);
+            rm = (uint32_t)__ldg(rr.res_meta + s * rr.units_per_row + col);
+          }
+          quad_transpose(rcw, lane);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int src = (lane & ~3) + i;
+            const uint32_t mi = (mm[u][i >> 1] >> (16 * (i & 1))) & 0xffffu;
+            const uint32_t rmi = __shfl_sync(0xffffffffu, rm, src);
+            const bool has_res = __shfl_sync(0xffffffffu, (int)(s >= 0), src) != 0;
+            if (qb + i < total_units) {
+              uint32_t pr[4];
+              decode_word(c[u][i], fb_bf16[(mi >> 8) & 31u], scale_bf16x2(mi), pr);
+              uint8_t* dst = reinterpret_cast<uint8_t*>(out) + ((qb + i) * 4 + qp) * kWordBytes;
+              if (has_res) {
+                uint32_t rd[4];
+                decode_word(rcw[i], fb_bf16[(rmi >> 8) & 31u], scale_bf16x2(rmi), rd);
+                store_sum_word<OUT_BF16>(dst, pr, rd, wide);
+              } else {
+                store_word<OUT_BF16>(dst, pr, wide);
+              }
+            }
+          }
+        }
+        continue;
+      }
+    }
 #pragma unroll
     for (int u = 0; u < kDecodeUnroll; ++u) {
       quad_transpose(c[u], lane);
@@ -199,36 +348,6 @@ fb4_dequantize_kernel(const uint32_t* __restrict__ codes, const uint16_t* __rest
         store_word<OUT_BF16>(reinterpret_cast<uint8_t*>(out) + (b * WPB + k) * kWordBytes, pr, wide);
       }
     }
-  }
-}
-
-// Sum of a decoded word and a decoded residual word (8 elements each as 4 x bf16x2), rounded once to
-// fp32, then stored as fp32 / bf16 / half at dst.
-template <int OUT_BF16>
-__device__ __forceinline__ void store_sum_word(uint8_t* dst, const uint32_t* pr, const uint32_t* rr, bool wide) {
-  uint32_t v[8];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    v[2 * j] = __float_as_uint(__fadd_rn(__uint_as_float(pr[j] << 16), __uint_as_float(rr[j] << 16)));
-    v[2 * j + 1] = __float_as_uint(
-        __fadd_rn(__uint_as_float(pr[j] & 0xffff0000u), __uint_as_float(rr[j] & 0xffff0000u)));
-  }
-  if (OUT_BF16 == 1) {
-    uint4 o;
-    o.x = f32_to_bf16_rne(__uint_as_float(v[0])) | (f32_to_bf16_rne(__uint_as_float(v[1])) << 16);
-    o.y = f32_to_bf16_rne(__uint_as_float(v[2])) | (f32_to_bf16_rne(__uint_as_float(v[3])) << 16);
-    o.z = f32_to_bf16_rne(__uint_as_float(v[4])) | (f32_to_bf16_rne(__uint_as_float(v[5])) << 16);
-    o.w = f32_to_bf16_rne(__uint_as_float(v[6])) | (f32_to_bf16_rne(__uint_as_float(v[7])) << 16);
-    *reinterpret_cast<uint4*>(dst) = o;
-  } else if (OUT_BF16 == 2) {
-    uint4 o;
-    o.x = f32x2_to_f16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
-    o.y = f32x2_to_f16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
-    o.z = f32x2_to_f16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
-    o.w = f32x2_to_f16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
-    *reinterpret_cast<uint4*>(dst) = o;
-  } else {
-    store_b32x8(dst, v, wide);
   }
 }
 
@@ -423,15 +542,30 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
     else if (out_dtype == 2) { CALL(2); } \
     else { CALL(0); }               \
   } while (0)
+  ResidualRows none{};
+  if (B == 32 && n_salient > 0 && blocks_per_row >= 32 && total < 0xffffffffLL) {
+    // residual rows added in the same pass: every row is written once
+    const ResidualRows rr{salient_idx, n_salient, rw, res_meta, (uint32_t)blocks_per_row,
+                          (float)((double)n_salient / (double)T), T, ctx->d_status};
+#define FB4_CALL(O) \
+  fb4_dequantize_b32_kernel<O, false, true><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32, rr)
+    FB4_BY_DTYPE(FB4_CALL);
+#undef FB4_CALL
+    const cudaError_t fe = cudaGetLastError();
+    if (fe == cudaSuccess) *launches = 1;
+    return fe;
+  }
   if (B == 32) {
-#define FB4_CALL(O) fb4_dequantize_b32_kernel<O, false><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32)
+#define FB4_CALL(O) \
+  fb4_dequantize_b32_kernel<O, false, false><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32, none)
     FB4_BY_DTYPE(FB4_CALL);
 #undef FB4_CALL
   } else if (C % 32 == 0) {   // block 16 in units of two blocks
     const int64_t units = total / 2;
     const int64_t uwant = (units + kStep - 1) / kStep;
     const unsigned ugrid = (unsigned)(uwant < cap ? uwant : cap);
-#define FB4_CALL(O) fb4_dequantize_b32_kernel<O, true><<<ugrid, kDecodeThreads, 0, stream>>>(cw, meta, units, tb, out, a32)
+#define FB4_CALL(O) \
+  fb4_dequantize_b32_kernel<O, true, false><<<ugrid, kDecodeThreads, 0, stream>>>(cw, meta, units, tb, out, a32, none)
     FB4_BY_DTYPE(FB4_CALL);
 #undef FB4_CALL
   } else {

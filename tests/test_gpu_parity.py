@@ -165,6 +165,31 @@ def test_decomposed_small(q32, T, tile):
     assert_same_bits_f32(q32.dequantize(got2), orc.dequantize(ref2, FB), "decomposed idx dequant")
 
 
+@pytest.mark.parametrize("T,C,tile", [(300, 1024, 1), (257, 2112, 3), (1000, 1024, 20), (130, 4096 + 32, 2)])
+def test_decode_adds_residual_rows_in_the_same_pass(q32, T, C, tile):
+    """At 32 or more blocks per row the decode adds the residual of salient rows inside its one kernel
+    (steps with several salient rows, runs of consecutive salient rows, ragged last step); every output
+    type against the oracle, and one launch per call."""
+    bits = heavy(T, C, T + C)
+    w = synth.Workload("t", T=T, C=C, seed=1, kind=1, n_outlier=0, outlier_gain=1.0, score_seed=T + tile)
+    score = synth.scores(w)
+    lists = [orc.select_salient(score, tile),
+             np.array(sorted(set(range(5, 12)) | {0, T // 2, T - 2, T - 1}), dtype=np.int32),
+             np.array([T - 1], dtype=np.int32)]
+    x = to_dev_bf16(bits)
+    for sal in lists:
+        ref = orc.quantize(bits, FB, salient_idx=sal)
+        got = q32.quantize_decomposed(x, salient_idx=torch.from_numpy(sal).cuda())
+        assert_same_quantized(got, ref, "given set")
+        before = q32.launch_count
+        assert_same_bits_f32(q32.dequantize(got), orc.dequantize(ref, FB), "fp32 decode with residual rows")
+        assert q32.launch_count == before + 1
+        for dt, name in ((torch.bfloat16, "bf16"), (torch.float16, "f16")):
+            o = q32.dequantize(got, dt)
+            assert np.array_equal(o.view(torch.int16).cpu().numpy().view(np.uint16),
+                                  orc.dequantize(ref, FB, out_dtype=name)), name
+
+
 def test_decomposed_with_seda_and_b16():
     q = fb4.Fb4(block_size=16)
     bits = heavy(60, 128, 21)
