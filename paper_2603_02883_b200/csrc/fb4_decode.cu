@@ -114,6 +114,12 @@ __device__ __forceinline__ void store_sum_word(uint8_t* dst, const uint32_t* pr,
   }
 }
 
+// Rows at least this wide (in 32-element units) get their residual added inside the flat decode.
+// A step of 1024 units then spans at most 5 rows, so most steps hold no salient token and run the
+// plain code; with narrower rows most steps would take the slower branch (at 96 units per row the
+// fused kernel took 85 us against 81 us for the two kernels, fp32 output, and 70 against 49 us, bf16).
+constexpr int64_t kFusedResidualMinUnitsPerRow = 256;
+
 // The residual tensor of salient rows, for the flat decode that adds it in the same pass
 struct ResidualRows {
   const int32_t* salient_idx;   // ascending token ids
@@ -543,7 +549,7 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
     else { CALL(0); }               \
   } while (0)
   ResidualRows none{};
-  if (B == 32 && n_salient > 0 && blocks_per_row >= 32 && total < 0xffffffffLL) {
+  if (B == 32 && n_salient > 0 && blocks_per_row >= kFusedResidualMinUnitsPerRow && total < 0xffffffffLL) {
     // residual rows added in the same pass: every row is written once
     const ResidualRows rr{salient_idx, n_salient, rw, res_meta, (uint32_t)blocks_per_row,
                           (float)((double)n_salient / (double)T), T, ctx->d_status};

@@ -56,7 +56,7 @@ def test_cluster_ids_out_of_range_are_unconstrained_and_reported(variant, T, C):
         q.close()
 
 
-@pytest.mark.parametrize("block_size,C", [(32, 1024), (32, 96), (16, 48)])
+@pytest.mark.parametrize("block_size,C", [(32, 8192), (32, 1024), (32, 96), (16, 48)])
 def test_decode_skips_salient_rows_outside_the_tensor(block_size, C):
     T = 200
     w = synth.Workload("idx", T=T, C=C, seed=C, kind=1, n_outlier=1, outlier_gain=50.0)

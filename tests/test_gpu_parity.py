@@ -165,9 +165,9 @@ def test_decomposed_small(q32, T, tile):
     assert_same_bits_f32(q32.dequantize(got2), orc.dequantize(ref2, FB), "decomposed idx dequant")
 
 
-@pytest.mark.parametrize("T,C,tile", [(300, 1024, 1), (257, 2112, 3), (1000, 1024, 20), (130, 4096 + 32, 2)])
+@pytest.mark.parametrize("T,C,tile", [(300, 8192, 1), (257, 8192 + 32, 3), (500, 12288, 20), (130, 16384 + 64, 2)])
 def test_decode_adds_residual_rows_in_the_same_pass(q32, T, C, tile):
-    """At 32 or more blocks per row the decode adds the residual of salient rows inside its one kernel
+    """At 256 or more blocks per row the decode adds the residual of salient rows inside its one kernel
     (steps with several salient rows, runs of consecutive salient rows, ragged last step); every output
     type against the oracle, and one launch per call."""
     bits = heavy(T, C, T + C)
