@@ -238,6 +238,15 @@ class Ops:
             return (lambda: fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, tile, cid, cmask, cmask.numel(),
                                                         codes, meta, sal, rc, rm)), \
                 algorithmic_bytes(T, C, n_res_rows=n_sal, seda=True, decomposed=True)
+        if name == "quantize_mxfp8_decomposed_seda":
+            # the whole configuration (decomposition + SeDA) straight to two MXFP8 operands
+            e8 = self.buf("e4m3", (T, C), torch.uint8)
+            sc = self.buf("sf", (fb4.fb4_mxfp8_scale_bytes(T, C, 1),), torch.uint8)
+            r8 = self.buf("res_e4m3", (n_sal, C), torch.uint8)
+            rs = self.buf("res_sf", (fb4.fb4_mxfp8_scale_bytes(n_sal, C, 1),), torch.uint8)
+            return (lambda: fb4.fb4_quantize_mxfp8_decomposed(q.ctx, x, T, C, C, score, tile, sal, 0, cid, cmask,
+                                                              cmask.numel(), e8, sc, r8, rs, 1)), \
+                T * C * 3.0 + T * (C // B) + n_sal * (C + C // B + 4) + 8 * T
         # the decode ops read what a decomposed quantization left in codes/meta/sal/rc/rm
         fb4.fb4_quantize_decomposed(q.ctx, x, T, C, C, score, tile, None, None, 0, codes, meta, sal, rc, rm)
         plain_bytes = T * C * 0.5 + T * (C // B) * 2
@@ -272,7 +281,7 @@ class Ops:
 
 OP_NAMES = ["plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
             "dequantize_bf16_plain", "dequantize_bf16_decomposed", "dequantize_f16_plain", "to_mxfp8_tiled_scales",
-            "quantize_mxfp8_tiled_scales"]
+            "quantize_mxfp8_tiled_scales", "quantize_mxfp8_decomposed_seda"]
 
 
 def main():
@@ -418,7 +427,8 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         ms = total / steps
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
                      "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_given_set",
-                                                                         "decomposed_seda", "quantize_mxfp8_tiled_scales")
+                                                                         "decomposed_seda", "quantize_mxfp8_tiled_scales",
+                                                                         "quantize_mxfp8_decomposed_seda")
                      else "decode"}
         if name == "dequantize_f32_decomposed":
             ops.drop("out32")

@@ -290,6 +290,29 @@ int fb4_quantize_mxfp8(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, i
                        const int32_t* cluster_id, const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* e4m3,
                        uint8_t* scales, int scale_layout, void* stream);
 
+/*
+ * fb4_quantize_mxfp8 with activation decomposition (Sec. 3.3: Act ~ Q(Act) + Q(Delta) for salient
+ * tokens; App. D.2: the consumer is an MXFP8 GEMM): one pass writes Q(Act) as an MXFP8 operand
+ * [T][C] and Q(Delta) of the salient tokens as a second, compact MXFP8 operand [n_salient][C].
+ * The sum of the two is not an e4m3 value in general, so the residual stays a separate operand:
+ * the consumer multiplies it as a second, small GEMM and adds the rows listed in salient_idx.
+ * The outputs equal fb4_to_mxfp8 applied to the main and to the residual output of
+ * fb4_quantize_decomposed[_idx], byte for byte.  Same restrictions as fb4_quantize_mxfp8.
+ *   score        : device float [T] -> one salient token per `tile` tokens is selected first
+ *                  (fb4_select_salient) and written to salient_idx (capacity ceil(T/tile));
+ *                  NULL -> salient_idx is an input: n_salient strictly ascending token ids
+ *   n_salient    : used only when score is NULL
+ *   cluster_id   : NULL = no SeDA restriction; else main and residual both use the token's mask
+ *   res_e4m3     : device uint8 [n_salient][C] (out), 32-byte aligned
+ *   res_scales   : device uint8 (out), fb4_mxfp8_scale_bytes(n_salient, C, scale_layout) bytes,
+ *                  the scale layout applied to the residual operand on its own
+ */
+int fb4_quantize_mxfp8_decomposed(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems,
+                                  const float* score, int32_t tile, int32_t* salient_idx, int64_t n_salient,
+                                  const int32_t* cluster_id, const uint32_t* cluster_mask, int32_t n_clusters,
+                                  uint8_t* e4m3, uint8_t* scales, uint8_t* res_e4m3, uint8_t* res_scales,
+                                  int scale_layout, void* stream);
+
 /* Size in bytes of the scale buffer of fb4_to_mxfp8 (-1 for invalid arguments).  Host only. */
 int64_t fb4_mxfp8_scale_bytes(int64_t T, int64_t C, int scale_layout);
 

@@ -392,10 +392,47 @@ int fb4_quantize_mxfp8(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_
   ex.cluster_id = cluster_id;
   ex.cluster_mask = cluster_id ? cluster_mask : nullptr;
   ex.n_clusters = cluster_id ? n_clusters : 0;
-  cudaError_t e = fb4_launch_quantize_fast_mx(ctx, x, T, C, ld, ex, e4m3, scales, scale_layout,
-                                              static_cast<cudaStream_t>(stream));
+  int launches = 0;
+  cudaError_t e = fb4_launch_quantize_fast_mx(ctx, x, T, C, ld, ex, e4m3, scales, nullptr, nullptr, scale_layout,
+                                              static_cast<cudaStream_t>(stream), &launches);
+  ctx->launches += launches;
   if (e != cudaSuccess) return fb4_set_cuda_error(e);
-  ctx->launches += 1;
+  ctx->last_variant = "fast";
+  return FB4_OK;
+}
+
+int fb4_quantize_mxfp8_decomposed(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const float* score,
+                                  int32_t tile, int32_t* salient_idx, int64_t n_salient, const int32_t* cluster_id,
+                                  const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* e4m3, uint8_t* scales,
+                                  uint8_t* res_e4m3, uint8_t* res_scales, int scale_layout, void* stream) {
+  if (!ctx) return FB4_ERR_INVALID_ARG;
+  if (scale_layout != 0 && scale_layout != 1) return FB4_ERR_INVALID_ARG;
+  if (T < 0 || C <= 0 || C % 64 != 0 || ld < C || T > 0x7fffffffLL) return FB4_ERR_SHAPE;
+  if (score ? tile <= 0 : (n_salient < 0 || n_salient > T)) return FB4_ERR_INVALID_ARG;
+  if (T == 0) return FB4_OK;
+  if (score) n_salient = (T + tile - 1) / tile;
+  if (!x || !e4m3 || !scales) return FB4_ERR_INVALID_ARG;
+  if (n_salient > 0 && (!salient_idx || !res_e4m3 || !res_scales)) return FB4_ERR_INVALID_ARG;
+  if (cluster_id && (!cluster_mask || n_clusters <= 0)) return FB4_ERR_INVALID_ARG;
+  if (!aligned16(x) || (ld & 7) || (reinterpret_cast<uintptr_t>(e4m3) & 31u)) return FB4_ERR_ALIGN;
+  if (n_salient > 0 && (reinterpret_cast<uintptr_t>(res_e4m3) & 31u)) return FB4_ERR_ALIGN;
+  if (!fb4_fast_mx_eligible(ctx, x, T, C, ld)) return FB4_ERR_INVALID_ARG;   // default configuration only
+  if (score) {
+    const int rc = fb4_select_salient(ctx, score, T, tile, salient_idx, stream);
+    if (rc != FB4_OK) return rc;
+  }
+  Fb4RowExtras ex{};
+  ex.cluster_id = cluster_id;
+  ex.cluster_mask = cluster_id ? cluster_mask : nullptr;
+  ex.n_clusters = cluster_id ? n_clusters : 0;
+  ex.salient_idx = salient_idx;
+  ex.n_salient = n_salient;
+  ex.tile = score ? tile : 0;
+  int launches = 0;
+  cudaError_t e = fb4_launch_quantize_fast_mx(ctx, x, T, C, ld, ex, e4m3, scales, res_e4m3, res_scales, scale_layout,
+                                              static_cast<cudaStream_t>(stream), &launches);
+  ctx->launches += launches;
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
   ctx->last_variant = "fast";
   return FB4_OK;
 }

@@ -78,6 +78,8 @@ struct FastParams {
   uint32_t ec_lo, ec_hi;   // clamp of the biased block exponent (CLAMP kernels): exp_min + 127, exp_max + 127
   uint8_t* e4m3;           // MX kernels: e4m3 bytes [T][C] and E8M0 scale bytes instead of codes / meta
   uint8_t* scales;
+  uint8_t* res_e4m3;       // MX kernels with residual pass: the residual rows in the same form
+  uint8_t* res_scales;
   int64_t scale_col_tiles;
   int32_t scale_tiled;
 };
@@ -593,7 +595,18 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
         uint32_t rcw[4], rmeta;
         residual_block<SEDA, B16, CLAMP>(w, cw, didh, Ech, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, rcw,
                                          &rmeta);
-        if (active) {
+        if (MX) {
+          // the residual block as e4m3 bytes + E8M0 scale, row srow of the residual operand
+          if (active) {
+            const uint2 fb = tb->fb_e4m3[(rmeta >> 8) & 31u];
+            uint32_t o[8];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) fb4dev::codes_to_e4m3(rcw[q], fb, o[2 * q], o[2 * q + 1]);
+            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p.res_e4m3 + srow * p.C + blk * 32),
+                         "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+            p.res_scales[fb4dev::mx_scale_offset(srow, blk, nblk, p.scale_col_tiles, p.scale_tiled)] = (uint8_t)rmeta;
+          }
+        } else if (active) {
           *reinterpret_cast<uint4*>(ex.res_codes + srow * code_row_bytes + blk * 16) =
               make_uint4(rcw[0], rcw[1], rcw[2], rcw[3]);
           if (B16) *reinterpret_cast<uint32_t*>(ex.res_meta + (srow * nblk + blk) * 2) = rmeta;
@@ -883,6 +896,8 @@ cudaError_t fb4_fast_prepare_device() {
   FB4_OPT_IN(true, true, true, true);
   FB4_OPT_IN(false, false, false, false, true);
   FB4_OPT_IN(true, false, false, false, true);
+  FB4_OPT_IN(false, true, false, false, true);
+  FB4_OPT_IN(true, true, false, false, true);
 #undef FB4_OPT_IN
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
   return e;
@@ -1011,27 +1026,46 @@ bool fb4_fast_mx_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t 
   return c.block_size == 32 && c.exp_min == -124 && c.exp_max == 127 && fb4_fast_eligible(ctx, x, T, C, ld);
 }
 
+// With ex.n_salient > 0 the residual of the salient rows goes to res_e4m3 [n_salient][C] and
+// res_scales (the scale layout applied to the [n_salient][C] operand); ex.res_codes / res_meta are
+// not used.
 cudaError_t fb4_launch_quantize_fast_mx(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
-                                        const Fb4RowExtras& ex, uint8_t* e4m3, uint8_t* scales, int tiled,
-                                        cudaStream_t stream) {
+                                        const Fb4RowExtras& ex, uint8_t* e4m3, uint8_t* scales, uint8_t* res_e4m3,
+                                        uint8_t* res_scales, int tiled, cudaStream_t stream, int* launches) {
+  const bool decomp = ex.n_salient > 0;
   CUtensorMap map;
   FastParams p;
   int grid = 0;
-  cudaError_t e = fast_setup(ctx, x, T, C, ld, false, &map, &p, &grid);
+  cudaError_t e = fast_setup(ctx, x, T, C, ld, decomp, &map, &p, &grid);
   if (e != cudaSuccess) return e;
   p.e4m3 = e4m3;
   p.scales = scales;
+  p.res_e4m3 = res_e4m3;
+  p.res_scales = res_scales;
   p.scale_tiled = tiled;
   const int64_t n_col = C / 32;
   p.scale_col_tiles = (n_col + 3) / 4;
-  if (tiled && ((T & 127) || (n_col & 3))) {   // the kernel writes real entries only: padding = scale 1
+  // the kernel writes real entries only: padding of the tiled layout = scale 1
+  if (tiled && ((T & 127) || (n_col & 3))) {
     e = cudaMemsetAsync(scales, 0x7f, (size_t)(((T + 127) / 128) * p.scale_col_tiles * 512), stream);
     if (e != cudaSuccess) return e;
   }
+  if (decomp && tiled && ((ex.n_salient & 127) || (n_col & 3))) {
+    e = cudaMemsetAsync(res_scales, 0x7f, (size_t)(((ex.n_salient + 127) / 128) * p.scale_col_tiles * 512), stream);
+    if (e != cudaSuccess) return e;
+  }
   const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
-  if (ex.cluster_id)
-    fb4_quantize_fast_kernel<true, false, false, false, true><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
-  else
-    fb4_quantize_fast_kernel<false, false, false, false, true><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
-  return cudaGetLastError();
+  const int variant = (ex.cluster_id ? 1 : 0) | (decomp ? 2 : 0);
+#define FB4_MX(S, D) \
+  fb4_quantize_fast_kernel<S, D, false, false, true><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex)
+  switch (variant) {
+    case 0: FB4_MX(false, false); break;
+    case 1: FB4_MX(true, false); break;
+    case 2: FB4_MX(false, true); break;
+    default: FB4_MX(true, true); break;
+  }
+#undef FB4_MX
+  e = cudaGetLastError();
+  if (e == cudaSuccess) *launches = 1;
+  return e;
 }

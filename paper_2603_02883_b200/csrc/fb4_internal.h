@@ -59,8 +59,8 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
 
 bool fb4_fast_mx_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld);
 cudaError_t fb4_launch_quantize_fast_mx(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
-                                        const Fb4RowExtras& ex, uint8_t* e4m3, uint8_t* scales, int tiled,
-                                        cudaStream_t stream);
+                                        const Fb4RowExtras& ex, uint8_t* e4m3, uint8_t* scales, uint8_t* res_e4m3,
+                                        uint8_t* res_scales, int tiled, cudaStream_t stream, int* launches);
 bool fb4_fast_f32_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld);
 cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
                                          uint8_t* codes, uint16_t* meta, cudaStream_t stream);

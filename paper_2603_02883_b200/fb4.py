@@ -23,7 +23,7 @@ STATIC_MAX_CLUSTERS = 1024
 EXPORTS = [
     "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
     "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_select_salient_topk", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
-    "fb4_quantize_weights", "fb4_quantize_mxfp8", "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
+    "fb4_quantize_weights", "fb4_quantize_mxfp8", "fb4_quantize_mxfp8_decomposed", "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
 
 
@@ -86,6 +86,9 @@ def lib() -> ctypes.CDLL:
     L.fb4_quantize_weights.restype = ci
     L.fb4_quantize_mxfp8.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, vp, vp, ci, vp]
     L.fb4_quantize_mxfp8.restype = ci
+    L.fb4_quantize_mxfp8_decomposed.argtypes = [vp, vp, i64, i64, i64, vp, i32, vp, i64, vp, vp, i32, vp, vp, vp, vp,
+                                                ci, vp]
+    L.fb4_quantize_mxfp8_decomposed.restype = ci
     L.fb4_to_mxfp8.argtypes = [vp, vp, vp, i64, i64, vp, vp, ci, vp]
     L.fb4_to_mxfp8.restype = ci
     L.fb4_mxfp8_scale_bytes.argtypes = [i64, i64, ci]
@@ -232,6 +235,14 @@ def fb4_quantize_mxfp8(ctx, x, T, C, ld_elems, cluster_id, cluster_mask, n_clust
                        stream=None) -> None:
     _check(lib().fb4_quantize_mxfp8(ctx, _ptr(x), T, C, ld_elems, _ptr(cluster_id), _ptr(cluster_mask), n_clusters,
                                     _ptr(e4m3), _ptr(scales), scale_layout, _stream(stream)), "fb4_quantize_mxfp8")
+
+
+def fb4_quantize_mxfp8_decomposed(ctx, x, T, C, ld_elems, score, tile, salient_idx, n_salient, cluster_id, cluster_mask,
+                                  n_clusters, e4m3, scales, res_e4m3, res_scales, scale_layout, stream=None) -> None:
+    _check(lib().fb4_quantize_mxfp8_decomposed(ctx, _ptr(x), T, C, ld_elems, _ptr(score), tile, _ptr(salient_idx),
+                                               n_salient, _ptr(cluster_id), _ptr(cluster_mask), n_clusters,
+                                               _ptr(e4m3), _ptr(scales), _ptr(res_e4m3), _ptr(res_scales),
+                                               scale_layout, _stream(stream)), "fb4_quantize_mxfp8_decomposed")
 
 
 def fb4_to_mxfp8(ctx, codes, meta, T, C, e4m3, scales, scale_layout, stream=None) -> None:
@@ -392,6 +403,25 @@ class Fb4:
         fb4_quantize_mxfp8(self.ctx, x, T, C, ld, cluster_id, cluster_mask,
                            0 if cluster_mask is None else cluster_mask.numel(), e4m3, scales, scale_layout)
         return e4m3, scales[:n]
+
+    def quantize_mxfp8_decomposed(self, x, score=None, tile: int = 20, salient_idx=None, scale_layout: int = 1,
+                                  cluster_id=None, cluster_mask=None):
+        """-> (e4m3 [T][C], scales, salient_idx, res_e4m3 [n][C], res_scales): main and residual MXFP8 operands"""
+        assert x.dtype == torch.bfloat16
+        T, C, ld = self._shape(x)
+        n = -(-T // tile) if salient_idx is None else salient_idx.numel()
+        if salient_idx is None:
+            salient_idx = torch.empty(max(n, 1), dtype=torch.int32, device=x.device)
+        dev = x.device
+        e4m3 = torch.empty((T, C), dtype=torch.uint8, device=dev)
+        scales = torch.empty(max(fb4_mxfp8_scale_bytes(T, C, scale_layout), 1), dtype=torch.uint8, device=dev)
+        res = torch.empty((max(n, 1), C), dtype=torch.uint8, device=dev)
+        nrs = fb4_mxfp8_scale_bytes(n, C, scale_layout)
+        res_scales = torch.empty(max(nrs, 1), dtype=torch.uint8, device=dev)
+        fb4_quantize_mxfp8_decomposed(self.ctx, x, T, C, ld, score, tile, salient_idx, n, cluster_id, cluster_mask,
+                                      0 if cluster_mask is None else cluster_mask.numel(), e4m3, scales, res,
+                                      res_scales, scale_layout)
+        return (e4m3, scales[:fb4_mxfp8_scale_bytes(T, C, scale_layout)], salient_idx[:n], res[:n], res_scales[:nrs])
 
     def to_mxfp8(self, q: Quantized, scale_layout: int = 0):
         """(e4m3 bytes [T][C], E8M0 scale bytes) of the main tensor of q."""

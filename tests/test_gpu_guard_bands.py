@@ -95,6 +95,16 @@ def test_all_entry_points_stay_inside_their_buffers(T, C, B):
             torch.cuda.synchronize()
             e8.check(f"e4m3 layout {layout}")
             sc.check(f"scales layout {layout}")
+            if C % 64 == 0 and B == 32:   # the one-pass form with residual rows (default configuration only)
+                e8, sc = Guarded(T * C), Guarded(fb4.fb4_mxfp8_scale_bytes(T, C, layout))
+                r8, rs = Guarded(ns * C), Guarded(fb4.fb4_mxfp8_scale_bytes(ns, C, layout))
+                si = Guarded(ns * 4)
+                fb4.fb4_quantize_mxfp8_decomposed(q.ctx, x, T, C, C, score, tile, si.tensor(torch.int32, (ns,)), 0,
+                                                  cid, cmask, cmask.numel(), e8.view, sc.view, r8.view, rs.view, layout)
+                torch.cuda.synchronize()
+                for g, what in ((e8, "e4m3"), (sc, "scales"), (r8, "residual e4m3"), (rs, "residual scales"),
+                                (si, "salient indices")):
+                    g.check(f"one-pass decomposed MXFP8, {what}, layout {layout}")
     ncl = cmask.numel()
     cnt, msk = Guarded(ncl * 32 * 4), Guarded(ncl * 4)
     tok = torch.arange(0, T, max(1, T // 5), dtype=torch.int32, device="cuda")

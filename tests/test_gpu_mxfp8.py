@@ -155,3 +155,106 @@ def test_tiled_scales_at_an_odd_address(q32, T, C):
         got = buf.cpu().numpy()
         assert np.array_equal(got[shift:shift + n], s_ref), f"scale bytes, shift {shift}"
         assert (got[:shift] == 0xEE).all() and (got[shift + n:] == 0xEE).all(), "bytes outside the scale array"
+
+
+@pytest.mark.parametrize("T,C,tile", [(1, 64, 20), (130, 3072, 20), (300, 1024 + 64, 7), (257, 128, 1), (2368, 64, 20)])
+def test_fused_quantize_to_mxfp8_with_decomposition(q32, T, C, tile):
+    """fb4_quantize_mxfp8_decomposed equals the decomposed quantizer (oracle) followed by the MXFP8 view of the main
+    and of the residual tensor: per-tile selection and a given salient set, with and without SeDA, both layouts."""
+    w = synth.Workload("m", T=T, C=C, seed=T + C, kind=1, n_outlier=2, outlier_gain=50.0, seda=True,
+                       n_clusters=min(4, T), cluster_seed=5, score_seed=T)
+    bits = synth.activation(w)
+    cid, masks = synth.clusters(w)
+    score = synth.scores(w)
+    x = to_dev_bf16(bits)
+    d_cid, d_masks = torch.from_numpy(cid).cuda(), torch.from_numpy(masks.view(np.int32)).cuda()
+    sal = orc.select_salient(score, tile)
+    mine = np.unique(np.random.default_rng(T).integers(0, T, size=max(1, T // 3))).astype(np.int32)
+    for seda in (False, True):
+        kw = dict(cluster_id=cid, cluster_mask=masks) if seda else {}
+        dkw = dict(cluster_id=d_cid, cluster_mask=d_masks) if seda else {}
+        for layout in (0, 1):
+            for given in (False, True):
+                want_idx = mine if given else sal
+                ref = orc.quantize(bits, FB, salient_idx=want_idx, **kw)
+                e_ref, s_ref = orc.to_mxfp8(orc.Quantized(ref.codes, ref.meta), FB, layout)
+                re_ref, rs_ref = orc.to_mxfp8(orc.Quantized(ref.res_codes, ref.res_meta), FB, layout)
+                if given:
+                    out = q32.quantize_mxfp8_decomposed(x, salient_idx=torch.from_numpy(mine).cuda(),
+                                                        scale_layout=layout, **dkw)
+                else:
+                    out = q32.quantize_mxfp8_decomposed(x, score=torch.from_numpy(score).cuda(), tile=tile,
+                                                        scale_layout=layout, **dkw)
+                e4m3, scales, idx, res, res_scales = out
+                what = f"seda {seda} layout {layout} given {given}"
+                assert np.array_equal(idx.cpu().numpy(), want_idx), what
+                assert np.array_equal(e4m3.cpu().numpy(), e_ref), what
+                assert np.array_equal(scales.cpu().numpy(), s_ref), what
+                assert np.array_equal(res.cpu().numpy(), re_ref), what
+                assert np.array_equal(res_scales.cpu().numpy(), rs_ref), what
+
+
+def test_library_block_scaled_gemm_with_residual_operand(q32):
+    """(Q(Act) + Q(Delta)) W (Sec. 3.3) as two block-scaled library GEMMs on the operands of
+    fb4_quantize_mxfp8_decomposed: the main one over all tokens, the residual one over the salient tokens, added
+    into their rows; compared with the product of the decoded sum and the decoded weights."""
+    if not hasattr(torch, "_scaled_mm") or not hasattr(torch, "float8_e8m0fnu"):
+        pytest.skip("this torch build has no block-scaled GEMM")
+    T, N, K, tile = 320, 128, 1024, 20
+    wl = synth.Workload("a", T=T, C=K, seed=3, kind=1, n_outlier=2, outlier_gain=50.0, score_seed=9)
+    a_bits, score = synth.activation(wl), synth.scores(wl)
+    w_bits = synth.activation(synth.Workload("w", T=N, C=K, seed=4, kind=1, n_outlier=0, outlier_gain=1.0))
+    x = to_dev_bf16(a_bits)
+    e4m3, scales, idx, res, res_scales = q32.quantize_mxfp8_decomposed(x, score=torch.from_numpy(score).cuda(), tile=tile)
+    qw = q32.quantize_weights(to_dev_bf16(w_bits))
+    ew, sw = q32.to_mxfp8(qw, 1)
+    f8, e8 = torch.float8_e4m3fn, torch.float8_e8m0fnu
+
+    def gemm(a, sa):
+        return torch._scaled_mm(a.view(f8), ew.view(f8).t(), scale_a=sa.view(e8), scale_b=sw.view(e8),
+                                out_dtype=torch.float32)
+
+    y = gemm(e4m3, scales)
+    y.index_add_(0, idx.long(), gemm(res.contiguous(), res_scales))
+    qa = q32.quantize_decomposed(x, score=torch.from_numpy(score).cuda(), tile=tile)
+    da, dw = q32.dequantize(qa).double(), q32.dequantize(qw).double()
+    want, bound = da @ dw.T, da.abs() @ dw.abs().T
+    assert bool(((y.double() - want).abs() <= bound * 2e-5).all())      # fp32 accumulation, two partial products
+    # the residual operand matters: without it the salient rows are off by more than that
+    y0 = gemm(e4m3, scales).double()
+    rows = idx.long()
+    assert not bool(((y0[rows] - want[rows]).abs() <= bound[rows] * 2e-5).all())
+
+
+def test_fused_decomposed_argument_checks(q32):
+    L = fb4.lib()
+    x = torch.zeros((8, 64), dtype=torch.bfloat16, device="cuda")
+    out = torch.zeros(8192, dtype=torch.uint8, device="cuda")
+    idx = torch.zeros(8, dtype=torch.int32, device="cuda")
+    sc = torch.zeros(8, dtype=torch.float32, device="cuda")
+    p = lambda t: ctypes.c_void_p(t.data_ptr())
+    f = L.fb4_quantize_mxfp8_decomposed
+    ok = (q32.ctx, p(x), 8, 64, 64, p(sc), 4, p(idx), 0, None, None, 0, p(out), p(out), p(out), p(out), 0, None)
+    assert f(*ok) == fb4.OK
+
+    def call(**kw):
+        a = list(ok)
+        names = ["ctx", "x", "T", "C", "ld", "score", "tile", "idx", "n", "cid", "cmask", "ncl", "e", "s", "re", "rs",
+                 "layout", "stream"]
+        for k, v in kw.items():
+            a[names.index(k)] = v
+        return f(*a)
+
+    assert call(tile=0) == fb4.ERR_INVALID_ARG
+    assert call(score=None, n=9) == fb4.ERR_INVALID_ARG          # more salient tokens than tokens
+    assert call(score=None, n=-1) == fb4.ERR_INVALID_ARG
+    assert call(score=None, n=2, re=None) == fb4.ERR_INVALID_ARG
+    assert call(score=None, n=0, idx=None, re=None, rs=None) == fb4.OK     # no salient tokens: plain call
+    assert call(C=32) == fb4.ERR_SHAPE
+    assert call(layout=2) == fb4.ERR_INVALID_ARG
+    assert call(cid=p(idx)) == fb4.ERR_INVALID_ARG               # cluster ids without masks
+    assert call(re=ctypes.c_void_p(out.data_ptr() + 16)) == fb4.ERR_ALIGN
+    assert call(T=0, x=None) == fb4.OK
+    q16 = fb4.Fb4(block_size=16)
+    assert call(ctx=q16.ctx) == fb4.ERR_INVALID_ARG
+    q16.close()
