@@ -493,9 +493,25 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         tot_g, _ = time_steps(graph.replay, 20, 3, torch)
         res["c1_256x3072_quantize_plus_decode"] = {"us_per_pair_launched_one_by_one": tot / 200 * 1e3,
                                                    "us_per_pair_in_a_cuda_graph": tot_g / (20 * 20) * 1e3}
+        # context for that size: a library copy that moves the same number of bytes (half read, half
+        # written), timed the same way with the same flush
+        half = torch.empty(int(alg) // 4, dtype=torch.int16, device="cuda")
+        half2 = torch.empty_like(half)
+        cevs = []
+        for i in range(warm + steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            half2.copy_(half)
+            b.record()
+            cevs.append((a, b))
+        torch.cuda.synchronize()
+        copy_ms = float(np.mean([a.elapsed_time(b) for a, b in cevs[warm:]]))
         res["c2_plain_32760x3072_l2_flushed"] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9,
                                                  "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
-                                                 "kernel_variant": q.last_variant}
+                                                 "kernel_variant": q.last_variant,
+                                                 "library_copy_of_the_same_bytes_ms": copy_ms,
+                                                 "frac_of_that_copy": copy_ms / ms}
     return res
 
 
