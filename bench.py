@@ -553,9 +553,29 @@ def run_cpu_baseline(w, synth):
         if time.perf_counter() - t0 > 10.0 or reps >= 20:
             break
     dt = (time.perf_counter() - t0) / reps
-    return {"value": algorithmic_bytes(rows, w.C) / dt / 1e9, "unit": UNIT, "cores": os.cpu_count(),
-            "kind": "oracle", "gelem_per_s": rows * w.C / dt / 1e9,
-            "sample": f"first {rows} of {w.T} rows, {reps} passes, OpenMP over rows on all host cores"}
+    out = {"value": algorithmic_bytes(rows, w.C) / dt / 1e9, "unit": UNIT, "cores": os.cpu_count(),
+           "kind": "oracle", "gelem_per_s": rows * w.C / dt / 1e9,
+           "sample": f"first {rows} of {w.T} rows, {reps} passes, OpenMP over rows on all host cores"}
+    # the same oracle on one core (its OpenMP runtime told to use one thread), on a 1024-row slab
+    try:
+        import ctypes
+        gomp = ctypes.CDLL("libgomp.so.1")
+        gomp.omp_get_max_threads.restype = ctypes.c_int
+        before = gomp.omp_get_max_threads()
+        gomp.omp_set_num_threads(1)
+        try:
+            slab = bits[:min(rows, 1024)]
+            t0 = time.perf_counter()
+            orc.quantize(slab, fbk)
+            dt1 = time.perf_counter() - t0
+        finally:
+            gomp.omp_set_num_threads(before)
+        out["one_core"] = {"value": algorithmic_bytes(slab.shape[0], w.C) / dt1 / 1e9, "unit": UNIT,
+                           "gelem_per_s": slab.shape[0] * w.C / dt1 / 1e9,
+                           "sample": f"first {slab.shape[0]} rows, one pass, one thread"}
+    except OSError:
+        pass
+    return out
 
 
 if __name__ == "__main__":
