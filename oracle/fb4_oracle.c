@@ -247,6 +247,7 @@ int64_t fb4o_select_salient_topk(const float *score, int64_t T, int64_t k, int32
     int64_t arg = -1;
     for (int64_t t = 0; t < T; ++t)
       if (!taken[t] && (arg < 0 || score[t] > score[arg])) arg = t;   /* first maximum = lowest index */
+    if (arg < 0) break;   /* cannot happen (k <= T): keeps the compiler's bounds analysis quiet */
     taken[arg] = 1;
   }
   int64_t n = 0;
