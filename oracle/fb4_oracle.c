@@ -361,6 +361,30 @@ int fb4o_quantize_f32(const float *x, int64_t T, int64_t C, int64_t ld, const fb
   return 0;
 }
 
+/*
+ * Per-channel affine producer in front of the quantizer (App. D.2: quantization is fused with the
+ * preceding operation, e.g. LayerNorm; the elementwise tail of a LayerNorm is y = x * gamma_c +
+ * beta_c, and the modulation of Open-Sora 2.0's blocks, Sec. 3.3, is y = x * (1 + scale_c) +
+ * shift_c):  y[t][c] = x[t][c] * g_c + bias_c  with  g_c = gain_c  or  1 + gain_c (plus_one),
+ * x, gain and bias given as bf16.  The arithmetic is float32 as in the fused kernel, stated
+ * exactly: g_c is the float32 nearest to 1 + gain_c, and y is the float32 nearest to the exact
+ * value of x * g_c + bias_c (one rounding: fmaf).  The result feeds fb4o_quantize_f32.
+ */
+int fb4o_affine_f32(const uint16_t *x, int64_t T, int64_t C, int64_t ld, const uint16_t *gain,
+                    const uint16_t *bias, int plus_one, float *y) {
+  if (T < 0 || C <= 0 || ld < C) return -1;
+  for (int64_t t = 0; t < T; ++t) {
+    for (int64_t c = 0; c < C; ++c) {
+      const float xf = (float)bf16_to_double(x[t * ld + c]);
+      float g = (float)bf16_to_double(gain[c]);
+      const float b = (float)bf16_to_double(bias[c]);
+      if (plus_one) g = 1.0f + g;
+      y[t * C + c] = fmaf(xf, g, b);
+    }
+  }
+  return 0;
+}
+
 static uint16_t f32_to_bf16_rne(float f) {
   uint32_t u;
   memcpy(&u, &f, 4);

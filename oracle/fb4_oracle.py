@@ -80,6 +80,8 @@ def lib():
         L.fb4o_quantize_block_f64.restype = ctypes.c_int
         L.fb4o_quantize_f32.argtypes = [vp, i64, i64, i64, ctypes.POINTER(_Cfg), vp, vp, vp, vp]
         L.fb4o_quantize_f32.restype = ctypes.c_int
+        L.fb4o_affine_f32.argtypes = [vp, i64, i64, i64, vp, vp, ctypes.c_int, vp]
+        L.fb4o_affine_f32.restype = ctypes.c_int
         L.fb4o_to_mxfp8.argtypes = [vp, vp, i64, i64, vp, vp, vp, ctypes.c_int]
         L.fb4o_to_mxfp8.restype = ctypes.c_int
         L.fb4o_mxfp8_scale_offset.argtypes = [i64, i64, i64, ctypes.c_int]
@@ -246,6 +248,21 @@ def quantize_f32(x, formatbook, cfg: Config = Config(), stage1=None) -> Quantize
     if r != 0:
         raise ValueError(f"fb4o_quantize_f32 failed: {r}")
     return Quantized(codes, meta)
+
+
+def affine_f32(x_bits, gain_bits, bias_bits, plus_one: bool) -> np.ndarray:
+    """y = x * g + bias per channel in float32 (one rounding), g = gain or 1 + gain; all inputs bf16 bit patterns."""
+    x = np.asarray(x_bits)
+    assert x.dtype == np.uint16 and x.ndim == 2 and x.strides[1] == 2
+    T, C = x.shape
+    ld = x.strides[0] // 2 if T > 1 else C
+    g, b = _c(gain_bits, np.uint16), _c(bias_bits, np.uint16)
+    assert g.shape == (C,) and b.shape == (C,)
+    y = np.zeros((T, C), dtype=np.float32)
+    r = lib().fb4o_affine_f32(_p(x), T, C, ld, _p(g), _p(b), int(bool(plus_one)), _p(y))
+    if r != 0:
+        raise ValueError(f"fb4o_affine_f32 failed: {r}")
+    return y
 
 
 def mxfp8_scale_offset(row: int, col: int, n_col: int, layout: int) -> int:

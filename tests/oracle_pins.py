@@ -336,6 +336,68 @@ def pin_seda_choice_inside_mask(seed=4, n=120):
     assert np.array_equal(qa.codes, qb.codes) and np.array_equal(qa.meta, qb.meta)
 
 
+def _round_to_f32(q):
+    """The binary32 number nearest to the rational q (ties to even), by integer arithmetic: returns a Fraction.
+    (Overflow is out of range for the pins that use it.)"""
+    from fractions import Fraction
+    if q == 0:
+        return Fraction(0)
+    sign, a = (-1 if q < 0 else 1), abs(q)
+    e = a.numerator.bit_length() - a.denominator.bit_length()      # a in [2^(e-1), 2^(e+1))
+    if Fraction(2) ** e > a:
+        e -= 1                                                     # now 2^e <= a < 2^(e+1)
+    e = max(e, -126)                                               # subnormals share the spacing of 2^-126
+    ulp = Fraction(2) ** (e - 23)
+    n = a / ulp
+    k = n.numerator // n.denominator
+    rem = n - k
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and k % 2 == 1):
+        k += 1
+    return sign * k * ulp
+
+
+def pin_affine_producer(seed=21, n=400):
+    """y = x * g + bias (App. D.2 fusion with the preceding operation; LayerNorm tail / modulation): g is the
+    float32 nearest to 1 + gain, y the float32 nearest to the EXACT x * g + bias (one rounding), checked in
+    rationals; identity for gain 1 / bias 0 (or gain 0 with plus_one), signed zeros included."""
+    from fractions import Fraction
+    rng = np.random.default_rng(seed)
+    bf = lambda a: synth.f32_to_bf16_bits(np.asarray(a, dtype=np.float32))
+    val = lambda bits: Fraction(float(synth.bf16_bits_to_f32(np.asarray(bits, dtype=np.uint16).reshape(1))[0]))
+    C = 8
+    for it in range(n):
+        k = rng.integers(-20, 20)
+        x = bf(rng.standard_normal((2, C)) * np.exp2(float(k)))
+        gain = bf(rng.standard_normal(C) * np.exp2(float(rng.integers(-30, 3))))
+        # biases near -x*g make the sum cancel, where a second rounding would show
+        bias = bf(-synth.bf16_bits_to_f32(x[0]) * (1 + synth.bf16_bits_to_f32(gain)) * (1 + rng.standard_normal(C) * 2.0 ** -9))
+        if it % 7 == 0:
+            bias = bf(rng.standard_normal(C) * np.exp2(float(rng.integers(-20, 20))))
+        for plus_one in (False, True):
+            y = orc.affine_f32(x, gain, bias, plus_one)
+            for t in range(2):
+                for c in range(C):
+                    g = _round_to_f32(1 + val(gain[c])) if plus_one else val(gain[c])
+                    want = _round_to_f32(val(x[t, c]) * g + val(bias[c]))
+                    assert Fraction(float(y[t, c])) == want, (it, t, c, plus_one)
+    # identity, bit for bit (signed zeros: -0 * 1 + 0 = +0 is the IEEE sum, so bias -0 keeps the sign)
+    x = bf(np.array([[1.5, -2.0, 0.0, -0.0, 3e-39, -1e38, 7.0, 0.25]], dtype=np.float32))
+    one, zero, nzero = bf(np.ones(8)), bf(np.zeros(8)), bf(np.full(8, -0.0))
+    for g, p1 in ((one, False), (zero, True)):
+        y = orc.affine_f32(x, g, nzero, p1)
+        assert np.array_equal(y.view(np.uint32), synth.bf16_bits_to_f32(x).view(np.uint32))
+    y = orc.affine_f32(x, one, zero, False)
+    assert np.signbit(y[0, 3]) == False and y[0, 3] == 0.0        # -0 + 0 = +0
+    # a row stride, and a gain that 1 + gain cannot hold in float32 (2^-30): g rounds to exactly 1
+    wide = np.zeros((2, 16), dtype=np.uint16)
+    wide[:, :8] = bf(rng.standard_normal((2, 8)))
+    tiny = bf(np.full(8, 2.0 ** -30))
+    y = orc.affine_f32(wide[:, :8], tiny, zero, True)
+    assert np.array_equal(y, synth.bf16_bits_to_f32(wide[:, :8]))
+    y = orc.affine_f32(wide[:, :8], tiny, zero, False)
+    assert np.array_equal(y, synth.bf16_bits_to_f32(wide[:, :8]) * np.float32(2.0 ** -30))
+
+
 def pin_f32_input(seed=9, n=30):
     """fp32 input: every block equals the block-wise definition on the exact values (pinned above
     through quantize_block_f64), values that happen to be bf16 give the bf16 result, and a value
@@ -664,7 +726,7 @@ ALL_PINS = [
     pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
     pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_salient_topk, pin_decomposition, pin_residual_uses_the_seda_mask,
-    pin_dequantize_formula, pin_dequantize_f16, pin_mse, pin_f32_input, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
+    pin_dequantize_formula, pin_dequantize_f16, pin_mse, pin_f32_input, pin_affine_producer, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
     pin_subformatbook_hand_counted,
     pin_subformatbook_one_dialect_per_bucket_and_closed_loop,
 ]

@@ -70,6 +70,14 @@ MUTANTS = {
     "subformatbook_all_anchors_one_cluster": ("if (anchor_cluster[a] != c) continue;", ";"),
     "subformatbook_last_block_skipped": ("for (int64_t b = 0; b < nblk; ++b) count[", "for (int64_t b = 0; b + 1 < nblk; ++b) count["),
     "subformatbook_counts_scale_byte": ("count[(meta[t * nblk + b] >> 8) & 31] += 1;", "count[meta[t * nblk + b] & 31] += 1;"),
+    "affine_two_roundings": ("y[t * C + c] = fmaf(xf, g, b);", "y[t * C + c] = (float)(xf * g) + b;"),
+    "affine_one_plus_gain_exact": ("if (plus_one) g = 1.0f + g;\n      y[t * C + c] = fmaf(xf, g, b);",
+                                   "y[t * C + c] = plus_one ? (float)((double)xf * (1.0 + (double)g) + (double)b) : fmaf(xf, g, b);"),
+    "affine_plus_one_ignored": ("if (plus_one) g = 1.0f + g;", "if (plus_one) g = g;"),
+    "affine_bias_of_next_channel": ("const float b = (float)bf16_to_double(bias[c]);",
+                                    "const float b = (float)bf16_to_double(bias[c + 1 < C ? c + 1 : c]);"),
+    "affine_ignores_row_stride": ("const float xf = (float)bf16_to_double(x[t * ld + c]);",
+                                  "const float xf = (float)bf16_to_double(x[t * C + c]);"),
 }
 
 
