@@ -212,6 +212,14 @@ class Ops:
             sc = self.buf("sf", (fb4.fb4_mxfp8_scale_bytes(T, C, 1),), torch.uint8)
             return (lambda: fb4.fb4_quantize_mxfp8(q.ctx, x, T, C, C, None, None, 0, e8, sc, 1)), \
                 T * C * 3.0 + T * (C // B)
+        if name == "affine_plus_quantize":
+            # modulation y = x * (1 + scale_c) + shift_c fused in front of the quantizer
+            gen = torch.Generator(device="cuda").manual_seed(7)
+            sc = (0.5 * torch.randn(C, device="cuda", generator=gen)).to(torch.bfloat16)
+            sh = torch.randn(C, device="cuda", generator=gen).to(torch.bfloat16)
+            self._buf["affine"] = (sc, sh)
+            return (lambda: fb4.fb4_quantize_affine(q.ctx, x, T, C, C, sc, sh, 1, codes, meta)), \
+                algorithmic_bytes(T, C) + 4 * C
         if name == "plain_f32":
             xf = self.buf("x32", (T, C), torch.float32)
             xf.copy_(x)
@@ -279,7 +287,7 @@ class Ops:
         raise KeyError(name)
 
 
-OP_NAMES = ["plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
+OP_NAMES = ["plain", "plain_block16", "plain_f32", "affine_plus_quantize", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
             "dequantize_bf16_plain", "dequantize_bf16_decomposed", "dequantize_f16_plain", "to_mxfp8_tiled_scales",
             "quantize_mxfp8_tiled_scales", "quantize_mxfp8_decomposed_seda"]
 
@@ -426,7 +434,7 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         total, per = time_steps(fn, steps, warm, torch)
         ms = total / steps
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
-                     "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "seda", "decomposed", "decomposed_given_set",
+                     "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "affine_plus_quantize", "seda", "decomposed", "decomposed_given_set",
                                                                          "decomposed_seda", "quantize_mxfp8_tiled_scales",
                                                                          "quantize_mxfp8_decomposed_seda")
                      else "decode"}

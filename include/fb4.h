@@ -115,6 +115,25 @@ int fb4_quantize_f32(fb4_ctx* ctx, const float* x, int64_t T, int64_t C, int64_t
                      uint16_t* meta, void* stream);
 
 /*
+ * A per-channel affine producer fused in front of the quantizer (App. D.2: quantization is fused
+ * with the preceding operation such as LayerNorm; the elementwise tail of a LayerNorm is
+ * y = x * gamma_c + beta_c, the modulation in front of the linear layers of an adaLN block is
+ * y = x * (1 + scale_c) + shift_c):
+ *     y[t][c] = x[t][c] * g_c + bias_c,   g_c = gain_c (gain_plus_one 0) or 1 + gain_c (1),
+ * evaluated in float32 exactly as stated - g_c is the float32 nearest to 1 + gain_c, y the float32
+ * nearest to the exact x * g_c + bias_c (one fused multiply-add) - and quantized from registers as
+ * fb4_quantize_f32 quantizes a float32 tensor; y is never rounded to bfloat16 and never stored.
+ * Plain quantization (no SeDA, no residual pass).  The default configuration with C a multiple of
+ * 64 runs in one TMA-staged pass at 2.56 bytes per element; any other configuration runs in the
+ * generic kernel with the same result.
+ *   x    : device bfloat16 [T][ld_elems]
+ *   gain : device bfloat16 [C];  bias : device bfloat16 [C]   (per channel, shared by all tokens)
+ */
+int fb4_quantize_affine(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems,
+                        const void* gain_bf16, const void* bias_bf16, int gain_plus_one, uint8_t* codes,
+                        uint16_t* meta, void* stream);
+
+/*
  * SeDA-constrained quantization (Sec. 3.4): token t may only use the dialects in
  * cluster_mask[cluster_id[t]] (its cluster's sub-formatbook); cluster_id[t] == -1
  * means unconstrained.  Stage 1 is intersected with the mask; if the intersection

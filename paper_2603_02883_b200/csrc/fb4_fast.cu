@@ -758,6 +758,160 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Per-channel affine producer fused in front of the quantizer (App. D.2: quantization fused with the
+// preceding operation; the elementwise tail of a LayerNorm, or the modulation of an adaLN block):
+// y = x * g_c + bias_c in fp32 (one FMA, g_c = gain_c or 1 + gain_c), quantized from registers with
+// quantize_f32_block; y never reaches HBM.  Same ring, tables and tile shape as the bf16 kernel, but
+// the warps are column-stationary: a warp keeps one tile column (1024 channels) and walks down the
+// rows, so each lane holds the gain and bias of its 32 channels in 32 registers (two bf16 per
+// register) for the whole launch.  Warps beyond a multiple of the number of tile columns stay idle.
+template <bool PLUS_ONE>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
+                           FastParams p, const uint16_t* __restrict__ gain, const uint16_t* __restrict__ bias,
+                           int64_t n_active) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int64_t gwarp = (int64_t)blockIdx.x * kWarps + warp;
+  const int32_t tpr = (int32_t)p.tiles_per_row;
+
+  const uint32_t table_bar = smem_u32(bars + kWarps * kStages);
+  if (threadIdx.x == 0) {
+    for (int i = 0; i <= kWarps * kStages; ++i) mbar_init(smem_u32(bars + i), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
+    bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+  }
+  __syncthreads();
+
+  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytes);
+  const uint32_t my_bars = smem_u32(bars + warp * kStages);
+  // this warp's tiles: column `col`, rows row0, row0 + rstep, ...
+  const int32_t rstep = (int32_t)(n_active / tpr);
+  const int32_t col = (int32_t)(gwarp % tpr);
+  const int64_t row0 = gwarp / tpr;
+  const int32_t n_mine = (gwarp < n_active && row0 < p.T) ? (int32_t)((p.T - row0 + rstep - 1) / rstep) : 0;
+  int64_t pre_row = row0;
+  int32_t it_pre = 0;
+#pragma unroll
+  for (int s = 0; s < kStages; ++s) {
+    if (it_pre < n_mine && lane == 0) {
+      mbar_expect_tx(my_bars + 8 * s, kTileBytes);
+      tma_load_tile(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, col * 16, (int)pre_row);
+    }
+    ++it_pre;
+    pre_row += rstep;
+  }
+  const int64_t nblk = p.C >> 5;
+  const int64_t blk = (int64_t)col * 32 + lane;
+  const bool active = blk < nblk;
+  // gain and bias of this lane's 32 channels: fac[i] = gain bits | bias bits << 16
+  uint32_t fac[32];
+  {
+    uint32_t gw[16], bw[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) gw[k] = bw[k] = 0u;
+    if (active && n_mine > 0) {
+      const uint4* gp = reinterpret_cast<const uint4*>(gain + blk * 32);
+      const uint4* bp = reinterpret_cast<const uint4*>(bias + blk * 32);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 g = __ldg(gp + q), b = __ldg(bp + q);
+        gw[4 * q] = g.x; gw[4 * q + 1] = g.y; gw[4 * q + 2] = g.z; gw[4 * q + 3] = g.w;
+        bw[4 * q] = b.x; bw[4 * q + 1] = b.y; bw[4 * q + 2] = b.z; bw[4 * q + 3] = b.w;
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      fac[2 * k] = (gw[k] & 0xffffu) | (bw[k] << 16);
+      fac[2 * k + 1] = (gw[k] >> 16) | (bw[k] & 0xffff0000u);
+    }
+  }
+  {
+    uint32_t spins = 0;
+    bool ready = mbar_try_wait(table_bar, 0u);
+    while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(table_bar, 0u);
+    if (!__all_sync(0xffffffffu, ready)) {
+      if (lane == 0) atomicOr(p.status, 1u);
+      for (int j = 0; j < kStages && j < n_mine; ++j) {
+        uint32_t tries = 0;
+        while (!mbar_try_wait(my_bars + 8 * j, 0u) && ++tries < kSpinLimit) {}
+      }
+      return;
+    }
+  }
+  const uint32_t pair_base = smem_u32(tb->pairlut);
+  const uint32_t qerr_base = smem_u32(tb->qerr_private) + ((uint32_t)lane & 15u) * 8u;
+  const uint32_t r = (uint32_t)lane >> 1, c0 = ((uint32_t)lane & 1u) * 4u;
+  uint32_t chunk_off[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) chunk_off[j] = r * 128u + (((c0 + j) ^ (r & 7u)) << 4);
+  const int64_t code_row_bytes = p.C >> 1;
+
+  int s = 0;
+  uint32_t parity = 0;
+  int64_t row = row0;
+  for (int32_t it = 0; it < n_mine; ++it) {
+    const uint32_t bar = my_bars + 8 * s;
+    uint32_t spins = 0;
+    bool ready = mbar_try_wait(bar, parity);
+    while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(bar, parity);
+    if (!__all_sync(0xffffffffu, ready)) {
+      if (lane == 0) atomicOr(p.status, 1u);
+      int sj = s;
+      uint32_t pj = parity;
+      for (int j = 1; j < kStages; ++j) {
+        if (it + j >= n_mine) break;
+        if (++sj == kStages) { sj = 0; pj ^= 1u; }
+        uint32_t tries = 0;
+        while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
+      }
+      break;
+    }
+    uint32_t a[32], sg[4];
+    {
+      const uint32_t base = my_ring + s * kTileBytes;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 v = lds_v4(base + chunk_off[q]);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t sq = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xffff0000u) : (w[i >> 1] << 16);
+          const uint32_t f = fac[8 * q + i];
+          float g = __uint_as_float(f << 16);
+          if (PLUS_ONE) g = __fadd_rn(1.0f, g);
+          const uint32_t y = __float_as_uint(__fmaf_rn(__uint_as_float(xb), g, __uint_as_float(f & 0xffff0000u)));
+          a[8 * q + i] = y & 0x7fffffffu;
+          // sign bit 31 -> bit 4i+3 of the code word
+          sq |= (4 * i + 3 == 31) ? (y & 0x80000000u) : ((y >> (28 - 4 * i)) & (8u << (4 * i)));
+        }
+        sg[q] = sq;
+      }
+    }
+    uint32_t cw[4], m;
+    quantize_f32_block<false, false, false>(a, sg, 0xffffffffu, tb, qerr_base, pair_base, 3u, 254u, cw, &m);
+    if (active) {
+      *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      p.meta[row * nblk + blk] = (uint16_t)m;
+    }
+    __syncwarp();
+    if (lane == 0 && it_pre < n_mine) {
+      mbar_expect_tx(bar, kTileBytes);
+      tma_load_tile(my_ring + s * kTileBytes, &tmap, bar, col * 16, (int)pre_row);
+    }
+    ++it_pre;
+    pre_row += rstep;
+    row += rstep;
+    if (++s == kStages) { s = 0; parity ^= 1u; }
+  }
+}
+
 constexpr size_t kSmemBytesF32 =
     1024 + (size_t)kWarpsF32 * kStages * kTileBytesF32 + sizeof(SmemTables) + (kWarpsF32 * kStages + 1) * 8;
 static_assert(kSmemBytesF32 <= 227 * 1024, "shared memory budget of one CTA");
@@ -900,6 +1054,8 @@ cudaError_t fb4_fast_prepare_device() {
   FB4_OPT_IN(true, true, false, false, true);
 #undef FB4_OPT_IN
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true>, attr, bytes);
   return e;
 }
 
@@ -1069,3 +1225,42 @@ cudaError_t fb4_launch_quantize_fast_mx(const fb4_ctx* ctx, const void* x, int64
   if (e == cudaSuccess) *launches = 1;
   return e;
 }
+
+// Affine producer + quantizer in one pass: default configuration only, and at most as many tile
+// columns as the grid has warps (every warp keeps one tile column).
+bool fb4_fast_affine_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const void* gain,
+                              const void* bias) {
+  if (!fb4_fast_mx_eligible(ctx, x, T, C, ld)) return false;
+  if ((reinterpret_cast<uintptr_t>(gain) & 15) || (reinterpret_cast<uintptr_t>(bias) & 15)) return false;
+  return (C + 1023) / 1024 <= (int64_t)ctx->sm_count * kWarps;
+}
+
+cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
+                                            const void* gain, const void* bias, int plus_one, uint8_t* codes,
+                                            uint16_t* meta, cudaStream_t stream) {
+  CUtensorMap map;
+  FastParams p;
+  int grid = 0;
+  const cudaError_t e = fast_setup(ctx, x, T, C, ld, false, &map, &p, &grid);
+  if (e != cudaSuccess) return e;
+  p.codes = codes;
+  p.meta = meta;
+  // column-stationary warps: the largest multiple of the tile columns that the grid's warps cover;
+  // enough CTAs for one warp per (row, tile column) and never fewer than one full set of columns
+  const int64_t tpr = p.tiles_per_row;
+  int64_t want = (p.n_tiles + kWarps - 1) / kWarps;
+  const int64_t min_ctas = (tpr + kWarps - 1) / kWarps;
+  if (want < min_ctas) want = min_ctas;
+  grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
+  const int64_t n_active = ((int64_t)grid * kWarps / tpr) * tpr;
+  if (n_active <= 0) return cudaErrorInvalidValue;
+  const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
+  const uint16_t* g = static_cast<const uint16_t*>(gain);
+  const uint16_t* b = static_cast<const uint16_t*>(bias);
+  if (plus_one)
+    fb4_quantize_affine_kernel<true><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, g, b, n_active);
+  else
+    fb4_quantize_affine_kernel<false><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, g, b, n_active);
+  return cudaGetLastError();
+}
+

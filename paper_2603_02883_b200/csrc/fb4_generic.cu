@@ -116,11 +116,14 @@ __device__ __forceinline__ int64_t salient_row(const Fb4RowExtras& ex, int64_t t
   return -1;
 }
 
-template <int B, int GS, bool F32, bool RESID>
+// MOD 1 / 2: bf16 input goes through the per-channel affine producer first, y = x * g_c + bias_c in
+// fp32 with g_c = gain_c (1) or 1 + gain_c (2), one FMA; the block is quantized from y (App. D.2).
+template <int B, int GS, bool F32, bool RESID, int MOD = 0>
 __global__ void __launch_bounds__(128)
 fb4_quantize_generic_kernel(const void* __restrict__ xin, int64_t T, int64_t C, int64_t ld,
                             const Fb4DeviceTables* __restrict__ tables, GenericParams p, Fb4RowExtras ex,
-                            uint8_t* __restrict__ codes, uint16_t* __restrict__ meta, uint32_t* __restrict__ status) {
+                            uint8_t* __restrict__ codes, uint16_t* __restrict__ meta, uint32_t* __restrict__ status,
+                            const uint16_t* __restrict__ gain = nullptr, const uint16_t* __restrict__ bias = nullptr) {
   __shared__ SmemTables tb;
   {
     const uint32_t* src = reinterpret_cast<const uint32_t*>(tables);
@@ -163,6 +166,17 @@ fb4_quantize_generic_kernel(const void* __restrict__ xin, int64_t T, int64_t C, 
         sgn |= (hi >> 31) << (q * 8 + 2 * j + 1);
       }
     }
+    if (MOD != 0) {
+      sgn = 0;
+#pragma unroll
+      for (int i = 0; i < B; ++i) {
+        const int64_t c = blk * B + i;
+        float g = __uint_as_float((uint32_t)gain[c] << 16);
+        if (MOD == 2) g = __fadd_rn(1.0f, g);
+        xs[i] = __fmaf_rn(xs[i], g, __uint_as_float((uint32_t)bias[c] << 16));
+        sgn |= (__float_as_uint(xs[i]) >> 31) << i;
+      }
+    }
 #pragma unroll
     for (int i = 0; i < B; ++i) ax[i] = fabsf(xs[i]);
     uint32_t allowed = 0xffffffffu;
@@ -202,7 +216,7 @@ fb4_quantize_generic_kernel(const void* __restrict__ xin, int64_t T, int64_t C, 
 
 cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x_is_f32, int64_t T, int64_t C,
                                         int64_t ld, const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
-                                        cudaStream_t stream) {
+                                        cudaStream_t stream, const void* gain, const void* bias, int plus_one) {
   const int B = (int)ctx->cfg.block_size, G = (int)ctx->cfg.num_groups;
   const int64_t total = T * (C / B);
   if (total == 0) return cudaSuccess;
@@ -215,9 +229,17 @@ cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x
 #define FB4_LAUNCH_K(BB, GSZ, F, R) \
   fb4_quantize_generic_kernel<BB, GSZ, F, R><<<grid, threads, 0, stream>>>(x, T, C, ld, ctx->d_tables, p, ex, codes, meta, \
                                                                            ctx->d_status)
+  const uint16_t* g16 = static_cast<const uint16_t*>(gain);
+  const uint16_t* b16 = static_cast<const uint16_t*>(bias);
+  if (gain && (x_is_f32 || resid)) return cudaErrorInvalidValue;
+#define FB4_LAUNCH_MOD(BB, GSZ, M)                                                                       \
+  fb4_quantize_generic_kernel<BB, GSZ, false, false, M><<<grid, threads, 0, stream>>>(x, T, C, ld, ctx->d_tables, p, ex, \
+                                                                                      codes, meta, ctx->d_status, g16, b16)
 #define FB4_LAUNCH(BB, GSZ)                                  \
   do {                                                       \
-    if (x_is_f32) FB4_LAUNCH_K(BB, GSZ, true, false);        \
+    if (gain && plus_one) FB4_LAUNCH_MOD(BB, GSZ, 2);        \
+    else if (gain) FB4_LAUNCH_MOD(BB, GSZ, 1);               \
+    else if (x_is_f32) FB4_LAUNCH_K(BB, GSZ, true, false);   \
     else if (resid) FB4_LAUNCH_K(BB, GSZ, false, true);      \
     else FB4_LAUNCH_K(BB, GSZ, false, false);                \
   } while (0)
@@ -227,6 +249,7 @@ cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x
   else if (B == 16 && G == 16) FB4_LAUNCH(16, 1);
   else return cudaErrorInvalidValue;
 #undef FB4_LAUNCH
+#undef FB4_LAUNCH_MOD
 #undef FB4_LAUNCH_K
   return cudaGetLastError();
 }

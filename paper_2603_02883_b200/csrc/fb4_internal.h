@@ -61,6 +61,11 @@ bool fb4_fast_mx_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t 
 cudaError_t fb4_launch_quantize_fast_mx(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
                                         const Fb4RowExtras& ex, uint8_t* e4m3, uint8_t* scales, uint8_t* res_e4m3,
                                         uint8_t* res_scales, int tiled, cudaStream_t stream, int* launches);
+bool fb4_fast_affine_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const void* gain,
+                              const void* bias);
+cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
+                                            const void* gain, const void* bias, int plus_one, uint8_t* codes,
+                                            uint16_t* meta, cudaStream_t stream);
 bool fb4_fast_f32_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld);
 cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
                                          uint8_t* codes, uint16_t* meta, cudaStream_t stream);
@@ -68,7 +73,8 @@ cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int6
 // generic kernels (any supported config)
 cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x_is_f32, int64_t T, int64_t C,
                                         int64_t ld, const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
-                                        cudaStream_t stream);
+                                        cudaStream_t stream, const void* gain = nullptr, const void* bias = nullptr,
+                                        int plus_one = 0);   // gain/bias: affine producer in front (bf16 input only)
 cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T,
                                   int64_t C, const int32_t* salient_idx, int64_t n_salient,
                                   const uint8_t* res_codes, const uint16_t* res_meta, void* out, int out_dtype,

@@ -21,7 +21,7 @@ ERR_STATIC_LIMIT = -7
 STATIC_MAX_CLUSTERS = 1024
 
 EXPORTS = [
-    "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_seda",
+    "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_affine", "fb4_quantize_seda",
     "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_select_salient_topk", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
     "fb4_quantize_weights", "fb4_quantize_mxfp8", "fb4_quantize_mxfp8_decomposed", "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
     L.fb4_quantize.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.fb4_quantize_f32.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.fb4_quantize_f32.restype = ci
+    L.fb4_quantize_affine.argtypes = [vp, vp, i64, i64, i64, vp, vp, ci, vp, vp, vp]
+    L.fb4_quantize_affine.restype = ci
     L.fb4_quantize_seda.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, vp, vp, vp]
     L.fb4_build_subformatbook.argtypes = [vp, vp, i64, i64, vp, vp, i64, i32, vp, vp, vp]
     L.fb4_build_subformatbook.restype = ci
@@ -172,6 +174,11 @@ def fb4_quantize(ctx, x, T, C, ld_elems, codes, meta, stream=None) -> None:
 def fb4_quantize_f32(ctx, x, T, C, ld_elems, codes, meta, stream=None) -> None:
     _check(lib().fb4_quantize_f32(ctx, _ptr(x), T, C, ld_elems, _ptr(codes), _ptr(meta), _stream(stream)),
            "fb4_quantize_f32")
+
+
+def fb4_quantize_affine(ctx, x, T, C, ld_elems, gain, bias, gain_plus_one, codes, meta, stream=None) -> None:
+    _check(lib().fb4_quantize_affine(ctx, _ptr(x), T, C, ld_elems, _ptr(gain), _ptr(bias), int(bool(gain_plus_one)),
+                                     _ptr(codes), _ptr(meta), _stream(stream)), "fb4_quantize_affine")
 
 
 def fb4_quantize_seda(ctx, x, T, C, ld_elems, cluster_id, cluster_mask, n_clusters, codes, meta, stream=None) -> None:
@@ -336,6 +343,15 @@ class Fb4:
             fb4_quantize(self.ctx, x, T, C, ld, codes, meta)
         else:
             fb4_quantize_seda(self.ctx, x, T, C, ld, cluster_id, cluster_mask, cluster_mask.numel(), codes, meta)
+        return Quantized(codes, meta)
+
+    def quantize_affine(self, x, gain, bias, gain_plus_one: bool = False) -> Quantized:
+        """quantize(x * g + bias) with g = gain or 1 + gain per channel, the affine step evaluated in fp32 inside the kernel"""
+        assert x.dtype == torch.bfloat16 and gain.dtype == torch.bfloat16 and bias.dtype == torch.bfloat16
+        T, C, ld = self._shape(x)
+        assert gain.numel() == C and bias.numel() == C
+        codes, meta = self._outs(T, C)
+        fb4_quantize_affine(self.ctx, x, T, C, ld, gain, bias, gain_plus_one, codes, meta)
         return Quantized(codes, meta)
 
     def quantize_decomposed(self, x, score=None, tile: int = 20, salient_idx=None, cluster_id=None,
