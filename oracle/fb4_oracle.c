@@ -333,18 +333,25 @@ int fb4o_quantize(const uint16_t *x, int64_t T, int64_t C, int64_t ld,
 /*
  * The same quantization for float32 input (a producer handing over its fp32 result, App. D.2
  * fusion with the preceding operation): every value is taken as it is, nothing is rounded to
- * bf16 first.  Plain quantization only.
+ * bf16 first.  Optional SeDA tables as in fb4o_quantize (Sec. 3.4); no residual pass.
  */
 int fb4o_quantize_f32(const float *x, int64_t T, int64_t C, int64_t ld, const fb4o_config *cfg,
-                      const uint8_t *F, const uint32_t *stage1_in, uint8_t *codes, uint16_t *meta) {
+                      const uint8_t *F, const uint32_t *stage1_in,
+                      const int32_t *cluster_id, const uint32_t *cluster_mask, int32_t n_clusters,
+                      uint8_t *codes, uint16_t *meta) {
   if (!config_ok(cfg, C) || T < 0 || ld < C) return -1;
   if (!formatbook_ok(F)) return -2;
   uint32_t stage1[32];
   if (stage1_in) memcpy(stage1, stage1_in, sizeof stage1); else fb4o_default_stage1(F, stage1);
   const int B = cfg->block_size;
   const int64_t nblk = C / B;
+  if (cluster_id)
+    for (int64_t t = 0; t < T; ++t)
+      if (cluster_id[t] >= n_clusters || (cluster_id[t] >= 0 && cluster_mask[cluster_id[t]] == 0)) return -3;
 #pragma omp parallel for schedule(static)
   for (int64_t t = 0; t < T; ++t) {
+    /* Sec. 3.4: the token's sub-formatbook restricts the candidates, whatever the input type */
+    const uint32_t allowed = row_mask(cluster_id, cluster_mask, n_clusters, t);
     for (int64_t blk = 0; blk < nblk; ++blk) {
       double xv[FB4O_MAXB];
       uint8_t sg[FB4O_MAXB], code[FB4O_MAXB];
@@ -354,7 +361,7 @@ int fb4o_quantize_f32(const float *x, int64_t T, int64_t C, int64_t ld, const fb
         sg[i] = (uint8_t)(signbit(f) ? 1 : 0);
       }
       int did, e;
-      quantize_block(xv, sg, cfg, F, stage1, 0xffffffffu, code, &did, &e, NULL);
+      quantize_block(xv, sg, cfg, F, stage1, allowed, code, &did, &e, NULL);
       store_block(code, B, did, e, codes + t * (C / 2), meta + t * nblk, blk);
     }
   }

@@ -78,7 +78,7 @@ def lib():
         L.fb4o_mse.restype = ctypes.c_double
         L.fb4o_quantize_block_f64.argtypes = [vp, ctypes.POINTER(_Cfg), vp, vp, u32, vp, vp, vp, vp]
         L.fb4o_quantize_block_f64.restype = ctypes.c_int
-        L.fb4o_quantize_f32.argtypes = [vp, i64, i64, i64, ctypes.POINTER(_Cfg), vp, vp, vp, vp]
+        L.fb4o_quantize_f32.argtypes = [vp, i64, i64, i64, ctypes.POINTER(_Cfg), vp, vp, vp, vp, i32, vp, vp]
         L.fb4o_quantize_f32.restype = ctypes.c_int
         L.fb4o_affine_f32.argtypes = [vp, i64, i64, i64, vp, vp, ctypes.c_int, vp]
         L.fb4o_affine_f32.restype = ctypes.c_int
@@ -236,15 +236,17 @@ def build_subformatbook(meta, anchor_token, anchor_cluster, n_clusters: int, for
     return out[:n_clusters]
 
 
-def quantize_f32(x, formatbook, cfg: Config = Config(), stage1=None) -> Quantized:
-    """x: float32 [T][C], quantized as it is (no rounding to bf16)."""
+def quantize_f32(x, formatbook, cfg: Config = Config(), stage1=None, cluster_id=None, cluster_mask=None) -> Quantized:
+    """x: float32 [T][C], quantized as it is (no rounding to bf16); optional SeDA tables."""
     xv = np.ascontiguousarray(x, dtype=np.float32)
     T, C = xv.shape
     codes = np.zeros((T, C // 2), dtype=np.uint8)
     meta = np.zeros((T, C // cfg.block_size), dtype=np.uint16)
     ccfg = cfg.c()
+    cid, cm = _c(cluster_id, np.int32), _c(cluster_mask, np.uint32)
     r = lib().fb4o_quantize_f32(_p(xv), T, C, C, ctypes.byref(ccfg), _p(_c(formatbook, np.uint8)),
-                                _p(_c(stage1, np.uint32)), _p(codes), _p(meta))
+                                _p(_c(stage1, np.uint32)), _p(cid), _p(cm), 0 if cm is None else len(cm),
+                                _p(codes), _p(meta))
     if r != 0:
         raise ValueError(f"fb4o_quantize_f32 failed: {r}")
     return Quantized(codes, meta)

@@ -418,6 +418,27 @@ def pin_f32_input(seed=9, n=30):
         xb = synth.bf16_bits_to_f32(bits)
         qa, qb = orc.quantize_f32(xb, FB), orc.quantize(bits, FB)
         assert np.array_equal(qa.codes, qb.codes) and np.array_equal(qa.meta, qb.meta)
+    # SeDA tables restrict the fp32 path exactly as the bf16 path (Sec. 3.4): on bf16-representable values
+    # the two agree with the same masks (the bf16 path's SeDA behaviour is pinned on its own), every
+    # choice lies inside the token's mask, and a one-dialect mask forces that dialect
+    for it in range(10):
+        x = (rng.standard_normal((6, 64)) * np.exp2(rng.integers(-20, 20, size=(6, 1)))).astype(np.float32)
+        bits = synth.f32_to_bf16_bits(x)
+        xb = synth.bf16_bits_to_f32(bits)
+        masks = rng.integers(1, 2 ** 32, size=3, dtype=np.uint64).astype(np.uint32)
+        masks[2] = np.uint32(1) << np.uint32(rng.integers(0, 32))
+        cid = np.array([0, 1, 2, -1, 2, 0], dtype=np.int32)
+        qa = orc.quantize_f32(xb, FB, cluster_id=cid, cluster_mask=masks)
+        qb = orc.quantize(bits, FB, cluster_id=cid, cluster_mask=masks)
+        assert np.array_equal(qa.codes, qb.codes) and np.array_equal(qa.meta, qb.meta)
+        qf = orc.quantize_f32(x, FB, cluster_id=cid, cluster_mask=masks)
+        did = qf.meta >> 8
+        for t in range(6):
+            if cid[t] >= 0:
+                assert all((int(masks[cid[t]]) >> int(d)) & 1 for d in did[t])
+        assert all(int(d) == int(masks[2]).bit_length() - 1 for d in did[2]) and all(int(d) == int(masks[2]).bit_length() - 1 for d in did[4])
+        free = orc.quantize_f32(x, FB)
+        assert np.array_equal(free.meta[3], qf.meta[3]) and np.array_equal(free.codes[3], qf.codes[3])
     # 8.0 sets the scale (e = 3, v = x); 2.4990234375 = 2.5 - 2^-10 lies below the 2|3 boundary of
     # dialect d0..: as fp32 its bin is floor(4.998) = 4, while its bf16 rounding 2.5 has bin 5
     x = np.zeros((1, 32), np.float32)

@@ -78,6 +78,8 @@ MUTANTS = {
                                     "const float b = (float)bf16_to_double(bias[c + 1 < C ? c + 1 : c]);"),
     "affine_ignores_row_stride": ("const float xf = (float)bf16_to_double(x[t * ld + c]);",
                                   "const float xf = (float)bf16_to_double(x[t * C + c]);"),
+    "f32_path_ignores_seda_mask": ("    const uint32_t allowed = row_mask(cluster_id, cluster_mask, n_clusters, t);\n    for (int64_t blk = 0; blk < nblk; ++blk) {\n      double xv[FB4O_MAXB];\n      uint8_t sg[FB4O_MAXB], code[FB4O_MAXB];\n      for (int i = 0; i < B; ++i) {\n        float f",
+                                   "    const uint32_t allowed = 0xffffffffu;\n    for (int64_t blk = 0; blk < nblk; ++blk) {\n      double xv[FB4O_MAXB];\n      uint8_t sg[FB4O_MAXB], code[FB4O_MAXB];\n      for (int i = 0; i < B; ++i) {\n        float f"),
 }
 
 
