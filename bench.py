@@ -218,7 +218,7 @@ class Ops:
             sc = (0.5 * torch.randn(C, device="cuda", generator=gen)).to(torch.bfloat16)
             sh = torch.randn(C, device="cuda", generator=gen).to(torch.bfloat16)
             self._buf["affine"] = (sc, sh)
-            return (lambda: fb4.fb4_quantize_affine(q.ctx, x, T, C, C, sc, sh, 1, codes, meta)), \
+            return (lambda: fb4.fb4_quantize_affine(q.ctx, x, T, C, C, sc, sh, 1, None, None, 0, codes, meta)), \
                 algorithmic_bytes(T, C) + 4 * C
         if name == "plain_f32":
             xf = self.buf("x32", (T, C), torch.float32)

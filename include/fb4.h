@@ -123,15 +123,18 @@ int fb4_quantize_f32(fb4_ctx* ctx, const float* x, int64_t T, int64_t C, int64_t
  * evaluated in float32 exactly as stated - g_c is the float32 nearest to 1 + gain_c, y the float32
  * nearest to the exact x * g_c + bias_c (one fused multiply-add) - and quantized from registers as
  * fb4_quantize_f32 quantizes a float32 tensor; y is never rounded to bfloat16 and never stored.
- * Plain quantization (no SeDA, no residual pass).  The default configuration with C a multiple of
- * 64 runs in one TMA-staged pass at 2.56 bytes per element; any other configuration runs in the
+ * Optional SeDA restriction as in fb4_quantize_seda (Sec. 3.4; the layers the paper applies SeDA to sit
+ * behind such a producer); no residual pass.  The default configuration with C a multiple of 64
+ * runs in one TMA-staged pass at 2.56 bytes per element; any other configuration runs in the
  * generic kernel with the same result.
  *   x    : device bfloat16 [T][ld_elems]
  *   gain : device bfloat16 [C];  bias : device bfloat16 [C]   (per channel, shared by all tokens)
+ *   cluster_id : NULL = unconstrained (then cluster_mask is ignored); else as in fb4_quantize_seda
  */
 int fb4_quantize_affine(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems,
-                        const void* gain_bf16, const void* bias_bf16, int gain_plus_one, uint8_t* codes,
-                        uint16_t* meta, void* stream);
+                        const void* gain_bf16, const void* bias_bf16, int gain_plus_one,
+                        const int32_t* cluster_id, const uint32_t* cluster_mask, int32_t n_clusters,
+                        uint8_t* codes, uint16_t* meta, void* stream);
 
 /*
  * SeDA-constrained quantization (Sec. 3.4): token t may only use the dialects in

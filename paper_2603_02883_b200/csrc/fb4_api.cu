@@ -239,20 +239,25 @@ int fb4_quantize_f32(fb4_ctx* ctx, const float* x, int64_t T, int64_t C, int64_t
 }
 
 int fb4_quantize_affine(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const void* gain,
-                        const void* bias, int gain_plus_one, uint8_t* codes, uint16_t* meta, void* stream) {
+                        const void* bias, int gain_plus_one, const int32_t* cluster_id, const uint32_t* cluster_mask,
+                        int32_t n_clusters, uint8_t* codes, uint16_t* meta, void* stream) {
   const int rc = check_quantize_args(ctx, x, T, C, ld, codes, meta);
   if (rc != FB4_OK) return rc;
   if (gain_plus_one != 0 && gain_plus_one != 1) return FB4_ERR_INVALID_ARG;
   if (T == 0) return FB4_OK;
   if (!gain || !bias) return FB4_ERR_INVALID_ARG;
+  if (cluster_id && (!cluster_mask || n_clusters <= 0)) return FB4_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(gain) & 1u) || (reinterpret_cast<uintptr_t>(bias) & 1u)) return FB4_ERR_ALIGN;
   cudaError_t e;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  Fb4RowExtras ex{};
+  ex.cluster_id = cluster_id;
+  ex.cluster_mask = cluster_id ? cluster_mask : nullptr;
+  ex.n_clusters = cluster_id ? n_clusters : 0;
   if (!ctx->force_generic && fb4_fast_affine_eligible(ctx, x, T, C, ld, gain, bias)) {
-    e = fb4_launch_quantize_fast_affine(ctx, x, T, C, ld, gain, bias, gain_plus_one, codes, meta, st);
+    e = fb4_launch_quantize_fast_affine(ctx, x, T, C, ld, gain, bias, gain_plus_one, ex, codes, meta, st);
     ctx->last_variant = "fast";
   } else {
-    Fb4RowExtras ex{};
     e = fb4_launch_quantize_generic(ctx, x, 0, T, C, ld, ex, codes, meta, st, gain, bias, gain_plus_one);
     ctx->last_variant = "generic";
   }

@@ -766,11 +766,12 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
 // the warps are column-stationary: a warp keeps one tile column (1024 channels) and walks down the
 // rows, so each lane holds the gain and bias of its 32 channels in 32 registers (two bf16 per
 // register) for the whole launch.  Warps beyond a multiple of the number of tile columns stay idle.
-template <bool PLUS_ONE>
+// SEDA: the token's cluster mask restricts the candidates (Sec. 3.4); it is fetched one tile ahead.
+template <bool PLUS_ONE, bool SEDA>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
                            FastParams p, const uint16_t* __restrict__ gain, const uint16_t* __restrict__ bias,
-                           int64_t n_active) {
+                           int64_t n_active, Fb4RowExtras ex) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
@@ -852,10 +853,26 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
   for (int j = 0; j < 4; ++j) chunk_off[j] = r * 128u + (((c0 + j) ^ (r & 7u)) << 4);
   const int64_t code_row_bytes = p.C >> 1;
 
+  // cluster mask of a row; an id outside [-1, n_clusters) counts as -1 and is reported
+  bool bad_cid = false;
+  auto row_mask = [&](int64_t t) -> uint32_t {
+    const int32_t cid = __ldg(ex.cluster_id + t);
+    if ((uint32_t)cid < (uint32_t)ex.n_clusters) {
+      const uint32_t m = __ldg(ex.cluster_mask + cid);
+      return m ? m : 1u;   // a zero mask (precondition violated) yields dialect 0
+    }
+    if (cid != -1) bad_cid = true;
+    return 0xffffffffu;
+  };
+  uint32_t mask_next = 0xffffffffu;
+  if (SEDA && n_mine > 0) mask_next = row_mask(row0);
+
   int s = 0;
   uint32_t parity = 0;
   int64_t row = row0;
   for (int32_t it = 0; it < n_mine; ++it) {
+    const uint32_t allowed = mask_next;
+    if (SEDA && it + 1 < n_mine) mask_next = row_mask(row + rstep);
     const uint32_t bar = my_bars + 8 * s;
     uint32_t spins = 0;
     bool ready = mbar_try_wait(bar, parity);
@@ -895,7 +912,7 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
       }
     }
     uint32_t cw[4], m;
-    quantize_f32_block<false, false, false>(a, sg, 0xffffffffu, tb, qerr_base, pair_base, 3u, 254u, cw, &m);
+    quantize_f32_block<SEDA, false, false>(a, sg, allowed, tb, qerr_base, pair_base, 3u, 254u, cw, &m);
     if (active) {
       *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
       p.meta[row * nblk + blk] = (uint16_t)m;
@@ -910,6 +927,7 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
     row += rstep;
     if (++s == kStages) { s = 0; parity ^= 1u; }
   }
+  if (SEDA && bad_cid && lane == 0) atomicOr(p.status, 2u);
 }
 
 constexpr size_t kSmemBytesF32 =
@@ -1054,8 +1072,10 @@ cudaError_t fb4_fast_prepare_device() {
   FB4_OPT_IN(true, true, false, false, true);
 #undef FB4_OPT_IN
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false>, attr, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, true>, attr, bytes);
   return e;
 }
 
@@ -1236,8 +1256,9 @@ bool fb4_fast_affine_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int6
 }
 
 cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
-                                            const void* gain, const void* bias, int plus_one, uint8_t* codes,
-                                            uint16_t* meta, cudaStream_t stream) {
+                                            const void* gain, const void* bias, int plus_one,
+                                            const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
+                                            cudaStream_t stream) {
   CUtensorMap map;
   FastParams p;
   int grid = 0;
@@ -1257,10 +1278,15 @@ cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, i
   const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
   const uint16_t* g = static_cast<const uint16_t*>(gain);
   const uint16_t* b = static_cast<const uint16_t*>(bias);
-  if (plus_one)
-    fb4_quantize_affine_kernel<true><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, g, b, n_active);
-  else
-    fb4_quantize_affine_kernel<false><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, g, b, n_active);
+#define FB4_AFFINE(P, S) \
+  fb4_quantize_affine_kernel<P, S><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, g, b, n_active, ex)
+  switch ((plus_one ? 1 : 0) | (ex.cluster_id ? 2 : 0)) {
+    case 0: FB4_AFFINE(false, false); break;
+    case 1: FB4_AFFINE(true, false); break;
+    case 2: FB4_AFFINE(false, true); break;
+    default: FB4_AFFINE(true, true); break;
+  }
+#undef FB4_AFFINE
   return cudaGetLastError();
 }
 

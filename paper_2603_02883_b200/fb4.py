@@ -71,7 +71,7 @@ def lib() -> ctypes.CDLL:
     L.fb4_quantize.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.fb4_quantize_f32.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.fb4_quantize_f32.restype = ci
-    L.fb4_quantize_affine.argtypes = [vp, vp, i64, i64, i64, vp, vp, ci, vp, vp, vp]
+    L.fb4_quantize_affine.argtypes = [vp, vp, i64, i64, i64, vp, vp, ci, vp, vp, i32, vp, vp, vp]
     L.fb4_quantize_affine.restype = ci
     L.fb4_quantize_seda.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, vp, vp, vp]
     L.fb4_build_subformatbook.argtypes = [vp, vp, i64, i64, vp, vp, i64, i32, vp, vp, vp]
@@ -176,9 +176,11 @@ def fb4_quantize_f32(ctx, x, T, C, ld_elems, codes, meta, stream=None) -> None:
            "fb4_quantize_f32")
 
 
-def fb4_quantize_affine(ctx, x, T, C, ld_elems, gain, bias, gain_plus_one, codes, meta, stream=None) -> None:
+def fb4_quantize_affine(ctx, x, T, C, ld_elems, gain, bias, gain_plus_one, cluster_id, cluster_mask, n_clusters, codes,
+                        meta, stream=None) -> None:
     _check(lib().fb4_quantize_affine(ctx, _ptr(x), T, C, ld_elems, _ptr(gain), _ptr(bias), int(bool(gain_plus_one)),
-                                     _ptr(codes), _ptr(meta), _stream(stream)), "fb4_quantize_affine")
+                                     _ptr(cluster_id), _ptr(cluster_mask), n_clusters, _ptr(codes), _ptr(meta),
+                                     _stream(stream)), "fb4_quantize_affine")
 
 
 def fb4_quantize_seda(ctx, x, T, C, ld_elems, cluster_id, cluster_mask, n_clusters, codes, meta, stream=None) -> None:
@@ -345,13 +347,14 @@ class Fb4:
             fb4_quantize_seda(self.ctx, x, T, C, ld, cluster_id, cluster_mask, cluster_mask.numel(), codes, meta)
         return Quantized(codes, meta)
 
-    def quantize_affine(self, x, gain, bias, gain_plus_one: bool = False) -> Quantized:
+    def quantize_affine(self, x, gain, bias, gain_plus_one: bool = False, cluster_id=None, cluster_mask=None) -> Quantized:
         """quantize(x * g + bias) with g = gain or 1 + gain per channel, the affine step evaluated in fp32 inside the kernel"""
         assert x.dtype == torch.bfloat16 and gain.dtype == torch.bfloat16 and bias.dtype == torch.bfloat16
         T, C, ld = self._shape(x)
         assert gain.numel() == C and bias.numel() == C
         codes, meta = self._outs(T, C)
-        fb4_quantize_affine(self.ctx, x, T, C, ld, gain, bias, gain_plus_one, codes, meta)
+        fb4_quantize_affine(self.ctx, x, T, C, ld, gain, bias, gain_plus_one, cluster_id, cluster_mask,
+                            0 if cluster_mask is None else cluster_mask.numel(), codes, meta)
         return Quantized(codes, meta)
 
     def quantize_decomposed(self, x, score=None, tile: int = 20, salient_idx=None, cluster_id=None,

@@ -31,16 +31,25 @@ def factors(C, seed, kind):
     return synth.f32_to_bf16_bits(gain.astype(np.float32)), synth.f32_to_bf16_bits(bias.astype(np.float32))
 
 
-def run_case(q, cfg, T, C, ld, kind, plus_one, expect_variant=None):
+def run_case(q, cfg, T, C, ld, kind, plus_one, expect_variant=None, seda=False):
     w = synth.Workload("a", T=T, C=ld, seed=T + C, kind=1, n_outlier=max(1, C // 300), outlier_gain=50.0)
     bits = synth.activation(w)
     view = bits[:, :C]
     gain, bias = factors(C, C + T, kind)
-    ref = orc.quantize_f32(orc.affine_f32(view, gain, bias, plus_one), FB, cfg)
+    cid = masks = d_cid = d_masks = None
+    if seda:
+        rng = np.random.default_rng(T * 7 + C)
+        n_cl = 5
+        cid = rng.integers(-1, n_cl, size=T).astype(np.int32)
+        masks = rng.integers(1, 2 ** 32, size=n_cl, dtype=np.uint64).astype(np.uint32)
+        masks[1] = synth.clusters(synth.Workload("m", T=max(T, 8), C=C, seed=1, kind=1, n_outlier=0, outlier_gain=1.0, seda=True,
+                                                 n_clusters=2, cluster_seed=T))[1][0]      # one dialect per range
+        d_cid, d_masks = torch.from_numpy(cid).cuda(), torch.from_numpy(masks.view(np.int32)).cuda()
+    ref = orc.quantize_f32(orc.affine_f32(view, gain, bias, plus_one), FB, cfg, cluster_id=cid, cluster_mask=masks)
     x = to_dev_bf16(bits)[:, :C]
     got = q.quantize_affine(x, torch.from_numpy(gain.view(np.int16)).cuda().view(torch.bfloat16),
-                            torch.from_numpy(bias.view(np.int16)).cuda().view(torch.bfloat16), plus_one)
-    what = f"T={T} C={C} ld={ld} {kind} plus_one={plus_one} kernel={q.last_variant}"
+                            torch.from_numpy(bias.view(np.int16)).cuda().view(torch.bfloat16), plus_one, d_cid, d_masks)
+    what = f"T={T} C={C} ld={ld} {kind} plus_one={plus_one} seda={seda} kernel={q.last_variant}"
     if expect_variant:
         assert q.last_variant == expect_variant, what
     assert_same_quantized(got, ref, what)
@@ -53,6 +62,7 @@ def test_tma_staged_kernel(T, C, ld, kind, plus_one):
     q = fb4.Fb4()
     try:
         run_case(q, orc.Config(), T, C, ld, kind, plus_one, "fast")
+        run_case(q, orc.Config(), T, C, ld, kind, plus_one, "fast", seda=True)
         assert q.device_status == 0
     finally:
         q.close()
@@ -66,6 +76,7 @@ def test_other_configurations_run_in_the_generic_kernel(cfg, T, C, plus_one):
     q = fb4.Fb4(**cfg)
     try:
         run_case(q, orc.Config(**cfg), T, C, C, "wild" if plus_one else "modulation", plus_one, "generic")
+        run_case(q, orc.Config(**cfg), T, C, C, "modulation", plus_one, "generic", seda=True)
         assert q.device_status == 0
     finally:
         q.close()
@@ -99,16 +110,16 @@ def test_argument_checks():
     out = torch.zeros(4096, dtype=torch.uint8, device="cuda")
     p = lambda t: ctypes.c_void_p(t.data_ptr())
     f = L.fb4_quantize_affine
-    assert f(q.ctx, p(x), 4, 64, 64, p(v), p(v), 0, p(out), p(out), None) == fb4.OK
-    assert f(q.ctx, p(x), 4, 64, 64, None, p(v), 0, p(out), p(out), None) == fb4.ERR_INVALID_ARG
-    assert f(q.ctx, p(x), 4, 64, 64, p(v), p(v), 2, p(out), p(out), None) == fb4.ERR_INVALID_ARG
-    assert f(q.ctx, p(x), 4, 48, 64, p(v), p(v), 0, p(out), p(out), None) == fb4.ERR_SHAPE
-    assert f(q.ctx, p(x), 4, 64, 60, p(v), p(v), 0, p(out), p(out), None) == fb4.ERR_SHAPE
-    assert f(q.ctx, p(x), 4, 64, 64, ctypes.c_void_p(v.data_ptr() + 1), p(v), 0, p(out), p(out), None) == fb4.ERR_ALIGN
-    assert f(q.ctx, None, 0, 64, 64, None, None, 0, None, None, None) == fb4.OK
+    assert f(q.ctx, p(x), 4, 64, 64, p(v), p(v), 0, None, None, 0, p(out), p(out), None) == fb4.OK
+    assert f(q.ctx, p(x), 4, 64, 64, None, p(v), 0, None, None, 0, p(out), p(out), None) == fb4.ERR_INVALID_ARG
+    assert f(q.ctx, p(x), 4, 64, 64, p(v), p(v), 2, None, None, 0, p(out), p(out), None) == fb4.ERR_INVALID_ARG
+    assert f(q.ctx, p(x), 4, 48, 64, p(v), p(v), 0, None, None, 0, p(out), p(out), None) == fb4.ERR_SHAPE
+    assert f(q.ctx, p(x), 4, 64, 60, p(v), p(v), 0, None, None, 0, p(out), p(out), None) == fb4.ERR_SHAPE
+    assert f(q.ctx, p(x), 4, 64, 64, ctypes.c_void_p(v.data_ptr() + 1), p(v), 0, None, None, 0, p(out), p(out), None) == fb4.ERR_ALIGN
+    assert f(q.ctx, None, 0, 64, 64, None, None, 0, None, None, 0, None, None, None) == fb4.OK
     # gain / bias not 16-byte aligned: the generic kernel takes the call
     v2 = torch.zeros(72, dtype=torch.bfloat16, device="cuda")[1:65]
-    assert f(q.ctx, p(x), 4, 64, 64, p(v2), p(v2), 0, p(out), p(out), None) == fb4.OK
+    assert f(q.ctx, p(x), 4, 64, 64, p(v2), p(v2), 0, None, None, 0, p(out), p(out), None) == fb4.OK
     assert q.last_variant == "generic"
     assert q.device_status == 0
     q.close()

@@ -84,8 +84,8 @@ def test_all_entry_points_stay_inside_their_buffers(T, C, B):
             hm.check("meta, strided input")
     vec = torch.randn(C, device="cuda").to(torch.bfloat16)
     ac, am = Guarded(T * C // 2), Guarded(T * (C // B) * 2)
-    fb4.fb4_quantize_affine(q.ctx, x, T, C, C, vec, vec, 1, ac.tensor(torch.uint8, (T, C // 2)),
-                            am.tensor(torch.int16, (T, C // B)))
+    fb4.fb4_quantize_affine(q.ctx, x, T, C, C, vec, vec, 1, cid, cmask, cmask.numel(),
+                            ac.tensor(torch.uint8, (T, C // 2)), am.tensor(torch.int16, (T, C // B)))
     torch.cuda.synchronize()
     ac.check("codes, affine producer")
     am.check("meta, affine producer")
