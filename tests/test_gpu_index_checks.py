@@ -84,3 +84,28 @@ def test_decode_skips_salient_rows_outside_the_tensor(block_size, C):
         assert q.device_status == 2
     finally:
         q.close()
+
+
+@pytest.mark.parametrize("variant", [0, 1])
+def test_affine_entry_checks_cluster_ids_too(variant):
+    T, C = 150, 1024
+    w = _workload(T, C)
+    bits = synth.activation(w)
+    cid, masks = synth.clusters(w)
+    bad = cid.copy()
+    bad[::9] = 77
+    bad[4::13] = -3
+    clean = np.where((bad >= 0) & (bad < len(masks)), bad, -1).astype(np.int32)
+    gain = synth.f32_to_bf16_bits(np.linspace(-0.5, 0.5, C).astype(np.float32))
+    bias = synth.f32_to_bf16_bits(np.linspace(1.0, -1.0, C).astype(np.float32))
+    ref = orc.quantize_f32(orc.affine_f32(bits, gain, bias, True), FB, cluster_id=clean, cluster_mask=masks)
+    q = fb4.Fb4()
+    try:
+        q.set_kernel_variant(variant)
+        dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+        got = q.quantize_affine(to_dev_bf16(bits), dev(gain), dev(bias), True, torch.from_numpy(bad).cuda(),
+                                torch.from_numpy(masks.view(np.int32)).cuda())
+        assert_same_quantized(got, ref, "affine, ids out of range")
+        assert q.device_status == 2
+    finally:
+        q.close()
