@@ -184,6 +184,119 @@ __device__ __forceinline__ int choose_dialect(const float (&gm)[8], float sG, ui
   return select_general(cand, gb, tb);
 }
 
+// One lane's block(s) from 16 registers of two 16-bit values each - bf16 inputs, or any fp32 values cut
+// to their upper 16 bits: the scale exponent, the bins of the 0.5-wide tables and the sign are all
+// fixed by those bits (every bin boundary is a multiple of the cut's granularity), so the cut loses
+// nothing.  Scale, group maxima, dialect selection, LUT quantization; block size 32, or (B16) two
+// blocks of 16; CLAMP: clamped exponent range.  Out: the four code words, and per half the chosen
+// dialect and the biased exponent.
+template <bool SEDA, bool B16, bool CLAMP>
+__device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], uint32_t allowed, const SmemTables* tb,
+                                                      uint32_t qerr_lane, uint32_t pair_base, uint32_t ec_lo,
+                                                      uint32_t ec_hi, uint32_t (&cw)[4], int (&didh)[2],
+                                                      uint32_t (&Ech)[2]) {
+  // ---- magnitudes, group maxima (4 elements = 2 registers), block maximum
+  uint32_t a[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) a[i] = w[i] & 0x7fff7fffu;
+  // per half of the lane's 32 elements (block size 32: both halves belong to one block):
+  // biased exponent, the two bin scales of the Qvalue lookup, the chosen dialect's table address
+  float sHh[2], sLh[2], magich[2];
+  if (!B16) {
+    uint32_t g2[4];   // (group 2q+1 max << 16) | group 2q max
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const uint32_t m0 = __vmaxu2(a[4 * q], a[4 * q + 1]);
+      const uint32_t m1 = __vmaxu2(a[4 * q + 2], a[4 * q + 3]);
+      g2[q] = __vmaxu2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));
+    }
+    const uint32_t mm = __vmaxu2(__vmaxu2(g2[0], g2[1]), __vmaxu2(g2[2], g2[3]));
+    uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
+    // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
+    uint32_t Ec = max(amax16 >> 7, 3u);
+    if (CLAMP) {
+      // clamped exponent range: magnitudes that would normalise to 16 or more saturate at the
+      // largest value of bin 31 (biased exponent Ec, mantissa all ones)
+      Ec = min(max(amax16 >> 7, ec_lo), ec_hi);
+      const uint32_t bound = ((Ec << 7) | 0x7fu) * 0x10001u;
+      amax16 = min(amax16, bound & 0xffffu);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) a[i] = __vminu2(a[i], bound);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) g2[q] = __vminu2(g2[q], bound);
+    }
+    const float s2 = __uint_as_float((257u - Ec) << 23);   // 2^(3-e)
+    const float sG = s2 * 0x1p-21f;                        // bin in the mantissa of 2.0 + x
+    const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax16 << 16), sG, 2.0f)) & 31u;
+    // ---- dialect selection; the upper bf16 of a pair keeps the lower one as extra mantissa bits,
+    // which truncation discards
+    float gm[8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      gm[2 * q] = __uint_as_float(g2[q] << 16);
+      gm[2 * q + 1] = __uint_as_float(g2[q]);
+    }
+    const int did = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
+    Ech[0] = Ech[1] = Ec;
+    sHh[0] = sHh[1] = s2 * 0x1p-25f;                       // bin in the mantissa of 0.125 + x
+    sLh[0] = sLh[1] = s2 * 0x1p-5f;                        // bin in the mantissa of 2^17 + x
+    didh[0] = didh[1] = did;
+  } else {
+    // block size 16: the lane's two halves are two blocks; a group is the two elements of one register
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      uint32_t gx[8];   // group maximum in both halves of the register
+#pragma unroll
+      for (int k = 0; k < 8; ++k) gx[k] = __vmaxu2(a[8 * h + k], __byte_perm(a[8 * h + k], 0u, 0x1032));
+      uint32_t mm = __vmaxu2(__vmaxu2(__vmaxu2(gx[0], gx[1]), __vmaxu2(gx[2], gx[3])),
+                             __vmaxu2(__vmaxu2(gx[4], gx[5]), __vmaxu2(gx[6], gx[7])));
+      uint32_t Ec = max((mm & 0xffffu) >> 7, 3u);
+      if (CLAMP) {
+        Ec = min(max((mm & 0xffffu) >> 7, ec_lo), ec_hi);
+        const uint32_t bound = ((Ec << 7) | 0x7fu) * 0x10001u;
+        mm = __vminu2(mm, bound);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          a[8 * h + k] = __vminu2(a[8 * h + k], bound);
+          gx[k] = __vminu2(gx[k], bound);
+        }
+      }
+      const float s2 = __uint_as_float((257u - Ec) << 23);
+      const float sG = s2 * 0x1p-21f;
+      const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(mm), sG, 2.0f)) & 31u;
+      float gm[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) gm[k] = __uint_as_float(gx[k]);   // the low copy is truncated away
+      Ech[h] = Ec;
+      sHh[h] = s2 * 0x1p-25f;
+      sLh[h] = s2 * 0x1p-5f;
+      didh[h] = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
+    }
+  }
+  // ---- Qvalue: one lookup per element pair.  124*36 + 144 = 9*512, so the exponent fields of
+  // 36*bits(0.125 + ..) + bits(2^17 + ..) cancel mod 2^32 and leave table + 36*bin_hi + bin_lo.
+  magich[0] = __uint_as_float(0x48000000u + pair_base + (uint32_t)didh[0] * kPairStride);
+  magich[1] = B16 ? __uint_as_float(0x48000000u + pair_base + (uint32_t)didh[1] * kPairStride) : magich[0];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int h = B16 ? (q >> 1) : 0;
+    uint32_t b[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t av = a[4 * q + j];
+      const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sHh[h], 0.125f));
+      const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sLh[h], magich[h]));
+      b[j] = lds_u8(th * (uint32_t)kPairMul + tl);
+    }
+    const uint32_t idx = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
+    // sign bits: byte masks by sign replication, then to bit 3 of every nibble
+    const uint32_t sa = prmt(w[4 * q], w[4 * q + 1], 0xfdb9u);
+    const uint32_t sb = prmt(w[4 * q + 2], w[4 * q + 3], 0xfdb9u);
+    const uint32_t ev = __byte_perm(sa, sb, 0x6420), od = __byte_perm(sa, sb, 0x7531);
+    cw[q] = idx | (((ev & 0x0f0f0f0fu) | (od & 0xf0f0f0f0u)) & 0x88888888u);
+  }
+}
+
 // The lane's 32 elements given as fp32 magnitudes (bit patterns, sign cleared) plus their sign bits
 // already at bit 3 of every nibble of the four code words: scale, group maxima, dialect selection
 // and LUT quantization with the same tables as the bf16 path.  One block of 32, or (B16) two blocks
@@ -456,114 +569,14 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
         w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
       }
     }
-    // ---- magnitudes, group maxima (4 elements = 2 registers), block maximum
-    uint32_t a[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) a[i] = w[i] & 0x7fff7fffu;
+    uint32_t cw[4], Ech[2];
+    int didh[2];
     uint32_t allowed = 0xffffffffu;
     if (SEDA) {
       allowed = maskq[0];
       if (allowed == 0) allowed = 1u;   // precondition violated: stay in bounds
     }
-    // per half of the lane's 32 elements (block size 32: both halves belong to one block):
-    // biased exponent, the two bin scales of the Qvalue lookup, the chosen dialect's table address
-    uint32_t Ech[2];
-    float sHh[2], sLh[2], magich[2];
-    int didh[2];
-    if (!B16) {
-      uint32_t g2[4];   // (group 2q+1 max << 16) | group 2q max
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const uint32_t m0 = __vmaxu2(a[4 * q], a[4 * q + 1]);
-        const uint32_t m1 = __vmaxu2(a[4 * q + 2], a[4 * q + 3]);
-        g2[q] = __vmaxu2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));
-      }
-      const uint32_t mm = __vmaxu2(__vmaxu2(g2[0], g2[1]), __vmaxu2(g2[2], g2[3]));
-      uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
-      // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
-      uint32_t Ec = max(amax16 >> 7, 3u);
-      if (CLAMP) {
-        // clamped exponent range: magnitudes that would normalise to 16 or more saturate at the
-        // largest value of bin 31 (biased exponent Ec, mantissa all ones)
-        Ec = min(max(amax16 >> 7, p.ec_lo), p.ec_hi);
-        const uint32_t bound = ((Ec << 7) | 0x7fu) * 0x10001u;
-        amax16 = min(amax16, bound & 0xffffu);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) a[i] = __vminu2(a[i], bound);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) g2[q] = __vminu2(g2[q], bound);
-      }
-      const float s2 = __uint_as_float((257u - Ec) << 23);   // 2^(3-e)
-      const float sG = s2 * 0x1p-21f;                        // bin in the mantissa of 2.0 + x
-      const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax16 << 16), sG, 2.0f)) & 31u;
-      // ---- dialect selection; the upper bf16 of a pair keeps the lower one as extra mantissa bits,
-      // which truncation discards
-      float gm[8];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        gm[2 * q] = __uint_as_float(g2[q] << 16);
-        gm[2 * q + 1] = __uint_as_float(g2[q]);
-      }
-      const int did = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_base);
-      Ech[0] = Ech[1] = Ec;
-      sHh[0] = sHh[1] = s2 * 0x1p-25f;                       // bin in the mantissa of 0.125 + x
-      sLh[0] = sLh[1] = s2 * 0x1p-5f;                        // bin in the mantissa of 2^17 + x
-      didh[0] = didh[1] = did;
-    } else {
-      // block size 16: the lane's two halves are two blocks; a group is the two elements of one register
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        uint32_t gx[8];   // group maximum in both halves of the register
-#pragma unroll
-        for (int k = 0; k < 8; ++k) gx[k] = __vmaxu2(a[8 * h + k], __byte_perm(a[8 * h + k], 0u, 0x1032));
-        uint32_t mm = __vmaxu2(__vmaxu2(__vmaxu2(gx[0], gx[1]), __vmaxu2(gx[2], gx[3])),
-                               __vmaxu2(__vmaxu2(gx[4], gx[5]), __vmaxu2(gx[6], gx[7])));
-        uint32_t Ec = max((mm & 0xffffu) >> 7, 3u);
-        if (CLAMP) {
-          Ec = min(max((mm & 0xffffu) >> 7, p.ec_lo), p.ec_hi);
-          const uint32_t bound = ((Ec << 7) | 0x7fu) * 0x10001u;
-          mm = __vminu2(mm, bound);
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            a[8 * h + k] = __vminu2(a[8 * h + k], bound);
-            gx[k] = __vminu2(gx[k], bound);
-          }
-        }
-        const float s2 = __uint_as_float((257u - Ec) << 23);
-        const float sG = s2 * 0x1p-21f;
-        const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(mm), sG, 2.0f)) & 31u;
-        float gm[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) gm[k] = __uint_as_float(gx[k]);   // the low copy is truncated away
-        Ech[h] = Ec;
-        sHh[h] = s2 * 0x1p-25f;
-        sLh[h] = s2 * 0x1p-5f;
-        didh[h] = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_base);
-      }
-    }
-    // ---- Qvalue: one lookup per element pair.  124*36 + 144 = 9*512, so the exponent fields of
-    // 36*bits(0.125 + ..) + bits(2^17 + ..) cancel mod 2^32 and leave table + 36*bin_hi + bin_lo.
-    magich[0] = __uint_as_float(0x48000000u + pair_base + (uint32_t)didh[0] * kPairStride);
-    magich[1] = B16 ? __uint_as_float(0x48000000u + pair_base + (uint32_t)didh[1] * kPairStride) : magich[0];
-    uint32_t cw[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int h = B16 ? (q >> 1) : 0;
-      uint32_t b[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const uint32_t av = a[4 * q + j];
-        const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sHh[h], 0.125f));
-        const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sLh[h], magich[h]));
-        b[j] = lds_u8(th * (uint32_t)kPairMul + tl);
-      }
-      const uint32_t idx = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
-      // sign bits: byte masks by sign replication, then to bit 3 of every nibble
-      const uint32_t sa = prmt(w[4 * q], w[4 * q + 1], 0xfdb9u);
-      const uint32_t sb = prmt(w[4 * q + 2], w[4 * q + 3], 0xfdb9u);
-      const uint32_t ev = __byte_perm(sa, sb, 0x6420), od = __byte_perm(sa, sb, 0x7531);
-      cw[q] = idx | (((ev & 0x0f0f0f0fu) | (od & 0xf0f0f0f0u)) & 0x88888888u);
-    }
+    quantize_packed_block<SEDA, B16, CLAMP>(w, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, cw, didh, Ech);
     if (MX) {
       // MXFP8 output (block size 32): the codes become e4m3 bytes in registers, the scale byte is the
       // E8M0 scale; 32 contiguous bytes per lane, 1 KB per warp
