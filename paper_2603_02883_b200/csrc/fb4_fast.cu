@@ -297,69 +297,9 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
   }
 }
 
-// The lane's 32 elements given as fp32 magnitudes (bit patterns, sign cleared) plus their sign bits
-// already at bit 3 of every nibble of the four code words: scale, group maxima, dialect selection
-// and LUT quantization with the same tables as the bf16 path.  One block of 32, or (B16) two blocks
-// of 16 with a scale, a selection and a metadata record each; CLAMP: clamped exponent range,
-// magnitudes saturate at the largest value of bin 31.  Writes the code words and the metadata
-// (one record, or two records in one 32-bit word).
-template <bool SEDA, bool B16, bool CLAMP>
-__device__ __forceinline__ void quantize_f32_block(uint32_t (&a)[32], const uint32_t (&sg)[4], uint32_t allowed,
-                                                   const SmemTables* tb, uint32_t qerr_lane, uint32_t pair_base,
-                                                   uint32_t ec_lo, uint32_t ec_hi, uint32_t* rcw, uint32_t* rmeta) {
-  constexpr int NH = B16 ? 2 : 1;      // blocks in the lane's 32 elements
-  constexpr int NE = 32 / NH;          // elements per block
-  constexpr int GS = NE / 8;           // elements per group
-  uint32_t meta = 0;
-#pragma unroll
-  for (int h = 0; h < NH; ++h) {
-    uint32_t gmx[8];
-    uint32_t amax = 0;
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      uint32_t m = a[NE * h + GS * g];
-#pragma unroll
-      for (int i = 1; i < GS; ++i) m = max(m, a[NE * h + GS * g + i]);
-      gmx[g] = m;
-      amax = max(amax, m);
-    }
-    uint32_t Er = max(amax >> 23, 3u);
-    if (CLAMP) {
-      Er = min(max(amax >> 23, ec_lo), ec_hi);
-      const uint32_t bound = (Er << 23) | 0x7fffffu;
-      amax = min(amax, bound);
-#pragma unroll
-      for (int g = 0; g < 8; ++g) gmx[g] = min(gmx[g], bound);
-#pragma unroll
-      for (int i = 0; i < NE; ++i) a[NE * h + i] = min(a[NE * h + i], bound);
-    }
-    const float s2 = __uint_as_float((257u - Er) << 23);   // 2^(3-e)
-    const float sG = s2 * 0x1p-21f, sH = s2 * 0x1p-25f, sL = s2 * 0x1p-5f;
-    const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax), sG, 2.0f)) & 31u;
-    float gm[8];
-#pragma unroll
-    for (int g = 0; g < 8; ++g) gm[g] = __uint_as_float(gmx[g]);
-    const int rdid = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
-    const float magic_lo = __uint_as_float(0x48000000u + pair_base + (uint32_t)rdid * kPairStride);
-#pragma unroll
-    for (int q = (4 / NH) * h; q < (4 / NH) * (h + 1); ++q) {
-      uint32_t idx = 0;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j + 1]), sH, 0.125f));
-        const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(a[8 * q + 2 * j]), sL, magic_lo));
-        idx |= lds_u8(th * (uint32_t)kPairMul + tl) << (8 * j);
-      }
-      rcw[q] = idx | sg[q];
-    }
-    meta |= ((Er - 3u) | ((uint32_t)rdid << 8)) << (16 * h);
-  }
-  *rmeta = meta;
-}
-
 // Residual pass of the lane's block(s) (Sec. 3.3): Delta = x - Q(x) in fp32 (exact for the full
 // exponent range, the correctly rounded difference otherwise), quantized again with the same tables
-// as the main pass; the fp32 magnitudes take the place of the bf16 ones.
+// as the main pass, from the upper 16 bits of every Delta (see quantize_packed_block).
 // w = the 16 input registers (2 bf16 each), cw = the 4 code words, didh / Ech = dialect and biased
 // exponent per half (equal halves for block size 32).
 template <bool SEDA, bool B16, bool CLAMP>
@@ -367,8 +307,7 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
                                                const uint32_t* Ech, uint32_t allowed, const SmemTables* tb,
                                                uint32_t qerr_lane, uint32_t pair_base, uint32_t ec_lo, uint32_t ec_hi,
                                                uint32_t* rcw, uint32_t* rmeta) {
-  uint32_t a[32];      // |Delta| bit patterns
-  uint32_t sg[4];      // sign bits at bit 3 of every nibble
+  uint32_t dw[16];     // Delta cut to its upper 16 bits, two per register like the input
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     const int h = B16 ? (q >> 1) : 0;
@@ -376,24 +315,24 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
     const uint32_t sc2 = fb4dev::scale_bf16x2(Ech[h] - 3u);   // element scale 2^(e-3) as two bf16
     uint32_t xh[4];    // Q(x) of the word's 8 elements, two bf16 per register, signs included
     fb4dev::decode_word(cw[q], dt, sc2, xh);
-    uint32_t sq = 0;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const uint32_t xw = w[4 * q + j];
       const uint32_t d0 = __float_as_uint(__fsub_rn(__uint_as_float(xw << 16), __uint_as_float(xh[j] << 16)));
       const uint32_t d1 =
           __float_as_uint(__fsub_rn(__uint_as_float(xw & 0xffff0000u), __uint_as_float(xh[j] & 0xffff0000u)));
-      a[8 * q + 2 * j] = d0 & 0x7fffffffu;
-      a[8 * q + 2 * j + 1] = d1 & 0x7fffffffu;
-      sq |= (d0 >> (28 - 8 * j)) & (0x8u << (8 * j));
-      sq |= (d1 >> (24 - 8 * j)) & (0x80u << (8 * j));
+      dw[4 * q + j] = __byte_perm(d0, d1, 0x7632);
     }
-    sg[q] = sq;
   }
-  quantize_f32_block<SEDA, B16, CLAMP>(a, sg, allowed, tb, qerr_lane, pair_base, ec_lo, ec_hi, rcw, rmeta);
+  uint32_t rc[4], rE[2];
+  int rd[2];
+  quantize_packed_block<SEDA, B16, CLAMP>(dw, allowed, tb, qerr_lane, pair_base, ec_lo, ec_hi, rc, rd, rE);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) rcw[q] = rc[q];
+  *rmeta = B16 ? (((rE[0] - 3u) | ((uint32_t)rd[0] << 8)) | (((rE[1] - 3u) | ((uint32_t)rd[1] << 8)) << 16))
+               : ((rE[0] - 3u) | ((uint32_t)rd[0] << 8));
 }
 
-// Tile index -> (token row, tile column) without a division per tile: advance by a fixed step.
 struct TilePos {
   int32_t row;         // T < 2^31
   int32_t col;
@@ -652,7 +591,8 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
 // fp32 input (the hook for a producer that still holds its result in fp32): same ring and tables,
 // 8 warps per CTA, tiles of 1024 channels = 4 KB (view [T][C/32][32 floats], box 1 x 32 x 32,
 // 128-byte swizzle: row r of a stage is block r).  Lane i reads its block with eight conflict-free
-// 16-byte shared loads and quantizes it with quantize_f32_block.
+// 16-byte shared loads, keeps the upper 16 bits of every value and quantizes them with
+// quantize_packed_block.
 constexpr int kWarpsF32 = 8;
 constexpr int kTileBytesF32 = 4096;
 
@@ -736,25 +676,22 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
     }
     const int64_t row = cur.row;
     const int64_t blk = (int64_t)cur.col * 32 + lane;
-    uint32_t a[32], sg[4];
+    uint32_t xw[16];   // the upper 16 bits of every value, two per register (all the quantizer needs)
     {
       const uint32_t base = my_ring + s * kTileBytesF32;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const uint4 v0 = lds_v4(base + chunk_off[2 * q]), v1 = lds_v4(base + chunk_off[2 * q + 1]);
-        const uint32_t x[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
-        uint32_t sq = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          a[8 * q + i] = x[i] & 0x7fffffffu;
-          // sign bit 31 -> bit 4i+3 of the code word
-          sq |= (4 * i + 3 == 31) ? (x[i] & 0x80000000u) : ((x[i] >> (28 - 4 * i)) & (8u << (4 * i)));
-        }
-        sg[q] = sq;
+        xw[4 * q] = __byte_perm(v0.x, v0.y, 0x7632);
+        xw[4 * q + 1] = __byte_perm(v0.z, v0.w, 0x7632);
+        xw[4 * q + 2] = __byte_perm(v1.x, v1.y, 0x7632);
+        xw[4 * q + 3] = __byte_perm(v1.z, v1.w, 0x7632);
       }
     }
-    uint32_t cw[4], m;
-    quantize_f32_block<false, false, false>(a, sg, 0xffffffffu, tb, qerr_base, pair_base, 3u, 254u, cw, &m);
+    uint32_t cw[4], Eb[2];
+    int did[2];
+    quantize_packed_block<false, false, false>(xw, 0xffffffffu, tb, qerr_base, pair_base, 3u, 254u, cw, did, Eb);
+    const uint32_t m = (Eb[0] - 3u) | ((uint32_t)did[0] << 8);
     if (blk < nblk) {
       *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
       p.meta[row * nblk + blk] = (uint16_t)m;
@@ -775,7 +712,7 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
 // Per-channel affine producer fused in front of the quantizer (App. D.2: quantization fused with the
 // preceding operation; the elementwise tail of a LayerNorm, or the modulation of an adaLN block):
 // y = x * g_c + bias_c in fp32 (one FMA, g_c = gain_c or 1 + gain_c), quantized from registers with
-// quantize_f32_block; y never reaches HBM.  Same ring, tables and tile shape as the bf16 kernel, but
+// quantize_packed_block (on the upper 16 bits of y); y never reaches HBM.  Same ring, tables and tile shape as the bf16 kernel, but
 // the warps are column-stationary: a warp keeps one tile column (1024 channels) and walks down the
 // rows, so each lane holds the gain and bias of its 32 channels in 32 registers (two bf16 per
 // register) for the whole launch.  Warps beyond a multiple of the number of tile columns stay idle.
@@ -902,30 +839,32 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
       }
       break;
     }
-    uint32_t a[32], sg[4];
+    uint32_t yw[16];   // y cut to its upper 16 bits, two per register
     {
       const uint32_t base = my_ring + s * kTileBytes;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const uint4 v = lds_v4(base + chunk_off[q]);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-        uint32_t sq = 0;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const uint32_t xb = (i & 1) ? (w[i >> 1] & 0xffff0000u) : (w[i >> 1] << 16);
-          const uint32_t f = fac[8 * q + i];
-          float g = __uint_as_float(f << 16);
-          if (PLUS_ONE) g = __fadd_rn(1.0f, g);
-          const uint32_t y = __float_as_uint(__fmaf_rn(__uint_as_float(xb), g, __uint_as_float(f & 0xffff0000u)));
-          a[8 * q + i] = y & 0x7fffffffu;
-          // sign bit 31 -> bit 4i+3 of the code word
-          sq |= (4 * i + 3 == 31) ? (y & 0x80000000u) : ((y >> (28 - 4 * i)) & (8u << (4 * i)));
+        for (int j = 0; j < 4; ++j) {
+          uint32_t y[2];
+#pragma unroll
+          for (int hlf = 0; hlf < 2; ++hlf) {
+            const uint32_t xb = hlf ? (w[j] & 0xffff0000u) : (w[j] << 16);
+            const uint32_t f = fac[8 * q + 2 * j + hlf];
+            float g = __uint_as_float(f << 16);
+            if (PLUS_ONE) g = __fadd_rn(1.0f, g);
+            y[hlf] = __float_as_uint(__fmaf_rn(__uint_as_float(xb), g, __uint_as_float(f & 0xffff0000u)));
+          }
+          yw[4 * q + j] = __byte_perm(y[0], y[1], 0x7632);
         }
-        sg[q] = sq;
       }
     }
-    uint32_t cw[4], m;
-    quantize_f32_block<SEDA, false, false>(a, sg, allowed, tb, qerr_base, pair_base, 3u, 254u, cw, &m);
+    uint32_t cw[4], Eb[2];
+    int did[2];
+    quantize_packed_block<SEDA, false, false>(yw, allowed, tb, qerr_base, pair_base, 3u, 254u, cw, did, Eb);
+    const uint32_t m = (Eb[0] - 3u) | ((uint32_t)did[0] << 8);
     if (active) {
       *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
       p.meta[row * nblk + blk] = (uint16_t)m;
