@@ -212,8 +212,10 @@ int fb4_select_salient(fb4_ctx* ctx, const float* score, int64_t T, int32_t tile
  * sequence, ties to the lowest index, written in ascending token order (the input format of
  * fb4_quantize_decomposed_idx).  Sec. 3.3 selects per tile and App. F argues against a global
  * top-k; this call exists for workloads stated as "the top p % of the tokens by score".
- * One thread block does the work (a few passes over `score`): meant for sequence lengths, not
- * for large arrays.
+ * Sequences of 8192 to 16 Mi tokens run as a few small launches over many thread blocks (a radix
+ * select with histograms in scratch memory of the context, then an ordered write); others as one
+ * thread block.  Calls on one context must not overlap in time (different streams): they share
+ * that scratch.
  *   score       : device float [T] (finite; -0 counts as +0)
  *   salient_idx : device int32 [k] (out), 0 <= k <= T
  */

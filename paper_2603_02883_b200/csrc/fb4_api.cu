@@ -158,6 +158,7 @@ int fb4_init(fb4_ctx** out, int device, const uint8_t* formatbook, const uint32_
   ctx->fast_ok = 0;
   ctx->force_generic = 0;
   ctx->d_status = nullptr;
+  ctx->d_topk_scratch = nullptr;
   for (int i = 0; i < 3; ++i) { ctx->pipe_stream[i] = nullptr; ctx->pipe_event[i] = nullptr; }
   build_tables(ctx->host_tables, fb, stage1_mask);
 
@@ -168,7 +169,9 @@ int fb4_init(fb4_ctx** out, int device, const uint8_t* formatbook, const uint32_
     e = cudaMemcpy(ctx->d_tables, &ctx->host_tables, sizeof(Fb4DeviceTables), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMalloc(&ctx->d_status, sizeof(uint32_t));
   if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, sizeof(uint32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&ctx->d_topk_scratch, fb4_topk_scratch_bytes());
   if (e != cudaSuccess) {
+    if (ctx->d_topk_scratch) cudaFree(ctx->d_topk_scratch);
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->d_tables) cudaFree(ctx->d_tables);
     delete ctx;
@@ -191,6 +194,7 @@ int fb4_destroy(fb4_ctx* ctx) {
     if (ctx->pipe_stream[i]) cudaStreamDestroy(ctx->pipe_stream[i]);
   }
   if (ctx->d_fast_tables) cudaFree(ctx->d_fast_tables);
+  if (ctx->d_topk_scratch) cudaFree(ctx->d_topk_scratch);
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->d_tables) cudaFree(ctx->d_tables);
   delete ctx;
@@ -298,9 +302,15 @@ int fb4_select_salient_topk(fb4_ctx* ctx, const float* score, int64_t T, int64_t
   if (k < 0 || k > T) return FB4_ERR_INVALID_ARG;
   if (T == 0 || k == 0) return FB4_OK;
   if (!score || !salient_idx) return FB4_ERR_INVALID_ARG;
-  cudaError_t e = fb4_launch_select_salient_topk(score, T, k, salient_idx, static_cast<cudaStream_t>(stream));
+  cudaError_t e;
+  int launches = 1;
+  if (!ctx->force_generic && ctx->d_topk_scratch && fb4_topk_multi_eligible(T))
+    e = fb4_launch_select_salient_topk_multi(ctx, score, T, k, salient_idx, static_cast<cudaStream_t>(stream),
+                                             &launches);
+  else
+    e = fb4_launch_select_salient_topk(score, T, k, salient_idx, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return fb4_set_cuda_error(e);
-  ctx->launches += 1;
+  ctx->launches += launches;
   return FB4_OK;
 }
 

@@ -41,6 +41,7 @@ struct fb4_ctx {
   int force_generic;             // fb4_set_kernel_variant(ctx, 1): always take the generic kernel
   int fast_ok;                   // formatbook/stage-1 table fit the fast kernel's packed layout
   int sm_count;
+  void* d_topk_scratch;          // histograms and counters of the multi-CTA top-k selection (fb4_topk.cu)
   uint32_t* d_status;            // device status word (bit 0: a TMA wait ran out of tries; bit 1: an index argument out of range)
   int64_t launches;
   const char* last_variant;
@@ -88,6 +89,10 @@ cudaError_t fb4_launch_quantize_weights(const fb4_ctx* ctx, const void* w, int64
                                         uint8_t* codes, uint16_t* meta, cudaStream_t stream);
 cudaError_t fb4_launch_to_mxfp8(const fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int64_t T, int64_t C,
                                 uint8_t* e4m3, uint8_t* scales, int layout, cudaStream_t stream);
+size_t fb4_topk_scratch_bytes();
+bool fb4_topk_multi_eligible(int64_t T);
+cudaError_t fb4_launch_select_salient_topk_multi(const fb4_ctx* ctx, const float* score, int64_t T, int64_t k,
+                                                 int32_t* salient_idx, cudaStream_t stream, int* launches);
 cudaError_t fb4_launch_select_salient_topk(const float* score, int64_t T, int64_t k, int32_t* salient_idx,
                                            cudaStream_t stream);
 cudaError_t fb4_launch_select_salient(const float* score, int64_t T, int32_t tile, int32_t* salient_idx,

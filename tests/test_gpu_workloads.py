@@ -148,7 +148,8 @@ def test_c3_global_top5_percent_reading(q32, c2_bits):
     assert_same_bits_f32(q32.dequantize(got), orc.dequantize(ref, FB), "c3 global dequant")
 
 
-@pytest.mark.parametrize("T,k", [(1, 1), (7, 0), (7, 7), (1000, 50), (1024, 1), (5000, 4999), (75600, 3780)])
+@pytest.mark.parametrize("T,k", [(1, 1), (7, 0), (7, 7), (1000, 50), (1024, 1), (5000, 4999), (75600, 3780), (8192, 1),
+                                 (8192, 8192), (8193, 4000), (100001, 5000), (300000, 299999), (1 << 20, 52429)])
 def test_topk_selection_with_ties(q32, T, k):
     rng = np.random.default_rng(T + k)
     s = rng.random(T).astype(np.float32)
@@ -160,3 +161,25 @@ def test_topk_selection_with_ties(q32, T, k):
     want = orc.select_salient_topk(s, k) if T <= 5000 else np.sort(np.argsort(-s.astype(np.float64), kind="stable")[:k])
     got = q32.select_salient_topk(torch.from_numpy(s).cuda(), k)
     assert np.array_equal(got.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("variant", [0, 1])      # 0: several launches over many CTAs, 1: one CTA
+def test_topk_degenerate_scores_and_both_kernels(variant):
+    """All scores equal (every key ties at the threshold: the lowest indices win), two values only, and a
+    descending ramp; the many-CTA path and the single-CTA kernel give the same indices."""
+    q = fb4.Fb4()
+    try:
+        q.set_kernel_variant(variant)
+        T = 50000
+        for name, s in (("equal", np.full(T, 0.25, np.float32)),
+                        ("two values", (np.arange(T) % 3 == 0).astype(np.float32)),
+                        ("ramp", np.linspace(1.0, -1.0, T).astype(np.float32)),
+                        ("tiny differences", np.float32(1.0) + np.arange(T, dtype=np.float32) * np.float32(2.0 ** -23))):
+            for k in (1, 2500, T - 1):
+                want = np.sort(np.argsort(-s.astype(np.float64), kind="stable")[:k])
+                got = q.select_salient_topk(torch.from_numpy(s).cuda(), k)
+                assert np.array_equal(got.cpu().numpy(), want), f"{name} k={k}"
+        assert q.device_status == 0
+    finally:
+        q.close()
+
