@@ -220,6 +220,15 @@ class Ops:
             self._buf["affine"] = (sc, sh)
             return (lambda: fb4.fb4_quantize_affine(q.ctx, x, T, C, C, sc, sh, 1, None, None, 0, codes, meta)), \
                 algorithmic_bytes(T, C) + 4 * C
+        if name == "affine_plus_quantize_mxfp8":
+            gen = torch.Generator(device="cuda").manual_seed(7)
+            sc_v = (0.5 * torch.randn(C, device="cuda", generator=gen)).to(torch.bfloat16)
+            sh_v = torch.randn(C, device="cuda", generator=gen).to(torch.bfloat16)
+            self._buf["affine_mx"] = (sc_v, sh_v)
+            e8 = self.buf("e4m3", (T, C), torch.uint8)
+            sf = self.buf("sf", (fb4.fb4_mxfp8_scale_bytes(T, C, 1),), torch.uint8)
+            return (lambda: fb4.fb4_quantize_affine_mxfp8(q.ctx, x, T, C, C, sc_v, sh_v, 1, None, None, 0, e8, sf, 1)), \
+                T * C * 3.0 + T * (C // B) + 4 * C
         if name == "plain_f32":
             xf = self.buf("x32", (T, C), torch.float32)
             xf.copy_(x)
@@ -289,7 +298,7 @@ class Ops:
 
 OP_NAMES = ["plain", "plain_block16", "plain_f32", "affine_plus_quantize", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
             "dequantize_bf16_plain", "dequantize_bf16_decomposed", "dequantize_f16_plain", "to_mxfp8_tiled_scales",
-            "quantize_mxfp8_tiled_scales", "quantize_mxfp8_decomposed_seda"]
+            "quantize_mxfp8_tiled_scales", "quantize_mxfp8_decomposed_seda", "affine_plus_quantize_mxfp8"]
 
 
 def main():
@@ -436,7 +445,7 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
                      "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "affine_plus_quantize", "seda", "decomposed", "decomposed_given_set",
                                                                          "decomposed_seda", "quantize_mxfp8_tiled_scales",
-                                                                         "quantize_mxfp8_decomposed_seda")
+                                                                         "quantize_mxfp8_decomposed_seda", "affine_plus_quantize_mxfp8")
                      else "decode"}
         if name == "dequantize_f32_decomposed":
             ops.drop("out32")

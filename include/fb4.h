@@ -137,6 +137,19 @@ int fb4_quantize_affine(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, 
                         uint8_t* codes, uint16_t* meta, void* stream);
 
 /*
+ * fb4_quantize_affine with the result written as an MXFP8 operand (App. D.2): producer, quantizer
+ * and MXFP8 view in one pass - bf16 in, e4m3 bytes + E8M0 scales out, 3.03 bytes per element, and
+ * neither y nor the 4-bit codes reach memory.  The output equals fb4_to_mxfp8 applied to the output
+ * of fb4_quantize_affine, byte for byte.  Default configuration and C a multiple of 64 only, gain and
+ * bias 16-byte aligned (FB4_ERR_INVALID_ARG / FB4_ERR_SHAPE / FB4_ERR_ALIGN otherwise).
+ *   e4m3, scales, scale_layout : as in fb4_quantize_mxfp8
+ */
+int fb4_quantize_affine_mxfp8(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems,
+                              const void* gain_bf16, const void* bias_bf16, int gain_plus_one,
+                              const int32_t* cluster_id, const uint32_t* cluster_mask, int32_t n_clusters,
+                              uint8_t* e4m3, uint8_t* scales, int scale_layout, void* stream);
+
+/*
  * SeDA-constrained quantization (Sec. 3.4): token t may only use the dialects in
  * cluster_mask[cluster_id[t]] (its cluster's sub-formatbook); cluster_id[t] == -1
  * means unconstrained.  Stage 1 is intersected with the mask; if the intersection

@@ -270,6 +270,33 @@ int fb4_quantize_affine(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64
   return FB4_OK;
 }
 
+int fb4_quantize_affine_mxfp8(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const void* gain,
+                              const void* bias, int gain_plus_one, const int32_t* cluster_id,
+                              const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* e4m3, uint8_t* scales,
+                              int scale_layout, void* stream) {
+  if (!ctx) return FB4_ERR_INVALID_ARG;
+  if (scale_layout != 0 && scale_layout != 1) return FB4_ERR_INVALID_ARG;
+  if (gain_plus_one != 0 && gain_plus_one != 1) return FB4_ERR_INVALID_ARG;
+  if (T < 0 || C <= 0 || C % 64 != 0 || ld < C || T > 0x7fffffffLL) return FB4_ERR_SHAPE;
+  if (T == 0) return FB4_OK;
+  if (!x || !gain || !bias || !e4m3 || !scales) return FB4_ERR_INVALID_ARG;
+  if (cluster_id && (!cluster_mask || n_clusters <= 0)) return FB4_ERR_INVALID_ARG;
+  if (!aligned16(x) || (ld & 7) || (reinterpret_cast<uintptr_t>(e4m3) & 31u) || !aligned16(gain) || !aligned16(bias))
+    return FB4_ERR_ALIGN;
+  if (!fb4_fast_affine_eligible(ctx, x, T, C, ld, gain, bias)) return FB4_ERR_INVALID_ARG;   // default configuration only
+  Fb4RowExtras ex{};
+  ex.cluster_id = cluster_id;
+  ex.cluster_mask = cluster_id ? cluster_mask : nullptr;
+  ex.n_clusters = cluster_id ? n_clusters : 0;
+  const cudaError_t e = fb4_launch_quantize_fast_affine(ctx, x, T, C, ld, gain, bias, gain_plus_one, ex, nullptr,
+                                                        nullptr, static_cast<cudaStream_t>(stream), e4m3, scales,
+                                                        scale_layout);
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
+  ctx->launches += 1;
+  ctx->last_variant = "fast";
+  return FB4_OK;
+}
+
 int fb4_quantize_seda(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const int32_t* cluster_id,
                       const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* codes, uint16_t* meta,
                       void* stream) {

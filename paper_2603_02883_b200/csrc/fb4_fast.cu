@@ -717,7 +717,8 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
 // rows, so each lane holds the gain and bias of its 32 channels in 32 registers (two bf16 per
 // register) for the whole launch.  Warps beyond a multiple of the number of tile columns stay idle.
 // SEDA: the token's cluster mask restricts the candidates (Sec. 3.4); it is fetched one tile ahead.
-template <bool PLUS_ONE, bool SEDA>
+// MX: the result leaves as e4m3 bytes + E8M0 scales (p.e4m3 / p.scales) instead of codes / metadata.
+template <bool PLUS_ONE, bool SEDA, bool MX = false>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
                            FastParams p, const uint16_t* __restrict__ gain, const uint16_t* __restrict__ bias,
@@ -865,7 +866,17 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
     int did[2];
     quantize_packed_block<SEDA, false, false>(yw, allowed, tb, qerr_base, pair_base, 3u, 254u, cw, did, Eb);
     const uint32_t m = (Eb[0] - 3u) | ((uint32_t)did[0] << 8);
-    if (active) {
+    if (MX) {
+      if (active) {
+        const uint2 fb = tb->fb_e4m3[did[0]];
+        uint32_t o[8];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) fb4dev::codes_to_e4m3(cw[q], fb, o[2 * q], o[2 * q + 1]);
+        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p.e4m3 + row * p.C + blk * 32),
+                     "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+        p.scales[fb4dev::mx_scale_offset(row, blk, nblk, p.scale_col_tiles, p.scale_tiled)] = (uint8_t)m;
+      }
+    } else if (active) {
       *reinterpret_cast<uint4*>(p.codes + row * code_row_bytes + blk * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
       p.meta[row * nblk + blk] = (uint16_t)m;
     }
@@ -1028,6 +1039,10 @@ cudaError_t fb4_fast_prepare_device() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, false>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, false, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, false, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, true, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, true, true>, attr, bytes);
   return e;
 }
 
@@ -1210,7 +1225,7 @@ bool fb4_fast_affine_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int6
 cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
                                             const void* gain, const void* bias, int plus_one,
                                             const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
-                                            cudaStream_t stream) {
+                                            cudaStream_t stream, uint8_t* e4m3, uint8_t* scales, int tiled) {
   CUtensorMap map;
   FastParams p;
   int grid = 0;
@@ -1230,13 +1245,29 @@ cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, i
   const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
   const uint16_t* g = static_cast<const uint16_t*>(gain);
   const uint16_t* b = static_cast<const uint16_t*>(bias);
-#define FB4_AFFINE(P, S) \
-  fb4_quantize_affine_kernel<P, S><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, g, b, n_active, ex)
-  switch ((plus_one ? 1 : 0) | (ex.cluster_id ? 2 : 0)) {
-    case 0: FB4_AFFINE(false, false); break;
-    case 1: FB4_AFFINE(true, false); break;
-    case 2: FB4_AFFINE(false, true); break;
-    default: FB4_AFFINE(true, true); break;
+  if (e4m3) {   // MXFP8 output: padding of the tiled scale layout = scale 1, the kernel writes real entries only
+    p.e4m3 = e4m3;
+    p.scales = scales;
+    p.scale_tiled = tiled;
+    const int64_t n_col = C / 32;
+    p.scale_col_tiles = (n_col + 3) / 4;
+    if (tiled && ((T & 127) || (n_col & 3))) {
+      const cudaError_t me =
+          cudaMemsetAsync(scales, 0x7f, (size_t)(((T + 127) / 128) * p.scale_col_tiles * 512), stream);
+      if (me != cudaSuccess) return me;
+    }
+  }
+#define FB4_AFFINE(P, S, M) \
+  fb4_quantize_affine_kernel<P, S, M><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, g, b, n_active, ex)
+  switch ((plus_one ? 1 : 0) | (ex.cluster_id ? 2 : 0) | (e4m3 ? 4 : 0)) {
+    case 0: FB4_AFFINE(false, false, false); break;
+    case 1: FB4_AFFINE(true, false, false); break;
+    case 2: FB4_AFFINE(false, true, false); break;
+    case 3: FB4_AFFINE(true, true, false); break;
+    case 4: FB4_AFFINE(false, false, true); break;
+    case 5: FB4_AFFINE(true, false, true); break;
+    case 6: FB4_AFFINE(false, true, true); break;
+    default: FB4_AFFINE(true, true, true); break;
   }
 #undef FB4_AFFINE
   return cudaGetLastError();

@@ -67,7 +67,8 @@ bool fb4_fast_affine_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int6
 cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
                                             const void* gain, const void* bias, int plus_one,
                                             const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
-                                            cudaStream_t stream);
+                                            cudaStream_t stream, uint8_t* e4m3 = nullptr, uint8_t* scales = nullptr,
+                                            int tiled = 0);   // e4m3 != NULL: MXFP8 output instead of codes / meta
 bool fb4_fast_f32_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld);
 cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
                                          uint8_t* codes, uint16_t* meta, cudaStream_t stream);

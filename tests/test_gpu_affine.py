@@ -123,3 +123,49 @@ def test_argument_checks():
     assert q.last_variant == "generic"
     assert q.device_status == 0
     q.close()
+
+
+@pytest.mark.parametrize("T,C", [(1, 64), (130, 3072), (300, 1024 + 64), (257, 128), (2368 + 5, 2048)])
+@pytest.mark.parametrize("plus_one", [False, True])
+def test_affine_producer_straight_to_mxfp8(T, C, plus_one):
+    """fb4_quantize_affine_mxfp8 = affine producer (oracle, fp32) -> fp32 quantizer (oracle) -> MXFP8 view (oracle),
+    byte for byte, both scale layouts, with and without SeDA."""
+    w = synth.Workload("a", T=T, C=C, seed=T + C, kind=1, n_outlier=max(1, C // 300), outlier_gain=50.0, seda=True,
+                       n_clusters=min(4, T), cluster_seed=3)
+    bits = synth.activation(w)
+    cid, masks = synth.clusters(w)
+    gain, bias = factors(C, T, "modulation" if plus_one else "layernorm")
+    dev = lambda a: torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    y = orc.affine_f32(bits, gain, bias, plus_one)
+    q = fb4.Fb4()
+    try:
+        for seda in (False, True):
+            ref = orc.quantize_f32(y, FB, cluster_id=cid if seda else None, cluster_mask=masks if seda else None)
+            for layout in (0, 1):
+                e_ref, s_ref = orc.to_mxfp8(ref, FB, layout)
+                e4m3, scales = q.quantize_affine_mxfp8(
+                    to_dev_bf16(bits), dev(gain), dev(bias), plus_one, layout,
+                    torch.from_numpy(cid).cuda() if seda else None,
+                    torch.from_numpy(masks.view(np.int32)).cuda() if seda else None)
+                what = f"seda {seda} layout {layout}"
+                assert np.array_equal(e4m3.cpu().numpy(), e_ref), what
+                assert np.array_equal(scales.cpu().numpy(), s_ref), what
+        assert q.device_status == 0
+        # other configurations are refused, not approximated
+        L = fb4.lib()
+        x = to_dev_bf16(bits)
+        g, b = dev(gain), dev(bias)
+        p = lambda t: ctypes.c_void_p(t.data_ptr())
+        out = torch.zeros(T * C + 4096, dtype=torch.uint8, device="cuda")
+        q16 = fb4.Fb4(block_size=16)
+        assert L.fb4_quantize_affine_mxfp8(q16.ctx, p(x), T, C, C, p(g), p(b), 0, None, None, 0, p(out), p(out), 0,
+                                           None) == fb4.ERR_INVALID_ARG
+        q16.close()
+        assert L.fb4_quantize_affine_mxfp8(q.ctx, p(x), T, C, C, p(g), p(b), 0, None, None, 0, p(out), p(out), 2,
+                                           None) == fb4.ERR_INVALID_ARG
+        assert L.fb4_quantize_affine_mxfp8(q.ctx, p(x), T, C, C, p(g), None, 0, None, None, 0, p(out), p(out), 0,
+                                           None) == fb4.ERR_INVALID_ARG
+        assert L.fb4_quantize_affine_mxfp8(q.ctx, p(x), T, 32, C, p(g), p(b), 0, None, None, 0, p(out), p(out), 0,
+                                           None) == fb4.ERR_SHAPE
+    finally:
+        q.close()

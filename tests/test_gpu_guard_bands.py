@@ -102,6 +102,13 @@ def test_all_entry_points_stay_inside_their_buffers(T, C, B):
             torch.cuda.synchronize()
             e8.check(f"e4m3 layout {layout}")
             sc.check(f"scales layout {layout}")
+            if C % 64 == 0 and B == 32:   # producer + quantizer + MXFP8 view in one pass (default configuration only)
+                e8, sc = Guarded(T * C), Guarded(fb4.fb4_mxfp8_scale_bytes(T, C, layout))
+                fb4.fb4_quantize_affine_mxfp8(q.ctx, x, T, C, C, vec, vec, 1, cid, cmask, cmask.numel(), e8.view, sc.view,
+                                              layout)
+                torch.cuda.synchronize()
+                e8.check(f"affine MXFP8, e4m3, layout {layout}")
+                sc.check(f"affine MXFP8, scales, layout {layout}")
             if C % 64 == 0 and B == 32:   # the one-pass form with residual rows (default configuration only)
                 e8, sc = Guarded(T * C), Guarded(fb4.fb4_mxfp8_scale_bytes(T, C, layout))
                 r8, rs = Guarded(ns * C), Guarded(fb4.fb4_mxfp8_scale_bytes(ns, C, layout))
