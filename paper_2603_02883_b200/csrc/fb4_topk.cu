@@ -28,19 +28,33 @@ __device__ __forceinline__ uint32_t score_key(float f) {   // order-preserving; 
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// One histogram update per distinct bin of a warp (scores share their leading bits, and tie groups
+// share all of them: unaggregated, the updates of one address serialize).  All lanes take part.
+__device__ __forceinline__ void warp_hist_add(uint32_t* hist, uint32_t bin, bool counts) {
+  const uint32_t peers = __match_any_sync(0xffffffffu, counts ? bin : 0xffffffffu);
+  if (counts && (threadIdx.x & 31) == (uint32_t)(__ffs((int)peers) - 1)) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+}
+
 __global__ void __launch_bounds__(256)
 topk_hist_hi_kernel(const float* __restrict__ score, int64_t T, uint32_t* __restrict__ hist) {
-  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < T; t += (int64_t)gridDim.x * blockDim.x)
-    atomicAdd(&hist[score_key(__ldg(score + t)) >> 16], 1u);
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  // warp-uniform trip count: the first lane's index decides
+  for (int64_t t0 = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31); t0 < T; t0 += stride) {
+    const int64_t t = t0 + (threadIdx.x & 31);
+    const bool in = t < T;
+    warp_hist_add(hist, in ? score_key(__ldg(score + t)) >> 16 : 0u, in);
+  }
 }
 
 __global__ void __launch_bounds__(256)
 topk_hist_lo_kernel(const float* __restrict__ score, int64_t T, const uint32_t* __restrict__ state,
                     uint32_t* __restrict__ hist) {
   const uint32_t hi = state[0];
-  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < T; t += (int64_t)gridDim.x * blockDim.x) {
-    const uint32_t key = score_key(__ldg(score + t));
-    if ((key >> 16) == hi) atomicAdd(&hist[key & 0xffffu], 1u);
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t t0 = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31); t0 < T; t0 += stride) {
+    const int64_t t = t0 + (threadIdx.x & 31);
+    const uint32_t key = t < T ? score_key(__ldg(score + t)) : 0u;
+    warp_hist_add(hist, key & 0xffffu, t < T && (key >> 16) == hi);
   }
 }
 
