@@ -26,6 +26,9 @@
  *   App. D.2  MXFP8 view: the integer magnitudes 0..15 are exact in FP8 e4m3 and the
  *             power-of-two block scale is an E8M0 scale, so a quantized tensor can be
  *             re-expressed as an MXFP8 operand without any rounding.
+ *   App. D.2  fusion with the preceding operation: the per-channel affine step y = x * g_c +
+ *             bias_c (LayerNorm tail / modulation) in float32 with one rounding, and the
+ *             quantizer on float32 values taken as they are.
  *   Sec. 3.4  SeDA: the candidate set of a token is its cluster's sub-formatbook; a
  *             sub-formatbook is built by counting, over a cluster's anchor tokens, how
  *             often each dialect was chosen in each dynamic-range bucket and keeping
@@ -59,11 +62,11 @@
  * argmin invariant; decomposition never increases any element's error; SeDA
  * choices lie in the mask; per-tile argmax by brute force; sub-formatbooks on
  * hand-counted cases, one dialect per bucket, and a constrained tensor giving
- * back the sub-formatbook it was constrained to.
- * Parity unpinned: the formatbook VALUES (the paper's table is only in Fig. 2a),
- * any worked numeric example (the paper prints none), and the tiled order of the
- * MXFP8 scale bytes against a GEMM that consumes it (pinned only by its stated
- * properties).
+ * back the sub-formatbook it was constrained to; the affine step in exact rationals.
+ * Parity unpinned: the formatbook VALUES (the paper's table is only in Fig. 2a)
+ * and any worked numeric example (the paper prints none).  (The tiled order of the
+ * MXFP8 scale bytes is pinned here only by its stated properties; a GPU test hands
+ * it to a library block-scaled GEMM.)
  */
 #include <math.h>
 #include <stdint.h>
