@@ -535,7 +535,11 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
   if (blocks_per_row > 0x7fffffffLL) return cudaErrorInvalidValue;
   const int64_t total = T * blocks_per_row;
   constexpr int64_t kStep = (int64_t)kDecodeThreads * kDecodeUnroll;
-  const int64_t cap = (int64_t)ctx->sm_count * 8;          // up to 8 CTAs of 256 threads per SM
+  // One step per CTA, no persistent loop: with CTAs dispatched in order the whole GPU works on one
+  // narrow, advancing window of the output, which the memory system takes better than a few hundred
+  // resident CTAs streaming far apart (fp32 output: 0.695 -> 0.646 ms at 75600 x 12288).  The kernels
+  // keep their grid-stride loops for the few shapes whose step count exceeds the grid limit.
+  const int64_t cap = 0x7fffffff;
   const int64_t want = (total + kStep - 1) / kStep;
   const unsigned grid = (unsigned)(want < cap ? want : cap);
   const uint32_t* cw = reinterpret_cast<const uint32_t*>(codes);

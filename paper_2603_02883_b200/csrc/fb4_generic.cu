@@ -223,7 +223,7 @@ cudaError_t fb4_launch_quantize_generic(const fb4_ctx* ctx, const void* x, int x
   GenericParams p{ctx->cfg.exp_min, ctx->cfg.exp_max, ctx->cfg.select_mode == 1 ? 1 : 0};
   const int threads = 128;
   int64_t want = (total + threads - 1) / threads;
-  const int64_t cap = (int64_t)ctx->sm_count * 16;
+  const int64_t cap = 0x7fffffff;   // one block of work per thread, CTAs dispatched in order (see fb4_decode.cu)
   const int grid = (int)(want < cap ? want : cap);
   const bool resid = ex.n_salient > 0;
 #define FB4_LAUNCH_K(BB, GSZ, F, R) \

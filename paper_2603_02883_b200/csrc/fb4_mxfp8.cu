@@ -186,7 +186,7 @@ cudaError_t fb4_launch_to_mxfp8(const fb4_ctx* ctx, const uint8_t* codes, const 
   const int64_t n_col = C / 32, total = T * n_col;
   if (total == 0) return cudaSuccess;
   constexpr int64_t kStep = (int64_t)kThreads * kUnroll;
-  const int64_t want = (total + kStep - 1) / kStep, cap = (int64_t)ctx->sm_count * 8;
+  const int64_t want = (total + kStep - 1) / kStep, cap = 0x7fffffff;   // one step per CTA (see fb4_decode.cu)
   const int a32 = (reinterpret_cast<uintptr_t>(e4m3) & 31u) == 0 ? 1 : 0;
   if (layout == 1 && (reinterpret_cast<uintptr_t>(scales) & 15u) == 0) {
     const int64_t items = ((T + 127) >> 7) * ((n_col + 31) >> 5);
