@@ -142,7 +142,7 @@ struct ResidualRows {
 // CTA finds the first list entry at or after the step's first row; a step whose rows hold no
 // salient token (most of them) runs the plain code, the others look up each unit's row, load the
 // residual codes of salient rows and add.
-template <int OUT_BF16, bool B16, bool RESID>
+template <int OUT_BF16, bool B16, bool RESID, int UNROLL = kDecodeUnroll>
 __global__ void __launch_bounds__(kDecodeThreads, 3)
 fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __restrict__ meta, int64_t total_units,
                           const Fb4DeviceTables* __restrict__ tables, void* __restrict__ out, int out_aligned32,
@@ -155,7 +155,7 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
   const int qp = lane & 3;
   constexpr int RPU = B16 ? 2 : 1;   // metadata records per unit
   constexpr int kWordBytes = OUT_BF16 ? 16 : 32;
-  constexpr int64_t kStep = (int64_t)kDecodeThreads * kDecodeUnroll;
+  constexpr int64_t kStep = (int64_t)kDecodeThreads * UNROLL;
   int64_t base = (int64_t)blockIdx.x * kStep, end = total_units, stride = (int64_t)gridDim.x * kStep;
   int64_t pos = 0;   // RESID: first list entry at or after the current step's first row
   if (RESID && blockIdx.x == 0) {   // entries outside the tensor match no row; they are reported
@@ -169,11 +169,11 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
 
   // m = the metadata records of the lane's whole quad (4 units): after the transpose a lane decodes
   // one word of each of the quad's units and needs the record that covers it
-  uint32_t cw[kDecodeUnroll][4];
-  uint32_t m[kDecodeUnroll][2 * RPU];
+  uint32_t cw[UNROLL][4];
+  uint32_t m[UNROLL][2 * RPU];
   auto load = [&](int64_t base) {
 #pragma unroll
-    for (int u = 0; u < kDecodeUnroll; ++u) {
+    for (int u = 0; u < UNROLL; ++u) {
       const int64_t b = base + u * kDecodeThreads + threadIdx.x;
       const int64_t qb = b & ~3ll;
       cw[u][0] = cw[u][1] = cw[u][2] = cw[u][3] = 0u;
@@ -197,9 +197,9 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
   };
   if (base < end) load(base);
   for (; base < end; base += stride) {
-    uint32_t c[kDecodeUnroll][4], mm[kDecodeUnroll][2 * RPU];
+    uint32_t c[UNROLL][4], mm[UNROLL][2 * RPU];
 #pragma unroll
-    for (int u = 0; u < kDecodeUnroll; ++u) {
+    for (int u = 0; u < UNROLL; ++u) {
 #pragma unroll
       for (int k = 0; k < 2 * RPU; ++k) mm[u][k] = m[u][k];
 #pragma unroll
@@ -236,7 +236,7 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
         // rows load their residual codes and the quad adds the decoded residual.
         const bool more = pos + 1 < rr.n_salient && (int64_t)__ldg(rr.salient_idx + pos + 1) <= row_last;
 #pragma unroll
-        for (int u = 0; u < kDecodeUnroll; ++u) {
+        for (int u = 0; u < UNROLL; ++u) {
           const int64_t b = base + u * kDecodeThreads + threadIdx.x;
           int64_t s = -1;              // residual row of this lane's unit
           uint32_t col = 0;
@@ -300,7 +300,7 @@ fb4_dequantize_b32_kernel(const uint32_t* __restrict__ codes, const uint16_t* __
       }
     }
 #pragma unroll
-    for (int u = 0; u < kDecodeUnroll; ++u) {
+    for (int u = 0; u < UNROLL; ++u) {
       quad_transpose(c[u], lane);
       const int64_t qb = base + u * kDecodeThreads + (threadIdx.x & ~3);   // first unit of this quad
 #pragma unroll
@@ -565,7 +565,14 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
     if (fe == cudaSuccess) *launches = 1;
     return fe;
   }
-  if (B == 32) {
+  if (B == 32 && want < (int64_t)ctx->sm_count * 2) {
+    // small tensor: one unit per thread, so that the few units there are spread over all SMs
+    const unsigned sgrid = (unsigned)((total + kDecodeThreads - 1) / kDecodeThreads);
+#define FB4_CALL(O) \
+  fb4_dequantize_b32_kernel<O, false, false, 1><<<sgrid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32, none)
+    FB4_BY_DTYPE(FB4_CALL);
+#undef FB4_CALL
+  } else if (B == 32) {
 #define FB4_CALL(O) \
   fb4_dequantize_b32_kernel<O, false, false><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32, none)
     FB4_BY_DTYPE(FB4_CALL);
