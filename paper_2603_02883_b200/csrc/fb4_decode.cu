@@ -118,6 +118,8 @@ __device__ __forceinline__ void store_sum_word(uint8_t* dst, const uint32_t* pr,
 // A step of 1024 units then spans at most 5 rows, so most steps hold no salient token and run the
 // plain code; with narrower rows most steps would take the slower branch (at 96 units per row the
 // fused kernel took 85 us against 81 us for the two kernels, fp32 output, and 70 against 49 us, bf16).
+// The 16-bit outputs keep the two kernels at every width: their plain steps are short, the branch
+// with the residual is not (75600 x 12288: bf16 0.396 against 0.402 ms, half 0.402 against 0.427 ms).
 constexpr int64_t kFusedResidualMinUnitsPerRow = 256;
 
 // The residual tensor of salient rows, for the flat decode that adds it in the same pass
@@ -553,14 +555,12 @@ cudaError_t fb4_launch_dequantize(const fb4_ctx* ctx, const uint8_t* codes, cons
     else { CALL(0); }               \
   } while (0)
   ResidualRows none{};
-  if (B == 32 && n_salient > 0 && blocks_per_row >= kFusedResidualMinUnitsPerRow && total < 0xffffffffLL) {
+  if (B == 32 && n_salient > 0 && blocks_per_row >= kFusedResidualMinUnitsPerRow && total < 0xffffffffLL &&
+      out_dtype == 0) {   // fp32 output only: for the 16-bit outputs the two kernels measure faster
     // residual rows added in the same pass: every row is written once
     const ResidualRows rr{salient_idx, n_salient, rw, res_meta, (uint32_t)blocks_per_row,
                           (float)((double)n_salient / (double)T), T, ctx->d_status};
-#define FB4_CALL(O) \
-  fb4_dequantize_b32_kernel<O, false, true><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32, rr)
-    FB4_BY_DTYPE(FB4_CALL);
-#undef FB4_CALL
+    fb4_dequantize_b32_kernel<0, false, true><<<grid, kDecodeThreads, 0, stream>>>(cw, meta, total, tb, out, a32, rr);
     const cudaError_t fe = cudaGetLastError();
     if (fe == cudaSuccess) *launches = 1;
     return fe;

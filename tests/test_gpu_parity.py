@@ -183,7 +183,7 @@ def test_decode_adds_residual_rows_in_the_same_pass(q32, T, C, tile):
         assert_same_quantized(got, ref, "given set")
         before = q32.launch_count
         assert_same_bits_f32(q32.dequantize(got), orc.dequantize(ref, FB), "fp32 decode with residual rows")
-        assert q32.launch_count == before + 1
+        assert q32.launch_count == before + 1          # fp32 output: residual rows inside the one kernel
         for dt, name in ((torch.bfloat16, "bf16"), (torch.float16, "f16")):
             o = q32.dequantize(got, dt)
             assert np.array_equal(o.view(torch.int16).cpu().numpy().view(np.uint16),
