@@ -8,13 +8,15 @@ namespace {
 using fb4dev::decode_word;
 using fb4dev::scale_bf16x2;
 
-__device__ __forceinline__ uint32_t f32_to_bf16_rne(float f) {
-  const uint32_t u = __float_as_uint(f);
-  return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
-}
-
 constexpr int kDecodeThreads = 256;
 constexpr int kDecodeUnroll = 4;          // blocks in flight per thread
+
+// two fp32 -> two bf16 (round to nearest even), low half = a
+__device__ __forceinline__ uint32_t f32x2_to_bf16x2(float a, float b) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(b), "f"(a));
+  return d;
+}
 
 // two fp32 -> two IEEE halves (round to nearest even, overflow to infinity), low half = a
 __device__ __forceinline__ uint32_t f32x2_to_f16x2(float a, float b) {
@@ -97,10 +99,10 @@ __device__ __forceinline__ void store_sum_word(uint8_t* dst, const uint32_t* pr,
   }
   if (OUT_BF16 == 1) {
     uint4 o;
-    o.x = f32_to_bf16_rne(__uint_as_float(v[0])) | (f32_to_bf16_rne(__uint_as_float(v[1])) << 16);
-    o.y = f32_to_bf16_rne(__uint_as_float(v[2])) | (f32_to_bf16_rne(__uint_as_float(v[3])) << 16);
-    o.z = f32_to_bf16_rne(__uint_as_float(v[4])) | (f32_to_bf16_rne(__uint_as_float(v[5])) << 16);
-    o.w = f32_to_bf16_rne(__uint_as_float(v[6])) | (f32_to_bf16_rne(__uint_as_float(v[7])) << 16);
+    o.x = f32x2_to_bf16x2(__uint_as_float(v[0]), __uint_as_float(v[1]));
+    o.y = f32x2_to_bf16x2(__uint_as_float(v[2]), __uint_as_float(v[3]));
+    o.z = f32x2_to_bf16x2(__uint_as_float(v[4]), __uint_as_float(v[5]));
+    o.w = f32x2_to_bf16x2(__uint_as_float(v[6]), __uint_as_float(v[7]));
     *reinterpret_cast<uint4*>(dst) = o;
   } else if (OUT_BF16 == 2) {
     uint4 o;
