@@ -391,7 +391,8 @@ fb4_dequantize_residual_rows_kernel(const uint32_t* __restrict__ codes, const ui
     for (int k = 0; k < WPB; ++k) cw[k] = rcw[k] = 0u;
     int64_t b = -1;   // destination block; -1 = past the end
     if (rb < total) {
-      const int64_t srow = rb / blocks_per_row;
+      // 32-bit division whenever the block index fits (a 64-bit one costs about a hundred instructions)
+      const int64_t srow = total <= 0xffffffffLL ? (int64_t)((uint32_t)rb / blocks_per_row) : rb / blocks_per_row;
       const int64_t row = (int64_t)__ldg(salient_idx + srow);
       if (row >= 0 && row < T) {
         b = row * blocks_per_row + (rb - srow * blocks_per_row);
