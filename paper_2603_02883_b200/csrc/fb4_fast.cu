@@ -375,11 +375,17 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
   const int32_t tpr = (int32_t)p.tiles_per_row;
 
   const uint32_t table_bar = smem_u32(bars + kWarps * kStages);
-  if (threadIdx.x == 0) {
-    for (int i = 0; i <= kWarps * kStages; ++i) mbar_init(smem_u32(bars + i), 1);
+  // every warp initialises its own ring barriers; the first thread also the table barrier, and it
+  // starts the table copy at once (one thread doing all kWarps * kStages + 1 inits in a row used to
+  // hold the whole CTA for most of a microsecond)
+  if (lane == 0) {
+    for (int i = 0; i < kStages; ++i) mbar_init(smem_u32(bars + warp * kStages + i), 1);
+    if (warp == 0) mbar_init(table_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
-    bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+    if (warp == 0) {
+      mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
+      bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+    }
   }
   __syncthreads();
 
@@ -609,11 +615,17 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
   const int32_t tpr = (int32_t)p.tiles_per_row;
 
   const uint32_t table_bar = smem_u32(bars + kWarpsF32 * kStages);
-  if (threadIdx.x == 0) {
-    for (int i = 0; i <= kWarpsF32 * kStages; ++i) mbar_init(smem_u32(bars + i), 1);
+  // every warp initialises its own ring barriers; the first thread also the table barrier, and it
+  // starts the table copy at once (one thread doing all kWarpsF32 * kStages + 1 inits in a row used to
+  // hold the whole CTA for most of a microsecond)
+  if (lane == 0) {
+    for (int i = 0; i < kStages; ++i) mbar_init(smem_u32(bars + warp * kStages + i), 1);
+    if (warp == 0) mbar_init(table_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
-    bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+    if (warp == 0) {
+      mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
+      bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+    }
   }
   __syncthreads();
 
@@ -732,11 +744,17 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
   const int32_t tpr = (int32_t)p.tiles_per_row;
 
   const uint32_t table_bar = smem_u32(bars + kWarps * kStages);
-  if (threadIdx.x == 0) {
-    for (int i = 0; i <= kWarps * kStages; ++i) mbar_init(smem_u32(bars + i), 1);
+  // every warp initialises its own ring barriers; the first thread also the table barrier, and it
+  // starts the table copy at once (one thread doing all kWarps * kStages + 1 inits in a row used to
+  // hold the whole CTA for most of a microsecond)
+  if (lane == 0) {
+    for (int i = 0; i < kStages; ++i) mbar_init(smem_u32(bars + warp * kStages + i), 1);
+    if (warp == 0) mbar_init(table_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
-    bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+    if (warp == 0) {
+      mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
+      bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+    }
   }
   __syncthreads();
 
