@@ -32,7 +32,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this
 # workload, from the ncu capture summarised in profiles/fb4_quantize_fast_c5_plain_dram_bytes.md
 # (1 858 057 472 B read + 502 289 920 B written; set back to None whenever that kernel changes).
-NCU_TRAFFIC_BYTES = 2360810496
+NCU_TRAFFIC_BYTES = 2360395008
 
 
 def algorithmic_bytes(T: int, C: int, B: int = 32, n_res_rows: int = 0, seda: bool = False,
