@@ -508,6 +508,16 @@ def run_variants(ops, args, torch, fb4, synth, peak):
             for _ in range(20):
                 pair()
         tot_g, _ = time_steps(graph.replay, 20, 3, torch)
+        # salient-token selection, both readings, for the two sequence lengths of the workloads
+        sel = {}
+        for T_sel in (32760, 75600):
+            sc_sel = torch.rand(T_sel, device="cuda", generator=torch.Generator(device="cuda").manual_seed(T_sel))
+            out_sel = torch.empty(T_sel, dtype=torch.int32, device="cuda")
+            t_tile, _ = time_steps(lambda: fb4.fb4_select_salient(q.ctx, sc_sel, T_sel, 20, out_sel), 20, 3, torch)
+            t_topk, _ = time_steps(lambda: fb4.fb4_select_salient_topk(q.ctx, sc_sel, T_sel, T_sel // 20, out_sel), 20, 3,
+                                   torch)
+            sel[f"T={T_sel}"] = {"one_per_tile_of_20_us": t_tile / 20 * 1e3, "global_top_5_percent_us": t_topk / 20 * 1e3}
+        res["salient_selection_launched_from_a_stream"] = sel
         res["c1_256x3072_quantize_plus_decode"] = {"us_per_pair_launched_one_by_one": tot / 200 * 1e3,
                                                    "us_per_pair_in_a_cuda_graph": tot_g / (20 * 20) * 1e3}
         # context for that size: a library copy that moves the same number of bytes (half read, half
