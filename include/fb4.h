@@ -367,8 +367,9 @@ int fb4_quantize_host(fb4_ctx* ctx, const void* x_host, int64_t T, int64_t C, vo
 
 /* Kernel choice: 0 (default) = the TMA-staged kernel whenever the call qualifies (num_groups 8,
  * two-stage selection, a formatbook whose stage-1 groups hold at most 8 dialects, C a multiple
- * of 64; either block size, any exponent clamp, every extension), else the generic kernel; 1 = always the generic kernel.  Both produce identical
- * output; this exists for tests and measurements. */
+ * of 64; either block size, any exponent clamp, every extension), else the generic kernel;
+ * 1 = always the generic kernel (and the single-block form of fb4_select_salient_topk).  Both
+ * choices produce identical output; this exists for tests and measurements. */
 int fb4_set_kernel_variant(fb4_ctx* ctx, int variant);
 
 /* Device-side status word of the context, read back with a blocking copy: 0 = fine; bit 0 =
