@@ -435,7 +435,7 @@ def run_variants(ops, args, torch, fb4, synth, peak):
     """The other library paths on the same device, each timed like the headline step."""
     q, w, B = ops.q, ops.w, 32
     res = {}
-    steps, warm = max(3, min(args.steps // 2, 20)), 3
+    steps, warm = max(3, min(args.steps // 2, 20)), 5
     for name in OP_NAMES:
         if name == args.op:
             continue
