@@ -60,7 +60,9 @@
  * round-trips; closed form for the uniform dialect; exact-rational brute force
  * on tiny blocks and on all 65536 bf16 patterns; |E_d - exact error| <= G/4;
  * argmin invariant; decomposition never increases any element's error; SeDA
- * choices lie in the mask; per-tile argmax by brute force; sub-formatbooks on
+ * choices lie in the mask; per-tile argmax by brute force, the last token of the sequence
+ * included; bf16 decode of residual sums against integer round-to-nearest-even (hand-made
+ * ties); the residual under a clamped exponent range in exact rationals; sub-formatbooks on
  * hand-counted cases, one dialect per bucket, and a constrained tensor giving
  * back the sub-formatbook it was constrained to; the affine step in exact rationals.
  * Parity unpinned: the formatbook VALUES (the paper's table is only in Fig. 2a)

@@ -615,6 +615,16 @@ def pin_salient_is_per_tile_argmax(seed=5):
         for k, t0 in enumerate(range(0, T, tile)):
             assert int(idx[k]) == t0 + int(np.argmax(s[t0:t0 + tile]))   # numpy: first maximum
         assert np.all(np.diff(idx) > 0)
+    # the last token of the sequence as the unique maximum of its tile: a full last tile, a ragged one,
+    # and a last tile that holds that token alone
+    for T, tile, want in [(40, 20, [0, 39]), (47, 20, [0, 20, 46]), (41, 20, [0, 20, 40]), (7, 7, [6]), (3, 20, [2])]:
+        s = np.full(T, 0.125, dtype=np.float32)
+        s[T - 1] = 0.875
+        assert [int(i) for i in orc.select_salient(s, tile)] == want
+    # ... and as one of two equal maxima of the ragged last tile: the lower index wins
+    s = np.full(47, 0.125, dtype=np.float32)
+    s[[43, 46]] = 0.875
+    assert [int(i) for i in orc.select_salient(s, 20)] == [0, 20, 43]
 
 
 def pin_salient_topk(seed=12):
@@ -737,6 +747,118 @@ def pin_dequantize_f16(seed=13):
     assert np.isinf(want.view(np.float16)).any() and (want.view(np.float16) == 0).any()
 
 
+def _round_to_bf16_bits(q) -> int:
+    """bf16 bit pattern nearest to the rational q (round to nearest, ties to even), by integer arithmetic.
+    Normal range only (the pins that use it stay inside it)."""
+    sign, a = (1 if q < 0 else 0), abs(Fraction(q))
+    if a == 0:
+        return sign << 15
+    e = floor_log2(a)
+    assert -126 <= e <= 126
+    n = a / Fraction(2) ** (e - 7)                  # in [128, 256): 8 significant bits wanted
+    k = n.numerator // n.denominator
+    rem = n - k
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and k % 2 == 1):
+        k += 1
+    if k == 256:
+        k, e = 128, e + 1
+    return (sign << 15) | ((e + 127) << 7) | (k - 128)
+
+
+def pin_dequantize_bf16_rounds_sums_to_nearest_even(seed=17):
+    """bf16 decode of a salient row = Q(Act) + Q(Delta) rounded to nearest, ties to even.  A decoded FB4
+    value alone has 4 significant bits and is a bf16 number; the sum of two at different scales is not.
+    Expected bits come from the exact rational sum rounded by integer arithmetic written here."""
+    # hand-made: dialect 0 = {0 1 2 3 4 5 6 8}; main = 8 * 2^5 = 256 (index 7, scale byte 132), residual scale
+    # byte 127 = 2^0.  256 + 1 = 257 and 256 + 3 = 259 are exact ties of the 8-bit grid (spacing 2 above 256):
+    # 257 -> 256 (even mantissa), 259 -> 260; 256 + 2 = 258 is representable; 256 - 1 = 255 is representable
+    # (spacing 1 below 256); 256 + 5 = 261 -> tie -> 260; 256 + 6 = 262 stays; -256 - 3 -> -260.
+    assert [int(m) for m in FB[0]] == [0, 1, 2, 3, 4, 5, 6, 8]
+    n = 32
+    main_codes = np.full(n, 7, dtype=np.uint8)
+    res_idx = np.array([1, 3, 2, 1 | 8, 5, 6, 3 | 8, 0] * 4, dtype=np.uint8)
+    main_codes[6::8] = 7 | 8                                     # element 6 of every eight: -256
+    pack = lambda c: (c[0::2] | (c[1::2] << 4)).astype(np.uint8).reshape(1, -1)
+    q = orc.Quantized(pack(main_codes), np.array([[132 | (0 << 8)]], np.uint16),
+                      salient_idx=np.array([0], np.int32), res_codes=pack(res_idx),
+                      res_meta=np.array([[127 | (0 << 8)]], np.uint16))
+    got = orc.dequantize(q, FB, out_dtype="bf16")[0]
+    want_vals = [256, 260, 258, 255, 260, 262, -260, 256]
+    for i in range(n):
+        assert float(synth.bf16_bits_to_f32(got[i:i + 1])[0]) == want_vals[i % 8], (i, hex(int(got[i])))
+    # random codes, metadata and residuals at nearby scales: sums of up to 15 significant bits
+    rng = np.random.default_rng(seed)
+    T, C = 4, 64
+    codes = rng.integers(0, 256, size=(T, C // 2), dtype=np.uint8)
+    did = rng.integers(0, 32, size=(T, 2))
+    sb = rng.integers(100, 150, size=(T, 2))
+    meta = (sb | (did << 8)).astype(np.uint16)
+    sal = np.array([1, 2], np.int32)
+    rcodes = rng.integers(0, 256, size=(2, C // 2), dtype=np.uint8)
+    rdid = rng.integers(0, 32, size=(2, 2))
+    rsb = sb[sal] - rng.integers(5, 12, size=(2, 2))
+    rmeta = (rsb | (rdid << 8)).astype(np.uint16)
+    q = orc.Quantized(codes, meta, salient_idx=sal, res_codes=rcodes, res_meta=rmeta)
+    got = orc.dequantize(q, FB, out_dtype="bf16")
+    inexact = 0
+    for t in range(T):
+        cc = unpack_codes(codes[t])
+        for c in range(C):
+            mag = int(FB[did[t, c // 32], cc[c] & 7]) * Fraction(2) ** (int(sb[t, c // 32]) - 127)
+            val = -mag if cc[c] & 8 else mag
+            if t in (1, 2):
+                s_ = t - 1
+                rc = unpack_codes(rcodes[s_])
+                rmag = int(FB[rdid[s_, c // 32], rc[c] & 7]) * Fraction(2) ** (int(rsb[s_, c // 32]) - 127)
+                val += -rmag if rc[c] & 8 else rmag
+            if val == 0:
+                assert int(got[t, c]) & 0x7FFF == 0
+                continue
+            want = _round_to_bf16_bits(val)
+            assert int(got[t, c]) == want, (t, c, hex(int(got[t, c])), hex(want))
+            inexact += bf16_value(want) != val
+    assert inexact > 30, inexact                                  # the rounding was exercised
+
+
+def pin_decomposition_with_clamped_exponent(seed=18, n=30):
+    """Residual pass under the 5-bit exponent range (e in [-15, 16]): Delta is the difference between the input
+    and the decoded, possibly saturated, value; where that difference needs more than 24 significant bits it
+    is rounded to binary32 first.  Every residual block must equal the block-wise definition on those values,
+    and blocks with a saturated element must occur."""
+    rng = np.random.default_rng(seed)
+    cfg = orc.Config(exp_min=-15, exp_max=16)
+    saturated = rounded = 0
+    for it in range(n):
+        x = np.stack([rand_block_bits(rng, 64, (8, 44) if it % 2 == 0 else (-44, -8), zero_frac=0.05) for _ in range(3)])
+        if it % 3 == 0:
+            x[1, 5] = synth.f32_to_bf16_bits(np.array([1.9921875 * 2.0 ** 50], np.float32))[0]   # 8 bits at 2^50
+        sal = np.array([0, 1, 2], dtype=np.int32)
+        q = orc.quantize(x, FB, cfg, salient_idx=sal)
+        main = orc.dequantize(orc.Quantized(q.codes, q.meta), FB)
+        for t in range(3):
+            for blk in range(2):
+                sl = slice(blk * 32, blk * 32 + 32)
+                e = int(q.meta[t, blk] & 0xFF) - 124
+                assert -15 <= e <= 16
+                delta = []
+                for b, m in zip(x[t, sl], main[t, sl]):
+                    xv = bf16_value(int(b))
+                    assert abs(f32_value(m)) <= 15 * Fraction(2) ** (e - 3)
+                    saturated += abs(xv) >= 16 * Fraction(2) ** (e - 3)
+                    exact = xv - f32_value(m)
+                    r = _round_to_f32(exact)
+                    rounded += r != exact
+                    delta.append(float(r))
+                code, did, re_, _ = orc.quantize_block_f64(np.array(delta), FB, cfg)
+                assert np.array_equal(unpack_codes(q.res_codes[t, blk * 16:(blk + 1) * 16]), code)
+                assert int(q.res_meta[t, blk]) == (re_ + 124) | (did << 8)
+                # the sign of a saturated element's residual is the sign of the element
+                for b, dl in zip(x[t, sl], delta):
+                    if abs(bf16_value(int(b))) >= 16 * Fraction(2) ** (e - 3):
+                        assert (dl < 0) == bool(int(b) >> 15) and dl != 0
+    assert saturated > 100 and rounded > 0
+
+
 def pin_mse():
     x = synth.f32_to_bf16_bits(np.array([[1.0, 2.0, -3.0, 0.5]], np.float32))
     r = np.array([[1.5, 2.0, -1.0, 0.5]], np.float32)
@@ -747,7 +869,8 @@ ALL_PINS = [
     pin_scale_is_floor_log2, pin_exponent_clamp, pin_zero_block, pin_rounding_is_nearest, pin_uniform_dialect_closed_form,
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
     pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_salient_topk, pin_decomposition, pin_residual_uses_the_seda_mask,
-    pin_dequantize_formula, pin_dequantize_f16, pin_mse, pin_f32_input, pin_affine_producer, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
+    pin_dequantize_formula, pin_dequantize_f16, pin_dequantize_bf16_rounds_sums_to_nearest_even,
+    pin_decomposition_with_clamped_exponent, pin_mse, pin_f32_input, pin_affine_producer, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
     pin_subformatbook_hand_counted,
     pin_subformatbook_one_dialect_per_bucket_and_closed_loop,
 ]

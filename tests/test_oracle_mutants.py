@@ -78,6 +78,14 @@ MUTANTS = {
                                     "const float b = (float)bf16_to_double(bias[c + 1 < C ? c + 1 : c]);"),
     "affine_ignores_row_stride": ("const float xf = (float)bf16_to_double(x[t * ld + c]);",
                                   "const float xf = (float)bf16_to_double(x[t * C + c]);"),
+    "bf16_by_truncation": ("u += 0x7fffu + lsb;", "u += 0u * lsb;"),
+    "bf16_ties_away_from_zero": ("u += 0x7fffu + lsb;", "u += 0x8000u + 0u * lsb;"),
+    "bf16_ties_toward_zero": ("u += 0x7fffu + lsb;", "u += 0x7fffu + 0u * lsb;"),
+    "salient_last_token_never_seen": ("int64_t t1 = t0 + tile < T ? t0 + tile : T, arg = t0;",
+                                      "int64_t t1 = t0 + tile < T ? t0 + tile : T - 1, arg = t0;"),
+    "residual_of_clamped_block_uses_unsaturated_value": (
+        "float df = (float)(xv[i] - dequant_value(F, did, e, code[i]));",
+        "float df = (float)(xv[i] - (fabs(xv[i]) >= ldexp(16.0, e - 3) ? xv[i] : dequant_value(F, did, e, code[i])));"),
     "f32_path_ignores_seda_mask": ("    const uint32_t allowed = row_mask(cluster_id, cluster_mask, n_clusters, t);\n    for (int64_t blk = 0; blk < nblk; ++blk) {\n      double xv[FB4O_MAXB];\n      uint8_t sg[FB4O_MAXB], code[FB4O_MAXB];\n      for (int i = 0; i < B; ++i) {\n        float f",
                                    "    const uint32_t allowed = 0xffffffffu;\n    for (int64_t blk = 0; blk < nblk; ++blk) {\n      double xv[FB4O_MAXB];\n      uint8_t sg[FB4O_MAXB], code[FB4O_MAXB];\n      for (int i = 0; i < B; ++i) {\n        float f"),
 }
