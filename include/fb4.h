@@ -79,8 +79,8 @@ void fb4_default_config(fb4_config* cfg);
  *   formatbook  : host, 32*8 bytes, dialect-major; NULL = the built-in stand-in
  *                 table (the paper gives its table only as Fig. 2a).
  *   stage1_mask : host, 32 words; entry k = bit mask of the dialects compared when
- *                 the block maximum falls in bin k = floor(2*vmax) (Sec. 3.2,
- *                 "sub-formatbook based on the block maximum").  NULL = dialects
+ *                 the block maximum falls in bin k = floor(2*vmax) (Sec. 3.2:
+ *                 stage 1 of the two-stage selection).  NULL = dialects
  *                 whose largest magnitude equals max(8, k/2).
  *   cfg         : NULL = defaults.
  * On success *out owns device memory until fb4_destroy().
@@ -105,9 +105,9 @@ int fb4_quantize(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t
                  uint16_t* meta, void* stream);
 
 /*
- * fb4_quantize for float32 input (App. D.2: "Quantization is fused with the preceding operation
- * (e.g., GeLU, LayerNorm) where possible" -- a producer that still holds its result in fp32 hands
- * it over without rounding it to bf16 first).  The values are quantized as they are: the block
+ * fb4_quantize for float32 input (App. D.2 runs the quantizer as the tail of the operation in
+ * front of it, an activation function or a normalisation: a producer that still holds its result
+ * in fp32 hands it over without rounding it to bf16 first).  The values are quantized as they are: the block
  * exponent is the fp32 exponent of the largest magnitude, bins come from the full fp32 mantissa.
  *   x : device float32 [T][ld_elems], finite; 16-byte aligned, ld_elems a multiple of 4
  */
@@ -165,9 +165,9 @@ int fb4_quantize_seda(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, in
                       uint16_t* meta, void* stream);
 
 /*
- * Sub-formatbook construction for SeDA (Sec. 3.4: "bin-count profiling on anchor tokens to
- * measure how often each dialect is selected in each dynamic range ... selecting the most
- * frequent dialect for each dynamic-range bucket").  `meta` is the metadata of a quantization of
+ * Sub-formatbook construction for SeDA (Sec. 3.4: a per-cluster histogram of the dialects chosen
+ * on the anchor tokens, of which every dynamic-range bucket keeps its most frequent member).
+ * `meta` is the metadata of a quantization of
  * the layer's activation (normally unconstrained); anchor a is token anchor_token[a] and belongs
  * to cluster anchor_cluster[a].  For every cluster the dialect ids of all blocks of its anchor
  * tokens are counted; for every dynamic-range bucket (a distinct entry of the context's stage-1
@@ -211,8 +211,8 @@ int fb4_build_subformatbook_static(fb4_ctx* ctx, const uint16_t* meta, int64_t T
                                    int32_t n_clusters, uint32_t* cluster_mask, void* stream);
 
 /*
- * Salient-token selection for activation decomposition (Sec. 3.3: "one salient
- * token per tile ... the highest-scoring token in each tile"): for every tile of
+ * Salient-token selection for activation decomposition (Sec. 3.3: every tile of
+ * tokens contributes its single highest-scoring token): for every tile of
  * `tile` consecutive tokens, the index of the largest score (ties: lowest index).
  *   score       : device float [T] (finite)
  *   salient_idx : device int32 [ceil(T/tile)], ascending on return
@@ -279,8 +279,8 @@ int fb4_dequantize(fb4_ctx* ctx, const uint8_t* codes, const uint16_t* meta, int
                    const uint16_t* res_meta, void* out, int out_dtype, void* stream);
 
 /*
- * Offline weight quantization (Sec. 3.3: weights are "quantized offline, allowing exhaustive
- * dialect selection without runtime approximations"; App. C: "an MSE-based criterion").  Same
+ * Offline weight quantization (Sec. 3.3: weights are known ahead of time, so their dialects can be
+ * searched exhaustively with no approximation; App. C: the criterion is the squared error).  Same
  * format and scale as fb4_quantize, but the dialect of a block is the one with the smallest
  * squared error over ALL its elements among ALL 32 dialects (no groups, no stage 1, no error
  * table), ties to the lowest id.  The errors are summed in double precision in element order.
@@ -291,9 +291,9 @@ int fb4_quantize_weights(fb4_ctx* ctx, const void* w_bf16, int64_t N, int64_t K,
                          uint16_t* meta, void* stream);
 
 /*
- * MXFP8 view of a quantized tensor (App. D.2: FB4's integer magnitudes 0..15 "are exactly
- * representable in FP8 e4m3" and its scaling is power-of-two, so it is "directly compatible with
- * MXFP8 GEMM").  Element -> the e4m3 byte of its signed magnitude; block -> the E8M0 byte of its
+ * MXFP8 view of a quantized tensor (App. D.2: every integer magnitude 0..15 is an e4m3 number and
+ * the block scale is a power of two, so an FB4 tensor is an MXFP8 GEMM operand as it stands).
+ * Element -> the e4m3 byte of its signed magnitude; block -> the E8M0 byte of its
  * element scale 2^(e-3), which is the scale byte of `meta`.  Exact: e4m3 * scale equals the value
  * fb4_dequantize gives.  Block size 32 only (FB4_ERR_INVALID_ARG otherwise); residual tensors
  * (res_codes / res_meta) are converted by a second call.

@@ -40,7 +40,7 @@
  * Readings taken where the paper is silent (the same list is in the design notes):
  *   - rounding ties (v exactly half-way between two magnitudes) go to the LARGER
  *     magnitude: bins are half-open [k/2,(k+1)/2) and a boundary is the left
- *     edge of its bin (Sec. 3.2, "shift-and-truncate");
+ *     edge of its bin (Sec. 3.2: the bin index comes from a shift that drops the low bits);
  *   - dialect ties go to the LOWEST dialect id;
  *   - the exponent is clamped to [exp_min, exp_max]; an all-zero block gets exp_min;
  *   - the sign bit is copied even when the magnitude rounds to 0;
@@ -119,7 +119,7 @@ static int nearest_index(const uint8_t *Fd, double u) {
 }
 
 /* Default stage-1 table: entry k (bin of the block maximum) -> dialects whose
- * largest magnitude is max(8, k/2)  (Sec. 3.2 two-stage; Sec. 3.4 "block maxima 8-15"). */
+ * largest magnitude is max(8, k/2)  (Sec. 3.2 two-stage; Sec. 3.4: one bucket per integer block maximum 8..15). */
 void fb4o_default_stage1(const uint8_t *F, uint32_t *stage1 /*32*/) {
   for (int k = 0; k < 32; ++k) {
     int bucket = k / 2 < 8 ? 8 : k / 2;
@@ -482,8 +482,8 @@ int fb4o_quantize_block_f64(const double *x, const fb4o_config *cfg, const uint8
 }
 
 /*
- * Sub-formatbook construction, Sec. 3.4 ("bin-count profiling on anchor tokens ...
- * selecting the most frequent dialect for each dynamic-range bucket").
+ * Sub-formatbook construction, Sec. 3.4 (a histogram of the dialects chosen on a cluster's anchor
+ * tokens; every dynamic-range bucket keeps its most frequent member).
  * meta [T][nblk] holds the dialect chosen for every block (bits 8-12).  Anchor a is
  * token anchor_token[a] and belongs to cluster anchor_cluster[a].  For every cluster:
  * count how often each dialect occurs in the blocks of its anchor tokens; then, for
@@ -521,9 +521,9 @@ int fb4o_build_subformatbook(const uint16_t *meta, int64_t T, int64_t nblk,
 }
 
 /*
- * MXFP8 view of a quantized tensor (App. D.2: FB4's "normalized integer values (0-15) are exactly
- * representable in FP8 e4m3" and its scaling is power-of-two, hence "directly compatible with
- * MXFP8 GEMM").  Every element becomes the e4m3 byte of its signed integer magnitude
+ * MXFP8 view of a quantized tensor (App. D.2: the integer magnitudes 0..15 are all e4m3 numbers
+ * and the block scale is a power of two, which makes an FB4 tensor an MXFP8 operand without any
+ * rounding).  Every element becomes the e4m3 byte of its signed integer magnitude
  * (sign, 4-bit exponent with bias 7, 3-bit mantissa), every 32-element block gets the E8M0 byte
  * of its element scale 2^(e-3), which is the block's scale byte itself (E8M0 of 2^k is k+127).
  *
@@ -576,9 +576,8 @@ int fb4o_to_mxfp8(const uint8_t *codes, const uint16_t *meta, int64_t T, int64_t
 }
 
 /*
- * Offline weight quantization (Sec. 3.3: weights "can be quantized offline, allowing exhaustive
- * dialect selection without runtime approximations"; App. C: "weight dialect selection and
- * quantization follow an MSE-based criterion").  Per block: the same power-of-two scale as for
+ * Offline weight quantization (Sec. 3.3: weights are available before inference, so every dialect
+ * can be tried on every element; App. C: the squared error decides).  Per block: the same power-of-two scale as for
  * activations; then for EVERY dialect the squared error of rounding every element to its nearest
  * magnitude, summed over the block's elements in index order in double precision (each term
  * (v - m)^2 is exact in double; only the running sum rounds); the dialect with the smallest sum

@@ -1,5 +1,5 @@
-// Offline weight quantization (Sec. 3.3: weights "can be quantized offline, allowing exhaustive
-// dialect selection"; App. C: an MSE-based criterion): for every block the squared error of every
+// Offline weight quantization (Sec. 3.3: exhaustive dialect search ahead of inference; App. C: the
+// squared error is the criterion): for every block the squared error of every
 // one of the 32 dialects over all elements, in double precision and in element order (so that the
 // minimum is decided exactly as the definition's sequential sum decides it), the smallest wins, ties
 // to the lowest id.  One thread per block; not a bandwidth path (about 3 K fp64 operations per block).
