@@ -594,6 +594,334 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
 }
 
 // ---------------------------------------------------------------------------------------------
+// Contiguous tensors (ld == C): the tensor is one run of 32-element units and a tile is a run of
+// consecutive units, whatever token they belong to, so every output address is linear in the unit
+// number and the per-tile bookkeeping of the row / column walk is gone (2-D view [N/64][64] for TMA).
+//  * Calls without a residual pass and with FB4 output: tiles of 4 KB = 64 units, two stages per warp;
+//    lane i owns units 2i and 2i+1 (128 contiguous bytes = row i of the stage under the 128-byte
+//    swizzle, eight conflict-free 16-byte shared loads).  One TMA load, one mbarrier wait, one 32-byte
+//    code store and one 4-byte metadata store per lane serve two blocks.
+//  * Calls with a residual pass or MXFP8 output: tiles of 2 KB = 32 units, four stages, lane i owns
+//    unit i (half a row of the stage) - the register budget of the residual pass, and 32-byte e4m3
+//    stores that cover whole lines, ask for one unit per lane.
+// Token-dependent state (SeDA mask, salient list, tiled scale layout) follows a per-lane
+// (token, unit-in-token) position; C is a multiple of 64, so the units 2i and 2i+1 share their token.
+// The stage loop is unrolled, so stage addresses are immediates.  With block size 16 a unit is two blocks.
+struct FlatParams {
+  uint32_t n_tiles;        // tiles; the last one may reach beyond the tensor (TMA fills zeros, stores are guarded)
+  uint32_t n_units;        // 32-element units in the tensor (even)
+  uint32_t units_row;      // units per token (even)
+  uint32_t step_rows;      // one warp step (units between a warp's consecutive tiles) = step_rows tokens + step_rem units
+  uint32_t step_rem;
+  uint8_t* codes;
+  uint16_t* meta;
+  uint32_t* status;
+  uint32_t ec_lo, ec_hi;
+  uint8_t* e4m3;           // MX: e4m3 bytes and E8M0 scale bytes instead of codes / meta
+  uint8_t* scales;
+  uint8_t* res_e4m3;
+  uint8_t* res_scales;
+  int64_t scale_col_tiles;
+  int32_t scale_tiled;
+};
+
+struct FlatPos {
+  int32_t row;      // token
+  uint32_t rem;     // unit inside the token
+  __device__ __forceinline__ void advance(const FlatParams& p) {
+    row += (int32_t)p.step_rows;
+    rem += p.step_rem;
+    if (rem >= p.units_row) { rem -= p.units_row; ++row; }
+  }
+};
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+// A load that stays where it is written (the compiler may not sink it towards its use): the per-token
+// inputs of the tiles ahead are requested before the wait on the current tile.
+__device__ __forceinline__ uint32_t ldg_early(const void* ptr) {
+  uint32_t v;
+  asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(ptr));
+  return v;
+}
+__device__ __forceinline__ void stg_v8(void* ptr, const uint32_t* o) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(o[0]), "r"(o[1]), "r"(o[2]),
+               "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+}
+
+// units per lane and tile of a flat kernel
+__host__ __device__ constexpr int flat_units(bool decomp, bool mx) { return (decomp || mx) ? 1 : 2; }
+
+template <bool SEDA, bool DECOMP, bool B16, bool CLAMP, bool MX = false>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
+                         FlatParams p, Fb4RowExtras ex) {
+  constexpr int U = flat_units(DECOMP, MX);     // units per lane
+  constexpr int kSt = kStages / U;              // stages per warp: the ring holds 8 KB per warp either way
+  constexpr int kTileB = kTileBytes * U;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // Tile -> warp assignment as in the strided kernel: interleaved over all warps of the grid, or (with a
+  // residual pass) a contiguous range per CTA dealt round-robin to its warps.
+  uint32_t g0, g_end, wstride;
+  if (DECOMP) {
+    const uint32_t per = p.n_tiles / gridDim.x, extra = p.n_tiles % gridDim.x, b = blockIdx.x;
+    const uint32_t t0 = b * per + (b < extra ? b : extra);
+    g0 = t0 + warp;
+    g_end = t0 + per + (b < extra ? 1u : 0u);
+    wstride = kWarps;
+  } else {
+    g0 = blockIdx.x * kWarps + warp;
+    g_end = p.n_tiles;
+    wstride = gridDim.x * kWarps;
+  }
+  const uint32_t table_bar = smem_u32(bars + kWarps * kStages);
+  if (lane == 0) {
+    for (int i = 0; i < kSt; ++i) mbar_init(smem_u32(bars + warp * kStages + i), 1);
+    if (warp == 0) mbar_init(table_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (warp == 0) {
+      mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
+      bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+    }
+  }
+  __syncthreads();
+  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytes);
+  const uint32_t my_bars = smem_u32(bars + warp * kStages);
+  const int32_t n_mine = g0 < g_end ? (int32_t)((g_end - g0 + wstride - 1) / wstride) : 0;
+  int32_t y_pre = (int32_t)(g0 * (16u * U));      // first 128-byte row of the next tile to request
+  const int32_t y_step = (int32_t)(wstride * (16u * U));
+#pragma unroll
+  for (int s = 0; s < kSt; ++s) {
+    if (s < n_mine && lane == 0) {
+      mbar_expect_tx(my_bars + 8 * s, kTileB);
+      tma_load_2d(my_ring + s * kTileB, &tmap, my_bars + 8 * s, 0, y_pre);
+    }
+    y_pre += y_step;
+  }
+  // this lane's first unit of the current tile, and (where a token-dependent input or layout needs it)
+  // the token / unit-in-token it falls in
+  constexpr bool kNeedPos = SEDA || DECOMP || MX;
+  uint32_t unit = g0 * (32u * U) + (uint32_t)(U * lane);
+  const uint32_t unit_step = wstride * (32u * U);
+  FlatPos pos{0, 0};
+  if (kNeedPos) {
+    pos.row = (int32_t)(unit / p.units_row);
+    pos.rem = unit - (uint32_t)pos.row * p.units_row;
+  }
+  // SeDA: the cluster id of a lane's token is fetched three tiles ahead, its mask two tiles ahead.  Where the
+  // value of a mask is first touched was settled by measurement: kernels with a residual pass run close to
+  // their issue limit and must not wait for the mask when it is requested (the zero check waits for the use);
+  // the others have slack there, and holding two more loads in flight across tiles cost them 3 to 5 %.
+  constexpr bool kDeferMask = DECOMP;
+  const bool use_seda = SEDA && ex.cluster_id != nullptr;
+  const uint32_t n_cl = (uint32_t)ex.n_clusters;
+  bool bad_cid = false;
+  auto mask_of = [&](int32_t cid) -> uint32_t {
+    if ((uint32_t)cid < n_cl) {
+      const uint32_t m = ldg_early(ex.cluster_mask + cid);
+      return kDeferMask ? m : (m ? m : 1u);   // a zero mask (precondition violated) yields dialect 0: stay in bounds
+    }
+    if (cid != -1) bad_cid = true;  // outside [-1, n_clusters): unconstrained, reported in bit 1 of the status word
+    return 0xffffffffu;
+  };
+  uint32_t mask_cur = 0xffffffffu, mask_nx = 0xffffffffu;
+  int32_t cid_n2 = -1;
+  FlatPos pos_pf = pos;
+  uint32_t unit_pf = unit;
+  if (SEDA) {
+    if (use_seda) {
+      auto cid_at = [&](int k) -> int32_t { return (k < n_mine && unit_pf < p.n_units) ? (int32_t)ldg_early(ex.cluster_id + pos_pf.row) : -1; };
+      mask_cur = mask_of(cid_at(0));
+      pos_pf.advance(p); unit_pf += unit_step;
+      mask_nx = mask_of(cid_at(1));
+      pos_pf.advance(p); unit_pf += unit_step;
+      cid_n2 = cid_at(2);
+      pos_pf.advance(p); unit_pf += unit_step;
+    }
+  }
+  // salient tokens: an ascending list; a lane's tokens never decrease, so a cursor walks it
+  int64_t list_pos = 0;
+  int32_t list_next = 0x7fffffff;
+  if (DECOMP && n_mine > 0) {
+    int64_t lo = 0, hi = ex.n_salient;
+    while (lo < hi) {
+      const int64_t mid = (lo + hi) >> 1;
+      if (ex.salient_idx[mid] < pos.row) lo = mid + 1; else hi = mid;
+    }
+    list_pos = lo;
+    if (lo < ex.n_salient) list_next = ex.salient_idx[lo];
+  }
+  {
+    uint32_t spins = 0;
+    bool ready = mbar_try_wait(table_bar, 0u);
+    while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(table_bar, 0u);
+    if (!__all_sync(0xffffffffu, ready)) {
+      if (lane == 0) atomicOr(p.status, 1u);
+      for (int j = 0; j < kSt && j < n_mine; ++j) {
+        uint32_t tries = 0;
+        while (!mbar_try_wait(my_bars + 8 * j, 0u) && ++tries < kSpinLimit) {}
+      }
+      return;
+    }
+  }
+  const uint32_t pair_base = smem_u32(tb->pairlut);
+  const uint32_t qerr_base = smem_u32(tb->qerr_private) + ((uint32_t)lane & 15u) * 8u;
+  // this lane's 16-byte chunks in stage 0.  Two units: row `lane` of 128 B, chunk j at position j ^ (lane & 7).
+  // One unit: row lane / 2, chunks (lane & 1) * 4 + j.
+  uint32_t chunk[4 * U];
+#pragma unroll
+  for (int j = 0; j < 4 * U; ++j) {
+    const uint32_t r = U == 2 ? (uint32_t)lane : ((uint32_t)lane >> 1);
+    const uint32_t c = U == 2 ? (uint32_t)j : (((uint32_t)lane & 1u) * 4u + (uint32_t)j);
+    chunk[j] = my_ring + r * 128u + ((c ^ (r & 7u)) << 4);
+  }
+
+  // The stage loop is unrolled (stage addresses become immediates) except with a residual pass, whose
+  // body is too long to be worth several copies (measured: 0.38 ms against 0.39 and 0.42 ms for two and four).
+  constexpr int kUnroll = DECOMP ? 1 : kSt;
+  uint32_t parity = 0;
+  int s_dyn = 0;
+  bool failed = false;
+  for (int32_t it = 0; it < n_mine && !failed; it += kUnroll) {
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int s = kUnroll == kSt ? u : s_dyn;
+      if (it + u < n_mine && !failed) {
+        // ---- SeDA inputs of the tiles ahead
+        uint32_t mask_new = 0xffffffffu;
+        int32_t cid_new = -1;
+        if (SEDA) {
+          if (use_seda) {
+            mask_new = mask_of(cid_n2);
+            if (it + u + 3 < n_mine && unit_pf < p.n_units) cid_new = (int32_t)ldg_early(ex.cluster_id + pos_pf.row);
+            pos_pf.advance(p);
+            unit_pf += unit_step;
+          }
+        }
+        const uint32_t bar = my_bars + 8 * s;
+        uint32_t spins = 0;
+        bool ready = mbar_try_wait(bar, parity);
+        while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(bar, parity);
+        if (!__all_sync(0xffffffffu, ready)) {
+          // A load never arrived: raise the status bit, give the loads still in flight for this warp a
+          // bounded chance to land (so none writes into shared memory after the CTA has gone), stop.
+          if (lane == 0) atomicOr(p.status, 1u);
+          for (int j = 1; j < kSt; ++j) {
+            if (it + u + j >= n_mine) break;
+            const int sj = (s + j) % kSt;
+            const uint32_t pj = (s + j) >= kSt ? (parity ^ 1u) : parity;
+            uint32_t tries = 0;
+            while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
+          }
+          failed = true;
+        } else {
+          const bool active = unit < p.n_units;
+          const uint32_t allowed = SEDA ? (kDeferMask ? (mask_cur ? mask_cur : 1u) : mask_cur) : 0xffffffffu;
+          int64_t srow = -1;
+          if (DECOMP) {
+            while (list_next < pos.row) {
+              ++list_pos;
+              list_next = list_pos < ex.n_salient ? ex.salient_idx[list_pos] : 0x7fffffff;
+            }
+            if (list_next == pos.row && active) srow = list_pos;
+          }
+          uint32_t cw[4 * U], mrec[U];      // per unit: code words, metadata (one record, or two with block size 16)
+          int did0[U];
+#pragma unroll
+          for (int h = 0; h < U; ++h) {
+            uint32_t w[16];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint4 v = lds_v4(chunk[4 * h + j] + s * kTileB);
+              w[4 * j] = v.x; w[4 * j + 1] = v.y; w[4 * j + 2] = v.z; w[4 * j + 3] = v.w;
+            }
+            uint32_t c4[4], Ech[2];
+            int didh[2];
+            quantize_packed_block<SEDA, B16, CLAMP>(w, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, c4, didh, Ech);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) cw[4 * h + q] = c4[q];
+            did0[h] = didh[0];
+            mrec[h] = B16 ? (((Ech[0] - 3u) | ((uint32_t)didh[0] << 8)) | (((Ech[1] - 3u) | ((uint32_t)didh[1] << 8)) << 16))
+                          : ((Ech[0] - 3u) | ((uint32_t)didh[0] << 8));
+            if (DECOMP) {     // one unit per lane: the residual follows at once, from the same registers
+              if (srow >= 0) {
+                uint32_t rcw[4], rrec;
+                residual_block<SEDA, B16, CLAMP>(w, c4, didh, Ech, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi,
+                                                 rcw, &rrec);
+                const size_t ru = (size_t)srow * p.units_row + pos.rem;      // unit of the residual tensor
+                if (MX) {
+                  const uint2 fb = tb->fb_e4m3[(rrec >> 8) & 31u];
+                  uint32_t o[8];
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) fb4dev::codes_to_e4m3(rcw[q], fb, o[2 * q], o[2 * q + 1]);
+                  stg_v8(p.res_e4m3 + ru * 32u, o);
+                  p.res_scales[fb4dev::mx_scale_offset(srow, pos.rem, p.units_row, p.scale_col_tiles, p.scale_tiled)] =
+                      (uint8_t)rrec;
+                } else {
+                  *reinterpret_cast<uint4*>(ex.res_codes + ru * 16u) = make_uint4(rcw[0], rcw[1], rcw[2], rcw[3]);
+                  if (B16) *reinterpret_cast<uint32_t*>(ex.res_meta + ru * 2u) = rrec;
+                  else ex.res_meta[ru] = (uint16_t)rrec;
+                }
+              }
+            }
+          }
+          if (active) {
+            if (MX) {
+              // the codes become e4m3 bytes in registers, 32 contiguous bytes per lane; the scale byte is the E8M0 scale
+              const uint2 fb = tb->fb_e4m3[did0[0]];
+              uint32_t o[8];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) fb4dev::codes_to_e4m3(cw[q], fb, o[2 * q], o[2 * q + 1]);
+              stg_v8(p.e4m3 + (size_t)unit * 32u, o);
+              const int64_t so = p.scale_tiled ? fb4dev::mx_scale_offset(pos.row, pos.rem, p.units_row, p.scale_col_tiles, 1)
+                                               : (int64_t)unit;
+              p.scales[so] = (uint8_t)mrec[0];
+            } else if (U == 2) {
+              stg_v8(p.codes + (size_t)unit * 16u, cw);
+              if (B16) *reinterpret_cast<uint2*>(p.meta + (size_t)unit * 2u) = make_uint2(mrec[0], mrec[U - 1]);
+              else *reinterpret_cast<uint32_t*>(p.meta + unit) = mrec[0] | (mrec[U - 1] << 16);
+            } else {
+              *reinterpret_cast<uint4*>(p.codes + (size_t)unit * 16u) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+              if (B16) *reinterpret_cast<uint32_t*>(p.meta + (size_t)unit * 2u) = mrec[0];
+              else p.meta[unit] = (uint16_t)mrec[0];
+            }
+          }
+          // ---- refill this stage (all lanes have consumed their registers from it)
+          __syncwarp();
+          if (lane == 0 && it + u + kSt < n_mine) {
+            mbar_expect_tx(bar, kTileB);
+            tma_load_2d(my_ring + s * kTileB, &tmap, bar, 0, y_pre);
+          }
+          y_pre += y_step;
+          unit += unit_step;
+          if (kNeedPos) pos.advance(p);
+          if (SEDA) {
+            mask_cur = mask_nx;
+            mask_nx = mask_new;
+            cid_n2 = cid_new;
+          }
+        }
+      }
+    }
+    if (kUnroll == kSt) {
+      parity ^= 1u;
+    } else if (++s_dyn == kSt) {
+      s_dyn = 0;
+      parity ^= 1u;
+    }
+  }
+  if (SEDA && bad_cid) atomicOr(p.status, 2u);
+}
+
+
+// ---------------------------------------------------------------------------------------------
 // fp32 input (the hook for a producer that still holds its result in fp32): same ring and tables,
 // 8 warps per CTA, tiles of 1024 channels = 4 KB (view [T][C/32][32 floats], box 1 x 32 x 32,
 // 128-byte swizzle: row r of a stage is block r).  Lane i reads its block with eight conflict-free
@@ -1052,6 +1380,29 @@ cudaError_t fb4_fast_prepare_device() {
   FB4_OPT_IN(false, true, false, false, true);
   FB4_OPT_IN(true, true, false, false, true);
 #undef FB4_OPT_IN
+#define FB4_OPT_IN(...) \
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_flat_kernel<__VA_ARGS__>, attr, (int)kSmemBytes)
+  FB4_OPT_IN(false, false, false, false);
+  FB4_OPT_IN(true, false, false, false);
+  FB4_OPT_IN(false, true, false, false);
+  FB4_OPT_IN(true, true, false, false);
+  FB4_OPT_IN(false, false, true, false);
+  FB4_OPT_IN(true, false, true, false);
+  FB4_OPT_IN(false, true, true, false);
+  FB4_OPT_IN(true, true, true, false);
+  FB4_OPT_IN(false, false, false, true);
+  FB4_OPT_IN(true, false, false, true);
+  FB4_OPT_IN(false, true, false, true);
+  FB4_OPT_IN(true, true, false, true);
+  FB4_OPT_IN(false, false, true, true);
+  FB4_OPT_IN(true, false, true, true);
+  FB4_OPT_IN(false, true, true, true);
+  FB4_OPT_IN(true, true, true, true);
+  FB4_OPT_IN(false, false, false, false, true);
+  FB4_OPT_IN(true, false, false, false, true);
+  FB4_OPT_IN(false, true, false, false, true);
+  FB4_OPT_IN(true, true, false, false, true);
+#undef FB4_OPT_IN
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, false>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, false>, attr, bytes);
@@ -1104,10 +1455,83 @@ static cudaError_t fast_setup(const fb4_ctx* ctx, const void* x, int64_t T, int6
   return cudaSuccess;
 }
 
+// The flat kernel takes contiguous tensors whose unit count fits 31 bits.
+static bool flat_eligible(int64_t T, int64_t C, int64_t ld) {
+  return ld == C && C % 64 == 0 && T > 0 && T * (C / 32) < 0x7fffffffLL;
+}
+
+// Tensor map (2-D view [N/64][64] of the contiguous tensor), grid and walk parameters of one flat launch.
+static cudaError_t flat_setup(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, bool chunked, bool mx,
+                              CUtensorMap* map, FlatParams* p, int* grid_out) {
+  const uint32_t U = (uint32_t)flat_units(chunked, mx);   // units per lane: tiles of 32 * U units = 2 KB * U
+  const cuuint64_t dims[2] = {64, (cuuint64_t)(T * C / 64)};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {64, 16 * U};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = encode_tiled_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box,
+                                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  *p = FlatParams{};
+  p->units_row = (uint32_t)(C / 32);
+  p->n_units = (uint32_t)(T * (C / 32));
+  p->n_tiles = (p->n_units + 32u * U - 1u) / (32u * U);
+  p->status = ctx->d_status;
+  const int64_t want = ((int64_t)p->n_tiles + kWarps - 1) / kWarps;
+  const int grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
+  const uint64_t unit_step = (uint64_t)(chunked ? kWarps : grid * kWarps) * 32u * U;
+  p->step_rows = (uint32_t)(unit_step / p->units_row);
+  p->step_rem = (uint32_t)(unit_step % p->units_row);
+  p->ec_lo = (uint32_t)(ctx->cfg.exp_min + 127);
+  p->ec_hi = (uint32_t)(ctx->cfg.exp_max + 127);
+  *grid_out = grid;
+  return cudaSuccess;
+}
+
+template <bool SEDA, bool DECOMP, bool B16, bool CLAMP>
+static cudaError_t launch_flat(const CUtensorMap& map, const SmemTables* tables, const FlatParams& p,
+                               const Fb4RowExtras& ex, int grid, cudaStream_t stream) {
+  fb4_quantize_flat_kernel<SEDA, DECOMP, B16, CLAMP><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, p, ex);
+  return cudaGetLastError();
+}
+
 cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
                                      const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta, cudaStream_t stream) {
   const bool seda = ex.cluster_id != nullptr, decomp = ex.n_salient > 0;
   CUtensorMap map;
+  if (flat_eligible(T, C, ld)) {
+    FlatParams fp;
+    int grid = 0;
+    const cudaError_t e = flat_setup(ctx, x, T, C, decomp, false, &map, &fp, &grid);
+    if (e != cudaSuccess) return e;
+    fp.codes = codes;
+    fp.meta = meta;
+    const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
+    const bool b16 = ctx->cfg.block_size == 16;
+    const bool clamp = ctx->cfg.exp_min != -124 || ctx->cfg.exp_max != 127;
+    switch ((seda ? 1 : 0) | (decomp ? 2 : 0) | (b16 ? 4 : 0) | (clamp ? 8 : 0)) {
+#define FB4_CASE(V, S, D, B, K) \
+  case V: return launch_flat<S, D, B, K>(map, tables, fp, ex, grid, stream)
+      FB4_CASE(0, false, false, false, false);
+      FB4_CASE(1, true, false, false, false);
+      FB4_CASE(2, false, true, false, false);
+      FB4_CASE(3, true, true, false, false);
+      FB4_CASE(4, false, false, true, false);
+      FB4_CASE(5, true, false, true, false);
+      FB4_CASE(6, false, true, true, false);
+      FB4_CASE(7, true, true, true, false);
+      FB4_CASE(8, false, false, false, true);
+      FB4_CASE(9, true, false, false, true);
+      FB4_CASE(10, false, true, false, true);
+      FB4_CASE(11, true, true, false, true);
+      FB4_CASE(12, false, false, true, true);
+      FB4_CASE(13, true, false, true, true);
+      FB4_CASE(14, false, true, true, true);
+      FB4_CASE(15, true, true, true, true);
+#undef FB4_CASE
+    }
+    return cudaErrorInvalidValue;
+  }
   FastParams p;
   int grid = 0;
   const cudaError_t e = fast_setup(ctx, x, T, C, ld, decomp, &map, &p, &grid);
@@ -1195,6 +1619,41 @@ cudaError_t fb4_launch_quantize_fast_mx(const fb4_ctx* ctx, const void* x, int64
                                         uint8_t* res_scales, int tiled, cudaStream_t stream, int* launches) {
   const bool decomp = ex.n_salient > 0;
   CUtensorMap map;
+  if (flat_eligible(T, C, ld)) {
+    FlatParams fp;
+    int fgrid = 0;
+    cudaError_t fe = flat_setup(ctx, x, T, C, decomp, true, &map, &fp, &fgrid);
+    if (fe != cudaSuccess) return fe;
+    fp.e4m3 = e4m3;
+    fp.scales = scales;
+    fp.res_e4m3 = res_e4m3;
+    fp.res_scales = res_scales;
+    fp.scale_tiled = tiled;
+    const int64_t n_col = C / 32;
+    fp.scale_col_tiles = (n_col + 3) / 4;
+    // the kernel writes real entries only: padding of the tiled layout = scale 1
+    if (tiled && ((T & 127) || (n_col & 3))) {
+      fe = cudaMemsetAsync(scales, 0x7f, (size_t)(((T + 127) / 128) * fp.scale_col_tiles * 512), stream);
+      if (fe != cudaSuccess) return fe;
+    }
+    if (decomp && tiled && ((ex.n_salient & 127) || (n_col & 3))) {
+      fe = cudaMemsetAsync(res_scales, 0x7f, (size_t)(((ex.n_salient + 127) / 128) * fp.scale_col_tiles * 512), stream);
+      if (fe != cudaSuccess) return fe;
+    }
+    const SmemTables* ftables = static_cast<const SmemTables*>(ctx->d_fast_tables);
+#define FB4_MXF(S, D) \
+  fb4_quantize_flat_kernel<S, D, false, false, true><<<fgrid, kWarps * 32, kSmemBytes, stream>>>(map, ftables, fp, ex)
+    switch ((ex.cluster_id ? 1 : 0) | (decomp ? 2 : 0)) {
+      case 0: FB4_MXF(false, false); break;
+      case 1: FB4_MXF(true, false); break;
+      case 2: FB4_MXF(false, true); break;
+      default: FB4_MXF(true, true); break;
+    }
+#undef FB4_MXF
+    fe = cudaGetLastError();
+    if (fe == cudaSuccess) *launches = 1;
+    return fe;
+  }
   FastParams p;
   int grid = 0;
   cudaError_t e = fast_setup(ctx, x, T, C, ld, decomp, &map, &p, &grid);
