@@ -26,6 +26,13 @@
  *   - Alignment: x and every output pointer must be 16-byte aligned and
  *     ld_elems a multiple of 8; otherwise FB4_ERR_ALIGN.
  *   - The device of the context must be the current device of the calling thread.
+ *   - Host threads: a context is not internally locked.  Calls on ONE context must be serialised by
+ *     the caller (the context keeps a launch counter, the name of the last kernel variant, the
+ *     staging streams of fb4_quantize_host and scratch of the global top-k selection, all unguarded).
+ *     Different contexts, also on the same device, may be used from different threads at the
+ *     same time; one-time library set-up (driver entry points, the address of the built-in
+ *     scratch of the *_static call) is guarded inside the library.  fb4_init / fb4_destroy of
+ *     different contexts may run concurrently.
  *   - Device code has no unbounded wait loops: the only waits (for asynchronous loads into
  *     shared memory) give up after a fixed number of tries and raise a status bit
  *     (fb4_device_status); a call cannot hang.
