@@ -103,6 +103,16 @@ int fb4_get_tables(const fb4_ctx* ctx, uint8_t* formatbook, uint32_t* stage1_mas
                    uint8_t* qerror_q4);
 
 /*
+ * The table image that the device code of include/fb4_block.cuh reads (App. D.2: the quantizer as the
+ * tail of a producer kernel; that header holds the per-block routine the library's own kernels use).
+ * *device_image receives a DEVICE pointer owned by the context (valid until fb4_destroy), *bytes its
+ * size (= sizeof(fb4blk::Tables)).  FB4_ERR_INVALID_ARG if the context's configuration is not the one
+ * the header implements (block 32, 8 groups, two-stage selection, full exponent range) or its
+ * formatbook / stage-1 table does not fit the packed layout.
+ */
+int fb4_block_tables(const fb4_ctx* ctx, const void** device_image, uint64_t* bytes);
+
+/*
  * Plain FB4 quantization of x[T][C] (Sec. 3.1-3.2): per block, scale -> group
  * maxima -> LUT error sums over the stage-1 candidates -> argmin (ties: lowest
  * dialect id) -> LUT quantization.  Writes codes[T][C/2] and meta[T][C/B].

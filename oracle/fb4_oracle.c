@@ -64,7 +64,8 @@
  * included; bf16 decode of residual sums against integer round-to-nearest-even (hand-made
  * ties); the residual under a clamped exponent range in exact rationals; sub-formatbooks on
  * hand-counted cases, one dialect per bucket, and a constrained tensor giving
- * back the sub-formatbook it was constrained to; the affine step in exact rationals.
+ * back the sub-formatbook it was constrained to; the affine step and the LayerNorm producer in
+ * exact rationals (every operation rounded by integer arithmetic, the square root checked by squaring).
  * Parity unpinned: the formatbook VALUES (the paper's table is only in Fig. 2a)
  * and any worked numeric example (the paper prints none).  (The tiled order of the
  * MXFP8 scale bytes is pinned here only by its stated properties; a GPU test hands
@@ -394,6 +395,82 @@ int fb4o_affine_f32(const uint16_t *x, int64_t T, int64_t C, int64_t ld, const u
       y[t * C + c] = fmaf(xf, g, b);
     }
   }
+  return 0;
+}
+
+/*
+ * LayerNorm with per-channel modulation in front of the quantizer (App. D.2 names LayerNorm as an operation
+ * the quantizer is fused behind; in the adaLN blocks the normalised activation is modulated as
+ * y = n * (1 + scale_c) + shift_c before the linear layer).  Per token, in float32, with every operation
+ * rounded once (IEEE binary32, round to nearest even) and the order of the additions stated:
+ *   block sums    s_b = (((x_0 + x_1) + x_2) + ...) over the 32 consecutive channels of block b;
+ *   segment sums  the block sums of 32 consecutive blocks (1024 channels; a short last segment is filled
+ *                 up with +0) are added as a butterfly: for off = 16, 8, 4, 2, 1, all at once,
+ *                 v_i <- v_i + v_(i xor off); the segment sum is v_0;
+ *   row total     the segment sums added in order, ((S_0 + S_1) + S_2) + ...;
+ *   mean = total / C;  d_i = x_i - mean;
+ *   the sum of squares by the same three steps with q_b = fma(d, d, q) over the block's channels in order
+ *   (q = 0 at the start);  var = total of squares / C;  rstd = 1 / sqrt(var + eps);
+ *   y_i = fma(d_i * rstd, g_c, bias_c),  g_c = gain_c or 1 + gain_c (float32 sum).
+ * x, gain, bias are bf16 bit patterns; y feeds fb4o_quantize_f32.  C must be a multiple of 32.
+ */
+static float ln_segment_butterfly(const float *blocksum, int n) {
+  float v[32], u[32];
+  for (int i = 0; i < 32; ++i) v[i] = i < n ? blocksum[i] : 0.0f;
+  for (int off = 16; off >= 1; off >>= 1) {
+    for (int i = 0; i < 32; ++i) u[i] = v[i] + v[i ^ off];
+    memcpy(v, u, sizeof v);
+  }
+  return v[0];
+}
+
+static float ln_row_total(const float *blocksum, int64_t nblk) {
+  float total = 0.0f;
+  int first = 1;
+  for (int64_t b0 = 0; b0 < nblk; b0 += 32) {
+    int n = nblk - b0 < 32 ? (int)(nblk - b0) : 32;
+    float seg = ln_segment_butterfly(blocksum + b0, n);
+    total = first ? seg : total + seg;
+    first = 0;
+  }
+  return total;
+}
+
+int fb4o_layernorm_f32(const uint16_t *x, int64_t T, int64_t C, int64_t ld, const uint16_t *gain,
+                       const uint16_t *bias, int plus_one, float eps, float *y, float *stats /* optional [T][2]: mean, var */) {
+  if (T < 0 || C <= 0 || C % 32 || ld < C) return -1;
+  const int64_t nblk = C / 32;
+  float *bs = (float *)malloc((size_t)nblk * sizeof(float));
+  float *d = (float *)malloc((size_t)C * sizeof(float));
+  if (!bs || !d) { free(bs); free(d); return -1; }
+  for (int64_t t = 0; t < T; ++t) {
+    for (int64_t b = 0; b < nblk; ++b) {
+      float s = (float)bf16_to_double(x[t * ld + b * 32]);
+      for (int i = 1; i < 32; ++i) s = s + (float)bf16_to_double(x[t * ld + b * 32 + i]);
+      bs[b] = s;
+    }
+    const float mean = ln_row_total(bs, nblk) / (float)C;
+    for (int64_t b = 0; b < nblk; ++b) {
+      float q = 0.0f;
+      for (int i = 0; i < 32; ++i) {
+        float di = (float)bf16_to_double(x[t * ld + b * 32 + i]) - mean;
+        d[b * 32 + i] = di;
+        q = fmaf(di, di, q);
+      }
+      bs[b] = q;
+    }
+    const float var = ln_row_total(bs, nblk) / (float)C;
+    const float rstd = 1.0f / sqrtf(var + eps);
+    if (stats) { stats[2 * t] = mean; stats[2 * t + 1] = var; }
+    for (int64_t c = 0; c < C; ++c) {
+      float g = (float)bf16_to_double(gain[c]);
+      const float bc = (float)bf16_to_double(bias[c]);
+      if (plus_one) g = 1.0f + g;
+      y[t * C + c] = fmaf(d[c] * rstd, g, bc);
+    }
+  }
+  free(bs);
+  free(d);
   return 0;
 }
 

@@ -82,6 +82,8 @@ def lib():
         L.fb4o_quantize_f32.restype = ctypes.c_int
         L.fb4o_affine_f32.argtypes = [vp, i64, i64, i64, vp, vp, ctypes.c_int, vp]
         L.fb4o_affine_f32.restype = ctypes.c_int
+        L.fb4o_layernorm_f32.argtypes = [vp, i64, i64, i64, vp, vp, ctypes.c_int, ctypes.c_float, vp, vp]
+        L.fb4o_layernorm_f32.restype = ctypes.c_int
         L.fb4o_to_mxfp8.argtypes = [vp, vp, i64, i64, vp, vp, vp, ctypes.c_int]
         L.fb4o_to_mxfp8.restype = ctypes.c_int
         L.fb4o_mxfp8_scale_offset.argtypes = [i64, i64, i64, ctypes.c_int]
@@ -265,6 +267,22 @@ def affine_f32(x_bits, gain_bits, bias_bits, plus_one: bool) -> np.ndarray:
     if r != 0:
         raise ValueError(f"fb4o_affine_f32 failed: {r}")
     return y
+
+
+def layernorm_f32(x_bits, gain_bits, bias_bits, plus_one: bool, eps: float, want_stats: bool = False):
+    """LayerNorm + per-channel modulation in float32 with the stated order of operations; inputs bf16 bit patterns."""
+    x = np.asarray(x_bits)
+    assert x.dtype == np.uint16 and x.ndim == 2 and x.strides[1] == 2
+    T, C = x.shape
+    ld = x.strides[0] // 2 if T > 1 else C
+    g, b = _c(gain_bits, np.uint16), _c(bias_bits, np.uint16)
+    assert g.shape == (C,) and b.shape == (C,)
+    y = np.zeros((T, C), dtype=np.float32)
+    stats = np.zeros((T, 2), dtype=np.float32) if want_stats else None
+    r = lib().fb4o_layernorm_f32(_p(x), T, C, ld, _p(g), _p(b), int(bool(plus_one)), float(np.float32(eps)), _p(y), _p(stats))
+    if r != 0:
+        raise ValueError(f"fb4o_layernorm_f32 failed: {r}")
+    return (y, stats) if want_stats else y
 
 
 def mxfp8_scale_offset(row: int, col: int, n_col: int, layout: int) -> int:

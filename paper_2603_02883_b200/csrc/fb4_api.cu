@@ -181,6 +181,7 @@ int fb4_init(fb4_ctx** out, int device, const uint8_t* formatbook, const uint32_
   if (fb4_fast_build_tables(ctx->host_tables, &ctx->d_fast_tables, &fast_bytes) &&
       fb4_fast_prepare_device() == cudaSuccess)
     ctx->fast_ok = 1;
+  ctx->fast_table_bytes = fast_bytes;
   cudaGetLastError();
   *out = ctx;
   return FB4_OK;
@@ -198,6 +199,17 @@ int fb4_destroy(fb4_ctx* ctx) {
   if (ctx->d_status) cudaFree(ctx->d_status);
   if (ctx->d_tables) cudaFree(ctx->d_tables);
   delete ctx;
+  return FB4_OK;
+}
+
+int fb4_block_tables(const fb4_ctx* ctx, const void** device_image, uint64_t* bytes) {
+  if (!ctx || !device_image || !bytes) return FB4_ERR_INVALID_ARG;
+  const fb4_config& c = ctx->cfg;
+  if (!ctx->fast_ok || !ctx->d_fast_tables || c.block_size != 32 || c.num_groups != 8 || c.select_mode != 0 ||
+      c.exp_min != -124 || c.exp_max != 127)
+    return FB4_ERR_INVALID_ARG;
+  *device_image = ctx->d_fast_tables;
+  *bytes = ctx->fast_table_bytes;
   return FB4_OK;
 }
 

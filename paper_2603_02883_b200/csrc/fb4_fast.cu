@@ -28,6 +28,7 @@
 #include <mutex>
 #include <new>
 
+#include "fb4_block.cuh"
 #include "fb4_device.cuh"
 #include "fb4_internal.h"
 
@@ -35,38 +36,13 @@ namespace {
 
 using fb4dev::pow2f;
 using fb4dev::prmt;
+using namespace fb4blk;
+using SmemTables = fb4blk::Tables;
 
 constexpr int kWarps = 16;           // warps per CTA
 constexpr int kStages = 4;           // ring depth per warp
 constexpr int kTileBytes = 2048;     // 1024 bf16
-constexpr int kPairMul = 36;         // pair-table address = 36*bin_hi + bin_lo: spreads small bins over the banks
-constexpr int kPairStride = 1148;    // 36*31 + 32 bytes per dialect; 287 words: one bank of rotation per dialect
-constexpr int kMaxGroups = 8;        // distinct stage-1 groups the packed tables hold
 constexpr uint32_t kSpinLimit = 1u << 20;   // tries per wait before a warp gives up
-
-// Compact tables, built at init (the part of the shared-memory image that is read as is).
-struct FastTables {
-  uint8_t qvalue[32][32];                // [dialect][bin] -> index of the nearest magnitude
-  uint64_t qerr64[kMaxGroups][32];       // [group][bin] -> byte j = Qerror of candidate j (pad 31)
-  uint8_t did_of[kMaxGroups][8];         // [group][candidate] -> dialect id
-  uint8_t group_of_bin[32];              // [bin of block maximum] -> group
-  uint32_t stage1[32];                   // [bin of block maximum] -> candidate mask
-  uint8_t qerror[32][32];                // [dialect][bin], for masks that cut a group
-  uint8_t fb[32][8];
-};
-static_assert(sizeof(FastTables) % 16 == 0, "copied with 16-byte accesses");
-
-// The tables as they sit in shared memory.  The image is built once on the host at init, kept in
-// global memory, and copied by every CTA with one bulk asynchronous copy.
-struct SmemTables {
-  // [group][bin][lane & 15] -> the 8 candidate errors: each lane of a half-warp has its own
-  // 8-byte column, so the 64-bit loads of a warp never conflict
-  uint64_t qerr_private[kMaxGroups][32][16];
-  uint8_t pairlut[32 * kPairStride];     // [dialect][36*bin_hi + bin_lo] -> idx_lo | idx_hi<<4
-  uint4 fb_bf16[32];                     // [dialect] -> magnitudes as bf16, high bytes then low bytes (residual pass)
-  uint2 fb_e4m3[32];                     // [dialect] -> magnitudes as e4m3 bytes (MXFP8 output)
-  FastTables c;
-};
 
 struct FastParams {
   int64_t T, C;
@@ -84,8 +60,6 @@ struct FastParams {
   int64_t scale_col_tiles;
   int32_t scale_tiled;
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -113,191 +87,6 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
-  uint32_t v;
-  asm("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
-  uint2 v;
-  asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
-}
-
-// Score an arbitrary candidate mask over 8 group bins with the byte table (SeDA masks that
-// cut a stage-1 group).  Ascending ids: ties keep the lowest.
-__device__ __forceinline__ int select_general(uint32_t cand, const uint8_t* gb, const SmemTables* tb) {
-  int best = 0, best_err = 0x7fffffff;
-  for (uint32_t m = cand; m; m &= m - 1) {
-    const int d = __ffs((int)m) - 1;
-    int err = 0;
-#pragma unroll
-    for (int g = 0; g < 8; ++g) err += tb->c.qerror[d][gb[g]];
-    if (err < best_err) { best_err = err; best = d; }
-  }
-  return best;
-}
-
-// Dialect selection of one block (Sec. 3.2 two-stage; Sec. 3.4 restriction).  gm = the 8 group
-// maxima as fp32 magnitudes (mantissa bits below the bin resolution are truncated away),
-// sG = 2^(3-e) * 2^-21, bmax = bin of the block maximum, qerr_lane = this lane's column of the
-// packed error table.
-template <bool SEDA>
-__device__ __forceinline__ int choose_dialect(const float (&gm)[8], float sG, uint32_t bmax, uint32_t allowed,
-                                              const SmemTables* tb, uint32_t qerr_lane) {
-  const uint32_t grp = tb->c.group_of_bin[bmax];
-  bool packed_path = true;
-  uint32_t cand = 0;
-  if (SEDA) {
-    const uint32_t st1 = tb->c.stage1[bmax];
-    cand = st1 & allowed;
-    if (cand == 0) cand = allowed;
-    packed_path = (cand == st1);
-  }
-  if (!SEDA || packed_path) {
-    const uint32_t qb = qerr_lane + grp * 4096u;
-    uint32_t lo = 0, hi = 0;
-#pragma unroll
-    for (int g = 0; g < 8; ++g) {
-      const uint32_t t = __float_as_uint(__fmaf_rz(gm[g], sG, 2.0f));
-      const uint2 e = lds_v2((t << 7) + qb);   // 0x40000000 << 7 vanishes mod 2^32: 128 B per bin
-      lo += e.x;
-      hi += e.y;
-    }
-    // argmin over 8 byte sums, ties to the lowest candidate: keys (err << 3 | j) in 16-bit lanes
-    const uint32_t k02 = (lo & 0x00ff00ffu) * 8u + 0x00020000u;
-    const uint32_t k13 = ((lo >> 8) & 0x00ff00ffu) * 8u + 0x00030001u;
-    const uint32_t k46 = (hi & 0x00ff00ffu) * 8u + 0x00060004u;
-    const uint32_t k57 = ((hi >> 8) & 0x00ff00ffu) * 8u + 0x00070005u;
-    const uint32_t km = __vminu2(__vminu2(k02, k13), __vminu2(k46, k57));
-    const uint32_t key = min(km & 0xffffu, km >> 16);
-    return tb->c.did_of[grp][key & 7u];
-  }
-  if (__popc(cand) == 1) return __ffs((int)cand) - 1;
-  uint8_t gb[8];
-#pragma unroll
-  for (int g = 0; g < 8; ++g) gb[g] = (uint8_t)(__float_as_uint(__fmaf_rz(gm[g], sG, 2.0f)) & 31u);
-  return select_general(cand, gb, tb);
-}
-
-// One lane's block(s) from 16 registers of two 16-bit values each - bf16 inputs, or any fp32 values cut
-// to their upper 16 bits: the scale exponent, the bins of the 0.5-wide tables and the sign are all
-// fixed by those bits (every bin boundary is a multiple of the cut's granularity), so the cut loses
-// nothing.  Scale, group maxima, dialect selection, LUT quantization; block size 32, or (B16) two
-// blocks of 16; CLAMP: clamped exponent range.  Out: the four code words, and per half the chosen
-// dialect and the biased exponent.
-template <bool SEDA, bool B16, bool CLAMP>
-__device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], uint32_t allowed, const SmemTables* tb,
-                                                      uint32_t qerr_lane, uint32_t pair_base, uint32_t ec_lo,
-                                                      uint32_t ec_hi, uint32_t (&cw)[4], int (&didh)[2],
-                                                      uint32_t (&Ech)[2]) {
-  // ---- magnitudes, group maxima (4 elements = 2 registers), block maximum
-  uint32_t a[16];
-#pragma unroll
-  for (int i = 0; i < 16; ++i) a[i] = w[i] & 0x7fff7fffu;
-  // per half of the lane's 32 elements (block size 32: both halves belong to one block):
-  // biased exponent, the two bin scales of the Qvalue lookup, the chosen dialect's table address
-  float sHh[2], sLh[2], magich[2];
-  if (!B16) {
-    uint32_t g2[4];   // (group 2q+1 max << 16) | group 2q max
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const uint32_t m0 = __vmaxu2(a[4 * q], a[4 * q + 1]);
-      const uint32_t m1 = __vmaxu2(a[4 * q + 2], a[4 * q + 3]);
-      g2[q] = __vmaxu2(__byte_perm(m0, m1, 0x5410), __byte_perm(m0, m1, 0x7632));
-    }
-    const uint32_t mm = __vmaxu2(__vmaxu2(g2[0], g2[1]), __vmaxu2(g2[2], g2[3]));
-    uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
-    // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
-    uint32_t Ec = max(amax16 >> 7, 3u);
-    if (CLAMP) {
-      // clamped exponent range: magnitudes that would normalise to 16 or more saturate at the
-      // largest value of bin 31 (biased exponent Ec, mantissa all ones)
-      Ec = min(max(amax16 >> 7, ec_lo), ec_hi);
-      const uint32_t bound = ((Ec << 7) | 0x7fu) * 0x10001u;
-      amax16 = min(amax16, bound & 0xffffu);
-#pragma unroll
-      for (int i = 0; i < 16; ++i) a[i] = __vminu2(a[i], bound);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) g2[q] = __vminu2(g2[q], bound);
-    }
-    const float s2 = __uint_as_float((257u - Ec) << 23);   // 2^(3-e)
-    const float sG = s2 * 0x1p-21f;                        // bin in the mantissa of 2.0 + x
-    const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(amax16 << 16), sG, 2.0f)) & 31u;
-    // ---- dialect selection; the upper bf16 of a pair keeps the lower one as extra mantissa bits,
-    // which truncation discards
-    float gm[8];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      gm[2 * q] = __uint_as_float(g2[q] << 16);
-      gm[2 * q + 1] = __uint_as_float(g2[q]);
-    }
-    const int did = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
-    Ech[0] = Ech[1] = Ec;
-    sHh[0] = sHh[1] = s2 * 0x1p-25f;                       // bin in the mantissa of 0.125 + x
-    sLh[0] = sLh[1] = s2 * 0x1p-5f;                        // bin in the mantissa of 2^17 + x
-    didh[0] = didh[1] = did;
-  } else {
-    // block size 16: the lane's two halves are two blocks; a group is the two elements of one register
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      uint32_t gx[8];   // group maximum in both halves of the register
-#pragma unroll
-      for (int k = 0; k < 8; ++k) gx[k] = __vmaxu2(a[8 * h + k], __byte_perm(a[8 * h + k], 0u, 0x1032));
-      uint32_t mm = __vmaxu2(__vmaxu2(__vmaxu2(gx[0], gx[1]), __vmaxu2(gx[2], gx[3])),
-                             __vmaxu2(__vmaxu2(gx[4], gx[5]), __vmaxu2(gx[6], gx[7])));
-      uint32_t Ec = max((mm & 0xffffu) >> 7, 3u);
-      if (CLAMP) {
-        Ec = min(max((mm & 0xffffu) >> 7, ec_lo), ec_hi);
-        const uint32_t bound = ((Ec << 7) | 0x7fu) * 0x10001u;
-        mm = __vminu2(mm, bound);
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          a[8 * h + k] = __vminu2(a[8 * h + k], bound);
-          gx[k] = __vminu2(gx[k], bound);
-        }
-      }
-      const float s2 = __uint_as_float((257u - Ec) << 23);
-      const float sG = s2 * 0x1p-21f;
-      const uint32_t bmax = __float_as_uint(__fmaf_rz(__uint_as_float(mm), sG, 2.0f)) & 31u;
-      float gm[8];
-#pragma unroll
-      for (int k = 0; k < 8; ++k) gm[k] = __uint_as_float(gx[k]);   // the low copy is truncated away
-      Ech[h] = Ec;
-      sHh[h] = s2 * 0x1p-25f;
-      sLh[h] = s2 * 0x1p-5f;
-      didh[h] = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
-    }
-  }
-  // ---- Qvalue: one lookup per element pair.  124*36 + 144 = 9*512, so the exponent fields of
-  // 36*bits(0.125 + ..) + bits(2^17 + ..) cancel mod 2^32 and leave table + 36*bin_hi + bin_lo.
-  magich[0] = __uint_as_float(0x48000000u + pair_base + (uint32_t)didh[0] * kPairStride);
-  magich[1] = B16 ? __uint_as_float(0x48000000u + pair_base + (uint32_t)didh[1] * kPairStride) : magich[0];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const int h = B16 ? (q >> 1) : 0;
-    uint32_t b[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t av = a[4 * q + j];
-      const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sHh[h], 0.125f));
-      const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sLh[h], magich[h]));
-      b[j] = lds_u8(th * (uint32_t)kPairMul + tl);
-    }
-    const uint32_t idx = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
-    // sign bits: byte masks by sign replication, then to bit 3 of every nibble
-    const uint32_t sa = prmt(w[4 * q], w[4 * q + 1], 0xfdb9u);
-    const uint32_t sb = prmt(w[4 * q + 2], w[4 * q + 3], 0xfdb9u);
-    const uint32_t ev = __byte_perm(sa, sb, 0x6420), od = __byte_perm(sa, sb, 0x7531);
-    cw[q] = idx | (((ev & 0x0f0f0f0fu) | (od & 0xf0f0f0f0u)) & 0x88888888u);
-  }
-}
-
 // Residual pass of the lane's block(s) (Sec. 3.3): Delta = x - Q(x) in fp32 (exact for the full
 // exponent range, the correctly rounded difference otherwise), quantized again with the same tables
 // as the main pass, from the upper 16 bits of every Delta (see quantize_packed_block).

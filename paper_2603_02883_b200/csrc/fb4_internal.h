@@ -38,6 +38,7 @@ struct fb4_ctx {
   Fb4DeviceTables host_tables;   // host copy
   Fb4DeviceTables* d_tables;     // device copy
   void* d_fast_tables;           // packed tables of the TMA-staged kernel (NULL if not eligible)
+  size_t fast_table_bytes;
   int force_generic;             // fb4_set_kernel_variant(ctx, 1): always take the generic kernel
   int fast_ok;                   // formatbook/stage-1 table fit the fast kernel's packed layout
   int sm_count;

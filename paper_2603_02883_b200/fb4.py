@@ -21,7 +21,7 @@ ERR_STATIC_LIMIT = -7
 STATIC_MAX_CLUSTERS = 1024
 
 EXPORTS = [
-    "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_affine", "fb4_quantize_affine_mxfp8", "fb4_quantize_seda",
+    "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_block_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_affine", "fb4_quantize_affine_mxfp8", "fb4_quantize_seda",
     "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_select_salient_topk", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
     "fb4_quantize_weights", "fb4_quantize_mxfp8", "fb4_quantize_mxfp8_decomposed", "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
     L.fb4_init.argtypes = [ctypes.POINTER(vp), ci, vp, vp, ctypes.POINTER(Fb4Config)]
     L.fb4_destroy.argtypes = [vp]
     L.fb4_get_tables.argtypes = [vp, vp, vp, vp, vp]
+    L.fb4_block_tables.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_uint64)]
+    L.fb4_block_tables.restype = ci
     L.fb4_quantize.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.fb4_quantize_f32.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.fb4_quantize_f32.restype = ci
@@ -167,6 +169,13 @@ def fb4_get_tables(ctx):
     p = lambda a: a.ctypes.data_as(ctypes.c_void_p)
     _check(lib().fb4_get_tables(ctx, p(fb), p(s1), p(qv), p(qe)), "fb4_get_tables")
     return fb, s1, qv, qe
+
+
+def fb4_block_tables(ctx):
+    """(device pointer, size in bytes) of the table image that include/fb4_block.cuh reads"""
+    ptr, n = ctypes.c_void_p(), ctypes.c_uint64(0)
+    _check(lib().fb4_block_tables(ctx, ctypes.byref(ptr), ctypes.byref(n)), "fb4_block_tables")
+    return int(ptr.value), int(n.value)
 
 
 def fb4_quantize(ctx, x, T, C, ld_elems, codes, meta, stream=None) -> None:

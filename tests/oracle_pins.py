@@ -398,6 +398,114 @@ def pin_affine_producer(seed=21, n=400):
     assert np.array_equal(y, synth.bf16_bits_to_f32(wide[:, :8]) * np.float32(2.0 ** -30))
 
 
+def _sqrt_to_f32(q):
+    """The binary32 number nearest to sqrt(q) for a positive rational q (ties cannot occur: the midpoint of two
+    neighbouring floats has 25 significant bits, its square at most 50, so it is never the exact root of a
+    49-bit argument unless representable).  Candidate from the double square root, verified by squaring
+    the midpoints to its neighbours in exact rationals."""
+    from fractions import Fraction
+    assert q > 0
+    c = np.float32(math.sqrt(float(q)))
+    for _ in range(4):
+        lo, hi = np.nextafter(c, np.float32(0)), np.nextafter(c, np.float32(np.inf))
+        mlo = (Fraction(float(lo)) + Fraction(float(c))) / 2
+        mhi = (Fraction(float(c)) + Fraction(float(hi))) / 2
+        if mlo * mlo <= q <= mhi * mhi:
+            assert mlo * mlo != q and mhi * mhi != q
+            return Fraction(float(c))
+        c = lo if q < mlo * mlo else hi
+    raise AssertionError("square root candidate did not settle")
+
+
+def _layernorm_rational(xv, gv, bv, plus_one, eps):
+    """The stated LayerNorm order in exact rationals, every operation rounded to binary32 by _round_to_f32."""
+    from fractions import Fraction
+    R = _round_to_f32
+    C = len(xv)
+    nblk = C // 32
+
+    def total(bs):
+        acc = None
+        for b0 in range(0, nblk, 32):
+            v = [bs[b0 + i] if b0 + i < nblk else Fraction(0) for i in range(32)]
+            for off in (16, 8, 4, 2, 1):
+                v = [R(v[i] + v[i ^ off]) for i in range(32)]
+            acc = v[0] if acc is None else R(acc + v[0])
+        return acc
+
+    bs = []
+    for b in range(nblk):
+        s_ = xv[b * 32]
+        for i in range(1, 32):
+            s_ = R(s_ + xv[b * 32 + i])
+        bs.append(s_)
+    mean = R(total(bs) / C)
+    d = [R(x - mean) for x in xv]
+    bs = []
+    for b in range(nblk):
+        q = Fraction(0)
+        for i in range(32):
+            q = R(d[b * 32 + i] * d[b * 32 + i] + q)
+        bs.append(q)
+    var = R(total(bs) / C)
+    rstd = R(1 / _sqrt_to_f32(R(var + eps)))
+    out = []
+    for c in range(C):
+        g = R(1 + gv[c]) if plus_one else gv[c]
+        out.append(R(R(d[c] * rstd) * g + bv[c]))
+    return out, mean, var
+
+
+def pin_layernorm_producer(seed=22):
+    """LayerNorm + modulation (App. D.2 fusion with the preceding operation): the float32 result equals the stated
+    order of operations carried out in exact rationals with one rounding per operation (square root checked by
+    squaring); it stays within a few units in the last place of the exact LayerNorm; a row of equal values
+    normalises to the bias; the row stride is honoured."""
+    from fractions import Fraction
+    rng = np.random.default_rng(seed)
+    bf = lambda a: synth.f32_to_bf16_bits(np.asarray(a, dtype=np.float32))
+    val = lambda bits: [Fraction(float(v)) for v in synth.bf16_bits_to_f32(np.asarray(bits, dtype=np.uint16))]
+    eps = float(np.float32(1e-6))
+    # 1, 3, 33, 65 blocks: short last segments.  "wide": magnitudes spread over 2^-12 .. 2^12 inside a block, so that
+    # the additions round, the mean has 24 significant bits and the squares are not representable - with a single
+    # block (C = 32) mean and variance are the block's own sums divided by a power of two, nothing hides a rounding
+    for C, plus_one, wide in [(32, False, False), (32, True, True), (64, False, True), (96, True, False), (1056, False, True),
+                              (2080, True, False)]:
+        x = bf(rng.standard_t(3, size=(2, C)) * np.exp2(float(rng.integers(-6, 6))) + rng.standard_normal())
+        if wide:
+            x = bf(rng.standard_normal((2, C)) * np.exp2(rng.integers(-12, 13, size=(2, C)).astype(np.float64)))
+        gain = bf(rng.standard_normal(C) * 0.5)
+        bias = bf(rng.standard_normal(C))
+        y, stats = orc.layernorm_f32(x, gain, bias, plus_one, eps, want_stats=True)
+        for t in range(2):
+            want, mean, var = _layernorm_rational(val(x[t]), val(gain), val(bias), plus_one, Fraction(eps))
+            assert Fraction(float(stats[t, 0])) == mean and Fraction(float(stats[t, 1])) == var, (C, t)
+            got = [Fraction(float(v)) for v in y[t]]
+            assert got == want, (C, t, next(i for i in range(C) if got[i] != want[i]))
+            # against the exact LayerNorm: mean and variance in rationals, the root in double precision
+            xv = val(x[t])
+            m = sum(xv) / C
+            v = sum((a - m) ** 2 for a in xv) / C
+            assert abs(mean - m) <= Fraction(1, 2 ** 18) * max(abs(a) for a in xv)
+            assert abs(var - v) <= Fraction(1, 2 ** 17) * v
+            r = 1.0 / math.sqrt(float(v) + eps)
+            for c in range(0, C, 7):
+                g = float(val(gain[c:c + 1])[0]) + (1.0 if plus_one else 0.0)
+                exact = float(xv[c] - m) * r * g + float(val(bias[c:c + 1])[0])
+                assert abs(float(y[t, c]) - exact) <= 3e-5 * (1.0 + abs(exact)), (C, t, c)
+    # a row of equal values: d = 0 everywhere, y = bias bit for bit (fma(+-0, g, b) = b)
+    x = bf(np.full((1, 64), 3.0))
+    gain, bias = bf(rng.standard_normal(64)), bf(rng.standard_normal(64) + 2.0)
+    y = orc.layernorm_f32(x, gain, bias, True, eps)
+    assert np.array_equal(y[0], synth.bf16_bits_to_f32(bias))
+    # row stride
+    wide = bf(rng.standard_normal((3, 128)))
+    gain, bias = bf(np.ones(64)), bf(np.zeros(64))
+    a = orc.layernorm_f32(wide[:, :64], gain, bias, False, eps)
+    b = orc.layernorm_f32(np.ascontiguousarray(wide[:, :64]), gain, bias, False, eps)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
 def pin_f32_input(seed=9, n=30):
     """fp32 input: every block equals the block-wise definition on the exact values (pinned above
     through quantize_block_f64), values that happen to be bf16 give the bf16 result, and a value
@@ -870,7 +978,7 @@ ALL_PINS = [
     pin_representable_values_roundtrip, pin_error_terms_and_argmin, pin_groups_are_contiguous,
     pin_select_all_mode, pin_seda_choice_inside_mask, pin_salient_is_per_tile_argmax, pin_salient_topk, pin_decomposition, pin_residual_uses_the_seda_mask,
     pin_dequantize_formula, pin_dequantize_f16, pin_dequantize_bf16_rounds_sums_to_nearest_even,
-    pin_decomposition_with_clamped_exponent, pin_mse, pin_f32_input, pin_affine_producer, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
+    pin_decomposition_with_clamped_exponent, pin_mse, pin_f32_input, pin_affine_producer, pin_layernorm_producer, pin_mxfp8_view, pin_mxfp8_scale_layout, pin_weight_quantization,
     pin_subformatbook_hand_counted,
     pin_subformatbook_one_dialect_per_bucket_and_closed_loop,
 ]

@@ -78,6 +78,17 @@ MUTANTS = {
                                     "const float b = (float)bf16_to_double(bias[c + 1 < C ? c + 1 : c]);"),
     "affine_ignores_row_stride": ("const float xf = (float)bf16_to_double(x[t * ld + c]);",
                                   "const float xf = (float)bf16_to_double(x[t * C + c]);"),
+    "layernorm_block_sums_in_double": ("for (int i = 1; i < 32; ++i) s = s + (float)bf16_to_double(x[t * ld + b * 32 + i]);",
+                                       "{ double s_ = s; for (int i = 1; i < 32; ++i) s_ += bf16_to_double(x[t * ld + b * 32 + i]); s = (float)s_; }"),
+    "layernorm_butterfly_replaced_by_a_running_sum": ("  return v[0];\n}\n\nstatic float ln_row_total",
+                                                     "  { float r_ = 0.0f; for (int i = 0; i < n; ++i) r_ += blocksum[i]; return r_; }\n}\n\nstatic float ln_row_total"),
+    "layernorm_square_not_fused": ("q = fmaf(di, di, q);", "q = q + di * di;"),
+    "layernorm_eps_dropped": ("const float rstd = 1.0f / sqrtf(var + eps);", "const float rstd = 1.0f / sqrtf(var);"),
+    "layernorm_rsqrt_in_double": ("const float rstd = 1.0f / sqrtf(var + eps);", "const float rstd = (float)(1.0 / sqrt((double)var + (double)eps));"),
+    "layernorm_variance_unbiased": ("const float var = ln_row_total(bs, nblk) / (float)C;", "const float var = ln_row_total(bs, nblk) / (float)(C - 1);"),
+    "layernorm_modulation_two_roundings": ("y[t * C + c] = fmaf(d[c] * rstd, g, bc);", "y[t * C + c] = (d[c] * rstd) * g + bc;"),
+    "layernorm_short_segment_padded_with_first_block": ("v[i] = i < n ? blocksum[i] : 0.0f;", "v[i] = i < n ? blocksum[i] : blocksum[0];"),
+    "layernorm_segments_added_last_to_first": ("total = first ? seg : total + seg;", "total = first ? seg : seg + total * 1.0000001f;"),
     "bf16_by_truncation": ("u += 0x7fffu + lsb;", "u += 0u * lsb;"),
     "bf16_ties_away_from_zero": ("u += 0x7fffu + lsb;", "u += 0x8000u + 0u * lsb;"),
     "bf16_ties_toward_zero": ("u += 0x7fffu + lsb;", "u += 0x7fffu + 0u * lsb;"),
