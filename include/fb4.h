@@ -167,6 +167,30 @@ int fb4_quantize_affine_mxfp8(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64
                               uint8_t* e4m3, uint8_t* scales, int scale_layout, void* stream);
 
 /*
+ * LayerNorm with per-channel modulation fused in front of the quantizer (App. D.2 lists LayerNorm among the
+ * operations the quantizer runs behind; in the adaLN blocks the normalised activation is modulated as
+ * y = n * (1 + scale_c) + shift_c before the linear layer).  Per token, in float32:
+ *     mean = sum(x) / C,  d = x - mean,  var = sum(d * d) / C,  rstd = 1 / sqrt(var + eps),
+ *     y[c] = (d[c] * rstd) * g_c + bias_c,   g_c = gain_c (gain_plus_one 0) or 1 + gain_c (1),
+ * every operation rounded once (IEEE binary32, nearest even; square root and divisions correctly rounded),
+ * d * d + q and (d * rstd) * g + bias as fused multiply-adds, and the additions in a fixed order: the
+ * 32 channels of a block in index order; the 32 block sums of a run of 1024 channels by an xor butterfly
+ * (v_i <- v_i + v_(i xor off) for off = 16, 8, 4, 2, 1, all i at once; the run's sum is v_0); the runs of a
+ * token in order.  The result is therefore reproducible bit for bit; it is quantized from registers as
+ * fb4_quantize_f32 quantizes a float32 tensor, so the token is read once and y never exists in memory.
+ * Optional SeDA restriction as in fb4_quantize_seda.  One fused pass; default configuration only,
+ * contiguous rows (ld_elems == C), C a multiple of 1024 and at most 16384, gain and bias 16-byte
+ * aligned: FB4_ERR_INVALID_ARG for another configuration, FB4_ERR_SHAPE for another shape.
+ *   x    : device bfloat16 [T][C]
+ *   gain : device bfloat16 [C];  bias : device bfloat16 [C]
+ *   eps  : added to the variance (>= 0, finite)
+ */
+int fb4_quantize_layernorm(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64_t C, int64_t ld_elems,
+                           const void* gain_bf16, const void* bias_bf16, int gain_plus_one, float eps,
+                           const int32_t* cluster_id, const uint32_t* cluster_mask, int32_t n_clusters,
+                           uint8_t* codes, uint16_t* meta, void* stream);
+
+/*
  * SeDA-constrained quantization (Sec. 3.4): token t may only use the dialects in
  * cluster_mask[cluster_id[t]] (its cluster's sub-formatbook); cluster_id[t] == -1
  * means unconstrained.  Stage 1 is intersected with the mask; if the intersection

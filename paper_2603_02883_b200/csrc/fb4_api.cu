@@ -254,6 +254,36 @@ int fb4_quantize_f32(fb4_ctx* ctx, const float* x, int64_t T, int64_t C, int64_t
   return FB4_OK;
 }
 
+int fb4_quantize_layernorm(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const void* gain,
+                           const void* bias, int gain_plus_one, float eps, const int32_t* cluster_id,
+                           const uint32_t* cluster_mask, int32_t n_clusters, uint8_t* codes, uint16_t* meta,
+                           void* stream) {
+  const int rc = check_quantize_args(ctx, x, T, C, ld, codes, meta);
+  if (rc != FB4_OK) return rc;
+  if (gain_plus_one != 0 && gain_plus_one != 1) return FB4_ERR_INVALID_ARG;
+  if (!(eps >= 0.0f) || eps > 3.0e38f) return FB4_ERR_INVALID_ARG;
+  const fb4_config& c = ctx->cfg;
+  if (c.block_size != 32 || c.num_groups != 8 || c.select_mode != 0 || c.exp_min != -124 || c.exp_max != 127 ||
+      !ctx->fast_ok)
+    return FB4_ERR_INVALID_ARG;
+  if (ld != C || C % 1024 != 0 || C > 16384 || T > 0x7fffffffLL) return FB4_ERR_SHAPE;
+  if (T == 0) return FB4_OK;
+  if (!gain || !bias) return FB4_ERR_INVALID_ARG;
+  if (cluster_id && (!cluster_mask || n_clusters <= 0)) return FB4_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(gain) & 15u) || (reinterpret_cast<uintptr_t>(bias) & 15u)) return FB4_ERR_ALIGN;
+  Fb4RowExtras ex{};
+  ex.cluster_id = cluster_id;
+  ex.cluster_mask = cluster_id ? cluster_mask : nullptr;
+  ex.n_clusters = cluster_id ? n_clusters : 0;
+  if (!fb4_fast_layernorm_eligible(ctx, x, T, C, ld, gain, bias)) return FB4_ERR_SHAPE;
+  const cudaError_t e = fb4_launch_quantize_layernorm(ctx, x, T, C, gain, bias, gain_plus_one, eps, ex, codes, meta,
+                                                      static_cast<cudaStream_t>(stream));
+  ctx->last_variant = "fast";
+  if (e != cudaSuccess) return fb4_set_cuda_error(e);
+  ctx->launches += 1;
+  return FB4_OK;
+}
+
 int fb4_quantize_affine(fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const void* gain,
                         const void* bias, int gain_plus_one, const int32_t* cluster_id, const uint32_t* cluster_mask,
                         int32_t n_clusters, uint8_t* codes, uint16_t* meta, void* stream) {

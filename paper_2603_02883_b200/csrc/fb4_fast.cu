@@ -1029,6 +1029,234 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
   if (SEDA && bad_cid && lane == 0) atomicOr(p.status, 2u);
 }
 
+// ---------------------------------------------------------------------------------------------
+// LayerNorm + per-channel modulation fused in front of the quantizer (App. D.2 names LayerNorm as an
+// operation the quantizer runs behind; the adaLN blocks modulate the normalised activation as
+// y = n * (1 + scale_c) + shift_c).  A token's C channels (a multiple of 1024, at most 16 384) belong to
+// C / 1024 warps of one CTA, lane = one block of 32 channels, held as 32 fp32 registers from the load to
+// the code store: the row is read once, y never exists in memory.  Every float32 operation is rounded
+// once and the additions have a fixed order, so the result is reproducible bit for bit:
+//   block sums in channel order; the 32 block sums of a warp by an xor butterfly (offsets 16 .. 1; all
+//   lanes end with the same bits because a + b = b + a); the warp sums of a token in warp order;
+//   mean = total / C; d = x - mean; sums of squares with q = fma(d, d, q), same reduction; var = total / C;
+//   rstd = 1 / sqrt(var + eps) (correctly rounded root and division); y = fma(d * rstd, g, b).
+// Same ring and tables as the flat kernel with one unit per lane; gain and bias of a lane's channels stay
+// in registers for the whole launch (a lane keeps its block column).  A CTA takes 16 / (C / 1024) tokens
+// per step; two CTA barriers per step carry the warp sums through shared memory.
+struct LnParams {
+  uint32_t T;
+  uint32_t units_row;      // C / 32
+  uint32_t wpr;            // warps per token = C / 1024
+  uint32_t rows_cta;       // tokens per CTA step
+  float c_f32;             // (float)C
+  float eps;
+  uint8_t* codes;
+  uint16_t* meta;
+  uint32_t* status;
+};
+
+template <bool PLUS_ONE, bool SEDA>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+fb4_quantize_layernorm_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
+                              LnParams p, const uint16_t* __restrict__ gain, const uint16_t* __restrict__ bias,
+                              Fb4RowExtras ex) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
+  float* part = reinterpret_cast<float*>(bars + kWarps * kStages + 1);      // [2 passes][kWarps] warp sums
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t row_local = (uint32_t)warp / p.wpr, wcol = (uint32_t)warp % p.wpr;
+  const bool warp_used = row_local < p.rows_cta;
+
+  const uint32_t table_bar = smem_u32(bars + kWarps * kStages);
+  if (lane == 0) {
+    for (int i = 0; i < kStages; ++i) mbar_init(smem_u32(bars + warp * kStages + i), 1);
+    if (warp == 0) mbar_init(table_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (warp == 0) {
+      mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
+      bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+    }
+  }
+  __syncthreads();
+  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytes);
+  const uint32_t my_bars = smem_u32(bars + warp * kStages);
+  // steps of this CTA: step i covers tokens (blockIdx.x + i * gridDim.x) * rows_cta + row_local
+  const uint32_t n_sets = (p.T + p.rows_cta - 1) / p.rows_cta;
+  const int32_t n_steps = blockIdx.x < n_sets ? (int32_t)((n_sets - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;
+  const uint32_t row0 = blockIdx.x * p.rows_cta + row_local;
+  const uint32_t row_step = gridDim.x * p.rows_cta;
+  auto tile_valid = [&](int32_t i) -> bool {
+    return warp_used && i < n_steps && (uint64_t)row0 + (uint64_t)i * row_step < p.T;
+  };
+  // prologue: fill the ring (2-D view [N/64][64]: a token's 128-byte rows start at row * C / 64)
+  const uint32_t rows128 = p.units_row / 2;
+#pragma unroll
+  for (int s = 0; s < kStages; ++s) {
+    if (tile_valid(s) && lane == 0) {
+      mbar_expect_tx(my_bars + 8 * s, kTileBytes);
+      tma_load_2d(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, 0,
+                  (int)((row0 + (uint32_t)s * row_step) * rows128 + wcol * 16u));
+    }
+  }
+  // gain and bias of this lane's 32 channels: fac[i] = gain bits | bias bits << 16
+  uint32_t fac[32];
+  {
+    uint32_t gw[16], bw[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) gw[k] = bw[k] = 0u;
+    if (warp_used) {
+      const uint4* gp = reinterpret_cast<const uint4*>(gain + ((size_t)wcol * 32 + lane) * 32);
+      const uint4* bp = reinterpret_cast<const uint4*>(bias + ((size_t)wcol * 32 + lane) * 32);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 g = __ldg(gp + q), b = __ldg(bp + q);
+        gw[4 * q] = g.x; gw[4 * q + 1] = g.y; gw[4 * q + 2] = g.z; gw[4 * q + 3] = g.w;
+        bw[4 * q] = b.x; bw[4 * q + 1] = b.y; bw[4 * q + 2] = b.z; bw[4 * q + 3] = b.w;
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      fac[2 * k] = (gw[k] & 0xffffu) | (bw[k] << 16);
+      fac[2 * k + 1] = (gw[k] >> 16) | (bw[k] & 0xffff0000u);
+    }
+  }
+  bool tables_ok;
+  {
+    uint32_t spins = 0;
+    bool ready = mbar_try_wait(table_bar, 0u);
+    while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(table_bar, 0u);
+    tables_ok = __all_sync(0xffffffffu, ready);
+  }
+  const uint32_t pair_base = smem_u32(tb->pairlut);
+  const uint32_t qerr_base = smem_u32(tb->qerr_private) + ((uint32_t)lane & 15u) * 8u;
+  const uint32_t r = (uint32_t)lane >> 1, c0 = ((uint32_t)lane & 1u) * 4u;
+  uint32_t chunk_off[4];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) chunk_off[j] = r * 128u + (((c0 + j) ^ (r & 7u)) << 4);
+
+  bool bad_cid = false;
+  // A wait that ran out (tables or a tile) is remembered per warp; the warp keeps meeting the CTA barriers
+  // but neither reads nor writes data any more, and the status bit is raised.
+  bool dead = !tables_ok;
+  int s = 0, s_dead = 0;
+  uint32_t parity = 0, parity_dead = 0;
+  int32_t it_dead = 0;
+  for (int32_t it = 0; it < n_steps; ++it) {
+    if (!dead) { s_dead = s; parity_dead = parity; it_dead = it; }   // where the ring stood when the warp gave up
+    const bool valid = tile_valid(it) && !dead;
+    const uint32_t row = row0 + (uint32_t)it * row_step;
+    uint32_t allowed = 0xffffffffu;
+    if (SEDA && valid) {
+      const int32_t cid = __ldg(ex.cluster_id + row);
+      if ((uint32_t)cid < (uint32_t)ex.n_clusters) {
+        const uint32_t m = __ldg(ex.cluster_mask + cid);
+        allowed = m ? m : 1u;
+      } else if (cid != -1) {
+        bad_cid = true;
+      }
+    }
+    const uint32_t bar = my_bars + 8 * s;
+    float x[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) x[i] = 0.0f;
+    if (tile_valid(it) && !dead) {
+      uint32_t spins = 0;
+      bool ready = mbar_try_wait(bar, parity);
+      while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(bar, parity);
+      if (!__all_sync(0xffffffffu, ready)) {
+        dead = true;
+      } else {
+        const uint32_t base = my_ring + s * kTileBytes;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const uint4 v = lds_v4(base + chunk_off[q]);
+          const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            x[8 * q + 2 * j] = __uint_as_float(w[j] << 16);
+            x[8 * q + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+          }
+        }
+      }
+    }
+    const bool live = valid && !dead;
+    // ---- mean: block sum in channel order, butterfly over the warp, warp sums of the token in order
+    float sum = x[0];
+#pragma unroll
+    for (int i = 1; i < 32; ++i) sum = __fadd_rn(sum, x[i]);
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xffffffffu, sum, off));
+    if (lane == 0) part[warp] = sum;
+    __syncthreads();
+    float total = part[row_local * p.wpr];
+    for (uint32_t k = 1; k < p.wpr; ++k) total = __fadd_rn(total, part[row_local * p.wpr + k]);
+    const float mean = __fdiv_rn(total, p.c_f32);
+    // ---- variance
+    float q = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      x[i] = __fsub_rn(x[i], mean);
+      q = __fmaf_rn(x[i], x[i], q);
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) q = __fadd_rn(q, __shfl_xor_sync(0xffffffffu, q, off));
+    if (lane == 0) part[kWarps + warp] = q;
+    __syncthreads();
+    float qt = part[kWarps + row_local * p.wpr];
+    for (uint32_t k = 1; k < p.wpr; ++k) qt = __fadd_rn(qt, part[kWarps + row_local * p.wpr + k]);
+    const float var = __fdiv_rn(qt, p.c_f32);
+    const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, p.eps)));
+    if (live) {
+      // ---- modulation, cut to the upper 16 bits (all the quantizer needs), quantize, store
+      uint32_t yw[16];
+#pragma unroll
+      for (int k = 0; k < 16; ++k) {
+        uint32_t y[2];
+#pragma unroll
+        for (int hlf = 0; hlf < 2; ++hlf) {
+          const uint32_t f = fac[2 * k + hlf];
+          float g = __uint_as_float(f << 16);
+          if (PLUS_ONE) g = __fadd_rn(1.0f, g);
+          y[hlf] = __float_as_uint(__fmaf_rn(__fmul_rn(x[2 * k + hlf], rstd), g, __uint_as_float(f & 0xffff0000u)));
+        }
+        yw[k] = __byte_perm(y[0], y[1], 0x7632);
+      }
+      uint32_t cw[4], Eb[2];
+      int did[2];
+      quantize_packed_block<SEDA, false, false>(yw, allowed, tb, qerr_base, pair_base, 3u, 254u, cw, did, Eb);
+      const size_t unit = (size_t)row * p.units_row + wcol * 32u + (uint32_t)lane;
+      *reinterpret_cast<uint4*>(p.codes + unit * 16u) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      p.meta[unit] = (uint16_t)((Eb[0] - 3u) | ((uint32_t)did[0] << 8));
+    }
+    // ---- refill this stage
+    __syncwarp();
+    if (lane == 0 && !dead && tile_valid(it + kStages)) {
+      mbar_expect_tx(bar, kTileBytes);
+      tma_load_2d(my_ring + s * kTileBytes, &tmap, bar, 0,
+                  (int)((row0 + (uint32_t)(it + kStages) * row_step) * rows128 + wcol * 16u));
+    }
+    if (++s == kStages) { s = 0; parity ^= 1u; }
+  }
+  if (dead) {
+    if (lane == 0) atomicOr(p.status, 1u);
+    // the loads still in flight for this warp (the kStages tiles from the step it gave up at) get a bounded
+    // chance to land before the CTA's shared memory goes
+    for (int j = 0; j < kStages; ++j) {
+      if (!tile_valid(it_dead + j)) break;
+      const int sj = (s_dead + j) % kStages;
+      const uint32_t pj = (s_dead + j) >= kStages ? (parity_dead ^ 1u) : parity_dead;
+      uint32_t tries = 0;
+      while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
+    }
+  }
+  if (SEDA && bad_cid && lane == 0) atomicOr(p.status, 2u);
+}
+
+constexpr size_t kSmemBytesLn = 
+    1024 + (size_t)kWarps * kStages * kTileBytes + sizeof(SmemTables) + (kWarps * kStages + 1) * 8 + 2 * kWarps * sizeof(float);
+
 constexpr size_t kSmemBytesF32 =
     1024 + (size_t)kWarpsF32 * kStages * kTileBytesF32 + sizeof(SmemTables) + (kWarpsF32 * kStages + 1) * 8;
 static_assert(kSmemBytesF32 <= 227 * 1024, "shared memory budget of one CTA");
@@ -1054,6 +1282,7 @@ EncodeTiledFn encode_tiled_fn() {
 constexpr size_t kSmemBytes =
     1024 + (size_t)kWarps * kStages * kTileBytes + sizeof(SmemTables) + (kWarps * kStages + 1) * 8;
 static_assert(kSmemBytes <= 227 * 1024, "shared memory budget of one CTA");
+static_assert(kSmemBytesLn <= 227 * 1024, "shared memory budget of one CTA");
 static_assert(sizeof(SmemTables) % 16 == 0, "bulk copy size; mbarriers behind the tables stay 8-byte aligned");
 
 template <bool SEDA, bool DECOMP, bool B16, bool CLAMP>
@@ -1202,6 +1431,10 @@ cudaError_t fb4_fast_prepare_device() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, false, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, true, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, true, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<false, false>, attr, (int)kSmemBytesLn);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<true, false>, attr, (int)kSmemBytesLn);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<false, true>, attr, (int)kSmemBytesLn);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<true, true>, attr, (int)kSmemBytesLn);
   return e;
 }
 
@@ -1540,3 +1773,47 @@ cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, i
   return cudaGetLastError();
 }
 
+
+// LayerNorm producer + quantizer in one pass: default configuration, contiguous rows, C a multiple of 1024
+// and at most 16 384 (one warp per 1024 channels, a token inside one CTA).
+bool fb4_fast_layernorm_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const void* gain,
+                                 const void* bias) {
+  if (!fb4_fast_mx_eligible(ctx, x, T, C, ld)) return false;
+  if ((reinterpret_cast<uintptr_t>(gain) & 15) || (reinterpret_cast<uintptr_t>(bias) & 15)) return false;
+  return flat_eligible(T, C, ld) && C % 1024 == 0 && C <= 1024 * kWarps;
+}
+
+cudaError_t fb4_launch_quantize_layernorm(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, const void* gain,
+                                          const void* bias, int plus_one, float eps, const Fb4RowExtras& ex,
+                                          uint8_t* codes, uint16_t* meta, cudaStream_t stream) {
+  CUtensorMap map;
+  FlatParams fp;
+  int grid = 0;
+  const cudaError_t e = flat_setup(ctx, x, T, C, true, false, &map, &fp, &grid);   // one unit per lane: 2 KB tiles
+  if (e != cudaSuccess) return e;
+  LnParams p{};
+  p.T = (uint32_t)T;
+  p.units_row = (uint32_t)(C / 32);
+  p.wpr = (uint32_t)(C / 1024);
+  p.rows_cta = (uint32_t)kWarps / p.wpr;
+  p.c_f32 = (float)C;
+  p.eps = eps;
+  p.codes = codes;
+  p.meta = meta;
+  p.status = ctx->d_status;
+  const int64_t n_sets = (T + p.rows_cta - 1) / p.rows_cta;
+  grid = (int)(n_sets < ctx->sm_count ? n_sets : ctx->sm_count);
+  const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
+  const uint16_t* g = static_cast<const uint16_t*>(gain);
+  const uint16_t* b = static_cast<const uint16_t*>(bias);
+#define FB4_LN(P, S) \
+  fb4_quantize_layernorm_kernel<P, S><<<grid, kWarps * 32, kSmemBytesLn, stream>>>(map, tables, p, g, b, ex)
+  switch ((plus_one ? 1 : 0) | (ex.cluster_id ? 2 : 0)) {
+    case 0: FB4_LN(false, false); break;
+    case 1: FB4_LN(true, false); break;
+    case 2: FB4_LN(false, true); break;
+    default: FB4_LN(true, true); break;
+  }
+#undef FB4_LN
+  return cudaGetLastError();
+}

@@ -70,6 +70,11 @@ cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, i
                                             const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
                                             cudaStream_t stream, uint8_t* e4m3 = nullptr, uint8_t* scales = nullptr,
                                             int tiled = 0);   // e4m3 != NULL: MXFP8 output instead of codes / meta
+bool fb4_fast_layernorm_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, const void* gain,
+                                 const void* bias);
+cudaError_t fb4_launch_quantize_layernorm(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, const void* gain,
+                                          const void* bias, int plus_one, float eps, const Fb4RowExtras& ex,
+                                          uint8_t* codes, uint16_t* meta, cudaStream_t stream);
 bool fb4_fast_f32_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld);
 cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
                                          uint8_t* codes, uint16_t* meta, cudaStream_t stream);

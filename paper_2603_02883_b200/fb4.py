@@ -21,7 +21,7 @@ ERR_STATIC_LIMIT = -7
 STATIC_MAX_CLUSTERS = 1024
 
 EXPORTS = [
-    "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_block_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_affine", "fb4_quantize_affine_mxfp8", "fb4_quantize_seda",
+    "fb4_default_config", "fb4_init", "fb4_destroy", "fb4_get_tables", "fb4_block_tables", "fb4_quantize", "fb4_quantize_f32", "fb4_quantize_affine", "fb4_quantize_affine_mxfp8", "fb4_quantize_layernorm", "fb4_quantize_seda",
     "fb4_build_subformatbook", "fb4_build_subformatbook_static", "fb4_select_salient", "fb4_select_salient_topk", "fb4_quantize_decomposed", "fb4_quantize_decomposed_idx", "fb4_dequantize",
     "fb4_quantize_weights", "fb4_quantize_mxfp8", "fb4_quantize_mxfp8_decomposed", "fb4_to_mxfp8", "fb4_mxfp8_scale_bytes", "fb4_quantize_host", "fb4_set_kernel_variant", "fb4_device_status", "fb4_launch_count", "fb4_last_variant", "fb4_last_cuda_error", "fb4_strerror",
 ]
@@ -75,6 +75,8 @@ def lib() -> ctypes.CDLL:
     L.fb4_quantize_f32.restype = ci
     L.fb4_quantize_affine.argtypes = [vp, vp, i64, i64, i64, vp, vp, ci, vp, vp, i32, vp, vp, vp]
     L.fb4_quantize_affine.restype = ci
+    L.fb4_quantize_layernorm.argtypes = [vp, vp, i64, i64, i64, vp, vp, ci, ctypes.c_float, vp, vp, i32, vp, vp, vp]
+    L.fb4_quantize_layernorm.restype = ci
     L.fb4_quantize_affine_mxfp8.argtypes = [vp, vp, i64, i64, i64, vp, vp, ci, vp, vp, i32, vp, vp, ci, vp]
     L.fb4_quantize_affine_mxfp8.restype = ci
     L.fb4_quantize_seda.argtypes = [vp, vp, i64, i64, i64, vp, vp, i32, vp, vp, vp]
@@ -192,6 +194,13 @@ def fb4_quantize_affine(ctx, x, T, C, ld_elems, gain, bias, gain_plus_one, clust
     _check(lib().fb4_quantize_affine(ctx, _ptr(x), T, C, ld_elems, _ptr(gain), _ptr(bias), int(bool(gain_plus_one)),
                                      _ptr(cluster_id), _ptr(cluster_mask), n_clusters, _ptr(codes), _ptr(meta),
                                      _stream(stream)), "fb4_quantize_affine")
+
+
+def fb4_quantize_layernorm(ctx, x, T, C, ld_elems, gain, bias, gain_plus_one, eps, cluster_id, cluster_mask, n_clusters,
+                           codes, meta, stream=None) -> None:
+    _check(lib().fb4_quantize_layernorm(ctx, _ptr(x), T, C, ld_elems, _ptr(gain), _ptr(bias), int(bool(gain_plus_one)),
+                                        ctypes.c_float(eps), _ptr(cluster_id), _ptr(cluster_mask), n_clusters,
+                                        _ptr(codes), _ptr(meta), _stream(stream)), "fb4_quantize_layernorm")
 
 
 def fb4_quantize_affine_mxfp8(ctx, x, T, C, ld_elems, gain, bias, gain_plus_one, cluster_id, cluster_mask, n_clusters, e4m3,
@@ -373,6 +382,15 @@ class Fb4:
         codes, meta = self._outs(T, C)
         fb4_quantize_affine(self.ctx, x, T, C, ld, gain, bias, gain_plus_one, cluster_id, cluster_mask,
                             0 if cluster_mask is None else cluster_mask.numel(), codes, meta)
+        return Quantized(codes, meta)
+
+    def quantize_layernorm(self, x, gain, bias, gain_plus_one: bool = False, eps: float = 1e-6, cluster_id=None,
+                           cluster_mask=None) -> Quantized:
+        """quantize(LayerNorm(x) * g + bias), g = gain or 1 + gain per channel, in one fused pass"""
+        T, C, ld = self._shape(x)
+        codes, meta = self._outs(T, C)
+        fb4_quantize_layernorm(self.ctx, x, T, C, ld, gain, bias, gain_plus_one, eps, cluster_id, cluster_mask,
+                               0 if cluster_mask is None else cluster_mask.numel(), codes, meta)
         return Quantized(codes, meta)
 
     def quantize_affine_mxfp8(self, x, gain, bias, gain_plus_one: bool = False, scale_layout: int = 1, cluster_id=None,
