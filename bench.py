@@ -220,6 +220,14 @@ class Ops:
             self._buf["affine"] = (sc, sh)
             return (lambda: fb4.fb4_quantize_affine(q.ctx, x, T, C, C, sc, sh, 1, None, None, 0, codes, meta)), \
                 algorithmic_bytes(T, C) + 4 * C
+        if name == "layernorm_plus_quantize":
+            # LayerNorm statistics + modulation y = n * (1 + scale_c) + shift_c fused in front of the quantizer
+            gen = torch.Generator(device="cuda").manual_seed(7)
+            sc = (0.5 * torch.randn(C, device="cuda", generator=gen)).to(torch.bfloat16)
+            sh = torch.randn(C, device="cuda", generator=gen).to(torch.bfloat16)
+            self._buf["layernorm"] = (sc, sh)
+            return (lambda: fb4.fb4_quantize_layernorm(q.ctx, x, T, C, C, sc, sh, 1, 1e-6, None, None, 0, codes, meta)), \
+                algorithmic_bytes(T, C) + 4 * C
         if name == "affine_plus_quantize_mxfp8":
             gen = torch.Generator(device="cuda").manual_seed(7)
             sc_v = (0.5 * torch.randn(C, device="cuda", generator=gen)).to(torch.bfloat16)
@@ -296,7 +304,7 @@ class Ops:
         raise KeyError(name)
 
 
-OP_NAMES = ["plain", "plain_block16", "plain_f32", "affine_plus_quantize", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
+OP_NAMES = ["plain", "plain_block16", "plain_f32", "affine_plus_quantize", "layernorm_plus_quantize", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
             "dequantize_bf16_plain", "dequantize_bf16_decomposed", "dequantize_f16_plain", "to_mxfp8_tiled_scales",
             "quantize_mxfp8_tiled_scales", "quantize_mxfp8_decomposed_seda", "affine_plus_quantize_mxfp8"]
 
@@ -315,6 +323,8 @@ def main():
     ap.add_argument("--no-variants", action="store_true", help="time only the step")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sustained-steps", type=int, default=1500,
+                    help="length of the clock-binned run of the step (0 = skip)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -395,6 +405,8 @@ def main():
         out["quality"] = quality_report(ops, torch, fb4)
     if rank == 0 and not args.no_variants:
         out["variants"] = run_variants(ops, args, torch, fb4, synth, peak)
+    if rank == 0 and world == 1 and args.sustained_steps > 0:
+        out["sustained"] = run_sustained(step, alg, args.sustained_steps, visible_index(local_rank), torch, peak)
     del ops
     if not args.no_e2e:
         e2e = run_e2e(q, bits, w, args, torch, fb4, barrier)
@@ -406,11 +418,66 @@ def main():
         out["e2e"] = e2e
     if rank == 0 and not args.no_cpu_baseline:
         out["cpu_baseline"] = run_cpu_baseline(w, synth)
+    if rank == 0 and world == 1 and not args.no_variants:
+        out["c_abi_host_cost"] = run_host_cost()
     if rank == 0:
         print(json.dumps(out))
     q.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_sustained(step, alg, steps, index, torch, peak):
+    """The step repeated for about half a second and longer, timed in chunks of 25 launches with CUDA events, the
+    SM clock read through NVML once per chunk: throughput binned by the clock the GPU settled at.  On a 1 kW part
+    the power cap pulls the clock down after some tens of milliseconds of this kernel; nothing is set or reset
+    here, the clocks are only read."""
+    chunk = 25
+    n = max(steps // chunk, 8)
+    try:
+        import pynvml
+        pynvml.nvmlInit()
+        h = pynvml.nvmlDeviceGetHandleByIndex(index)
+    except Exception:
+        return None
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+    clocks, power = [], []
+    ev[0].record()
+    for c in range(n):
+        for _ in range(chunk):
+            step()
+        ev[c + 1].record()
+        if c >= 4:
+            ev[c - 3].synchronize()          # a short queue, so that the sample belongs to the chunks around it
+            clocks.append(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+            power.append(pynvml.nvmlDeviceGetPowerUsage(h) / 1000.0)
+    torch.cuda.synchronize()
+    ms = [ev[c].elapsed_time(ev[c + 1]) / chunk for c in range(n)]
+    bins = {}
+    for c, mhz in enumerate(clocks):
+        bins.setdefault(int(round(mhz / 50.0) * 50), []).append(ms[c + 1])
+    out = {str(k): {"chunks": len(v), "frac_hbm_measured": alg / (sum(v) / len(v) * 1e-3) / 1e9 / peak,
+                    "ms_times_mhz": sum(v) / len(v) * k} for k, v in sorted(bins.items())}
+    lowest = min(bins) if bins else None
+    return {"steps": n * chunk, "seconds": sum(ms) * chunk * 1e-3, "chunk_launches": chunk, "by_sm_mhz": out,
+            "lowest_sm_mhz": lowest, "frac_at_lowest_clock": out[str(lowest)]["frac_hbm_measured"] if bins else None,
+            "first_chunk_frac": alg / (ms[0] * 1e-3) / 1e9 / peak, "last_chunk_frac": alg / (ms[-1] * 1e-3) / 1e9 / peak,
+            "power_w_max": max(power) if power else None}
+
+
+def run_host_cost():
+    """Host microseconds per C-ABI call on the small tensor, measured by the C program of the package (no Python in
+    the timed loop); None if it cannot be built or run."""
+    import subprocess
+    try:
+        from paper_2603_02883_b200 import build as _b
+        exe = _b.build_hostcost()
+        r = subprocess.run([exe, "200", "20"], capture_output=True, text=True, timeout=120)
+        if r.returncode != 0:
+            return {"error": (r.stderr or r.stdout).strip()[-200:]}
+        return json.loads(r.stdout.strip().splitlines()[-1])
+    except Exception as e:   # no gcc / no CUDA headers on this machine
+        return {"error": str(e)[-200:]}
 
 
 def quality_report(ops, torch, fb4):
@@ -443,7 +510,7 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         total, per = time_steps(fn, steps, warm, torch)
         ms = total / steps
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
-                     "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "affine_plus_quantize", "seda", "decomposed", "decomposed_given_set",
+                     "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "affine_plus_quantize", "layernorm_plus_quantize", "seda", "decomposed", "decomposed_given_set",
                                                                          "decomposed_seda", "quantize_mxfp8_tiled_scales",
                                                                          "quantize_mxfp8_decomposed_seda", "affine_plus_quantize_mxfp8")
                      else "decode"}

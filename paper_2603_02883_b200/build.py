@@ -66,5 +66,21 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+HOSTCOST = os.path.join(HERE, "fb4_hostcost")
+
+
+def build_hostcost(force: bool = False) -> str:
+    """The C program that times the host side of the ABI (hostcost/fb4_hostcost.c), linked against libfb4.so."""
+    src = os.path.join(HERE, "hostcost", "fb4_hostcost.c")
+    if not force and os.path.exists(HOSTCOST) and os.path.getmtime(HOSTCOST) >= max(os.path.getmtime(src), os.path.getmtime(LIB)):
+        return HOSTCOST
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    subprocess.check_call(["gcc", "-O2", "-std=c99", "-I", INCLUDE, "-I", os.path.join(cuda, "include"), src, "-o", HOSTCOST,
+                           "-L", HERE, "-lfb4", "-L", os.path.join(cuda, "lib64"), "-lcudart",
+                           "-Wl,-rpath," + HERE, "-Wl,-rpath," + os.path.join(cuda, "lib64")])
+    return HOSTCOST
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build_hostcost(force="--force" in sys.argv))

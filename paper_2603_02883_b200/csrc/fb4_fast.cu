@@ -1450,6 +1450,25 @@ bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, 
   return encode_tiled_fn() != nullptr;
 }
 
+static_assert(sizeof(CUtensorMap) == sizeof(Fb4TensorMapSlot::map), "slot size");
+
+// The encoded tensor map of (x, T, C, ld) for kernel family `kind`: from the context's slot if the last launch
+// of that family had the same arguments, else encoded by `encode` and kept.
+template <typename Encode>
+static cudaError_t cached_tensor_map(const fb4_ctx* ctx, int kind, const void* x, int64_t T, int64_t C, int64_t ld,
+                                     CUtensorMap* map, Encode encode) {
+  Fb4TensorMapSlot& sl = ctx->tmap_slot[kind];
+  if (sl.valid && sl.x == x && sl.T == T && sl.C == C && sl.ld == ld) {
+    std::memcpy(map, sl.map, sizeof(CUtensorMap));
+    return cudaSuccess;
+  }
+  if (encode(map) != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  sl.x = x; sl.T = T; sl.C = C; sl.ld = ld;
+  std::memcpy(sl.map, map, sizeof(CUtensorMap));
+  sl.valid = 1;
+  return cudaSuccess;
+}
+
 // Tensor map, grid and tile-walk parameters of one launch of the bf16-input kernels.
 static cudaError_t fast_setup(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld, bool chunked,
                               CUtensorMap* map, FastParams* p, int* grid_out) {
@@ -1457,10 +1476,12 @@ static cudaError_t fast_setup(const fb4_ctx* ctx, const void* x, int64_t T, int6
   const cuuint64_t strides[2] = {128, (cuuint64_t)ld * 2};
   const cuuint32_t box[3] = {64, 16, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = encode_tiled_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides,
-                                       box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  const cudaError_t ce = cached_tensor_map(ctx, 0, x, T, C, ld, map, [&](CUtensorMap* m) {
+    return encode_tiled_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  });
+  if (ce != cudaSuccess) return ce;
   *p = FastParams{};
   p->T = T;
   p->C = C;
@@ -1491,10 +1512,12 @@ static cudaError_t flat_setup(const fb4_ctx* ctx, const void* x, int64_t T, int6
   const cuuint64_t strides[1] = {128};
   const cuuint32_t box[2] = {64, 16 * U};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = encode_tiled_fn()(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box,
-                                       estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  const cudaError_t ce = cached_tensor_map(ctx, (int)U, x, T, C, C, map, [&](CUtensorMap* m) {
+    return encode_tiled_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  });
+  if (ce != cudaSuccess) return ce;
   *p = FlatParams{};
   p->units_row = (uint32_t)(C / 32);
   p->n_units = (uint32_t)(T * (C / 32));
@@ -1606,10 +1629,12 @@ cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int6
   const cuuint64_t strides[2] = {128, (cuuint64_t)ld * 4};
   const cuuint32_t box[3] = {32, 32, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  const CUresult r = encode_tiled_fn()(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(x), dims, strides,
-                                       box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+  const cudaError_t ce = cached_tensor_map(ctx, 3, x, T, C, ld, &map, [&](CUtensorMap* m) {
+    return encode_tiled_fn()(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(x), dims, strides, box, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  });
+  if (ce != cudaSuccess) return ce;
   FastParams p{};
   p.T = T;
   p.C = C;

@@ -32,8 +32,18 @@ struct Fb4RowExtras {
   uint16_t* res_meta;           // [n_salient][C/B]
 };
 
+// The tensor map of the last launch of each kernel family (encoding one costs a good part of a microsecond on the
+// host; a layer quantizes the same buffer step after step).
+struct Fb4TensorMapSlot {
+  const void* x;
+  int64_t T, C, ld;
+  int valid;
+  alignas(64) unsigned char map[128];
+};
+
 struct fb4_ctx {
   int device;
+  mutable Fb4TensorMapSlot tmap_slot[4];   // 0: strided bf16, 1: flat, 2 KB tiles, 2: flat, 4 KB tiles, 3: fp32 input
   fb4_config cfg;
   Fb4DeviceTables host_tables;   // host copy
   Fb4DeviceTables* d_tables;     // device copy
