@@ -176,7 +176,7 @@ int fb4_quantize_affine_mxfp8(fb4_ctx* ctx, const void* x_bf16, int64_t T, int64
  * d * d + q and (d * rstd) * g + bias as fused multiply-adds, and the additions in a fixed order: the
  * 32 channels of a block in index order; the 32 block sums of a run of 1024 channels by an xor butterfly
  * (v_i <- v_i + v_(i xor off) for off = 16, 8, 4, 2, 1, all i at once; the run's sum is v_0); the runs of a
- * token in order.  The result is therefore reproducible bit for bit; it is quantized from registers as
+ * token added to +0 in order.  The result is therefore reproducible bit for bit; it is quantized from registers as
  * fb4_quantize_f32 quantizes a float32 tensor, so the token is read once and y never exists in memory.
  * Optional SeDA restriction as in fb4_quantize_seda.  One fused pass; default configuration only,
  * contiguous rows (ld_elems == C), C a multiple of 1024 and at most 16384, gain and bias 16-byte

@@ -407,7 +407,7 @@ int fb4o_affine_f32(const uint16_t *x, int64_t T, int64_t C, int64_t ld, const u
  *   segment sums  the block sums of 32 consecutive blocks (1024 channels; a short last segment is filled
  *                 up with +0) are added as a butterfly: for off = 16, 8, 4, 2, 1, all at once,
  *                 v_i <- v_i + v_(i xor off); the segment sum is v_0;
- *   row total     the segment sums added in order, ((S_0 + S_1) + S_2) + ...;
+ *   row total     the segment sums added to +0 in order, (((0 + S_0) + S_1) + S_2) + ...;
  *   mean = total / C;  d_i = x_i - mean;
  *   the sum of squares by the same three steps with q_b = fma(d, d, q) over the block's channels in order
  *   (q = 0 at the start);  var = total of squares / C;  rstd = 1 / sqrt(var + eps);
@@ -426,12 +426,9 @@ static float ln_segment_butterfly(const float *blocksum, int n) {
 
 static float ln_row_total(const float *blocksum, int64_t nblk) {
   float total = 0.0f;
-  int first = 1;
   for (int64_t b0 = 0; b0 < nblk; b0 += 32) {
     int n = nblk - b0 < 32 ? (int)(nblk - b0) : 32;
-    float seg = ln_segment_butterfly(blocksum + b0, n);
-    total = first ? seg : total + seg;
-    first = 0;
+    total = total + ln_segment_butterfly(blocksum + b0, n);
   }
   return total;
 }

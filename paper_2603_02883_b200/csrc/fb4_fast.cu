@@ -1033,21 +1033,23 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
 // LayerNorm + per-channel modulation fused in front of the quantizer (App. D.2 names LayerNorm as an
 // operation the quantizer runs behind; the adaLN blocks modulate the normalised activation as
 // y = n * (1 + scale_c) + shift_c).  A token's C channels (a multiple of 1024, at most 16 384) belong to
-// C / 1024 warps of one CTA, lane = one block of 32 channels, held as 32 fp32 registers from the load to
-// the code store: the row is read once, y never exists in memory.  Every float32 operation is rounded
-// once and the additions have a fixed order, so the result is reproducible bit for bit:
+// C / 1024 warps of one CTA, lane = one block of 32 channels, held in registers (as the 16 packed input
+// words) from the load to the code store: the row is read once, y never exists in memory.  Every float32
+// operation is rounded once and the additions have a fixed order, so the result is reproducible bit for bit:
 //   block sums in channel order; the 32 block sums of a warp by an xor butterfly (offsets 16 .. 1; all
-//   lanes end with the same bits because a + b = b + a); the warp sums of a token in warp order;
+//   lanes end with the same bits because a + b = b + a); the warp sums of a token added to +0 in warp order;
 //   mean = total / C; d = x - mean; sums of squares with q = fma(d, d, q), same reduction; var = total / C;
 //   rstd = 1 / sqrt(var + eps) (correctly rounded root and division); y = fma(d * rstd, g, b).
 // Same ring and tables as the flat kernel with one unit per lane; gain and bias of a lane's channels stay
-// in registers for the whole launch (a lane keeps its block column).  A CTA takes 16 / (C / 1024) tokens
-// per step; two CTA barriers per step carry the warp sums through shared memory.
+// in registers for the whole launch (a lane keeps its block column).  The warp sums travel through shared
+// memory behind two CTA barriers per step, and between barriers every chain of additions is a latency
+// chain, so a step takes TWO tokens per team of warps (a CTA takes 2 * 16 / (C / 1024) tokens per step):
+// the chains of the two tokens interleave and a token costs one barrier.
 struct LnParams {
   uint32_t T;
   uint32_t units_row;      // C / 32
   uint32_t wpr;            // warps per token = C / 1024
-  uint32_t rows_cta;       // tokens per CTA step
+  uint32_t teams;          // teams of wpr warps per CTA; a team takes two tokens per step
   float c_f32;             // (float)C
   float eps;
   uint8_t* codes;
@@ -1055,8 +1057,10 @@ struct LnParams {
   uint32_t* status;
 };
 
-template <bool PLUS_ONE, bool SEDA>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+// NW = warps per CTA: 12 where the warps of a token divide 12 (170 registers per thread, room for two tokens and
+// the factors), 16 otherwise.
+template <bool PLUS_ONE, bool SEDA, int NW>
+__global__ void __launch_bounds__(NW * 32, 1)
 fb4_quantize_layernorm_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
                               LnParams p, const uint16_t* __restrict__ gain, const uint16_t* __restrict__ bias,
                               Fb4RowExtras ex) {
@@ -1064,10 +1068,11 @@ fb4_quantize_layernorm_kernel(const __grid_constant__ CUtensorMap tmap, const Sm
   uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
-  float* part = reinterpret_cast<float*>(bars + kWarps * kStages + 1);      // [2 passes][kWarps] warp sums
+  // warp sums: [2 passes][2 tokens][team][16], a team's entries padded with +0 to 16 (written once, below)
+  float* part = reinterpret_cast<float*>(bars + kWarps * kStages + 2);      // 16-byte aligned: the barriers are an odd count
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t row_local = (uint32_t)warp / p.wpr, wcol = (uint32_t)warp % p.wpr;
-  const bool warp_used = row_local < p.rows_cta;
+  const uint32_t team = (uint32_t)warp / p.wpr, wcol = (uint32_t)warp % p.wpr;
+  const bool warp_used = team < p.teams;
 
   const uint32_t table_bar = smem_u32(bars + kWarps * kStages);
   if (lane == 0) {
@@ -1079,31 +1084,37 @@ fb4_quantize_layernorm_kernel(const __grid_constant__ CUtensorMap tmap, const Sm
       bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
     }
   }
+  for (int i = threadIdx.x; i < 4 * kWarps * 16; i += blockDim.x) part[i] = 0.0f;
   __syncthreads();
   const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytes);
   const uint32_t my_bars = smem_u32(bars + warp * kStages);
-  // steps of this CTA: step i covers tokens (blockIdx.x + i * gridDim.x) * rows_cta + row_local
-  const uint32_t n_sets = (p.T + p.rows_cta - 1) / p.rows_cta;
+  // Step i of this CTA covers the token pairs (blockIdx.x + i * gridDim.x) * teams + team; a pair is the tokens
+  // 2 * pair and 2 * pair + 1.  Ring stage 2 * (i mod 2) + ab holds this warp's 1024 channels of token ab of step i.
+  const uint32_t n_pairs = (p.T + 1u) / 2u;
+  const uint32_t n_sets = (n_pairs + p.teams - 1) / p.teams;
   const int32_t n_steps = blockIdx.x < n_sets ? (int32_t)((n_sets - blockIdx.x + gridDim.x - 1) / gridDim.x) : 0;
-  const uint32_t row0 = blockIdx.x * p.rows_cta + row_local;
-  const uint32_t row_step = gridDim.x * p.rows_cta;
-  auto tile_valid = [&](int32_t i) -> bool {
-    return warp_used && i < n_steps && (uint64_t)row0 + (uint64_t)i * row_step < p.T;
+  const uint32_t pair0 = blockIdx.x * p.teams + team;
+  const uint32_t pair_step = gridDim.x * p.teams;
+  auto row_of = [&](int32_t i, int ab) -> uint64_t { return 2u * ((uint64_t)pair0 + (uint64_t)i * pair_step) + (uint64_t)ab; };
+  auto tile_valid = [&](int32_t i, int ab) -> bool { return warp_used && i < n_steps && row_of(i, ab) < p.T; };
+  const uint32_t rows128 = p.units_row / 2;      // 128-byte rows of the 2-D view per token
+  auto request = [&](int32_t i, int ab) {
+    const uint32_t st = (uint32_t)(2 * (i & 1) + ab);
+    mbar_expect_tx(my_bars + 8 * st, kTileBytes);
+    tma_load_2d(my_ring + st * kTileBytes, &tmap, my_bars + 8 * st, 0, (int)((uint32_t)row_of(i, ab) * rows128 + wcol * 16u));
   };
-  // prologue: fill the ring (2-D view [N/64][64]: a token's 128-byte rows start at row * C / 64)
-  const uint32_t rows128 = p.units_row / 2;
+  if (lane == 0) {
 #pragma unroll
-  for (int s = 0; s < kStages; ++s) {
-    if (tile_valid(s) && lane == 0) {
-      mbar_expect_tx(my_bars + 8 * s, kTileBytes);
-      tma_load_2d(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, 0,
-                  (int)((row0 + (uint32_t)s * row_step) * rows128 + wcol * 16u));
-    }
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int ab = 0; ab < 2; ++ab)
+        if (tile_valid(i, ab)) request(i, ab);
   }
-  // gain and bias of this lane's 32 channels: fac[i] = gain bits | bias bits << 16
-  uint32_t fac[32];
+  // this lane's 32 channels: the factor g = gain or 1 + gain in float32, the bias as loaded (two bf16 per register)
+  float gf[32];
+  uint32_t bw[16];
   {
-    uint32_t gw[16], bw[16];
+    uint32_t gw[16];
 #pragma unroll
     for (int k = 0; k < 16; ++k) gw[k] = bw[k] = 0u;
     if (warp_used) {
@@ -1118,8 +1129,12 @@ fb4_quantize_layernorm_kernel(const __grid_constant__ CUtensorMap tmap, const Sm
     }
 #pragma unroll
     for (int k = 0; k < 16; ++k) {
-      fac[2 * k] = (gw[k] & 0xffffu) | (bw[k] << 16);
-      fac[2 * k + 1] = (gw[k] >> 16) | (bw[k] & 0xffff0000u);
+      gf[2 * k] = __uint_as_float(gw[k] << 16);
+      gf[2 * k + 1] = __uint_as_float(gw[k] & 0xffff0000u);
+      if (PLUS_ONE) {
+        gf[2 * k] = __fadd_rn(1.0f, gf[2 * k]);
+        gf[2 * k + 1] = __fadd_rn(1.0f, gf[2 * k + 1]);
+      }
     }
   }
   bool tables_ok;
@@ -1135,127 +1150,175 @@ fb4_quantize_layernorm_kernel(const __grid_constant__ CUtensorMap tmap, const Sm
   uint32_t chunk_off[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) chunk_off[j] = r * 128u + (((c0 + j) ^ (r & 7u)) << 4);
-
+  // the warp sums of this warp's team, added to +0 in warp order; the entries behind the team's last warp hold +0,
+  // which leaves the sum as it is, so whole groups of four are read and added
+  auto team_total = [&](const float* ps) -> float {
+    const float4* v4 = reinterpret_cast<const float4*>(ps + team * 16u);
+    float t = 0.0f;
+#pragma unroll
+    for (int k4 = 0; k4 < kWarps / 4; ++k4) {
+      if ((uint32_t)(4 * k4) >= p.wpr) break;
+      const float4 v = v4[k4];
+      t = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(t, v.x), v.y), v.z), v.w);
+    }
+    return t;
+  };
+  // The warps of a team meet at a barrier of their own (hardware barrier 1 + team), so the teams of a CTA drift
+  // apart and one team's additions overlap another team's quantization; warps outside every team meet nobody.
+  auto team_sync = [&]() {
+    if (warp_used) asm volatile("bar.sync %0, %1;" ::"r"(team + 1u), "r"(p.wpr * 32u) : "memory");
+  };
   bool bad_cid = false;
-  // A wait that ran out (tables or a tile) is remembered per warp; the warp keeps meeting the CTA barriers
+  // A wait that ran out (tables or a tile) is remembered per warp; the warp keeps meeting its team's barriers
   // but neither reads nor writes data any more, and the status bit is raised.
   bool dead = !tables_ok;
-  int s = 0, s_dead = 0;
   uint32_t parity = 0, parity_dead = 0;
   int32_t it_dead = 0;
   for (int32_t it = 0; it < n_steps; ++it) {
-    if (!dead) { s_dead = s; parity_dead = parity; it_dead = it; }   // where the ring stood when the warp gave up
-    const bool valid = tile_valid(it) && !dead;
-    const uint32_t row = row0 + (uint32_t)it * row_step;
-    uint32_t allowed = 0xffffffffu;
-    if (SEDA && valid) {
-      const int32_t cid = __ldg(ex.cluster_id + row);
-      if ((uint32_t)cid < (uint32_t)ex.n_clusters) {
-        const uint32_t m = __ldg(ex.cluster_mask + cid);
-        allowed = m ? m : 1u;
-      } else if (cid != -1) {
-        bad_cid = true;
+    if (!dead) { parity_dead = parity; it_dead = it; }   // where the ring stood when the warp gave up
+    const uint32_t st0 = (uint32_t)(2 * (it & 1));
+    bool live[2];
+    uint32_t allowed[2] = {0xffffffffu, 0xffffffffu};
+    uint32_t w[2][16];       // the two tokens' blocks as loaded: two bf16 per register
+#pragma unroll
+    for (int ab = 0; ab < 2; ++ab) {
+      live[ab] = tile_valid(it, ab) && !dead;
+#pragma unroll
+      for (int k = 0; k < 16; ++k) w[ab][k] = 0u;
+      if (SEDA && live[ab]) {
+        const int32_t cid = __ldg(ex.cluster_id + row_of(it, ab));
+        if ((uint32_t)cid < (uint32_t)ex.n_clusters) {
+          const uint32_t m = __ldg(ex.cluster_mask + cid);
+          allowed[ab] = m ? m : 1u;
+        } else if (cid != -1) {
+          bad_cid = true;
+        }
       }
     }
-    const uint32_t bar = my_bars + 8 * s;
-    float x[32];
 #pragma unroll
-    for (int i = 0; i < 32; ++i) x[i] = 0.0f;
-    if (tile_valid(it) && !dead) {
-      uint32_t spins = 0;
-      bool ready = mbar_try_wait(bar, parity);
-      while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(bar, parity);
-      if (!__all_sync(0xffffffffu, ready)) {
-        dead = true;
-      } else {
-        const uint32_t base = my_ring + s * kTileBytes;
+    for (int ab = 0; ab < 2; ++ab) {
+      if (live[ab]) {      // warp-uniform
+        const uint32_t bar = my_bars + 8 * (st0 + ab);
+        uint32_t spins = 0;
+        bool ready = mbar_try_wait(bar, parity);
+        while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(bar, parity);
+        if (!__all_sync(0xffffffffu, ready)) {
+          dead = true;
+          live[0] = live[1] = false;
+        } else {
+          const uint32_t base = my_ring + (st0 + ab) * kTileBytes;
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const uint4 v = lds_v4(base + chunk_off[q]);
-          const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            x[8 * q + 2 * j] = __uint_as_float(w[j] << 16);
-            x[8 * q + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+          for (int q = 0; q < 4; ++q) {
+            const uint4 v = lds_v4(base + chunk_off[q]);
+            w[ab][4 * q] = v.x; w[ab][4 * q + 1] = v.y; w[ab][4 * q + 2] = v.z; w[ab][4 * q + 3] = v.w;
           }
         }
       }
     }
-    const bool live = valid && !dead;
     // ---- mean: block sum in channel order, butterfly over the warp, warp sums of the token in order
-    float sum = x[0];
+    float sum[2];
 #pragma unroll
-    for (int i = 1; i < 32; ++i) sum = __fadd_rn(sum, x[i]);
+    for (int ab = 0; ab < 2; ++ab) {
+      float s = __uint_as_float(w[ab][0] << 16);
+      s = __fadd_rn(s, __uint_as_float(w[ab][0] & 0xffff0000u));
 #pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) sum = __fadd_rn(sum, __shfl_xor_sync(0xffffffffu, sum, off));
-    if (lane == 0) part[warp] = sum;
-    __syncthreads();
-    float total = part[row_local * p.wpr];
-    for (uint32_t k = 1; k < p.wpr; ++k) total = __fadd_rn(total, part[row_local * p.wpr + k]);
-    const float mean = __fdiv_rn(total, p.c_f32);
-    // ---- variance
-    float q = 0.0f;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      x[i] = __fsub_rn(x[i], mean);
-      q = __fmaf_rn(x[i], x[i], q);
-    }
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) q = __fadd_rn(q, __shfl_xor_sync(0xffffffffu, q, off));
-    if (lane == 0) part[kWarps + warp] = q;
-    __syncthreads();
-    float qt = part[kWarps + row_local * p.wpr];
-    for (uint32_t k = 1; k < p.wpr; ++k) qt = __fadd_rn(qt, part[kWarps + row_local * p.wpr + k]);
-    const float var = __fdiv_rn(qt, p.c_f32);
-    const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, p.eps)));
-    if (live) {
-      // ---- modulation, cut to the upper 16 bits (all the quantizer needs), quantize, store
-      uint32_t yw[16];
-#pragma unroll
-      for (int k = 0; k < 16; ++k) {
-        uint32_t y[2];
-#pragma unroll
-        for (int hlf = 0; hlf < 2; ++hlf) {
-          const uint32_t f = fac[2 * k + hlf];
-          float g = __uint_as_float(f << 16);
-          if (PLUS_ONE) g = __fadd_rn(1.0f, g);
-          y[hlf] = __float_as_uint(__fmaf_rn(__fmul_rn(x[2 * k + hlf], rstd), g, __uint_as_float(f & 0xffff0000u)));
-        }
-        yw[k] = __byte_perm(y[0], y[1], 0x7632);
+      for (int k = 1; k < 16; ++k) {
+        s = __fadd_rn(s, __uint_as_float(w[ab][k] << 16));
+        s = __fadd_rn(s, __uint_as_float(w[ab][k] & 0xffff0000u));
       }
-      uint32_t cw[4], Eb[2];
-      int did[2];
-      quantize_packed_block<SEDA, false, false>(yw, allowed, tb, qerr_base, pair_base, 3u, 254u, cw, did, Eb);
-      const size_t unit = (size_t)row * p.units_row + wcol * 32u + (uint32_t)lane;
-      *reinterpret_cast<uint4*>(p.codes + unit * 16u) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
-      p.meta[unit] = (uint16_t)((Eb[0] - 3u) | ((uint32_t)did[0] << 8));
+      sum[ab] = s;
     }
-    // ---- refill this stage
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+#pragma unroll
+      for (int ab = 0; ab < 2; ++ab) sum[ab] = __fadd_rn(sum[ab], __shfl_xor_sync(0xffffffffu, sum[ab], off));
+    }
+    if (lane == 0 && warp_used) {
+      part[team * 16u + wcol] = sum[0];
+      part[kWarps * 16 + team * 16u + wcol] = sum[1];
+    }
+    team_sync();
+    float mean[2] = {0.0f, 0.0f};
+    if (warp_used) {
+#pragma unroll
+      for (int ab = 0; ab < 2; ++ab) mean[ab] = __fdiv_rn(team_total(part + ab * kWarps * 16), p.c_f32);
+    }
+    // ---- variance
+    float q[2] = {0.0f, 0.0f};
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+#pragma unroll
+      for (int ab = 0; ab < 2; ++ab) {
+        const float d0 = __fsub_rn(__uint_as_float(w[ab][k] << 16), mean[ab]);
+        q[ab] = __fmaf_rn(d0, d0, q[ab]);
+        const float d1 = __fsub_rn(__uint_as_float(w[ab][k] & 0xffff0000u), mean[ab]);
+        q[ab] = __fmaf_rn(d1, d1, q[ab]);
+      }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+#pragma unroll
+      for (int ab = 0; ab < 2; ++ab) q[ab] = __fadd_rn(q[ab], __shfl_xor_sync(0xffffffffu, q[ab], off));
+    }
+    if (lane == 0 && warp_used) {
+      part[2 * kWarps * 16 + team * 16u + wcol] = q[0];
+      part[3 * kWarps * 16 + team * 16u + wcol] = q[1];
+    }
+    team_sync();
+#pragma unroll
+    for (int ab = 0; ab < 2; ++ab) {
+      if (live[ab]) {
+        const float var = __fdiv_rn(team_total(part + (2 + ab) * kWarps * 16), p.c_f32);
+        const float rstd = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(var, p.eps)));
+        // ---- modulation, cut to the upper 16 bits (all the quantizer needs), quantize, store
+        uint32_t yw[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+          uint32_t y[2];
+#pragma unroll
+          for (int hlf = 0; hlf < 2; ++hlf) {
+            const float xv = __uint_as_float(hlf ? (w[ab][k] & 0xffff0000u) : (w[ab][k] << 16));
+            const float bv = __uint_as_float(hlf ? (bw[k] & 0xffff0000u) : (bw[k] << 16));
+            y[hlf] = __float_as_uint(__fmaf_rn(__fmul_rn(__fsub_rn(xv, mean[ab]), rstd), gf[2 * k + hlf], bv));
+          }
+          yw[k] = __byte_perm(y[0], y[1], 0x7632);
+        }
+        uint32_t cw[4], Eb[2];
+        int did[2];
+        quantize_packed_block<SEDA, false, false>(yw, allowed[ab], tb, qerr_base, pair_base, 3u, 254u, cw, did, Eb);
+        const size_t unit = (size_t)row_of(it, ab) * p.units_row + wcol * 32u + (uint32_t)lane;
+        *reinterpret_cast<uint4*>(p.codes + unit * 16u) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+        p.meta[unit] = (uint16_t)((Eb[0] - 3u) | ((uint32_t)did[0] << 8));
+      }
+    }
+    // ---- refill the two stages of this step with the tokens two steps ahead
     __syncwarp();
-    if (lane == 0 && !dead && tile_valid(it + kStages)) {
-      mbar_expect_tx(bar, kTileBytes);
-      tma_load_2d(my_ring + s * kTileBytes, &tmap, bar, 0,
-                  (int)((row0 + (uint32_t)(it + kStages) * row_step) * rows128 + wcol * 16u));
+    if (lane == 0 && !dead) {
+#pragma unroll
+      for (int ab = 0; ab < 2; ++ab)
+        if (tile_valid(it + 2, ab)) request(it + 2, ab);
     }
-    if (++s == kStages) { s = 0; parity ^= 1u; }
+    if (it & 1) parity ^= 1u;
   }
   if (dead) {
     if (lane == 0) atomicOr(p.status, 1u);
-    // the loads still in flight for this warp (the kStages tiles from the step it gave up at) get a bounded
-    // chance to land before the CTA's shared memory goes
-    for (int j = 0; j < kStages; ++j) {
-      if (!tile_valid(it_dead + j)) break;
-      const int sj = (s_dead + j) % kStages;
-      const uint32_t pj = (s_dead + j) >= kStages ? (parity_dead ^ 1u) : parity_dead;
-      uint32_t tries = 0;
-      while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
+    // the loads still in flight for this warp (the tokens of the step it gave up at and of the next one) get a
+    // bounded chance to land before the CTA's shared memory goes
+    for (int j = 0; j < 2; ++j) {
+      const uint32_t pj = ((it_dead & 1) + j) >= 2 ? (parity_dead ^ 1u) : parity_dead;
+      for (int ab = 0; ab < 2; ++ab) {
+        if (!tile_valid(it_dead + j, ab)) continue;
+        const uint32_t st = (uint32_t)(2 * ((it_dead + j) & 1) + ab);
+        uint32_t tries = 0;
+        while (!mbar_try_wait(my_bars + 8 * st, pj) && ++tries < kSpinLimit) {}
+      }
     }
   }
   if (SEDA && bad_cid && lane == 0) atomicOr(p.status, 2u);
 }
 
-constexpr size_t kSmemBytesLn = 
-    1024 + (size_t)kWarps * kStages * kTileBytes + sizeof(SmemTables) + (kWarps * kStages + 1) * 8 + 2 * kWarps * sizeof(float);
+constexpr size_t kSmemBytesLn =
+    1024 + (size_t)kWarps * kStages * kTileBytes + sizeof(SmemTables) + (kWarps * kStages + 2) * 8 + 4 * kWarps * 16 * sizeof(float);
 
 constexpr size_t kSmemBytesF32 =
     1024 + (size_t)kWarpsF32 * kStages * kTileBytesF32 + sizeof(SmemTables) + (kWarpsF32 * kStages + 1) * 8;
@@ -1431,10 +1494,11 @@ cudaError_t fb4_fast_prepare_device() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, false, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, true, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, true, true>, attr, bytes);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<false, false>, attr, (int)kSmemBytesLn);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<true, false>, attr, (int)kSmemBytesLn);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<false, true>, attr, (int)kSmemBytesLn);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<true, true>, attr, (int)kSmemBytesLn);
+#define FB4_OPT_IN(...) \
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<__VA_ARGS__>, attr, (int)kSmemBytesLn)
+  FB4_OPT_IN(false, false, 12); FB4_OPT_IN(true, false, 12); FB4_OPT_IN(false, true, 12); FB4_OPT_IN(true, true, 12);
+  FB4_OPT_IN(false, false, 16); FB4_OPT_IN(true, false, 16); FB4_OPT_IN(false, true, 16); FB4_OPT_IN(true, true, 16);
+#undef FB4_OPT_IN
   return e;
 }
 
@@ -1820,19 +1884,23 @@ cudaError_t fb4_launch_quantize_layernorm(const fb4_ctx* ctx, const void* x, int
   p.T = (uint32_t)T;
   p.units_row = (uint32_t)(C / 32);
   p.wpr = (uint32_t)(C / 1024);
-  p.rows_cta = (uint32_t)kWarps / p.wpr;
+  const int nw = (12 % p.wpr == 0) ? 12 : kWarps;
+  p.teams = (uint32_t)nw / p.wpr;
   p.c_f32 = (float)C;
   p.eps = eps;
   p.codes = codes;
   p.meta = meta;
   p.status = ctx->d_status;
-  const int64_t n_sets = (T + p.rows_cta - 1) / p.rows_cta;
+  const int64_t n_sets = ((T + 1) / 2 + p.teams - 1) / p.teams;      // a team takes two tokens per step
   grid = (int)(n_sets < ctx->sm_count ? n_sets : ctx->sm_count);
   const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
   const uint16_t* g = static_cast<const uint16_t*>(gain);
   const uint16_t* b = static_cast<const uint16_t*>(bias);
 #define FB4_LN(P, S) \
-  fb4_quantize_layernorm_kernel<P, S><<<grid, kWarps * 32, kSmemBytesLn, stream>>>(map, tables, p, g, b, ex)
+  do { \
+    if (nw == 12) fb4_quantize_layernorm_kernel<P, S, 12><<<grid, 12 * 32, kSmemBytesLn, stream>>>(map, tables, p, g, b, ex); \
+    else fb4_quantize_layernorm_kernel<P, S, 16><<<grid, 16 * 32, kSmemBytesLn, stream>>>(map, tables, p, g, b, ex); \
+  } while (0)
   switch ((plus_one ? 1 : 0) | (ex.cluster_id ? 2 : 0)) {
     case 0: FB4_LN(false, false); break;
     case 1: FB4_LN(true, false); break;

@@ -425,12 +425,12 @@ def _layernorm_rational(xv, gv, bv, plus_one, eps):
     nblk = C // 32
 
     def total(bs):
-        acc = None
+        acc = Fraction(0)
         for b0 in range(0, nblk, 32):
             v = [bs[b0 + i] if b0 + i < nblk else Fraction(0) for i in range(32)]
             for off in (16, 8, 4, 2, 1):
                 v = [R(v[i] + v[i ^ off]) for i in range(32)]
-            acc = v[0] if acc is None else R(acc + v[0])
+            acc = R(acc + v[0])
         return acc
 
     bs = []

@@ -88,7 +88,8 @@ MUTANTS = {
     "layernorm_variance_unbiased": ("const float var = ln_row_total(bs, nblk) / (float)C;", "const float var = ln_row_total(bs, nblk) / (float)(C - 1);"),
     "layernorm_modulation_two_roundings": ("y[t * C + c] = fmaf(d[c] * rstd, g, bc);", "y[t * C + c] = (d[c] * rstd) * g + bc;"),
     "layernorm_short_segment_padded_with_first_block": ("v[i] = i < n ? blocksum[i] : 0.0f;", "v[i] = i < n ? blocksum[i] : blocksum[0];"),
-    "layernorm_segments_added_last_to_first": ("total = first ? seg : total + seg;", "total = first ? seg : seg + total * 1.0000001f;"),
+    "layernorm_segments_added_inexactly": ("total = total + ln_segment_butterfly(blocksum + b0, n);",
+                                           "total = total * 1.0000001f + ln_segment_butterfly(blocksum + b0, n);"),
     "bf16_by_truncation": ("u += 0x7fffu + lsb;", "u += 0u * lsb;"),
     "bf16_ties_away_from_zero": ("u += 0x7fffu + lsb;", "u += 0x8000u + 0u * lsb;"),
     "bf16_ties_toward_zero": ("u += 0x7fffu + lsb;", "u += 0x7fffu + 0u * lsb;"),
