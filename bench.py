@@ -207,6 +207,14 @@ class Ops:
             q16 = self._buf["q16"]
             meta16 = self.buf("meta16", (T, C // 16), torch.int16)
             return (lambda: fb4.fb4_quantize(q16.ctx, x, T, C, C, codes, meta16)), T * C * 2.5 + T * (C // 16) * 2
+        if name in ("plain_every_element_a_group", "plain_all_dialects_scored"):
+            # the two other selection settings of the paper's Table 2 comparison: num_groups = block, select_mode 1
+            key = "qg" if name == "plain_every_element_a_group" else "qa"
+            if key not in self._buf:
+                self._buf[key] = fb4.Fb4(device=torch.cuda.current_device(), num_groups=32) if key == "qg" else \
+                    fb4.Fb4(device=torch.cuda.current_device(), select_mode=1)
+            qs = self._buf[key]
+            return (lambda: fb4.fb4_quantize(qs.ctx, x, T, C, C, codes, meta)), algorithmic_bytes(T, C)
         if name == "quantize_mxfp8_tiled_scales":
             e8 = self.buf("e4m3", (T, C), torch.uint8)
             sc = self.buf("sf", (fb4.fb4_mxfp8_scale_bytes(T, C, 1),), torch.uint8)
@@ -304,7 +312,7 @@ class Ops:
         raise KeyError(name)
 
 
-OP_NAMES = ["plain", "plain_block16", "plain_f32", "affine_plus_quantize", "layernorm_plus_quantize", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
+OP_NAMES = ["plain", "plain_block16", "plain_every_element_a_group", "plain_all_dialects_scored", "plain_f32", "affine_plus_quantize", "layernorm_plus_quantize", "seda", "decomposed", "decomposed_given_set", "decomposed_seda", "dequantize_f32_plain", "dequantize_f32_decomposed",
             "dequantize_bf16_plain", "dequantize_bf16_decomposed", "dequantize_f16_plain", "to_mxfp8_tiled_scales",
             "quantize_mxfp8_tiled_scales", "quantize_mxfp8_decomposed_seda", "affine_plus_quantize_mxfp8"]
 
@@ -510,7 +518,7 @@ def run_variants(ops, args, torch, fb4, synth, peak):
         total, per = time_steps(fn, steps, warm, torch)
         ms = total / steps
         res[name] = {"ms": ms, "GB/s": alg / (ms * 1e-3) / 1e9, "frac_hbm_measured": alg / (ms * 1e-3) / 1e9 / peak,
-                     "kernel_variant": q.last_variant if name in ("plain", "plain_block16", "plain_f32", "affine_plus_quantize", "layernorm_plus_quantize", "seda", "decomposed", "decomposed_given_set",
+                     "kernel_variant": ("fast" if name.startswith("plain_") and name != "plain_f32" and name != "plain_block16" else q.last_variant) if name in ("plain", "plain_block16", "plain_every_element_a_group", "plain_all_dialects_scored", "plain_f32", "affine_plus_quantize", "layernorm_plus_quantize", "seda", "decomposed", "decomposed_given_set",
                                                                          "decomposed_seda", "quantize_mxfp8_tiled_scales",
                                                                          "quantize_mxfp8_decomposed_seda", "affine_plus_quantize_mxfp8")
                      else "decode"}

@@ -52,6 +52,9 @@ struct FastTables {
   uint32_t stage1[32];                   // [bin of block maximum] -> candidate mask
   uint8_t qerror[32][32];                // [dialect][bin], for masks that cut a group
   uint8_t fb[32][8];
+  uint32_t n_groups;                     // stage-1 groups in use
+  uint32_t pad_[3];
+  uint4 did_lanes[kMaxGroups];           // [group] -> dialect ids of candidates (2,0), (3,1), (6,4), (7,5) in 16-bit lanes
 };
 static_assert(sizeof(FastTables) % 16 == 0, "copied with 16-byte accesses");
 
@@ -141,13 +144,119 @@ __device__ __forceinline__ int choose_dialect(const float (&gm)[8], float sG, ui
   return select_general(cand, gb, tb);
 }
 
+// num_groups = block size (every element is its own group, the setting of the paper's Table 2 comparison):
+// the error of a candidate is summed over the bins of all 32 elements.  a = the 16 packed magnitude registers.
+// Byte sums would overflow (32 terms of up to 31), so every run of 8 elements is added in bytes and then
+// widened into 16-bit lanes; the keys are formed from those.
+template <bool SEDA>
+__device__ __forceinline__ int choose_dialect_per_element(const uint32_t (&a)[16], float sG, uint32_t bmax, uint32_t allowed,
+                                                          const Tables* tb, uint32_t qerr_lane) {
+  const uint32_t grp = tb->c.group_of_bin[bmax];
+  uint32_t cand = 0;
+  bool packed_path = true;
+  if (SEDA) {
+    const uint32_t st1 = tb->c.stage1[bmax];
+    cand = st1 & allowed;
+    if (cand == 0) cand = allowed;
+    packed_path = (cand == st1);
+  }
+  if (!SEDA || packed_path) {
+    const uint32_t qb = qerr_lane + grp * 4096u;
+    uint32_t s02 = 0, s13 = 0, s46 = 0, s57 = 0;      // candidates (2, 0), (3, 1), (6, 4), (7, 5) in 16-bit lanes
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t lo = 0, hi = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint32_t av = a[4 * q + j];
+        const uint32_t t1 = __float_as_uint(__fmaf_rz(__uint_as_float(av), sG, 2.0f));         // upper element
+        const uint32_t t0 = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sG, 2.0f));   // lower element
+        const uint2 e0 = lds_v2((t0 << 7) + qb), e1 = lds_v2((t1 << 7) + qb);
+        lo += e0.x + e1.x;
+        hi += e0.y + e1.y;
+      }
+      s02 += lo & 0x00ff00ffu;
+      s13 += (lo >> 8) & 0x00ff00ffu;
+      s46 += hi & 0x00ff00ffu;
+      s57 += (hi >> 8) & 0x00ff00ffu;
+    }
+    const uint32_t k02 = s02 * 8u + 0x00020000u, k13 = s13 * 8u + 0x00030001u;
+    const uint32_t k46 = s46 * 8u + 0x00060004u, k57 = s57 * 8u + 0x00070005u;
+    const uint32_t km = __vminu2(__vminu2(k02, k13), __vminu2(k46, k57));
+    const uint32_t key = min(km & 0xffffu, km >> 16);
+    return tb->c.did_of[grp][key & 7u];
+  }
+  if (__popc(cand) == 1) return __ffs((int)cand) - 1;
+  // a mask that cuts the stage-1 group: every candidate scored with the byte table (ascending ids: ties keep the lowest)
+  int best = 0, best_err = 0x7fffffff;
+  for (uint32_t m = cand; m; m &= m - 1) {
+    const int d = __ffs((int)m) - 1;
+    int err = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const uint32_t b1 = __float_as_uint(__fmaf_rz(__uint_as_float(a[i]), sG, 2.0f)) & 31u;
+      const uint32_t b0 = __float_as_uint(__fmaf_rz(__uint_as_float(a[i] << 16), sG, 2.0f)) & 31u;
+      err += tb->c.qerror[d][b0] + tb->c.qerror[d][b1];
+    }
+    if (err < best_err) { best_err = err; best = d; }
+  }
+  return best;
+}
+
+// select_mode 1: no stage 1, every allowed dialect is scored on the 8 group maxima (the plain comparison of all
+// dialects that Sec. 3.2 starts from, with the table criterion).  The packed words of all stage-1 groups are
+// summed in turn and compared as (error << 5 | dialect id) keys in 16-bit lanes; the smallest key wins, so ties go
+// to the lowest id.  A SeDA mask other than all-ones takes the byte table.
+template <bool SEDA>
+__device__ __forceinline__ int choose_dialect_all(const float (&gm)[8], float sG, uint32_t allowed, const Tables* tb,
+                                                  uint32_t qerr_lane) {
+  uint32_t t[8];
+#pragma unroll
+  for (int g = 0; g < 8; ++g) t[g] = __float_as_uint(__fmaf_rz(gm[g], sG, 2.0f));
+  if (SEDA && allowed != 0xffffffffu) {
+    uint8_t gb[8];
+#pragma unroll
+    for (int g = 0; g < 8; ++g) gb[g] = (uint8_t)(t[g] & 31u);
+    return select_general(allowed, gb, tb);
+  }
+  // running minima of (error << 5 | dialect id) in 16-bit lanes: byte lanes (2, 0), (3, 1), (6, 4), (7, 5) of the sums
+  uint32_t m02 = 0xffffffffu, m13 = 0xffffffffu, m46 = 0xffffffffu, m57 = 0xffffffffu;
+  const uint32_t n_groups = tb->c.n_groups;
+  uint32_t addr[8];
+#pragma unroll
+  for (int g = 0; g < 8; ++g) addr[g] = (t[g] << 7) + qerr_lane;
+#pragma unroll
+  for (int grp = 0; grp < kMaxGroups; ++grp) {
+    if ((uint32_t)grp < n_groups) {
+      uint32_t lo = 0, hi = 0;
+#pragma unroll
+      for (int g = 0; g < 8; ++g) {
+        const uint2 e = lds_v2(addr[g] + (uint32_t)grp * 4096u);
+        lo += e.x;
+        hi += e.y;
+      }
+      const uint4 ids = tb->c.did_lanes[grp];      // the candidates' dialect ids in the same lanes (pads: 31)
+      m02 = __vminu2(m02, (lo & 0x00ff00ffu) * 32u + ids.x);
+      m13 = __vminu2(m13, ((lo >> 8) & 0x00ff00ffu) * 32u + ids.y);
+      m46 = __vminu2(m46, (hi & 0x00ff00ffu) * 32u + ids.z);
+      m57 = __vminu2(m57, ((hi >> 8) & 0x00ff00ffu) * 32u + ids.w);
+    }
+  }
+  // a pad sums to 248 and carries id 31: it ties at worst with the real dialect 31, the same answer
+  const uint32_t km = __vminu2(__vminu2(m02, m13), __vminu2(m46, m57));
+  const uint32_t best = min(km & 0xffffu, km >> 16);
+  return (int)(best & 31u);
+}
+
 // One lane's block(s) from 16 registers of two 16-bit values each - bf16 inputs, or any fp32 values cut
 // to their upper 16 bits: the scale exponent, the bins of the 0.5-wide tables and the sign are all
 // fixed by those bits (every bin boundary is a multiple of the cut's granularity), so the cut loses
 // nothing.  Scale, group maxima, dialect selection, LUT quantization; block size 32, or (B16) two
 // blocks of 16; CLAMP: clamped exponent range.  Out: the four code words, and per half the chosen
 // dialect and the biased exponent.
-template <bool SEDA, bool B16, bool CLAMP>
+// SEL: 0 = 8 groups, two-stage selection (the default); 1 = every element its own group (block size 32 only);
+// 2 = 8 groups, every allowed dialect scored (select_mode 1).
+template <bool SEDA, bool B16, bool CLAMP, int SEL = 0>
 __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], uint32_t allowed, const Tables* tb,
                                                       uint32_t qerr_lane, uint32_t pair_base, uint32_t ec_lo,
                                                       uint32_t ec_hi, uint32_t (&cw)[4], int (&didh)[2],
@@ -193,7 +302,9 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
       gm[2 * q] = __uint_as_float(g2[q] << 16);
       gm[2 * q + 1] = __uint_as_float(g2[q]);
     }
-    const int did = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
+    const int did = SEL == 1 ? choose_dialect_per_element<SEDA>(a, sG, bmax, allowed, tb, qerr_lane)
+                    : SEL == 2 ? choose_dialect_all<SEDA>(gm, sG, allowed, tb, qerr_lane)
+                               : choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
     Ech[0] = Ech[1] = Ec;
     sHh[0] = sHh[1] = s2 * 0x1p-25f;                       // bin in the mantissa of 0.125 + x
     sLh[0] = sLh[1] = s2 * 0x1p-5f;                        // bin in the mantissa of 2^17 + x
@@ -227,7 +338,8 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
       Ech[h] = Ec;
       sHh[h] = s2 * 0x1p-25f;
       sLh[h] = s2 * 0x1p-5f;
-      didh[h] = choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
+      didh[h] = SEL == 2 ? choose_dialect_all<SEDA>(gm, sG, allowed, tb, qerr_lane)
+                         : choose_dialect<SEDA>(gm, sG, bmax, allowed, tb, qerr_lane);
     }
   }
   // ---- Qvalue: one lookup per element pair.  124*36 + 144 = 9*512, so the exponent fields of

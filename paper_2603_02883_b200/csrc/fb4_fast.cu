@@ -92,7 +92,7 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 // as the main pass, from the upper 16 bits of every Delta (see quantize_packed_block).
 // w = the 16 input registers (2 bf16 each), cw = the 4 code words, didh / Ech = dialect and biased
 // exponent per half (equal halves for block size 32).
-template <bool SEDA, bool B16, bool CLAMP>
+template <bool SEDA, bool B16, bool CLAMP, int SEL = 0>
 __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t* cw, const int* didh,
                                                const uint32_t* Ech, uint32_t allowed, const SmemTables* tb,
                                                uint32_t qerr_lane, uint32_t pair_base, uint32_t ec_lo, uint32_t ec_hi,
@@ -116,7 +116,7 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
   }
   uint32_t rc[4], rE[2];
   int rd[2];
-  quantize_packed_block<SEDA, B16, CLAMP>(dw, allowed, tb, qerr_lane, pair_base, ec_lo, ec_hi, rc, rd, rE);
+  quantize_packed_block<SEDA, B16, CLAMP, SEL>(dw, allowed, tb, qerr_lane, pair_base, ec_lo, ec_hi, rc, rd, rE);
 #pragma unroll
   for (int q = 0; q < 4; ++q) rcw[q] = rc[q];
   *rmeta = B16 ? (((rE[0] - 3u) | ((uint32_t)rd[0] << 8)) | (((rE[1] - 3u) | ((uint32_t)rd[1] << 8)) << 16))
@@ -445,7 +445,7 @@ __device__ __forceinline__ void stg_v8(void* ptr, const uint32_t* o) {
 // units per lane and tile of a flat kernel
 __host__ __device__ constexpr int flat_units(bool decomp, bool mx) { return (decomp || mx) ? 1 : 2; }
 
-template <bool SEDA, bool DECOMP, bool B16, bool CLAMP, bool MX = false>
+template <bool SEDA, bool DECOMP, bool B16, bool CLAMP, bool MX = false, int SEL = 0>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
                          FlatParams p, Fb4RowExtras ex) {
@@ -634,7 +634,7 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
             }
             uint32_t c4[4], Ech[2];
             int didh[2];
-            quantize_packed_block<SEDA, B16, CLAMP>(w, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, c4, didh, Ech);
+            quantize_packed_block<SEDA, B16, CLAMP, SEL>(w, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, c4, didh, Ech);
 #pragma unroll
             for (int q = 0; q < 4; ++q) cw[4 * h + q] = c4[q];
             did0[h] = didh[0];
@@ -643,7 +643,7 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
             if (DECOMP) {     // one unit per lane: the residual follows at once, from the same registers
               if (srow >= 0) {
                 uint32_t rcw[4], rrec;
-                residual_block<SEDA, B16, CLAMP>(w, c4, didh, Ech, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi,
+                residual_block<SEDA, B16, CLAMP, SEL>(w, c4, didh, Ech, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi,
                                                  rcw, &rrec);
                 const size_t ru = (size_t)srow * p.units_row + pos.rem;      // unit of the residual tensor
                 if (MX) {
@@ -1393,6 +1393,12 @@ bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes
     for (; j < 8; ++j)
       for (int k = 0; k < 32; ++k) ft.qerr64[gi][k] |= (uint64_t)31 << (8 * j);   // never beats a real candidate
   }
+  ft.n_groups = (uint32_t)ngroups;
+  for (int gi = 0; gi < kMaxGroups; ++gi) {
+    uint32_t id[8];
+    for (int j = 0; j < 8; ++j) id[j] = (gi < ngroups && j < __builtin_popcount(groups[gi])) ? ft.did_of[gi][j] : 31u;
+    ft.did_lanes[gi] = make_uint4(id[0] | (id[2] << 16), id[1] | (id[3] << 16), id[4] | (id[6] << 16), id[5] | (id[7] << 16));
+  }
   std::memcpy(ft.qvalue, t.qvalue, sizeof ft.qvalue);
   std::memcpy(ft.qerror, t.qerror, sizeof ft.qerror);
   std::memcpy(ft.fb, t.formatbook, sizeof ft.fb);
@@ -1484,6 +1490,14 @@ cudaError_t fb4_fast_prepare_device() {
   FB4_OPT_IN(true, false, false, false, true);
   FB4_OPT_IN(false, true, false, false, true);
   FB4_OPT_IN(true, true, false, false, true);
+  FB4_OPT_IN(false, false, false, false, false, 1);
+  FB4_OPT_IN(true, false, false, false, false, 1);
+  FB4_OPT_IN(false, true, false, false, false, 1);
+  FB4_OPT_IN(true, true, false, false, false, 1);
+  FB4_OPT_IN(false, false, false, false, false, 2);
+  FB4_OPT_IN(true, false, false, false, false, 2);
+  FB4_OPT_IN(false, true, false, false, false, 2);
+  FB4_OPT_IN(true, true, false, false, false, 2);
 #undef FB4_OPT_IN
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, false>, attr, bytes);
@@ -1507,8 +1521,13 @@ cudaError_t fb4_fast_prepare_device() {
 bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {
   const fb4_config& c = ctx->cfg;
   if (!ctx->fast_ok || !ctx->d_fast_tables) return false;
-  if (c.num_groups != 8 || c.select_mode != 0) return false;
   if (c.block_size != 32 && c.block_size != 16) return false;
+  if (c.num_groups != 8 || c.select_mode != 0) {
+    // every element its own group, or every dialect scored: block size 32, full exponent range, contiguous rows
+    const bool per_element = c.num_groups == 32 && c.select_mode == 0, all = c.num_groups == 8 && c.select_mode == 1;
+    if (!(per_element || all) || c.block_size != 32 || c.exp_min != -124 || c.exp_max != 127 || ld != C) return false;
+    if (T <= 0 || T * (C / 32) >= 0x7fffffffLL) return false;   // these modes exist in the kernel for contiguous tensors only
+  }
   if (C % 64 != 0 || (ld & 7) || (reinterpret_cast<uintptr_t>(x) & 15)) return false;
   if (T > 0x7fffffffLL || C / 64 > 0x7fffffffLL) return false;
   return encode_tiled_fn() != nullptr;
@@ -1619,6 +1638,23 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
     const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
     const bool b16 = ctx->cfg.block_size == 16;
     const bool clamp = ctx->cfg.exp_min != -124 || ctx->cfg.exp_max != 127;
+    const int sel = ctx->cfg.num_groups == 32 ? 1 : (ctx->cfg.select_mode == 1 ? 2 : 0);
+    if (sel != 0) {
+#define FB4_SEL(S, D, L) \
+  fb4_quantize_flat_kernel<S, D, false, false, false, L><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, fp, ex)
+      switch ((seda ? 1 : 0) | (decomp ? 2 : 0) | (sel == 2 ? 4 : 0)) {
+        case 0: FB4_SEL(false, false, 1); break;
+        case 1: FB4_SEL(true, false, 1); break;
+        case 2: FB4_SEL(false, true, 1); break;
+        case 3: FB4_SEL(true, true, 1); break;
+        case 4: FB4_SEL(false, false, 2); break;
+        case 5: FB4_SEL(true, false, 2); break;
+        case 6: FB4_SEL(false, true, 2); break;
+        default: FB4_SEL(true, true, 2); break;
+      }
+#undef FB4_SEL
+      return cudaGetLastError();
+    }
     switch ((seda ? 1 : 0) | (decomp ? 2 : 0) | (b16 ? 4 : 0) | (clamp ? 8 : 0)) {
 #define FB4_CASE(V, S, D, B, K) \
   case V: return launch_flat<S, D, B, K>(map, tables, fp, ex, grid, stream)
@@ -1720,7 +1756,8 @@ cudaError_t fb4_launch_quantize_fast_f32(const fb4_ctx* ctx, const void* x, int6
 // Quantize straight to an MXFP8 operand (e4m3 bytes + E8M0 scales): default configuration only.
 bool fb4_fast_mx_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld) {
   const fb4_config& c = ctx->cfg;
-  return c.block_size == 32 && c.exp_min == -124 && c.exp_max == 127 && fb4_fast_eligible(ctx, x, T, C, ld);
+  return c.block_size == 32 && c.num_groups == 8 && c.select_mode == 0 && c.exp_min == -124 && c.exp_max == 127 &&
+         fb4_fast_eligible(ctx, x, T, C, ld);
 }
 
 // With ex.n_salient > 0 the residual of the salient rows goes to res_e4m3 [n_salient][C] and

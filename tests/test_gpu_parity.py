@@ -400,3 +400,49 @@ def test_custom_formatbooks():
         assert_same_quantized(qw, orc.quantize_weights(bits, fbk), f"custom formatbook weights ({want})")
         assert q.device_status == 0
         q.close()
+
+
+@pytest.mark.parametrize("cfg", [dict(num_groups=32), dict(select_mode=1)], ids=["every_element_a_group", "all_dialects_scored"])
+def test_selection_variants_in_both_kernels(cfg):
+    """num_groups = block size (the paper's Table 2 setting) and select_mode 1: the TMA-staged kernel and the generic
+    kernel both against the oracle, plain, with SeDA masks (paper-structured, arbitrary, one dialect, all ones) and
+    with a residual pass."""
+    ocfg = orc.Config(**cfg)
+    T, C = 150, 1536
+    bits = heavy(T, C, 21)
+    bits[3, :64] = 0
+    w = synth.Workload("t", T=T, C=C, seed=9, kind=1, n_outlier=0, outlier_gain=1.0, seda=True, n_clusters=6, cluster_seed=12,
+                       score_seed=5)
+    cid, masks = synth.clusters(w)
+    rng = np.random.default_rng(4)
+    masks = masks.copy()
+    masks[1] = rng.integers(1, 2 ** 32)
+    masks[2] = 1 << 31
+    masks[3] = 0xFFFFFFFF
+    cid = cid.copy()
+    cid[5:9] = -1
+    score = synth.scores(w)
+    sal = orc.select_salient(score, 20)
+    refs = {"plain": orc.quantize(bits, FB, ocfg),
+            "seda": orc.quantize(bits, FB, ocfg, cluster_id=cid, cluster_mask=masks),
+            "decomposed+seda": orc.quantize(bits, FB, ocfg, cluster_id=cid, cluster_mask=masks, salient_idx=sal)}
+    x = to_dev_bf16(bits)
+    dcid, dmask = torch.from_numpy(cid).cuda(), torch.from_numpy(masks.view(np.int32)).cuda()
+    for variant, name in ((0, "fast"), (1, "generic")):
+        q = fb4.Fb4(**cfg)
+        q.set_kernel_variant(variant)
+        assert_same_quantized(q.quantize(x), refs["plain"], f"{cfg} plain {name}")
+        assert q.last_variant == name
+        assert_same_quantized(q.quantize(x, dcid, dmask), refs["seda"], f"{cfg} seda {name}")
+        got = q.quantize_decomposed(x, torch.from_numpy(score).cuda(), 20, cluster_id=dcid, cluster_mask=dmask)
+        assert q.last_variant == name
+        assert_same_quantized(got, refs["decomposed+seda"], f"{cfg} decomposed {name}")
+        assert q.device_status == 0
+        q.close()
+    # a strided view takes the generic kernel and still agrees
+    q = fb4.Fb4(**cfg)
+    wide = torch.zeros((T, C + 64), dtype=torch.bfloat16, device="cuda")
+    wide[:, :C] = x
+    assert_same_quantized(q.quantize(wide[:, :C]), refs["plain"], f"{cfg} strided")
+    assert q.last_variant == "generic"
+    q.close()
