@@ -29,10 +29,13 @@ import numpy as np
 METRIC = "fb4_quantize_throughput"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this
-# workload, from the ncu capture summarised in profiles/fb4_quantize_fast_c5_plain_dram_bytes.md
-# (1 858 057 472 B read + 502 289 920 B written; set back to None whenever that kernel changes).
-NCU_TRAFFIC_BYTES = 2360395008
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel on this workload, from the
+# ncu capture summarised in profiles/fb4_quantize_flat_c5_plain_dram_bytes.md (1 858 046 464 B read +
+# 499 021 056 B written).  The capture's date and the kernel's register count travel with it in the bench line,
+# so that a constant that has outlived the kernel shows; set it back to None whenever that kernel changes.
+NCU_TRAFFIC_BYTES = 2357067520
+NCU_TRAFFIC_SOURCE = {"profile": "profiles/fb4_quantize_flat_c5_plain_dram_bytes.md", "captured": "2026-11-28",
+                      "kernel": "fb4_quantize_flat_kernel<0,0,0,0,0,0>", "registers_per_thread": 115}
 
 
 def algorithmic_bytes(T: int, C: int, B: int = 32, n_res_rows: int = 0, seda: bool = False,
@@ -404,6 +407,8 @@ def main():
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES if (args.op == "plain" and args.workload == "c5_plain"
                                                       and not args.generic_kernel) else None,
+                     "traffic_source": NCU_TRAFFIC_SOURCE if (args.op == "plain" and args.workload == "c5_plain"
+                                                                and not args.generic_kernel) else None,
                      "peak_kind": f"{peak_kind} copy bandwidth",
                      "kernel": f"fb4 {args.op} ({variant})", "algorithmic_bytes_per_launch": alg,
                      "launch_ms_mean": kernel_ms, "launch_ms_min": float(np.min(per))},
