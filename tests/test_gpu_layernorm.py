@@ -92,3 +92,18 @@ def test_layernorm_argument_checks(q32):
                                     p(codes), p(meta), None) == fb4.ERR_INVALID_ARG
     q16.close()
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("T,C", [(1, 1024), (7, 3072), (33, 5120), (3, 16384)])
+def test_layernorm_stays_inside_its_buffers(q32, T, C):
+    """codes and metadata between guard bands: odd token counts leave the second token of the last step empty"""
+    from test_gpu_guard_bands import Guarded
+    bits, gain, bias = _inputs(T, C, seed=T)
+    codes, meta = Guarded(T * C // 2), Guarded(T * (C // 32) * 2)
+    fb4.fb4_quantize_layernorm(q32.ctx, to_dev_bf16(bits), T, C, C, to_dev_bf16(gain), to_dev_bf16(bias), 1, 1e-6, None, None,
+                               0, codes.tensor(torch.uint8, (T, C // 2)), meta.tensor(torch.int16, (T, C // 32)))
+    torch.cuda.synchronize()
+    codes.check("codes, layernorm producer")
+    meta.check("meta, layernorm producer")
+    ref = orc.quantize_f32(orc.layernorm_f32(bits, gain, bias, True, 1e-6), FB)
+    assert np.array_equal(codes.tensor(torch.uint8, (T, C // 2)).cpu().numpy(), ref.codes)

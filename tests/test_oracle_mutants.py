@@ -73,7 +73,10 @@ MUTANTS = {
     "affine_two_roundings": ("y[t * C + c] = fmaf(xf, g, b);", "y[t * C + c] = (float)(xf * g) + b;"),
     "affine_one_plus_gain_exact": ("if (plus_one) g = 1.0f + g;\n      y[t * C + c] = fmaf(xf, g, b);",
                                    "y[t * C + c] = plus_one ? (float)((double)xf * (1.0 + (double)g) + (double)b) : fmaf(xf, g, b);"),
-    "affine_plus_one_ignored": ("if (plus_one) g = 1.0f + g;", "if (plus_one) g = g;"),
+    "affine_plus_one_ignored": ("if (plus_one) g = 1.0f + g;\n      y[t * C + c] = fmaf(xf, g, b);",
+                                "if (plus_one) g = g;\n      y[t * C + c] = fmaf(xf, g, b);"),
+    "layernorm_plus_one_ignored": ("if (plus_one) g = 1.0f + g;\n      y[t * C + c] = fmaf(d[c] * rstd, g, bc);",
+                                   "if (plus_one) g = g;\n      y[t * C + c] = fmaf(d[c] * rstd, g, bc);"),
     "affine_bias_of_next_channel": ("const float b = (float)bf16_to_double(bias[c]);",
                                     "const float b = (float)bf16_to_double(bias[c + 1 < C ? c + 1 : c]);"),
     "affine_ignores_row_stride": ("const float xf = (float)bf16_to_double(x[t * ld + c]);",
