@@ -178,7 +178,7 @@ int fb4_init(fb4_ctx** out, int device, const uint8_t* formatbook, const uint32_
     return fb4_set_cuda_error(e);
   }
   size_t fast_bytes = 0;
-  if (fb4_fast_build_tables(ctx->host_tables, &ctx->d_fast_tables, &fast_bytes) &&
+  if (fb4_fast_build_tables(ctx->host_tables, c.select_mode, &ctx->d_fast_tables, &fast_bytes) &&
       fb4_fast_prepare_device() == cudaSuccess)
     ctx->fast_ok = 1;
   ctx->fast_table_bytes = fast_bytes;

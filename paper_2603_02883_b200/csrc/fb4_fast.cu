@@ -1360,12 +1360,19 @@ cudaError_t launch(const CUtensorMap& map, const SmemTables* tables, const FastP
 // Builds the packed tables of this kernel from the plain ones; returns false when the formatbook /
 // stage-1 table does not fit them (more than 8 groups, a group with 0 or more than 8 dialects, or
 // error sums that could overflow a byte): those contexts use the generic kernel.
-bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes) {
+bool fb4_fast_build_tables(const Fb4DeviceTables& t, int select_mode, void** d_out, size_t* bytes) {
   FastTables ft;
   std::memset(&ft, 0, sizeof ft);
   uint32_t groups[kMaxGroups];
   int ngroups = 0;
-  for (int k = 0; k < 32; ++k) {
+  // A context that scores every dialect never looks a stage-1 group up: its error words hold the 32 dialects
+  // once, eight to a word in id order, instead of the (padded) stage-1 groups.
+  if (select_mode == 1) {
+    for (int i = 0; i < 4; ++i) groups[i] = 0xffu << (8 * i);
+    ngroups = 4;
+  }
+  for (int k = 0; k < 32 && select_mode == 1; ++k) ft.stage1[k] = t.stage1[k];
+  for (int k = 0; k < 32 && select_mode != 1; ++k) {
     const uint32_t m = t.stage1[k];
     const int pc = __builtin_popcount(m);
     if (pc == 0 || pc > 8) return false;

@@ -63,7 +63,7 @@ struct fb4_ctx {
 int fb4_set_cuda_error(cudaError_t e);   // records e, returns FB4_ERR_CUDA
 
 // TMA-staged kernel of the default configuration (fb4_fast.cu)
-bool fb4_fast_build_tables(const Fb4DeviceTables& t, void** d_out, size_t* bytes);
+bool fb4_fast_build_tables(const Fb4DeviceTables& t, int select_mode, void** d_out, size_t* bytes);
 cudaError_t fb4_fast_prepare_device();
 bool fb4_fast_eligible(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld);
 cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, int64_t ld,
