@@ -1029,6 +1029,28 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
   if (SEDA && bad_cid && lane == 0) atomicOr(p.status, 2u);
 }
 
+// Float32 sum / difference with one bf16 half of a packed register as the first operand (HALF 0 = low, 1 = high):
+// the half is converted exactly and the result rounded once, as for __fadd_rn / __fsub_rn on the unpacked
+// value, but the instruction reads the half where it lies, without the shift or mask that unpacks it.
+template <int HALF>
+__device__ __forceinline__ float bf16_plus_f32(uint32_t w, float c) {
+  float d;
+  if (HALF == 0)
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tadd.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
+  else
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tadd.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
+  return d;
+}
+template <int HALF>
+__device__ __forceinline__ float bf16_minus_f32(uint32_t w, float c) {
+  float d;
+  if (HALF == 0)
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
+  else
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
+  return d;
+}
+
 // ---------------------------------------------------------------------------------------------
 // LayerNorm + per-channel modulation fused in front of the quantizer (App. D.2 names LayerNorm as an
 // operation the quantizer runs behind; the adaLN blocks modulate the normalised activation as
@@ -1220,11 +1242,11 @@ fb4_quantize_layernorm_kernel(const __grid_constant__ CUtensorMap tmap, const Sm
 #pragma unroll
     for (int ab = 0; ab < 2; ++ab) {
       float s = __uint_as_float(w[ab][0] << 16);
-      s = __fadd_rn(s, __uint_as_float(w[ab][0] & 0xffff0000u));
+      s = bf16_plus_f32<1>(w[ab][0], s);
 #pragma unroll
       for (int k = 1; k < 16; ++k) {
-        s = __fadd_rn(s, __uint_as_float(w[ab][k] << 16));
-        s = __fadd_rn(s, __uint_as_float(w[ab][k] & 0xffff0000u));
+        s = bf16_plus_f32<0>(w[ab][k], s);
+        s = bf16_plus_f32<1>(w[ab][k], s);
       }
       sum[ab] = s;
     }
@@ -1249,9 +1271,9 @@ fb4_quantize_layernorm_kernel(const __grid_constant__ CUtensorMap tmap, const Sm
     for (int k = 0; k < 16; ++k) {
 #pragma unroll
       for (int ab = 0; ab < 2; ++ab) {
-        const float d0 = __fsub_rn(__uint_as_float(w[ab][k] << 16), mean[ab]);
+        const float d0 = bf16_minus_f32<0>(w[ab][k], mean[ab]);
         q[ab] = __fmaf_rn(d0, d0, q[ab]);
-        const float d1 = __fsub_rn(__uint_as_float(w[ab][k] & 0xffff0000u), mean[ab]);
+        const float d1 = bf16_minus_f32<1>(w[ab][k], mean[ab]);
         q[ab] = __fmaf_rn(d1, d1, q[ab]);
       }
     }
@@ -1277,9 +1299,9 @@ fb4_quantize_layernorm_kernel(const __grid_constant__ CUtensorMap tmap, const Sm
           uint32_t y[2];
 #pragma unroll
           for (int hlf = 0; hlf < 2; ++hlf) {
-            const float xv = __uint_as_float(hlf ? (w[ab][k] & 0xffff0000u) : (w[ab][k] << 16));
+            const float dv = hlf ? bf16_minus_f32<1>(w[ab][k], mean[ab]) : bf16_minus_f32<0>(w[ab][k], mean[ab]);
             const float bv = __uint_as_float(hlf ? (bw[k] & 0xffff0000u) : (bw[k] << 16));
-            y[hlf] = __float_as_uint(__fmaf_rn(__fmul_rn(__fsub_rn(xv, mean[ab]), rstd), gf[2 * k + hlf], bv));
+            y[hlf] = __float_as_uint(__fmaf_rn(__fmul_rn(dv, rstd), gf[2 * k + hlf], bv));
           }
           yw[k] = __byte_perm(y[0], y[1], 0x7632);
         }
