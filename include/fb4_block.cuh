@@ -82,6 +82,30 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
   asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
   return v;
 }
+// Float32 sum / difference with one bf16 half of a packed register as the first operand (HALF 0 = low, 1 = high):
+// the half is converted exactly and the result rounded once, as for __fadd_rn / __fsub_rn on the unpacked
+// value, but the instruction reads the half where it lies, without the shift or mask that unpacks it.
+template <int HALF>
+__device__ __forceinline__ float bf16_plus_f32(uint32_t w, float c) {
+  float d;
+  if (HALF == 0)
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tadd.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
+  else
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tadd.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
+  return d;
+}
+template <int HALF>
+__device__ __forceinline__ float bf16_minus_f32(uint32_t w, float c) {
+  float d;
+  if (HALF == 0)
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
+  else
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
+  return d;
+}
+// The low bf16 of a packed register as float32 (x + -0 = x for every x): the FMA pipe instead of a shift on the
+// busier ALU pipe.
+__device__ __forceinline__ float bf16_lo_as_f32(uint32_t w) { return bf16_plus_f32<0>(w, -0.0f); }
 __device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
   uint4 v;
   asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -170,7 +194,7 @@ __device__ __forceinline__ int choose_dialect_per_element(const uint32_t (&a)[16
       for (int j = 0; j < 4; ++j) {
         const uint32_t av = a[4 * q + j];
         const uint32_t t1 = __float_as_uint(__fmaf_rz(__uint_as_float(av), sG, 2.0f));         // upper element
-        const uint32_t t0 = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sG, 2.0f));   // lower element
+        const uint32_t t0 = __float_as_uint(__fmaf_rz(bf16_lo_as_f32(av), sG, 2.0f));   // lower element
         const uint2 e0 = lds_v2((t0 << 7) + qb), e1 = lds_v2((t1 << 7) + qb);
         lo += e0.x + e1.x;
         hi += e0.y + e1.y;
@@ -299,7 +323,7 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
     float gm[8];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
-      gm[2 * q] = __uint_as_float(g2[q] << 16);
+      gm[2 * q] = bf16_lo_as_f32(g2[q]);
       gm[2 * q + 1] = __uint_as_float(g2[q]);
     }
     const int did = SEL == 1 ? choose_dialect_per_element<SEDA>(a, sG, bmax, allowed, tb, qerr_lane)
@@ -354,7 +378,7 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
     for (int j = 0; j < 4; ++j) {
       const uint32_t av = a[4 * q + j];
       const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sHh[h], 0.125f));
-      const uint32_t tl = __float_as_uint(__fmaf_rz(__uint_as_float(av << 16), sLh[h], magich[h]));
+      const uint32_t tl = __float_as_uint(__fmaf_rz(bf16_lo_as_f32(av), sLh[h], magich[h]));
       b[j] = lds_u8(th * (uint32_t)kPairMul + tl);
     }
     const uint32_t idx = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);

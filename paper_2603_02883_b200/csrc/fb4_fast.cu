@@ -108,9 +108,10 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const uint32_t xw = w[4 * q + j];
-      const uint32_t d0 = __float_as_uint(__fsub_rn(__uint_as_float(xw << 16), __uint_as_float(xh[j] << 16)));
-      const uint32_t d1 =
-          __float_as_uint(__fsub_rn(__uint_as_float(xw & 0xffff0000u), __uint_as_float(xh[j] & 0xffff0000u)));
+      // x - Q(x) by the mixed-precision add and sub (the halves are read where they lie; same bits as the
+      // float32 subtraction of the unpacked values)
+      const uint32_t d0 = __float_as_uint(bf16_minus_f32<0>(xw, bf16_plus_f32<0>(xh[j], -0.0f)));
+      const uint32_t d1 = __float_as_uint(bf16_minus_f32<1>(xw, bf16_plus_f32<1>(xh[j], -0.0f)));
       dw[4 * q + j] = __byte_perm(d0, d1, 0x7632);
     }
   }
@@ -988,11 +989,13 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
           uint32_t y[2];
 #pragma unroll
           for (int hlf = 0; hlf < 2; ++hlf) {
-            const uint32_t xb = hlf ? (w[j] & 0xffff0000u) : (w[j] << 16);
+            // x as float32 by the mixed-precision add (x + -0 = x): the FMA pipe instead of a shift or mask on
+            // the busier ALU pipe
+            const float xv = hlf ? bf16_plus_f32<1>(w[j], -0.0f) : bf16_plus_f32<0>(w[j], -0.0f);
             const uint32_t f = fac[8 * q + 2 * j + hlf];
             float g = __uint_as_float(f << 16);
             if (PLUS_ONE) g = __fadd_rn(1.0f, g);
-            y[hlf] = __float_as_uint(__fmaf_rn(__uint_as_float(xb), g, __uint_as_float(f & 0xffff0000u)));
+            y[hlf] = __float_as_uint(__fmaf_rn(xv, g, __uint_as_float(f & 0xffff0000u)));
           }
           yw[4 * q + j] = __byte_perm(y[0], y[1], 0x7632);
         }
@@ -1027,28 +1030,6 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
     if (++s == kStages) { s = 0; parity ^= 1u; }
   }
   if (SEDA && bad_cid && lane == 0) atomicOr(p.status, 2u);
-}
-
-// Float32 sum / difference with one bf16 half of a packed register as the first operand (HALF 0 = low, 1 = high):
-// the half is converted exactly and the result rounded once, as for __fadd_rn / __fsub_rn on the unpacked
-// value, but the instruction reads the half where it lies, without the shift or mask that unpacks it.
-template <int HALF>
-__device__ __forceinline__ float bf16_plus_f32(uint32_t w, float c) {
-  float d;
-  if (HALF == 0)
-    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tadd.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
-  else
-    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tadd.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
-  return d;
-}
-template <int HALF>
-__device__ __forceinline__ float bf16_minus_f32(uint32_t w, float c) {
-  float d;
-  if (HALF == 0)
-    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, lo, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
-  else
-    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %1;\n\tsub.rn.f32.bf16 %0, hi, %2;\n\t}" : "=f"(d) : "r"(w), "f"(c));
-  return d;
 }
 
 // ---------------------------------------------------------------------------------------------
