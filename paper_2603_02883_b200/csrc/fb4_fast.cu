@@ -1033,6 +1033,193 @@ fb4_quantize_affine_kernel(const __grid_constant__ CUtensorMap tmap, const SmemT
 }
 
 // ---------------------------------------------------------------------------------------------
+// The same producer on the flat tiles, for contiguous tensors whose tokens are whole tiles (C a multiple of
+// 1024): the flat kernel's loop with one unit per lane (2 KB tiles, four stages, stage addresses as immediates,
+// output addresses linear in the unit number) and a grid whose warp count is a multiple of the tiles per token,
+// so a warp still keeps its tile column - and its lanes the factors of their 32 channels - while it walks down
+// the tokens.
+template <bool PLUS_ONE, bool SEDA, bool MX = false>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+fb4_quantize_affine_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
+                                FlatParams p, const uint16_t* __restrict__ gain, const uint16_t* __restrict__ bias,
+                                Fb4RowExtras ex) {
+  constexpr int kSt = kStages;
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t g0 = blockIdx.x * kWarps + warp;
+  const uint32_t wstride = gridDim.x * kWarps;          // a multiple of the tiles per token (chosen by the host)
+  const uint32_t tpr = p.units_row >> 5;                // tiles per token
+  const uint32_t table_bar = smem_u32(bars + kWarps * kStages);
+  if (lane == 0) {
+    for (int i = 0; i < kSt; ++i) mbar_init(smem_u32(bars + warp * kStages + i), 1);
+    if (warp == 0) mbar_init(table_bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (warp == 0) {
+      mbar_expect_tx(table_bar, (uint32_t)sizeof(SmemTables));
+      bulk_load(smem_u32(tb), g_tables, (uint32_t)sizeof(SmemTables), table_bar);
+    }
+  }
+  __syncthreads();
+  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytes);
+  const uint32_t my_bars = smem_u32(bars + warp * kStages);
+  const int32_t n_mine = g0 < p.n_tiles ? (int32_t)((p.n_tiles - g0 + wstride - 1) / wstride) : 0;
+  int32_t y_pre = (int32_t)(g0 * 16u);                  // first 128-byte row of the next tile to request
+  const int32_t y_step = (int32_t)(wstride * 16u);
+#pragma unroll
+  for (int s = 0; s < kSt; ++s) {
+    if (s < n_mine && lane == 0) {
+      mbar_expect_tx(my_bars + 8 * s, kTileBytes);
+      tma_load_2d(my_ring + s * kTileBytes, &tmap, my_bars + 8 * s, 0, y_pre);
+    }
+    y_pre += y_step;
+  }
+  const uint32_t col = g0 % tpr;                        // this warp's tile column, for the whole launch
+  uint32_t row = g0 / tpr;
+  const uint32_t row_step = wstride / tpr;
+  const uint32_t rem = col * 32u + (uint32_t)lane;      // this lane's unit inside a token = its block of channels
+  uint32_t unit = g0 * 32u + (uint32_t)lane;
+  const uint32_t unit_step = wstride * 32u;
+  // gain and bias of this lane's 32 channels: fac[i] = gain bits | bias bits << 16
+  uint32_t fac[32];
+  {
+    uint32_t gw[16], bw[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) gw[k] = bw[k] = 0u;
+    if (n_mine > 0) {
+      const uint4* gp = reinterpret_cast<const uint4*>(gain + (size_t)rem * 32);
+      const uint4* bp = reinterpret_cast<const uint4*>(bias + (size_t)rem * 32);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint4 g = __ldg(gp + q), b = __ldg(bp + q);
+        gw[4 * q] = g.x; gw[4 * q + 1] = g.y; gw[4 * q + 2] = g.z; gw[4 * q + 3] = g.w;
+        bw[4 * q] = b.x; bw[4 * q + 1] = b.y; bw[4 * q + 2] = b.z; bw[4 * q + 3] = b.w;
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      fac[2 * k] = (gw[k] & 0xffffu) | (bw[k] << 16);
+      fac[2 * k + 1] = (gw[k] >> 16) | (bw[k] & 0xffff0000u);
+    }
+  }
+  {
+    uint32_t spins = 0;
+    bool ready = mbar_try_wait(table_bar, 0u);
+    while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(table_bar, 0u);
+    if (!__all_sync(0xffffffffu, ready)) {
+      if (lane == 0) atomicOr(p.status, 1u);
+      for (int j = 0; j < kSt && j < n_mine; ++j) {
+        uint32_t tries = 0;
+        while (!mbar_try_wait(my_bars + 8 * j, 0u) && ++tries < kSpinLimit) {}
+      }
+      return;
+    }
+  }
+  const uint32_t pair_base = smem_u32(tb->pairlut);
+  const uint32_t qerr_base = smem_u32(tb->qerr_private) + ((uint32_t)lane & 15u) * 8u;
+  uint32_t chunk[4];      // this lane's 16-byte chunks in stage 0: row lane / 2, chunks (lane & 1) * 4 + j
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t r = (uint32_t)lane >> 1, c = ((uint32_t)lane & 1u) * 4u + (uint32_t)j;
+    chunk[j] = my_ring + r * 128u + ((c ^ (r & 7u)) << 4);
+  }
+  // cluster mask of a token, fetched one tile ahead; an id outside [-1, n_clusters) counts as -1 and is reported
+  bool bad_cid = false;
+  auto row_mask = [&](uint32_t t) -> uint32_t {
+    const int32_t cid = __ldg(ex.cluster_id + t);
+    if ((uint32_t)cid < (uint32_t)ex.n_clusters) {
+      const uint32_t m = __ldg(ex.cluster_mask + cid);
+      return m ? m : 1u;   // a zero mask (precondition violated) yields dialect 0
+    }
+    if (cid != -1) bad_cid = true;
+    return 0xffffffffu;
+  };
+  uint32_t mask_next = 0xffffffffu;
+  if (SEDA && n_mine > 0) mask_next = row_mask(row);
+
+  uint32_t parity = 0;
+  bool failed = false;
+  for (int32_t it = 0; it < n_mine && !failed; it += kSt) {
+#pragma unroll
+    for (int s = 0; s < kSt; ++s) {
+      if (it + s < n_mine && !failed) {
+        const uint32_t allowed = mask_next;
+        if (SEDA && it + s + 1 < n_mine) mask_next = row_mask(row + row_step);
+        const uint32_t bar = my_bars + 8 * s;
+        uint32_t spins = 0;
+        bool ready = mbar_try_wait(bar, parity);
+        while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(bar, parity);
+        if (!__all_sync(0xffffffffu, ready)) {
+          // A load never arrived: raise the status bit, give the loads still in flight for this warp a
+          // bounded chance to land, stop.
+          if (lane == 0) atomicOr(p.status, 1u);
+          for (int j = 1; j < kSt; ++j) {
+            if (it + s + j >= n_mine) break;
+            const int sj = (s + j) % kSt;
+            const uint32_t pj = (s + j) >= kSt ? (parity ^ 1u) : parity;
+            uint32_t tries = 0;
+            while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
+          }
+          failed = true;
+        } else {
+          uint32_t yw[16];     // y cut to its upper 16 bits, two per register
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const uint4 v = lds_v4(chunk[q] + s * kTileBytes);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint32_t y[2];
+#pragma unroll
+              for (int hlf = 0; hlf < 2; ++hlf) {
+                const float xv = hlf ? bf16_plus_f32<1>(w[j], -0.0f) : bf16_plus_f32<0>(w[j], -0.0f);
+                const uint32_t f = fac[8 * q + 2 * j + hlf];
+                float g = __uint_as_float(f << 16);
+                if (PLUS_ONE) g = __fadd_rn(1.0f, g);
+                y[hlf] = __float_as_uint(__fmaf_rn(xv, g, __uint_as_float(f & 0xffff0000u)));
+              }
+              yw[4 * q + j] = __byte_perm(y[0], y[1], 0x7632);
+            }
+          }
+          uint32_t cw[4], Eb[2];
+          int did[2];
+          quantize_packed_block<SEDA, false, false>(yw, allowed, tb, qerr_base, pair_base, 3u, 254u, cw, did, Eb);
+          const uint32_t m = (Eb[0] - 3u) | ((uint32_t)did[0] << 8);
+          if (unit < p.n_units) {
+            if (MX) {
+              const uint2 fb = tb->fb_e4m3[did[0]];
+              uint32_t o[8];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) fb4dev::codes_to_e4m3(cw[q], fb, o[2 * q], o[2 * q + 1]);
+              stg_v8(p.e4m3 + (size_t)unit * 32u, o);
+              const int64_t so = p.scale_tiled ? fb4dev::mx_scale_offset(row, rem, p.units_row, p.scale_col_tiles, 1)
+                                               : (int64_t)unit;
+              p.scales[so] = (uint8_t)m;
+            } else {
+              *reinterpret_cast<uint4*>(p.codes + (size_t)unit * 16u) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+              p.meta[unit] = (uint16_t)m;
+            }
+          }
+          // ---- refill this stage (all lanes have consumed their registers from it)
+          __syncwarp();
+          if (lane == 0 && it + s + kSt < n_mine) {
+            mbar_expect_tx(bar, kTileBytes);
+            tma_load_2d(my_ring + s * kTileBytes, &tmap, bar, 0, y_pre);
+          }
+          y_pre += y_step;
+          unit += unit_step;
+          row += row_step;
+        }
+      }
+    }
+    parity ^= 1u;
+  }
+  if (SEDA && bad_cid && lane == 0) atomicOr(p.status, 2u);
+}
+
+// ---------------------------------------------------------------------------------------------
 // LayerNorm + per-channel modulation fused in front of the quantizer (App. D.2 names LayerNorm as an
 // operation the quantizer runs behind; the adaLN blocks modulate the normalised activation as
 // y = n * (1 + scale_c) + shift_c).  A token's C channels (a multiple of 1024, at most 16 384) belong to
@@ -1518,6 +1705,14 @@ cudaError_t fb4_fast_prepare_device() {
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, false, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<false, true, true>, attr, bytes);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_kernel<true, true, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_flat_kernel<false, false, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_flat_kernel<true, false, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_flat_kernel<false, true, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_flat_kernel<true, true, false>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_flat_kernel<false, false, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_flat_kernel<true, false, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_flat_kernel<false, true, true>, attr, bytes);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_affine_flat_kernel<true, true, true>, attr, bytes);
 #define FB4_OPT_IN(...) \
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_layernorm_kernel<__VA_ARGS__>, attr, (int)kSmemBytesLn)
   FB4_OPT_IN(false, false, 12); FB4_OPT_IN(true, false, 12); FB4_OPT_IN(false, true, 12); FB4_OPT_IN(true, true, 12);
@@ -1862,7 +2057,52 @@ cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, i
                                             const void* gain, const void* bias, int plus_one,
                                             const Fb4RowExtras& ex, uint8_t* codes, uint16_t* meta,
                                             cudaStream_t stream, uint8_t* e4m3, uint8_t* scales, int tiled) {
+  const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
+  const uint16_t* g = static_cast<const uint16_t*>(gain);
+  const uint16_t* b = static_cast<const uint16_t*>(bias);
   CUtensorMap map;
+  // Contiguous tensors whose tokens are whole tiles take the flat tiles, on the largest grid whose warps are a
+  // multiple of the tiles per token (147 CTAs for 12 or 3 tiles per token on 148 SMs).
+  if (flat_eligible(T, C, ld) && C % 1024 == 0) {
+    const int64_t tpr = C / 1024, n_tiles = T * tpr;
+    int64_t fgrid = (n_tiles + kWarps - 1) / kWarps;
+    if (fgrid > ctx->sm_count) fgrid = ctx->sm_count;
+    while (fgrid > 0 && (fgrid * kWarps) % tpr != 0) --fgrid;
+    if (fgrid > 0 && fgrid * 8 >= ctx->sm_count * 7) {     // else too few SMs would work: the strided kernel below
+      FlatParams fp;
+      int unused = 0;
+      const cudaError_t fe = flat_setup(ctx, x, T, C, true, false, &map, &fp, &unused);   // one unit per lane
+      if (fe != cudaSuccess) return fe;
+      fp.codes = codes;
+      fp.meta = meta;
+      if (e4m3) {   // MXFP8 output: padding of the tiled scale layout = scale 1, the kernel writes real entries only
+        fp.e4m3 = e4m3;
+        fp.scales = scales;
+        fp.scale_tiled = tiled;
+        const int64_t n_col = C / 32;
+        fp.scale_col_tiles = (n_col + 3) / 4;
+        if (tiled && ((T & 127) || (n_col & 3))) {
+          const cudaError_t me =
+              cudaMemsetAsync(scales, 0x7f, (size_t)(((T + 127) / 128) * fp.scale_col_tiles * 512), stream);
+          if (me != cudaSuccess) return me;
+        }
+      }
+#define FB4_AFFINE_FLAT(P, S, M)                                                                                   \
+  fb4_quantize_affine_flat_kernel<P, S, M><<<(int)fgrid, kWarps * 32, kSmemBytes, stream>>>(map, tables, fp, g, b, ex)
+      switch ((plus_one ? 1 : 0) | (ex.cluster_id ? 2 : 0) | (e4m3 ? 4 : 0)) {
+        case 0: FB4_AFFINE_FLAT(false, false, false); break;
+        case 1: FB4_AFFINE_FLAT(true, false, false); break;
+        case 2: FB4_AFFINE_FLAT(false, true, false); break;
+        case 3: FB4_AFFINE_FLAT(true, true, false); break;
+        case 4: FB4_AFFINE_FLAT(false, false, true); break;
+        case 5: FB4_AFFINE_FLAT(true, false, true); break;
+        case 6: FB4_AFFINE_FLAT(false, true, true); break;
+        default: FB4_AFFINE_FLAT(true, true, true); break;
+      }
+#undef FB4_AFFINE_FLAT
+      return cudaGetLastError();
+    }
+  }
   FastParams p;
   int grid = 0;
   const cudaError_t e = fast_setup(ctx, x, T, C, ld, false, &map, &p, &grid);
@@ -1878,9 +2118,6 @@ cudaError_t fb4_launch_quantize_fast_affine(const fb4_ctx* ctx, const void* x, i
   grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
   const int64_t n_active = ((int64_t)grid * kWarps / tpr) * tpr;
   if (n_active <= 0) return cudaErrorInvalidValue;
-  const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
-  const uint16_t* g = static_cast<const uint16_t*>(gain);
-  const uint16_t* b = static_cast<const uint16_t*>(bias);
   if (e4m3) {   // MXFP8 output: padding of the tiled scale layout = scale 1, the kernel writes real entries only
     p.e4m3 = e4m3;
     p.scales = scales;

@@ -56,7 +56,8 @@ def run_case(q, cfg, T, C, ld, kind, plus_one, expect_variant=None, seda=False):
 
 
 @pytest.mark.parametrize("T,C,ld", [(1, 64, 64), (130, 3072, 3072), (300, 1024 + 64, 1024 + 64 + 8), (257, 12288 + 64, 12288 + 64),
-                                    (5000, 64, 64), (2368 + 5, 2048, 2048), (37, 40 * 1024, 40 * 1024)])
+                                    (5000, 64, 64), (2368 + 5, 2048, 2048), (37, 40 * 1024, 40 * 1024),
+                                    (1600, 3072, 3072), (401, 12288, 12288)])   # the last three shapes: flat tiles
 @pytest.mark.parametrize("kind,plus_one", [("layernorm", False), ("modulation", True), ("wild", False), ("wild", True)])
 def test_tma_staged_kernel(T, C, ld, kind, plus_one):
     q = fb4.Fb4()
@@ -125,7 +126,7 @@ def test_argument_checks():
     q.close()
 
 
-@pytest.mark.parametrize("T,C", [(1, 64), (130, 3072), (300, 1024 + 64), (257, 128), (2368 + 5, 2048)])
+@pytest.mark.parametrize("T,C", [(1, 64), (130, 3072), (300, 1024 + 64), (257, 128), (2368 + 5, 2048), (1600, 3072)])
 @pytest.mark.parametrize("plus_one", [False, True])
 def test_affine_producer_straight_to_mxfp8(T, C, plus_one):
     """fb4_quantize_affine_mxfp8 = affine producer (oracle, fp32) -> fp32 quantizer (oracle) -> MXFP8 view (oracle),
