@@ -1,5 +1,6 @@
 // FB4 decode (4-bit codes + block metadata -> fp32 / bf16, optionally adding the decoded
 // residual of salient tokens) and the per-tile salient-token selection.
+#include "fb4_block.cuh"
 #include "fb4_device.cuh"
 #include "fb4_internal.h"
 
@@ -93,9 +94,10 @@ __device__ __forceinline__ void store_sum_word(uint8_t* dst, const uint32_t* pr,
   uint32_t v[8];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    v[2 * j] = __float_as_uint(__fadd_rn(__uint_as_float(pr[j] << 16), __uint_as_float(rr[j] << 16)));
-    v[2 * j + 1] = __float_as_uint(
-        __fadd_rn(__uint_as_float(pr[j] & 0xffff0000u), __uint_as_float(rr[j] & 0xffff0000u)));
+    // float32 sums by the mixed-precision add (the bf16 halves are read where they lie: two operations on the
+    // FMA pipe per element instead of two unpacking operations on the ALU pipe and an add)
+    v[2 * j] = __float_as_uint(fb4blk::bf16_plus_f32<0>(pr[j], fb4blk::bf16_plus_f32<0>(rr[j], -0.0f)));
+    v[2 * j + 1] = __float_as_uint(fb4blk::bf16_plus_f32<1>(pr[j], fb4blk::bf16_plus_f32<1>(rr[j], -0.0f)));
   }
   if (OUT_BF16 == 1) {
     uint4 o;
