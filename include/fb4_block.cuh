@@ -302,6 +302,16 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
     }
     const uint32_t mm = __vmaxu2(__vmaxu2(g2[0], g2[1]), __vmaxu2(g2[2], g2[3]));
     uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
+    if (!CLAMP && amax16 >= 0x7f80u) {
+      // An infinity or NaN in the block (inputs are required to be finite): every magnitude saturates at the
+      // largest finite bf16, so that the exponent, the bins and with them every table address below stay in
+      // range.  The block's output means nothing, but nothing is read or written out of bounds.
+      amax16 = 0x7f7fu;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) a[i] = __vminu2(a[i], 0x7f7f7f7fu);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) g2[q] = __vminu2(g2[q], 0x7f7f7f7fu);
+    }
     // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
     uint32_t Ec = max(amax16 >> 7, 3u);
     if (CLAMP) {
@@ -342,6 +352,14 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
       for (int k = 0; k < 8; ++k) gx[k] = __vmaxu2(a[8 * h + k], __byte_perm(a[8 * h + k], 0u, 0x1032));
       uint32_t mm = __vmaxu2(__vmaxu2(__vmaxu2(gx[0], gx[1]), __vmaxu2(gx[2], gx[3])),
                              __vmaxu2(__vmaxu2(gx[4], gx[5]), __vmaxu2(gx[6], gx[7])));
+      if (!CLAMP && (mm & 0xffffu) >= 0x7f80u) {      // an infinity or NaN: saturate, as for block size 32
+        mm = 0x7f7f7f7fu;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          a[8 * h + k] = __vminu2(a[8 * h + k], 0x7f7f7f7fu);
+          gx[k] = __vminu2(gx[k], 0x7f7f7f7fu);
+        }
+      }
       uint32_t Ec = max((mm & 0xffffu) >> 7, 3u);
       if (CLAMP) {
         Ec = min(max((mm & 0xffffu) >> 7, ec_lo), ec_hi);
