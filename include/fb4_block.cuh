@@ -77,6 +77,10 @@ __device__ __forceinline__ uint32_t lds_u8(uint32_t addr) {
   asm("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
   return v;
 }
+// A byte load that a flag switches off: with ok == 0 nothing is read and dst keeps the value it came with.
+__device__ __forceinline__ void lds_u8_if(uint32_t& dst, uint32_t addr, uint32_t ok) {
+  asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t@p ld.shared.u8 %0, [%1];\n\t}" : "+r"(dst) : "r"(addr), "r"(ok));
+}
 __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
   uint2 v;
   asm("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
@@ -280,7 +284,7 @@ __device__ __forceinline__ int choose_dialect_all(const float (&gm)[8], float sG
 // dialect and the biased exponent.
 // SEL: 0 = 8 groups, two-stage selection (the default); 1 = every element its own group (block size 32 only);
 // 2 = 8 groups, every allowed dialect scored (select_mode 1).
-template <bool SEDA, bool B16, bool CLAMP, int SEL = 0>
+template <bool SEDA, bool B16, bool CLAMP, int SEL = 0, bool BRANCHY = false>
 __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], uint32_t allowed, const Tables* tb,
                                                       uint32_t qerr_lane, uint32_t pair_base, uint32_t ec_lo,
                                                       uint32_t ec_hi, uint32_t (&cw)[4], int (&didh)[2],
@@ -292,6 +296,7 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
   // per half of the lane's 32 elements (block size 32: both halves belong to one block):
   // biased exponent, the two bin scales of the Qvalue lookup, the chosen dialect's table address
   float sHh[2], sLh[2], magich[2];
+  uint32_t finite = 1u;     // block size 32 without exponent clamp: 0 switches the value lookups off
   if (!B16) {
     uint32_t g2[4];   // (group 2q+1 max << 16) | group 2q max
 #pragma unroll
@@ -302,15 +307,30 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
     }
     const uint32_t mm = __vmaxu2(__vmaxu2(g2[0], g2[1]), __vmaxu2(g2[2], g2[3]));
     uint32_t amax16 = max(mm & 0xffffu, mm >> 16);
-    if (!CLAMP && amax16 >= 0x7f80u) {
-      // An infinity or NaN in the block (inputs are required to be finite): every magnitude saturates at the
-      // largest finite bf16, so that the exponent, the bins and with them every table address below stay in
-      // range.  The block's output means nothing, but nothing is read or written out of bounds.
-      amax16 = 0x7f7fu;
+    // An infinity or NaN in the block (inputs are required to be finite) must not turn into a table address out of
+    // range.  The group maxima and the block maximum saturate at the largest finite bf16, so the exponent and the
+    // error lookups stay in range; the value lookups further down are switched off for such a block (`finite` = 0).
+    // Its output means nothing, but nothing is read or written out of bounds.  No branch: one in the middle of the
+    // block's dependency chain cost the one-unit-per-lane kernels 3 to 15 %.
+    // BRANCHY: the same protection as a rare branch that saturates every magnitude; cheaper (3 instead of 13
+    // instructions per block) where a lane works on two blocks at a time and the branch does not hold anything up.
+    if (!CLAMP && BRANCHY) {
+      if (amax16 >= 0x7f80u) {
+        amax16 = 0x7f7fu;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) a[i] = __vminu2(a[i], 0x7f7f7f7fu);
+        for (int i = 0; i < 16; ++i) a[i] = __vminu2(a[i], 0x7f7f7f7fu);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) g2[q] = __vminu2(g2[q], 0x7f7f7f7fu);
+      }
+    } else if (!CLAMP) {
+      finite = amax16 < 0x7f80u ? 1u : 0u;
+      amax16 = min(amax16, 0x7f7fu);
 #pragma unroll
       for (int q = 0; q < 4; ++q) g2[q] = __vminu2(g2[q], 0x7f7f7f7fu);
+      if (SEL == 1) {     // every element is a group maximum here
+#pragma unroll
+        for (int i = 0; i < 16; ++i) a[i] = __vminu2(a[i], 0x7f7f7f7fu);
+      }
     }
     // ---- exponent: e = max(field,3) - 127 >= -124; element scale byte = field - 3
     uint32_t Ec = max(amax16 >> 7, 3u);
@@ -397,7 +417,12 @@ __device__ __forceinline__ void quantize_packed_block(const uint32_t (&w)[16], u
       const uint32_t av = a[4 * q + j];
       const uint32_t th = __float_as_uint(__fmaf_rz(__uint_as_float(av), sHh[h], 0.125f));
       const uint32_t tl = __float_as_uint(__fmaf_rz(bf16_lo_as_f32(av), sLh[h], magich[h]));
-      b[j] = lds_u8(th * (uint32_t)kPairMul + tl);
+      if (B16 || CLAMP || BRANCHY) {
+        b[j] = lds_u8(th * (uint32_t)kPairMul + tl);
+      } else {
+        b[j] = th;      // any defined value: the load replaces it unless the block holds an infinity or NaN
+        lds_u8_if(b[j], th * (uint32_t)kPairMul + tl, finite);
+      }
     }
     const uint32_t idx = b[0] | (b[1] << 8) | (b[2] << 16) | (b[3] << 24);
     // sign bits: byte masks by sign replication, then to bit 3 of every nibble

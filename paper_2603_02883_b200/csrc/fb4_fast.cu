@@ -543,7 +543,8 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
             }
             uint32_t c4[4], Ech[2];
             int didh[2];
-            quantize_packed_block<SEDA, B16, CLAMP, SEL>(w, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, c4, didh, Ech);
+            quantize_packed_block<SEDA, B16, CLAMP, SEL, U == 2>(w, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, c4, didh,
+                                                                 Ech);
 #pragma unroll
             for (int q = 0; q < 4; ++q) cw[4 * h + q] = c4[q];
             did0[h] = didh[0];
