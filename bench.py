@@ -33,9 +33,9 @@ FALLBACK_HBM_GBS = 6650.0
 # ncu capture summarised in profiles/fb4_quantize_flat_c5_plain_dram_bytes.md (1 858 046 464 B read +
 # 499 021 056 B written).  The capture's date and the kernel's register count travel with it in the bench line,
 # so that a constant that has outlived the kernel shows; set it back to None whenever that kernel changes.
-NCU_TRAFFIC_BYTES = 2357283584
+NCU_TRAFFIC_BYTES = 2357105152
 NCU_TRAFFIC_SOURCE = {"profile": "profiles/fb4_quantize_flat_c5_plain_dram_bytes.md", "captured": "2026-11-30",
-                      "kernel": "fb4_quantize_flat_kernel<0,0,0,0,0,0>", "registers_per_thread": 117}
+                      "kernel": "fb4_quantize_flat_kernel<0,0,0,0,0,0>", "registers_per_thread": 115}
 
 
 def algorithmic_bytes(T: int, C: int, B: int = 32, n_res_rows: int = 0, seda: bool = False,
