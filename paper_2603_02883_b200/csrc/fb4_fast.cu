@@ -45,7 +45,7 @@ using namespace fb4stage;
 // as the main pass, from the upper 16 bits of every Delta (see quantize_packed_block).
 // w = the 16 input registers (2 bf16 each), cw = the 4 code words, didh / Ech = dialect and biased
 // exponent per half (equal halves for block size 32).
-template <bool SEDA, bool B16, bool CLAMP, int SEL = 0>
+template <bool SEDA, bool B16, bool CLAMP, int SEL = 0, bool BRANCHY = false>
 __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t* cw, const int* didh,
                                                const uint32_t* Ech, uint32_t allowed, const SmemTables* tb,
                                                uint32_t qerr_lane, uint32_t pair_base, uint32_t ec_lo, uint32_t ec_hi,
@@ -70,7 +70,7 @@ __device__ __forceinline__ void residual_block(const uint32_t* w, const uint32_t
   }
   uint32_t rc[4], rE[2];
   int rd[2];
-  quantize_packed_block<SEDA, B16, CLAMP, SEL>(dw, allowed, tb, qerr_lane, pair_base, ec_lo, ec_hi, rc, rd, rE);
+  quantize_packed_block<SEDA, B16, CLAMP, SEL, BRANCHY>(dw, allowed, tb, qerr_lane, pair_base, ec_lo, ec_hi, rc, rd, rE);
 #pragma unroll
   for (int q = 0; q < 4; ++q) rcw[q] = rc[q];
   *rmeta = B16 ? (((rE[0] - 3u) | ((uint32_t)rd[0] << 8)) | (((rE[1] - 3u) | ((uint32_t)rd[1] << 8)) << 16))
@@ -361,6 +361,9 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
   constexpr int U = flat_units(DECOMP, MX);     // units per lane
   constexpr int kSt = kStages / U;              // stages per warp: the ring holds 8 KB per warp either way
   constexpr int kTileB = kTileBytes * U;
+  // which form the block routine's protection against non-finite input takes (by measurement: the branch costs
+  // nothing where a lane holds two blocks, and less than the switchable loads in the MXFP8 kernel with a residual pass)
+  constexpr bool kBranchy = U == 2 || (MX && DECOMP);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
@@ -543,8 +546,8 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
             }
             uint32_t c4[4], Ech[2];
             int didh[2];
-            quantize_packed_block<SEDA, B16, CLAMP, SEL, U == 2>(w, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, c4, didh,
-                                                                 Ech);
+            quantize_packed_block<SEDA, B16, CLAMP, SEL, kBranchy>(w, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi, c4,
+                                                                   didh, Ech);
 #pragma unroll
             for (int q = 0; q < 4; ++q) cw[4 * h + q] = c4[q];
             did0[h] = didh[0];
@@ -553,7 +556,7 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
             if (DECOMP) {     // one unit per lane: the residual follows at once, from the same registers
               if (srow >= 0) {
                 uint32_t rcw[4], rrec;
-                residual_block<SEDA, B16, CLAMP, SEL>(w, c4, didh, Ech, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi,
+                residual_block<SEDA, B16, CLAMP, SEL, kBranchy>(w, c4, didh, Ech, allowed, tb, qerr_base, pair_base, p.ec_lo, p.ec_hi,
                                                  rcw, &rrec);
                 const size_t ru = (size_t)srow * p.units_row + pos.rem;      // unit of the residual tensor
                 if (MX) {
