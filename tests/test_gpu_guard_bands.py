@@ -33,7 +33,8 @@ class Guarded:
         assert bool((a == FILL).all()) and bool((b == FILL).all()), f"guard band of {what} was written"
 
 
-SHAPES = [(1, 32), (3, 96), (37, 64), (19, 1024), (5, 1024 + 64), (130, 3072), (7, 12288 + 128), (2368, 64)]
+SHAPES = [(1, 32), (3, 96), (37, 64), (19, 1024), (5, 1024 + 64), (130, 3072), (7, 12288 + 128), (2368, 64),
+          (2373, 2048)]      # the last one is large enough for the grids of the flat producer kernels
 
 
 @pytest.mark.parametrize("T,C", SHAPES)
