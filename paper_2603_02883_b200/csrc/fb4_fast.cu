@@ -626,11 +626,12 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
 
 // ---------------------------------------------------------------------------------------------
 // fp32 input (the hook for a producer that still holds its result in fp32): same ring and tables,
-// 8 warps per CTA, tiles of 1024 channels = 4 KB (view [T][C/32][32 floats], box 1 x 32 x 32,
+// 12 warps per CTA, tiles of 1024 channels = 4 KB (view [T][C/32][32 floats], box 1 x 32 x 32,
 // 128-byte swizzle: row r of a stage is block r).  Lane i reads its block with eight conflict-free
 // 16-byte shared loads, keeps the upper 16 bits of every value and quantizes them with
 // quantize_packed_block.
-constexpr int kWarpsF32 = 8;
+constexpr int kWarpsF32 = 12;      // 80 registers: three warps per scheduler; three stages of 4 KB each keep the ring at 144 KB
+constexpr int kStagesF32 = 3;
 constexpr int kTileBytesF32 = 4096;
 
 __global__ void __launch_bounds__(kWarpsF32 * 32, 1)
@@ -638,19 +639,19 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
                         FastParams p) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarpsF32 * kStages * kTileBytesF32);
+  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarpsF32 * kStagesF32 * kTileBytesF32);
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t gwarp = (int64_t)blockIdx.x * kWarpsF32 + warp;
   const int64_t wstride = (int64_t)gridDim.x * kWarpsF32;
   const int32_t tpr = (int32_t)p.tiles_per_row;
 
-  const uint32_t table_bar = smem_u32(bars + kWarpsF32 * kStages);
+  const uint32_t table_bar = smem_u32(bars + kWarpsF32 * kStagesF32);
   // every warp initialises its own ring barriers; the first thread also the table barrier, and it
-  // starts the table copy at once (one thread doing all kWarpsF32 * kStages + 1 inits in a row used to
+  // starts the table copy at once (one thread doing all kWarpsF32 * kStagesF32 + 1 inits in a row used to
   // hold the whole CTA for most of a microsecond)
   if (lane == 0) {
-    for (int i = 0; i < kStages; ++i) mbar_init(smem_u32(bars + warp * kStages + i), 1);
+    for (int i = 0; i < kStagesF32; ++i) mbar_init(smem_u32(bars + warp * kStagesF32 + i), 1);
     if (warp == 0) mbar_init(table_bar, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (warp == 0) {
@@ -660,8 +661,8 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
   }
   __syncthreads();
 
-  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytesF32);
-  const uint32_t my_bars = smem_u32(bars + warp * kStages);
+  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStagesF32 * kTileBytesF32);
+  const uint32_t my_bars = smem_u32(bars + warp * kStagesF32);
   TilePos cur, pre;
   cur.row = (int32_t)(gwarp / tpr);
   cur.col = (int32_t)(gwarp - (int64_t)cur.row * tpr);
@@ -669,7 +670,7 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
   const int32_t n_mine = gwarp < p.n_tiles ? (int32_t)((p.n_tiles - gwarp + wstride - 1) / wstride) : 0;
   int32_t it_pre = 0;
 #pragma unroll
-  for (int s = 0; s < kStages; ++s) {
+  for (int s = 0; s < kStagesF32; ++s) {
     if (it_pre < n_mine && lane == 0) {
       mbar_expect_tx(my_bars + 8 * s, kTileBytesF32);
       tma_load_tile(my_ring + s * kTileBytesF32, &tmap, my_bars + 8 * s, pre.col * 32, pre.row);
@@ -683,7 +684,7 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
     while (!ready && ++spins < kSpinLimit) ready = mbar_try_wait(table_bar, 0u);
     if (!__all_sync(0xffffffffu, ready)) {
       if (lane == 0) atomicOr(p.status, 1u);
-      for (int j = 0; j < kStages && j < n_mine; ++j) {
+      for (int j = 0; j < kStagesF32 && j < n_mine; ++j) {
         uint32_t tries = 0;
         while (!mbar_try_wait(my_bars + 8 * j, 0u) && ++tries < kSpinLimit) {}
       }
@@ -709,9 +710,9 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
       if (lane == 0) atomicOr(p.status, 1u);
       int sj = s;
       uint32_t pj = parity;
-      for (int j = 1; j < kStages; ++j) {
+      for (int j = 1; j < kStagesF32; ++j) {
         if (it + j >= n_mine) break;
-        if (++sj == kStages) { sj = 0; pj ^= 1u; }
+        if (++sj == kStagesF32) { sj = 0; pj ^= 1u; }
         uint32_t tries = 0;
         while (!mbar_try_wait(my_bars + 8 * sj, pj) && ++tries < kSpinLimit) {}
       }
@@ -747,12 +748,12 @@ fb4_quantize_f32_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTabl
     ++it_pre;
     pre.advance(p, tpr);
     cur.advance(p, tpr);
-    if (++s == kStages) { s = 0; parity ^= 1u; }
+    if (++s == kStagesF32) { s = 0; parity ^= 1u; }
   }
 }
 
 constexpr size_t kSmemBytesF32 =
-    1024 + (size_t)kWarpsF32 * kStages * kTileBytesF32 + sizeof(SmemTables) + (kWarpsF32 * kStages + 1) * 8;
+    1024 + (size_t)kWarpsF32 * kStagesF32 * kTileBytesF32 + sizeof(SmemTables) + (kWarpsF32 * kStagesF32 + 1) * 8;
 static_assert(kSmemBytesF32 <= 227 * 1024, "shared memory budget of one CTA");
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
