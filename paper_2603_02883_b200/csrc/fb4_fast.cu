@@ -354,19 +354,21 @@ fb4_quantize_fast_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
 // units per lane and tile of a flat kernel
 __host__ __device__ constexpr int flat_units(bool decomp, bool mx) { return (decomp || mx) ? 1 : 2; }
 
-template <bool SEDA, bool DECOMP, bool B16, bool CLAMP, bool MX = false, int SEL = 0>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+// NW warps per CTA: 16, or 20 for the kernels with a residual pass that fit 96 registers (three stages per warp then).
+template <bool SEDA, bool DECOMP, bool B16, bool CLAMP, bool MX = false, int SEL = 0, int NW = kWarps>
+__global__ void __launch_bounds__(NW * 32, 1)
 fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTables* __restrict__ g_tables,
                          FlatParams p, Fb4RowExtras ex) {
   constexpr int U = flat_units(DECOMP, MX);     // units per lane
-  constexpr int kSt = kStages / U;              // stages per warp: the ring holds 8 KB per warp either way
+  constexpr int kSt = NW == kWarps ? kStages / U : 3;   // stages per warp: 8 KB of ring per warp with 16 warps, 6 KB with 20
+  constexpr int kRing = kSt * kTileBytes * U;           // ring bytes per warp
   constexpr int kTileB = kTileBytes * U;
   // which form the block routine's protection against non-finite input takes (by measurement: the branch costs
   // nothing where a lane holds two blocks, and less than the switchable loads in the MXFP8 kernel with a residual pass)
   constexpr bool kBranchy = U == 2 || (MX && DECOMP);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + kWarps * kStages * kTileBytes);
+  SmemTables* tb = reinterpret_cast<SmemTables*>(ring + NW * kRing);
   uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(tb) + sizeof(SmemTables));
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // Tile -> warp assignment as in the strided kernel: interleaved over all warps of the grid, or (with a
@@ -377,13 +379,13 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
     const uint32_t t0 = b * per + (b < extra ? b : extra);
     g0 = t0 + warp;
     g_end = t0 + per + (b < extra ? 1u : 0u);
-    wstride = kWarps;
+    wstride = NW;
   } else {
-    g0 = blockIdx.x * kWarps + warp;
+    g0 = blockIdx.x * NW + warp;
     g_end = p.n_tiles;
-    wstride = gridDim.x * kWarps;
+    wstride = gridDim.x * NW;
   }
-  const uint32_t table_bar = smem_u32(bars + kWarps * kStages);
+  const uint32_t table_bar = smem_u32(bars + NW * kStages);
   if (lane == 0) {
     for (int i = 0; i < kSt; ++i) mbar_init(smem_u32(bars + warp * kStages + i), 1);
     if (warp == 0) mbar_init(table_bar, 1);
@@ -394,7 +396,7 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
     }
   }
   __syncthreads();
-  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kStages * kTileBytes);
+  const uint32_t my_ring = smem_u32(ring + (size_t)warp * kRing);
   const uint32_t my_bars = smem_u32(bars + warp * kStages);
   const int32_t n_mine = g0 < g_end ? (int32_t)((g_end - g0 + wstride - 1) / wstride) : 0;
   int32_t y_pre = (int32_t)(g0 * (16u * U));      // first 128-byte row of the next tile to request
@@ -774,6 +776,11 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+constexpr int kWarpsWide = 20;
+constexpr size_t kSmemBytesWide =
+    1024 + (size_t)kWarpsWide * 3 * kTileBytes + sizeof(SmemTables) + (kWarpsWide * kStages + 1) * 8;
+static_assert(kSmemBytesWide <= 227 * 1024, "shared memory budget of one CTA");
+
 template <bool SEDA, bool DECOMP, bool B16, bool CLAMP>
 cudaError_t launch(const CUtensorMap& map, const SmemTables* tables, const FastParams& p, const Fb4RowExtras& ex,
                    int grid, cudaStream_t stream) {
@@ -932,6 +939,10 @@ cudaError_t fb4_fast_prepare_device() {
   FB4_OPT_IN(false, true, false, false, false, 2);
   FB4_OPT_IN(true, true, false, false, false, 2);
 #undef FB4_OPT_IN
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(fb4_quantize_flat_kernel<false, true, false, false, false, 0, kWarpsWide>, attr, (int)kSmemBytesWide);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(fb4_quantize_flat_kernel<true, true, false, false, false, 0, kWarpsWide>, attr, (int)kSmemBytesWide);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(fb4_quantize_f32_kernel, attr, (int)kSmemBytesF32);
   if (e == cudaSuccess) e = fb4_producers_prepare_device();
   return e;
@@ -1010,7 +1021,7 @@ static bool flat_eligible(int64_t T, int64_t C, int64_t ld) {
 
 // Tensor map (2-D view [N/64][64] of the contiguous tensor), grid and walk parameters of one flat launch.
 static cudaError_t flat_setup(const fb4_ctx* ctx, const void* x, int64_t T, int64_t C, bool chunked, bool mx,
-                              CUtensorMap* map, FlatParams* p, int* grid_out) {
+                              CUtensorMap* map, FlatParams* p, int* grid_out, int nw = kWarps) {
   const uint32_t U = (uint32_t)flat_units(chunked, mx);   // units per lane: tiles of 32 * U units = 2 KB * U
   const cuuint64_t dims[2] = {64, (cuuint64_t)(T * C / 64)};
   const cuuint64_t strides[1] = {128};
@@ -1027,9 +1038,9 @@ static cudaError_t flat_setup(const fb4_ctx* ctx, const void* x, int64_t T, int6
   p->n_units = (uint32_t)(T * (C / 32));
   p->n_tiles = (p->n_units + 32u * U - 1u) / (32u * U);
   p->status = ctx->d_status;
-  const int64_t want = ((int64_t)p->n_tiles + kWarps - 1) / kWarps;
+  const int64_t want = ((int64_t)p->n_tiles + nw - 1) / nw;
   const int grid = (int)(want < ctx->sm_count ? want : ctx->sm_count);
-  const uint64_t unit_step = (uint64_t)(chunked ? kWarps : grid * kWarps) * 32u * U;
+  const uint64_t unit_step = (uint64_t)(chunked ? nw : grid * nw) * 32u * U;
   p->step_rows = (uint32_t)(unit_step / p->units_row);
   p->step_rem = (uint32_t)(unit_step % p->units_row);
   p->ec_lo = (uint32_t)(ctx->cfg.exp_min + 127);
@@ -1052,14 +1063,25 @@ cudaError_t fb4_launch_quantize_fast(const fb4_ctx* ctx, const void* x, int64_t 
   if (flat_eligible(T, C, ld)) {
     FlatParams fp;
     int grid = 0;
-    const cudaError_t e = flat_setup(ctx, x, T, C, decomp, false, &map, &fp, &grid);
+    const bool b16 = ctx->cfg.block_size == 16;
+    const bool clamp = ctx->cfg.exp_min != -124 || ctx->cfg.exp_max != 127;
+    const int sel = ctx->cfg.num_groups == 32 ? 1 : (ctx->cfg.select_mode == 1 ? 2 : 0);
+    // the default configuration with a residual pass fits 96 registers: 20 warps per CTA
+    const bool wide = decomp && !b16 && !clamp && sel == 0;
+    const cudaError_t e = flat_setup(ctx, x, T, C, decomp, false, &map, &fp, &grid, wide ? kWarpsWide : kWarps);
     if (e != cudaSuccess) return e;
     fp.codes = codes;
     fp.meta = meta;
     const SmemTables* tables = static_cast<const SmemTables*>(ctx->d_fast_tables);
-    const bool b16 = ctx->cfg.block_size == 16;
-    const bool clamp = ctx->cfg.exp_min != -124 || ctx->cfg.exp_max != 127;
-    const int sel = ctx->cfg.num_groups == 32 ? 1 : (ctx->cfg.select_mode == 1 ? 2 : 0);
+    if (wide) {
+      if (seda)
+        fb4_quantize_flat_kernel<true, true, false, false, false, 0, kWarpsWide>
+            <<<grid, kWarpsWide * 32, kSmemBytesWide, stream>>>(map, tables, fp, ex);
+      else
+        fb4_quantize_flat_kernel<false, true, false, false, false, 0, kWarpsWide>
+            <<<grid, kWarpsWide * 32, kSmemBytesWide, stream>>>(map, tables, fp, ex);
+      return cudaGetLastError();
+    }
     if (sel != 0) {
 #define FB4_SEL(S, D, L) \
   fb4_quantize_flat_kernel<S, D, false, false, false, L><<<grid, kWarps * 32, kSmemBytes, stream>>>(map, tables, fp, ex)
