@@ -628,12 +628,12 @@ fb4_quantize_flat_kernel(const __grid_constant__ CUtensorMap tmap, const SmemTab
 
 // ---------------------------------------------------------------------------------------------
 // fp32 input (the hook for a producer that still holds its result in fp32): same ring and tables,
-// 12 warps per CTA, tiles of 1024 channels = 4 KB (view [T][C/32][32 floats], box 1 x 32 x 32,
+// 16 warps per CTA, tiles of 1024 channels = 4 KB (view [T][C/32][32 floats], box 1 x 32 x 32,
 // 128-byte swizzle: row r of a stage is block r).  Lane i reads its block with eight conflict-free
 // 16-byte shared loads, keeps the upper 16 bits of every value and quantizes them with
 // quantize_packed_block.
-constexpr int kWarpsF32 = 12;      // 80 registers: three warps per scheduler; three stages of 4 KB each keep the ring at 144 KB
-constexpr int kStagesF32 = 3;
+constexpr int kWarpsF32 = 16;      // 80 registers; two stages of 4 KB each keep the ring at 128 KB
+constexpr int kStagesF32 = 2;
 constexpr int kTileBytesF32 = 4096;
 
 __global__ void __launch_bounds__(kWarpsF32 * 32, 1)
